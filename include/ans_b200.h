@@ -1,0 +1,224 @@
+/*
+ * ans_b200 -- inference-time decoding of tabled-ANS (tANS) coded, zero-point quantised
+ * neural-network weights on NVIDIA B200 (sm_100a).
+ *
+ * The operation is the decoder of "Efficient Neural Compression with Inference-time
+ * Decoding" (Metz, Bichler, Dupret; ISCAS 2024):
+ *   - Section II-A, Fig. 2: a look-up table gives, for the current state, the decoded
+ *     symbol, a number of bits nb_bits to take from the compressed stream and a
+ *     transition integer newX; the next state is newX + the bits taken.  Transitions
+ *     that take no bits are what lets the rate fall under 1 bit per weight.
+ *   - Section III-B: many streams are decoded at once with ONE table per layer and a
+ *     VECTOR of states, one state per stream.
+ *   - Section II-B: weights come from a uniform quantiser with a zero-point, so a
+ *     decoded symbol q becomes the weight  w = scale * (q - zero_point).
+ *
+ * C ABI, plain pointers and sizes.  Pointer names say where the memory lives:
+ *   h_*  host memory,  d_*  device memory of the CURRENT CUDA device.
+ * The caller owns every buffer.  Unless a function says otherwise the library
+ * allocates nothing, keeps no state except the last CUDA error code, enqueues its
+ * device work on the caller's stream (`stream` is a cudaStream_t passed as void*;
+ * NULL is the default stream) and returns without waiting for it.
+ * Every function returns ANS_OK (0) or a negative ANS_ERR_* code; none throws, aborts
+ * or prints.
+ *
+ * Containers (how one layer's symbols are cut into independently decodable pieces;
+ * the paper leaves this open beyond "one state per stream"):
+ *   A layer of n symbols (the tensor flattened in memory order) is cut into chunks of
+ *   `chunk_symbols` consecutive symbols.  Inside a chunk, `lanes` = 32*G lanes take the
+ *   symbols round-robin (chunk-relative symbol q is the (q / lanes)-th symbol of lane
+ *   q % lanes); every lane is its own tANS stream with its own state, all lanes of a
+ *   layer share the layer's table.  Lane 32*g + k is lane k of sub-stream g; sub-streams
+ *   are numbered chunk-major: sub = chunk*G + g.  Every sub-stream's bytes start at a
+ *   16-byte aligned offset of d_stream, given by d_sub_offsets[sub] (n_sub + 1 entries).
+ *   Bits are packed least-significant first; a lane's encoder starts from state index 0,
+ *   so a sound stream makes its decoder END in state index 0.
+ *     ANS_LAYOUT_INTERLEAVED: the 32 lanes of a sub-stream share ONE sequence of
+ *       little-endian 16-bit units.  Before each round every lane that still has a
+ *       symbol to decode and holds fewer than 16 buffered bits takes the next unit
+ *       (lanes in ascending order); then each such lane decodes one symbol.
+ *       d_lane_meta is uint16_t[n_sub][32]: initial state index per lane.
+ *     ANS_LAYOUT_PRIVATE: every lane owns a contiguous run of little-endian 32-bit
+ *       words inside its sub-stream, lanes in ascending order.
+ *       d_lane_meta is uint32_t[n_sub][32]: initial state | (first word, counted from
+ *       the sub-stream's start) << 16.
+ */
+#ifndef ANS_B200_H
+#define ANS_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ANS_OK                    0
+#define ANS_ERR_INVALID_ARG      -1   /* null pointer, size out of range, misaligned buffer      */
+#define ANS_ERR_BAD_FREQS        -2   /* frequencies do not sum to 2^table_log / unusable symbol */
+#define ANS_ERR_UNSUPPORTED      -3   /* table_log outside [1,14], lanes not 32*G, unknown dtype */
+#define ANS_ERR_BUFFER_TOO_SMALL -4
+#define ANS_ERR_CUDA             -5   /* a CUDA call failed; raw code from ans_last_cuda_error() */
+#define ANS_ERR_CORRUPT          -6   /* device status word: a stream did not decode soundly     */
+
+#define ANS_U8   0   /* decoded symbols, one byte each             */
+#define ANS_F32  1   /* dequantised weights, IEEE single           */
+#define ANS_BF16 2   /* dequantised weights, bfloat16 (RNE of F32) */
+
+#define ANS_LAYOUT_INTERLEAVED 0
+#define ANS_LAYOUT_PRIVATE     1
+
+#define ANS_MAX_TABLE_LOG 14
+#define ANS_MAX_ALPHABET  256
+
+/* bits of the device status word (0 = every stream sound) */
+#define ANS_STATUS_BAD_FINAL_STATE 1u   /* a lane did not end in state index 0          */
+#define ANS_STATUS_BAD_LENGTH      2u   /* a sub-stream consumed more or fewer bytes than it holds */
+#define ANS_STATUS_BAD_SYMBOL      4u   /* a decoded symbol does not fit `bitwidth` bits  */
+
+/*
+ * One layer of a decode call.  For the *_batch call an array of these lives in device
+ * memory (with a host copy for validation); all pointers inside are device pointers.
+ */
+typedef struct ans_layer_desc {
+  const void*     d_table;        /* this layer's table, written by ans_build_decode_tables  */
+  const uint8_t*  d_stream;       /* compressed bytes of all the layer's sub-streams, 16-byte aligned */
+  const uint64_t* d_sub_offsets;  /* [n_sub + 1] byte offsets into d_stream, each a multiple of 16 */
+  const void*     d_lane_meta;    /* per-lane initial state (and first word): see the layouts above */
+  void*           d_out;          /* n_symbols elements of out_dtype, 16-byte aligned       */
+  uint64_t        stream_bytes;   /* bytes readable at d_stream (offsets beyond it are flagged) */
+  uint64_t        n_symbols;      /* weights in the layer; may be 0                          */
+  uint32_t        chunk_symbols;  /* symbols per chunk (last chunk may be shorter), >= 1    */
+  uint32_t        lanes;          /* 32*G, G in {1,2,4,8}                                    */
+  int32_t         table_log;      /* R: the table has 2^R states (paper: l = 64..256; here 1..14) */
+  int32_t         bitwidth;       /* b in [1,8]: symbols must be < 2^b (checked on the device) */
+  int32_t         zero_point;     /* symbol that dequantises to 0 (Section II-B)            */
+  float           scale;          /* quantisation step                                      */
+  int32_t         out_dtype;      /* ANS_U8 | ANS_F32 | ANS_BF16                            */
+  int32_t         layout;         /* ANS_LAYOUT_*                                           */
+  uint32_t        work_begin;     /* written by ans_plan_batch: first work item of the layer */
+  uint32_t        work_count;     /* written by ans_plan_batch: the layer's work items      */
+} ans_layer_desc;
+
+/* Library version (major*100 + minor). */
+int ans_version(void);
+
+/* Text for an ANS_* code; never NULL. */
+const char* ans_strerror(int code);
+
+/* The cudaError_t of the most recent failed CUDA call made by this library (0 if none). */
+int ans_last_cuda_error(void);
+
+/*
+ * Bytes one layer's device table takes for a given table_log (a multiple of 256).
+ * Section II-A sizes the paper's table at 3 bytes per state; this library stores 32-bit
+ * entries plus a pre-walked copy for chains of zero-bit transitions.
+ */
+int ans_table_bytes(int table_log, size_t* h_bytes_out);
+
+/*
+ * Build the decode tables of n_layers layers on the device (Section II-A: per state the
+ * symbol, nb_bits and newX).  States are handed to symbols in bit-reversal order and a
+ * symbol's states are numbered upwards, the same rule an encoder must use.
+ *   h_norm_freqs   [n_layers][256]  normalised frequencies; row l sums to 1 << h_table_log[l]
+ *   h_alphabet     [n_layers]       symbols in use (frequencies at or beyond it must be 0)
+ *   h_table_log    [n_layers]       R per layer, 1..14
+ *   d_tables       device buffer, 256-byte aligned, d_tables_bytes long; layer l's table
+ *                  is written at byte offset h_table_offsets_out[l]
+ *   h_table_offsets_out [n_layers]  filled on return
+ * The host arrays are read before the call returns.  Asynchronous on `stream`.
+ * Errors: INVALID_ARG, UNSUPPORTED (R), BAD_FREQS, BUFFER_TOO_SMALL, CUDA.
+ */
+int ans_build_decode_tables(const uint32_t* h_norm_freqs, const int32_t* h_alphabet,
+                            const int32_t* h_table_log, int n_layers,
+                            void* d_tables, size_t d_tables_bytes,
+                            uint64_t* h_table_offsets_out, void* stream);
+
+/*
+ * Fill work_begin / work_count of every descriptor (one work item per sub-stream) so that
+ * a batch can run as ONE launch.  Call it on the host array before copying it to the
+ * device.  h_total_work_out receives the number of work items.  Host only.
+ */
+int ans_plan_batch(ans_layer_desc* h_descs, int n_layers, uint64_t* h_total_work_out);
+
+/*
+ * Decode one layer to symbols (Section II-A decode rule over the layer's vector of states,
+ * Section III-B): d_symbols_out receives h_desc->n_symbols bytes; d_out/out_dtype/scale are
+ * ignored.  d_status (one uint32 in device memory, zeroed by the caller or by an earlier
+ * ans_read_status) receives ANS_STATUS_* bits by atomic OR.  Asynchronous on `stream`.
+ */
+int ans_decode_layer(const ans_layer_desc* h_desc, uint8_t* d_symbols_out,
+                     uint32_t* d_status, void* stream);
+
+/*
+ * Decode one layer and dequantise it in the same kernel (Section II-B):
+ * d_out[i] = (float)(q_i - zero_point) * scale, one IEEE single-precision multiply, then
+ * for ANS_BF16 a round-to-nearest-even to bfloat16; ANS_U8 stores q_i itself.
+ */
+int ans_decode_dequant(const ans_layer_desc* h_desc, uint32_t* d_status, void* stream);
+
+/*
+ * The same for n_layers layers in one kernel launch.  d_descs is the device copy of
+ * h_descs (after ans_plan_batch); the host copy is only used for validation and sizing.
+ * All layers of one call share `layout`; out_dtype, table_log and every other field may
+ * differ from layer to layer.
+ */
+int ans_decode_dequant_batch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs,
+                             int n_layers, uint32_t* d_status, void* stream);
+
+/*
+ * Wait for `stream`, copy the status word to *h_status_out, clear it on the device.
+ * Returns ANS_ERR_CORRUPT if any bit was set, ANS_OK otherwise.
+ */
+int ans_read_status(uint32_t* d_status, void* stream, uint32_t* h_status_out);
+
+/*
+ * End-to-end helper with HOST buffers: copies the layer's stream, offsets and lane
+ * metadata to the device scratch the caller provides, decodes + dequantises, copies the
+ * result back to h_out and waits.  h_desc's d_stream/d_sub_offsets/d_lane_meta/d_out are
+ * IGNORED; the host pointers given here are used instead.  d_table must already be on the
+ * device.  d_scratch must hold ans_host_scratch_bytes(...) bytes, 256-byte aligned.
+ * Synchronous: returns after h_out is complete; returns ANS_ERR_CORRUPT on a bad stream.
+ */
+int ans_host_scratch_bytes(const ans_layer_desc* h_desc, uint64_t stream_bytes, size_t* h_bytes_out);
+int ans_decode_dequant_host(const ans_layer_desc* h_desc,
+                            const uint8_t* h_stream, uint64_t stream_bytes,
+                            const uint64_t* h_sub_offsets, const void* h_lane_meta,
+                            void* h_out, void* d_scratch, size_t d_scratch_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Host-side packer: makes the streams the decoder reads.  Runs on the CPU, off the
+ * inference path (the paper compresses offline, Section III-A); it is here so that a
+ * user can produce containers without any other tool.
+ * ------------------------------------------------------------------------------------ */
+
+/*
+ * Histogram -> normalised frequencies summing to 1 << table_log; every symbol that occurs
+ * keeps at least one state.  h_counts[alphabet], h_freqs_out[256] (entries >= alphabet = 0).
+ */
+int ans_host_normalize_freqs(const uint64_t* h_counts, int alphabet, int table_log,
+                             uint32_t* h_freqs_out);
+
+/* Upper bound of the stream bytes ans_host_pack_layer can produce. */
+int ans_host_pack_bound(uint64_t n_symbols, uint32_t chunk_symbols, uint32_t lanes,
+                        int layout, uint64_t* h_bytes_out);
+
+/*
+ * Encode one layer (Section II-A: follow the automaton's transition for each symbol and
+ * append its label bits) into the chosen container.
+ *   h_symbols[n_symbols]; h_freqs[256] as given to ans_build_decode_tables
+ *   h_stream_out (capacity stream_cap), h_sub_offsets_out[n_sub + 1],
+ *   h_lane_meta_out: uint16_t[n_sub][32] (interleaved) or uint32_t[n_sub][32] (private)
+ *   n_threads: host threads to use (<= 0: all)
+ * *h_stream_bytes_out receives the bytes written.
+ */
+int ans_host_pack_layer(const uint8_t* h_symbols, uint64_t n_symbols,
+                        const uint32_t* h_freqs, int alphabet, int table_log,
+                        uint32_t chunk_symbols, uint32_t lanes, int layout,
+                        uint8_t* h_stream_out, uint64_t stream_cap, uint64_t* h_stream_bytes_out,
+                        uint64_t* h_sub_offsets_out, void* h_lane_meta_out, int n_threads);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ANS_B200_H */

@@ -1,0 +1,55 @@
+"""Parity at the benchmark's full sizes and launch configuration (library packer, one batched
+launch).  Every output element is compared with the oracle's dequantiser applied to the
+source symbols (what a correct decode must give back), and a sample of chunks is decoded by
+the oracle itself from the same bytes."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synthgen as sg
+import paper_2406_06237_b200 as ans
+from paper_2406_06237_b200.runtime import DeviceBatch, pack_layer
+from helpers import bits_view, expected_bits, parallel_map
+
+pytestmark = pytest.mark.gpu
+
+
+def full_size(specs, layout, lanes, sample_chunks=64):
+    def prep(spec):
+        sym = sg.draw_symbols(spec, threads=2)
+        pl = pack_layer(sym, spec.alphabet, spec.table_log, spec.chunk_symbols, lanes, layout,
+                        spec.bitwidth, spec.zero_point, spec.scale, ans.DTYPES[spec.out_dtype], n_threads=4)
+        return sym, pl
+
+    prepared = parallel_map(prep, specs, 8)
+    db = DeviceBatch([p[1] for p in prepared])
+    for o in db.out_sets[0]:
+        o.view(torch.uint8).fill_(0xA5)
+    db.decode()
+    assert db.read_status() == 0
+    rng = np.random.default_rng(1)
+    for i, (spec, (sym, pl)) in enumerate(zip(specs, prepared)):
+        want = oracle.dequant(sym, spec.zero_point, spec.scale, spec.out_dtype, threads=8)
+        got = bits_view(db.output(i))
+        assert np.array_equal(got, expected_bits(want)), f"layer {i}"
+        # the oracle decodes sampled chunks from the very bytes the GPU read
+        T = oracle.Table(pl.freqs[:spec.alphabet], spec.table_log)
+        P = oracle.Packed(layout, pl.stream, pl.sub_offsets, pl.lane_meta, pl.n_symbols, pl.chunk_symbols, lanes // 32)
+        per_layer = max(1, sample_chunks // len(specs))
+        for c in rng.choice(P.n_chunks, size=min(per_layer, P.n_chunks), replace=False):
+            osym, rc = oracle.unpack(T, P, chunk_range=(int(c), int(c) + 1))
+            a, b = int(c) * pl.chunk_symbols, min((int(c) + 1) * pl.chunk_symbols, pl.n_symbols)
+            assert rc == oracle.OK and (osym[a:b] == sym[a:b]).all()
+            assert np.array_equal(got[a:b], expected_bits(want)[a:b])
+
+
+@pytest.mark.parametrize("layout", [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE])
+def test_config5_large_layers_full(layout):
+    full_size(sg.workload_large(), layout, 32)
+
+
+@pytest.mark.parametrize("layout", [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE])
+@pytest.mark.parametrize("chunk,R", [(1024, 11), (65536, 14), (16384, 12)])
+def test_config4_sweep_full(layout, chunk, R):
+    full_size(sg.workload_sweep(table_log=R, chunk=chunk), layout, 32)

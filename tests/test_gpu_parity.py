@@ -1,0 +1,216 @@
+"""GPU vs oracle, element by element, through the C ABI.  Streams are encoded by the ORACLE;
+the library only decodes them.  Integer symbols, fp32 and bf16 outputs are compared as bit
+patterns: the decode is integer work and the dequantiser is one IEEE multiply plus one
+round-to-nearest-even, so the tolerance is zero."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synthgen as sg
+import paper_2406_06237_b200 as ans
+from paper_2406_06237_b200.runtime import DeviceBatch
+from helpers import (bits_view, expected_bits, oracle_expected, oracle_pack_spec, parallel_map, tiny_spec,
+                     to_packed_layer)
+
+pytestmark = pytest.mark.gpu
+LAYOUTS = [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE]
+
+
+def run_and_compare(specs, layout, lanes=32, per_layer=False, threads=8, chunk=None, table_log=None):
+    def prep(spec):
+        sym = sg.draw_symbols(spec, threads=1)
+        T, P, f256 = oracle_pack_spec(spec, sym, layout, lanes, chunk, table_log)
+        want_sym, want = oracle_expected(spec, T, P)
+        assert (want_sym == sym).all()
+        return to_packed_layer(spec, P, f256, table_log), want_sym, want
+
+    prepared = parallel_map(prep, specs, threads)
+    db = DeviceBatch([p[0] for p in prepared])
+    # canaries: outputs start poisoned so that an element the kernel skips cannot pass by luck
+    for o in db.out_sets[0]:
+        o.view(torch.uint8).fill_(0xA5)
+    (db.decode_per_layer if per_layer else db.decode)()
+    assert db.read_status() == 0
+    for i, (pl, want_sym, want) in enumerate(prepared):
+        got = bits_view(db.output(i))
+        assert got.shape == want.shape
+        bad = np.flatnonzero(got != expected_bits(want))
+        assert bad.size == 0, f"layer {i} ({specs[i].name}): {bad.size} mismatches, first at {bad[:5]}"
+    return db, prepared
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("lanes", [32, 64, 128, 256])
+def test_config1_single_conv_fp32(layout, lanes):
+    db, prepared = run_and_compare(sg.workload_conv3x3(), layout, lanes)
+    assert (db.decode_symbols(0).cpu().numpy() == prepared[0][1]).all()
+    assert db.read_status() == 0
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("n", [0, 1, 31, 32, 33, 63, 64, 65, 2047, 2048, 2049, 4096 + 17, 3 * 4096])
+def test_edge_sizes(layout, n):
+    for dt in ("u8", "bf16", "f32"):
+        run_and_compare([tiny_spec(n, out_dtype=dt, chunk=4096)], layout, 64)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("R", [1, 2, 3, 6, 7, 8, 11, 12, 13, 14])
+def test_table_sizes(layout, R):
+    b = 1 if R == 1 else min(8, R)
+    specs = [tiny_spec(50_000 + R, bitwidth=b, pzp=p, table_log=R, chunk=16384, out_dtype=dt, index=i)
+             for i, (p, dt) in enumerate([(0.55, "bf16"), (0.9, "u8"), (0.97, "f32")])]
+    run_and_compare(specs, layout, 32)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_single_symbol_layer_and_odd_chunks(layout):
+    """A layer whose every weight is the zero-point has one symbol with f = l: every
+    transition reads zero bits and the streams hold only padding."""
+    A, zp = sg.alphabet_for_bits(4)
+    spec = sg.LayerSpec("const", (10_000,), 4, A, zp, 1e-9, 0.5, 10, 1000, "bf16", sg.stream_key(5, 0))
+    sym = sg.draw_symbols(spec)
+    assert (sym == zp).all()
+    run_and_compare([spec], layout, 32)
+    # chunk sizes that are not multiples of the lane count or of 16
+    run_and_compare([tiny_spec(7001, chunk=c, out_dtype=dt, index=c) for c, dt in
+                     [(999, "u8"), (1001, "bf16"), (77, "f32"), (4099, "u8")]], layout, 64)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_batch_with_mixed_layers_one_launch(layout):
+    specs = [tiny_spec(20_000, 2, 0.8, 9, 4096, "bf16", index=0), tiny_spec(0, 4, 0.6, 12, 4096, "f32", index=1),
+             tiny_spec(4096, 8, 0.9, 14, 1024, "u8", index=2), tiny_spec(123_457, 6, 0.7, 11, 16384, "bf16", index=3),
+             tiny_spec(1, 1, 0.6, 1, 64, "f32", index=4), tiny_spec(70_000, 3, 0.95, 12, 32768, "bf16", index=5)]
+    run_and_compare(specs, layout, 32)
+    run_and_compare(specs, layout, 128, per_layer=True)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_config2_resnet18_bf16(layout):
+    run_and_compare(sg.workload_resnet18(), layout, 32)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("lanes", [32, 128])
+def test_config3_resnet50_bf16(layout, lanes):
+    run_and_compare(sg.workload_resnet50(), layout, lanes)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("chunk", [1024, 4096, 16384, 65536])
+@pytest.mark.parametrize("R", [11, 12, 14])
+def test_config4_sweep_reduced(layout, chunk, R):
+    """The granularity sweep at 2^22 symbols (the full 2^28 runs in test_gpu_full_size)."""
+    run_and_compare(sg.workload_sweep(table_log=R, chunk=chunk, n=(1 << 22) + 12345), layout, 32)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_config5_reduced(layout):
+    run_and_compare(sg.workload_large(n_mats=2, dim=2048), layout, 32)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_corrupt_streams_are_flagged_not_fatal(layout):
+    """Corruption is planted on the host.  Reads are clamped to the stream and every loop is
+    counted, so a bad stream yields wrong symbols and a status bit, never a fault."""
+    spec = tiny_spec(40_000, 4, 0.6, 12, 4096, "bf16")
+    sym = sg.draw_symbols(spec)
+    T, P, f256 = oracle_pack_spec(spec, sym, layout, 32)
+
+    def decode(P2):
+        db = DeviceBatch([to_packed_layer(spec, P2, f256)])
+        guard = torch.full((1 << 16,), 0x5A, dtype=torch.uint8, device="cuda")
+        db.decode()
+        st = db.read_status()
+        assert (guard == 0x5A).all()
+        return st, bits_view(db.output(0))
+
+    st, good = decode(P)
+    assert st == 0
+    flagged = 0
+    rng = np.random.default_rng(0)
+    for trial in range(6):
+        s = P.stream.copy()
+        pos = rng.integers(0, s.size, size=8)
+        s[pos] ^= rng.integers(1, 256, size=8).astype(np.uint8)
+        st, _ = decode(oracle.Packed(P.layout, s, P.sub_offsets, P.lane_meta, P.n, P.chunk, P.groups))
+        _, orc = oracle.unpack(T, oracle.Packed(P.layout, s, P.sub_offsets, P.lane_meta, P.n, P.chunk, P.groups))
+        assert (st != 0) == (orc != oracle.OK)
+        flagged += st != 0
+    assert flagged > 0
+    m = P.lane_meta.copy(); m[1, 3] ^= 1
+    st, _ = decode(oracle.Packed(P.layout, P.stream, P.sub_offsets, m, P.n, P.chunk, P.groups))
+    assert st & 1
+    o = P.sub_offsets.copy(); o[2] += 1 << 40            # offset far outside the stream
+    st, _ = decode(oracle.Packed(P.layout, P.stream, o, P.lane_meta, P.n, P.chunk, P.groups))
+    assert st & 2
+    short = P.stream[:P.stream.size - 16].copy()         # truncated stream
+    st, _ = decode(oracle.Packed(P.layout, short, P.sub_offsets, P.lane_meta, P.n, P.chunk, P.groups))
+    assert st & 2
+
+
+def test_bitwidth_check():
+    spec = tiny_spec(5000, 4, 0.6, 12, 4096, "u8")
+    sym = sg.draw_symbols(spec)
+    T, P, f256 = oracle_pack_spec(spec, sym, ans.ANS_LAYOUT_INTERLEAVED, 32)
+    pl = to_packed_layer(spec, P, f256)
+    pl.bitwidth, pl.zero_point = 2, 1                    # alphabet 15 does not fit 2 bits
+    db = DeviceBatch([pl])
+    db.decode()
+    assert db.read_status() & 4
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_host_buffer_entry_point(layout):
+    spec = tiny_spec(100_000, 3, 0.7, 12, 16384, "bf16")
+    sym = sg.draw_symbols(spec)
+    T, P, f256 = oracle_pack_spec(spec, sym, layout, 32)
+    _, want = oracle_expected(spec, T, P)
+    pl = to_packed_layer(spec, P, f256)
+    db = DeviceBatch([pl])                               # for the table only
+    d = db.h_descs[0][0]
+    need = ans.ans_host_scratch_bytes(d, pl.stream.nbytes)
+    scratch = torch.empty(need, dtype=torch.uint8, device="cuda")
+    out = np.zeros(spec.n, dtype=np.uint16)
+    rc = ans.ans_decode_dequant_host(d, pl.stream, pl.sub_offsets, pl.lane_meta, out, scratch.data_ptr(), need,
+                                     torch.cuda.current_stream().cuda_stream)
+    assert rc == ans.ANS_OK and (out == want).all()
+    bad = pl.stream.copy(); bad[100] ^= 0xFF
+    rc = ans.ans_decode_dequant_host(d, bad, pl.sub_offsets, pl.lane_meta, out, scratch.data_ptr(), need,
+                                     torch.cuda.current_stream().cuda_stream)
+    assert rc == ans.ANS_ERR_CORRUPT
+
+
+def test_device_tables_match_oracle_tables():
+    """ans_build_decode_tables against the oracle's table, entry by entry, and the pre-walked
+    entries against a walk of the oracle's table."""
+    specs = [tiny_spec(30_000, b, p, R, 4096, index=i) for i, (b, p, R) in
+             enumerate([(1, 0.6, 1), (2, 0.9, 2), (4, 0.6, 6), (5, 0.85, 8), (8, 0.95, 12), (3, 0.7, 12), (8, 0.5, 14)])]
+    layers = []
+    tabs = []
+    for spec in specs:
+        sym = sg.draw_symbols(spec)
+        T, P, f256 = oracle_pack_spec(spec, sym, ans.ANS_LAYOUT_PRIVATE, 32)
+        layers.append(to_packed_layer(spec, P, f256)); tabs.append(T)
+    db = DeviceBatch(layers)
+    raw = db.tables.cpu().numpy()
+    for spec, T, off in zip(specs, tabs, db.table_offsets):
+        L = 1 << spec.table_log
+        blob = raw[int(off):int(off) + ans.ans_table_bytes(spec.table_log)]
+        hdr = blob[:16].view(np.uint32)
+        single = blob[1040:1040 + 4 * L].view(np.uint32)
+        multi = blob[1040 + 4 * L:1040 + 8 * L].view(np.uint32)
+        ent = T.entries()
+        assert hdr[1] == spec.table_log and hdr[2] == spec.alphabet
+        dom = [s for s in range(spec.alphabet) if 2 * int(T.freqs[s]) > L]
+        assert hdr[3] == (dom[0] if dom else 0xFFFFFFFF)
+        for i, (s, nb, nx) in enumerate(ent):
+            assert single[i] == (s | nb << 8 | nx << 16)
+            cur, run = i, 0
+            while run < 15 and ent[cur][1] == 0:
+                assert ent[cur][0] == dom[0]
+                cur, run = ent[cur][2], run + 1
+            s2, nb2, nx2 = ent[cur]
+            assert multi[i] == (s2 | nb2 << 8 | run << 12 | nx2 << 16)
