@@ -1,0 +1,398 @@
+#!/usr/bin/env python
+"""Benchmark of the tANS decode + dequantise path on B200.
+
+One step = one pass of the whole hot path (stage tables, read compressed streams, decode,
+dequantise, store) over one synthetic workload, as ONE batched kernel launch.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload large|resnet50|resnet18|conv3x3|sweep]
+                  [--layout private|interleaved] [--lanes 32|64|128|256] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  With --impl reference the CPU oracle is timed instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synthgen as sg  # noqa: E402
+
+METRIC = "decoded weights/sec and achieved HBM GB/s (fraction of B200 peak), 1 GPU"
+NOMINAL_PEAK_GBS = 8000.0
+FALLBACK_PEAK_GBS = 6650.0
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_PEAK_GBS, "fallback"
+
+
+def make_specs(args):
+    if args.workload == "sweep":
+        return sg.workload_sweep(table_log=args.table_log or 12, chunk=args.chunk or 16384)
+    if args.workload == "large":
+        return sg.workload_large(n_mats=args.mats, dim=args.dim, chunk=args.chunk or 32768,
+                                 table_log=args.table_log or 12)
+    if args.workload in ("resnet18", "resnet50"):
+        return sg.WORKLOADS[args.workload](table_log=args.table_log or 12, chunk=args.chunk or 16384)
+    return sg.workload_conv3x3()
+
+
+WORKLOAD_TEXT = {
+    "conv3x3": "single 3x3 conv 64->64 (36,864 weights), 4-bit zero-point, 12-bit table, 4096-symbol chunks, fp32",
+    "resnet18": "ResNet-18 conv weights (20 layers, 11.2M), bitwidth {2,3,4,6}, 0.8-1.5 bit/weight, 16K chunks, bf16",
+    "resnet50": "ResNet-50 conv weights (53 layers, 23.5M), 1-8 bit mixed precision, P(zp) 0.85-0.95, 16K chunks, bf16",
+    "sweep": "256M 8-bit symbols, two-sided geometric (2.5 bit), decode-only to uint8",
+    "large": "large dense layers: 8 matrices of 8192x8192 (537M weights), 3-bit zero-point, P(zp)=0.7, 32K chunks, bf16",
+}
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+        sm = [float(r[1]) for r in self.rows if len(r) >= 9 and r[1].replace(".", "").isdigit()]
+        mx = [float(r[2]) for r in self.rows if len(r) >= 9 and r[2].replace(".", "").isdigit()]
+        reasons = set()
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cpu_baseline(specs, syms, layout_name, budget_s=12.0):
+    """The CPU oracle, as it stands, decoding + dequantising a bounded sample of the same
+    workload on this host's cores: single thread and all cores."""
+    import oracle
+    layout = oracle.PRIVATE if layout_name == "private" else oracle.INTERLEAVED
+    cores = os.cpu_count() or 1
+    target = 48_000_000                         # symbols in the sample (about 10-30 s of CPU work in all)
+    sample, total = [], 0
+    for spec, sym in zip(specs, syms):
+        take = min(sym.size, max(0, target - total))
+        take -= take % spec.chunk_symbols if take > spec.chunk_symbols else 0
+        if take <= 0:
+            break
+        s = sym[:take]
+        f = oracle.normalize_freqs(oracle.histogram(s), spec.alphabet, spec.table_log)
+        T = oracle.Table(f, spec.table_log)
+        sample.append((spec, T, oracle.pack(T, s, spec.chunk_symbols, 1, layout)))
+        total += take
+
+    def run(threads):
+        best = float("inf")
+        for _ in range(3):
+            t0 = time.perf_counter()
+            for spec, T, P in sample:
+                out, rc = oracle.unpack(T, P, threads=threads)
+                assert rc == 0
+                oracle.dequant(out, spec.zero_point, spec.scale, spec.out_dtype, threads=threads)
+            best = min(best, time.perf_counter() - t0)
+        return total / best
+
+    one = run(1)
+    many = run(cores) if cores > 1 else one
+    return {"value": many, "unit": "weights/s", "cores": cores, "kind": "oracle",
+            "single_thread_value": one,
+            "sample": f"first {total} weights of the workload ({len(sample)} layer(s)), {layout_name} container, "
+                      f"decode + dequant, best of 3"}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on the host cores, bounded sample per step."""
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    specs = make_specs(args)
+    layout = oracle.PRIVATE if args.layout == "private" else oracle.INTERLEAVED
+    cores = os.cpu_count() or 1
+    target = 24_000_000
+    sample, total = [], 0
+    for spec in specs:
+        take = min(spec.n, max(0, target - total))
+        if take <= 0:
+            break
+        sub = sg.LayerSpec(spec.name, (take,), spec.bitwidth, spec.alphabet, spec.zero_point, spec.theta, spec.scale,
+                           spec.table_log, spec.chunk_symbols, spec.out_dtype, spec.key)
+        s = sg.draw_symbols(sub)
+        T = oracle.Table(oracle.normalize_freqs(oracle.histogram(s), spec.alphabet, spec.table_log), spec.table_log)
+        sample.append((spec, T, oracle.pack(T, s, spec.chunk_symbols, 1, layout)))
+        total += take
+
+    def step():
+        for spec, T, P in sample:
+            out, rc = oracle.unpack(T, P, threads=cores)
+            assert rc == 0
+            oracle.dequant(out, spec.zero_point, spec.scale, spec.out_dtype, threads=cores)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / max(1, args.steps)
+    value = total / dt
+    sample_txt = f"first {total} weights of the workload per step, {args.layout} container, all {cores} cores"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "weights/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": WORKLOAD_TEXT[args.workload], "layout": args.layout, "sample": sample_txt},
+        "cpu_baseline": {"value": value, "unit": "weights/s", "cores": cores, "kind": "oracle", "sample": sample_txt},
+        "e2e": {"value": value, "unit": "weights/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def reduce_max(x: float, world: int) -> float:
+    """Max over ranks (identity for one rank)."""
+    if world <= 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda" if dist.get_backend() == "nccl" else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def time_workload(db, steps, warmup, flush, n_sets, world):
+    """K timed steps, each bracketed by CUDA events on the launching stream; the L2 flush (if
+    any) sits outside the brackets.  Returns per-step milliseconds (max over ranks of the sum)."""
+    import torch
+    import torch.distributed as dist
+    st = torch.cuda.current_stream()
+    for i in range(warmup):
+        if flush is not None:
+            flush.add_(1)
+        db.decode(i % n_sets)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for i in range(steps):
+        if flush is not None:
+            flush.add_(1)
+        ev[i][0].record(st)
+        db.decode(i % n_sets)
+        ev[i][1].record(st)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ms = [a.elapsed_time(b) for a, b in ev]
+    assert db.read_status() == 0, "decoder flagged a stream"
+    return ms
+
+
+def run_ours(args):
+    import torch
+    import paper_2406_06237_b200 as ans
+    from paper_2406_06237_b200.runtime import DeviceBatch, pack_layer
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    ans.lib()                                           # fail loudly if the library is missing
+
+    layout = ans.ANS_LAYOUT_PRIVATE if args.layout == "private" else ans.ANS_LAYOUT_INTERLEAVED
+    specs = make_specs(args)
+    t_setup = time.perf_counter()
+    from concurrent.futures import ThreadPoolExecutor
+    cores = os.cpu_count() or 1
+
+    def prep(spec):
+        sym = sg.draw_symbols(spec, threads=max(1, cores // 4))
+        pl = pack_layer(sym, spec.alphabet, spec.table_log, spec.chunk_symbols, args.lanes, layout, spec.bitwidth,
+                        spec.zero_point, spec.scale, ans.DTYPES[spec.out_dtype], n_threads=max(1, cores // 2))
+        return sym, pl
+
+    with ThreadPoolExecutor(4) as ex:
+        prepared = list(ex.map(prep, specs))
+    syms = [p[0] for p in prepared]
+    layers = [p[1] for p in prepared]
+    out_bytes = sum(L.n_symbols * ans.ELEM_SIZE[L.out_dtype] for L in layers)
+    # keep the working set out of L2 (126 MB): big workloads are larger than L2 by themselves,
+    # small ones rotate output sets and flush L2 between timed steps
+    small = out_bytes < (512 << 20)
+    n_sets = 4 if small else 1
+    db = DeviceBatch(layers, f"cuda:{local}", n_out_sets=n_sets)
+    flush = torch.zeros(256 << 20, dtype=torch.uint8, device="cuda") if small else None
+    setup_s = time.perf_counter() - t_setup
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms = time_workload(db, args.steps, args.warmup, flush, n_sets, world)
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = reduce_max(sum(ms), world)
+    ms_per_step = total_ms / args.steps
+    n_w = db.n_symbols()
+    value = world * n_w / (ms_per_step * 1e-3)
+
+    # algorithmic bytes of one launch: everything compressed read once, each layer's table
+    # once, every decoded element written once
+    table_read = sum(4 << L.table_log for L in layers)
+    algo_bytes = db.compressed_bytes() + table_read + out_bytes
+    peak, peak_kind = measured_peak()
+    kernel_ms = statistics.mean(ms)
+    achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
+    kname = "ans_decode_kernel<private>" if args.layout == "private" else "ans_decode_kernel<interleaved>"
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "kernel": kname, "peak_kind": f"of {peak_kind}",
+                "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms_mean": kernel_ms,
+                "kernel_ms_median": statistics.median(ms), "kernel_ms_min": min(ms),
+                "frac_of_nominal_8TBs": achieved / NOMINAL_PEAK_GBS}
+
+    # end to end through the host-buffer entry point: pinned host buffers in, pinned out
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(ans, db, layers, args, world)
+
+    if rank != 0:
+        return
+    hist = np.zeros(256, dtype=np.float64)
+    ent_bits = 0.0
+    for spec, sym in zip(specs, syms):
+        c = np.bincount(sym, minlength=256).astype(np.float64)
+        p = c[c > 0] / max(1, sym.size)
+        ent_bits += float(-(p * np.log2(p)).sum()) * sym.size
+    coded_bits = 8.0 * db.compressed_bytes()
+    cpu = cpu_baseline(specs, syms, args.layout) if world == 1 and not args.no_cpu_baseline else None
+    out = {
+        "metric": METRIC, "value": value, "unit": "weights/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": WORKLOAD_TEXT[args.workload], "name": args.workload, "layout": args.layout,
+                   "lanes": args.lanes, "table_log": layers[0].table_log, "chunk_symbols": layers[0].chunk_symbols,
+                   "layers": len(layers), "weights": n_w, "out_dtype": specs[0].out_dtype,
+                   "l2_policy": ("outputs rotate over 4 buffer sets and a 256 MB buffer is rewritten between timed steps"
+                                 if small else "working set (compressed + output) is larger than L2"),
+                   "per_gpu": "every rank decodes its own replica of the workload; no collective on the data path"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "roofline": roofline, "cpu_baseline": cpu,
+        "compression": {"coded_bits_per_weight": coded_bits / max(1, n_w), "entropy_bits_per_weight": ent_bits / max(1, n_w),
+                        "gap_bits_per_weight": (coded_bits - ent_bits) / max(1, n_w),
+                        "compressed_bytes": db.compressed_bytes(), "output_bytes": out_bytes},
+        "setup_s": setup_s,
+    }
+    print(json.dumps(out))
+
+
+def run_e2e(ans, db, layers, args, world):
+    """Same metric through ans_decode_dequant_host: per layer, compressed bytes go host -> device,
+    the layer is decoded, the weights come back device -> host, all inside the timed region."""
+    import torch
+    n_w = sum(L.n_symbols for L in layers)
+    st = torch.cuda.current_stream().cuda_stream
+    pinned_in, pinned_out, need = [], [], 0
+    for i, L in enumerate(layers):
+        bufs = []
+        for a in (L.stream, L.sub_offsets, L.lane_meta):
+            t = torch.empty(max(a.nbytes, 1), dtype=torch.uint8, pin_memory=True)
+            t.numpy()[:a.nbytes] = a.reshape(-1).view(np.uint8)
+            bufs.append(t)
+        pinned_in.append(bufs)
+        pinned_out.append(torch.empty(max(L.n_symbols * ans.ELEM_SIZE[L.out_dtype], 1), dtype=torch.uint8, pin_memory=True))
+        need = max(need, ans.ans_host_scratch_bytes(db.h_descs[0][i], L.stream.nbytes))
+    scratch = torch.empty(need, dtype=torch.uint8, device="cuda")
+    lib = ans.lib()
+    import ctypes
+
+    def step():
+        for i, L in enumerate(layers):
+            if L.n_symbols == 0:
+                continue
+            s, o, m = pinned_in[i]
+            rc = lib.ans_decode_dequant_host(ctypes.byref(db.h_descs[0][i]), s.data_ptr(), L.stream.nbytes,
+                                             o.data_ptr(), m.data_ptr(), pinned_out[i].data_ptr(),
+                                             scratch.data_ptr(), need, st)
+            assert rc == 0, rc
+
+    steps = max(1, min(args.steps, 5))
+    step()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    torch.cuda.synchronize()
+    dt = reduce_max((time.perf_counter() - t0) / steps, world)
+    h2d = sum(L.compressed_bytes() for L in layers)
+    d2h = sum(L.n_symbols * ans.ELEM_SIZE[L.out_dtype] for L in layers)
+    return {"value": world * n_w / dt, "unit": "weights/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "ms_per_step": dt * 1e3, "steps": steps, "api": "ans_decode_dequant_host (pinned host buffers)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large", choices=list(WORKLOAD_TEXT))
+    ap.add_argument("--layout", default="private", choices=["private", "interleaved"])
+    ap.add_argument("--lanes", type=int, default=32)
+    ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--table-log", type=int, default=0)
+    ap.add_argument("--mats", type=int, default=8, help="large workload: number of matrices (8 = full size)")
+    ap.add_argument("--dim", type=int, default=8192, help="large workload: matrix dimension (8192 = full size)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
