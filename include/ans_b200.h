@@ -97,7 +97,8 @@ typedef struct ans_layer_desc {
   int32_t         out_dtype;      /* ANS_U8 | ANS_F32 | ANS_BF16                            */
   int32_t         layout;         /* ANS_LAYOUT_*                                           */
   uint32_t        work_begin;     /* written by ans_plan_batch: first work item of the layer */
-  uint32_t        work_count;     /* written by ans_plan_batch: the layer's work items      */
+  uint32_t        work_count;     /* written by ans_plan_batch: the layer's work items (a work
+                                     item is a group of up to 4 consecutive sub-streams)     */
 } ans_layer_desc;
 
 /* Library version (major*100 + minor). */
@@ -135,8 +136,8 @@ int ans_build_decode_tables(const uint32_t* h_norm_freqs, const int32_t* h_alpha
                             uint64_t* h_table_offsets_out, void* stream);
 
 /*
- * Fill work_begin / work_count of every descriptor (one work item per sub-stream) so that
- * a batch can run as ONE launch.  Call it on the host array before copying it to the
+ * Fill work_begin / work_count of every descriptor (one work item per group of up to 4
+ * consecutive sub-streams of a layer) so that a batch can run as ONE launch.  Call it on the host array before copying it to the
  * device.  h_total_work_out receives the number of work items.  Host only.
  */
 int ans_plan_batch(ans_layer_desc* h_descs, int n_layers, uint64_t* h_total_work_out);

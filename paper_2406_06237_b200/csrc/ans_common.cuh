@@ -61,6 +61,8 @@ inline uint64_t chunks_of(const ans_layer_desc& d) {
   return d.n_symbols ? (d.n_symbols + d.chunk_symbols - 1) / d.chunk_symbols : 0;
 }
 inline uint64_t subs_of(const ans_layer_desc& d) { return chunks_of(d) * groups_of(d); }
+constexpr uint32_t kGranule = 4;   // sub-streams per work item of the batch plan
+inline uint64_t granules_of(const ans_layer_desc& d) { return (subs_of(d) + kGranule - 1) / kGranule; }
 inline size_t elem_size(int dtype) { return dtype == ANS_U8 ? 1 : dtype == ANS_F32 ? 4 : 2; }
 
 }  // namespace ansb

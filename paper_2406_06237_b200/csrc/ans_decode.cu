@@ -6,18 +6,17 @@
 // layer's table sits in shared memory; the decoded symbol goes through a 256-entry table of
 // already dequantised values (Section II-B: w = scale * (q - zero_point)) on its way out.
 //
-// Work item = one sub-stream (32 lanes) = one warp.  A CTA owns a contiguous range of the work
-// list, walks it kWarps items at a time and restages the table only when the layer changes.
+// One sub-stream (32 lanes) is decoded by one warp.  The work list counts granules of up to
+// kGranule consecutive sub-streams of a layer; a CTA owns a contiguous range of granules, walks
+// it one sub-stream per warp at a time and restages the table only when the layer changes.
 #include <cuda_bf16.h>
 
 #include "ans_common.cuh"
 
 namespace ansb {
 
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
-constexpr int kTileRows = 64;          // private layout: rows of 32 symbols staged per warp
 constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr uint32_t kStatusTimeout = 8u;   // a bounded wait on an asynchronous copy ran out
 
 struct LaunchArgs {
   const ans_layer_desc* d_descs;   // device array, or nullptr when `one` is the only layer
@@ -28,6 +27,7 @@ struct LaunchArgs {
   uint32_t* d_status;
   uint8_t* d_symbols_override;     // ans_decode_layer: write symbols here instead of d_out
   uint32_t table_words;            // shared-memory words reserved for the table
+  uint32_t stage_bytes;            // private layout: per-warp staging buffer for compressed bytes
 };
 
 __device__ __forceinline__ const ans_layer_desc& layer_at(const LaunchArgs& a, int l) {
@@ -51,10 +51,57 @@ __device__ __forceinline__ uint32_t lane_symbols(uint32_t nc, uint32_t W, uint32
   return nc > lambda ? (nc - lambda + W - 1) / W : 0u;
 }
 
-// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// ---- work list walking shared by both kernels ----------------------------------------------
+struct Item {
+  uint64_t sub;        // sub-stream index inside the layer
+  uint64_t c0;         // first symbol of the chunk
+  uint32_t nc;         // symbols in the chunk
+  uint32_t g;          // sub-stream inside the chunk
+  uint64_t off0;       // byte offset of the sub-stream
+  uint64_t extent;     // its bytes (0 if the offsets are unusable)
+  uint32_t bad;
+};
+
+__device__ __forceinline__ Item make_item(const ans_layer_desc& L, uint64_t sub) {
+  Item it;
+  const uint32_t G = L.lanes / 32u;
+  it.sub = sub;
+  const uint64_t chunk = sub / G;
+  it.g = static_cast<uint32_t>(sub % G);
+  it.c0 = chunk * L.chunk_symbols;
+  it.nc = static_cast<uint32_t>(min(uint64_t(L.chunk_symbols), L.n_symbols - it.c0));
+  it.off0 = __ldg(L.d_sub_offsets + sub);
+  const uint64_t off1 = __ldg(L.d_sub_offsets + sub + 1);
+  it.extent = off1 - it.off0;
+  it.bad = 0;
+  if (off1 < it.off0 || off1 > L.stream_bytes || (it.off0 & 15u)) {   // never read outside the stream
+    it.extent = 0;
+    it.off0 = 0;
+    it.bad = ANS_STATUS_BAD_LENGTH;
+  }
+  return it;
+}
+
+// layer that holds work item `cursor`: the last layer with work_begin <= cursor
+__device__ __forceinline__ int find_layer(const LaunchArgs& a, uint64_t cursor) {
+  int lo = 0, hi = a.n_layers;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (layer_at(a, mid).work_begin <= cursor) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// =============================================================================================
 // Interleaved container: the warp's 32 lanes share one sequence of 16-bit units; a lane whose
 // buffer holds fewer than 16 bits takes the next unit, its place found by ballot + popcount.
-// ---------------------------------------------------------------------------------------------
+// =============================================================================================
+constexpr int kIWarps = 8;
+
 template <int ES>
 __device__ __forceinline__ uint32_t decode_interleaved(
     const uint32_t* __restrict__ tab, const uint32_t* __restrict__ vals,
@@ -92,131 +139,18 @@ __device__ __forceinline__ uint32_t decode_interleaved(
   return bad;
 }
 
-// ---------------------------------------------------------------------------------------------
-// Private container: every lane reads its own run of 32-bit words.  Look-ups go through the
-// pre-walked table, so one look-up may stand for several symbols: `run` copies of the layer's
-// dominant symbol followed by one more.  The warp stages kTileRows rows of output in shared
-// memory, pre-filled with the dominant value, drops the other symbols into place and writes
-// the rows out with 16-byte stores.
-// ---------------------------------------------------------------------------------------------
-template <int ES>
-__device__ __forceinline__ void flush_rows(const uint8_t* tile, uint8_t* out_row0, size_t row_stride_bytes,
-                                           uint32_t full_rows, uint32_t part_row_lanes, uint32_t lane) {
-  constexpr uint32_t RB = 32u * ES;                 // bytes per row
-  constexpr uint32_t PPR = RB / 16u;                // 16-byte pieces per row
-  if ((reinterpret_cast<uintptr_t>(out_row0) & 15u) == 0 && (row_stride_bytes & 15u) == 0) {
-    for (uint32_t idx = lane; idx < full_rows * PPR; idx += 32u) {
-      const uint32_t row = idx / PPR, piece = idx % PPR;
-      const uint4 v = *reinterpret_cast<const uint4*>(tile + size_t(idx) * 16u);
-      *reinterpret_cast<uint4*>(out_row0 + size_t(row) * row_stride_bytes + piece * 16u) = v;
-    }
-  } else {
-    using E = typename ElemT<ES>::type;
-    for (uint32_t row = 0; row < full_rows; ++row)
-      reinterpret_cast<E*>(out_row0 + size_t(row) * row_stride_bytes)[lane] =
-          reinterpret_cast<const E*>(tile)[row * 32u + lane];
-  }
-  if (lane < part_row_lanes) {
-    using E = typename ElemT<ES>::type;
-    reinterpret_cast<E*>(out_row0 + size_t(full_rows) * row_stride_bytes)[lane] =
-        reinterpret_cast<const E*>(tile)[full_rows * 32u + lane];
-  }
-}
-
-template <int ES>
-__device__ __forceinline__ uint32_t decode_private(
-    const uint32_t* __restrict__ mtab, const uint32_t* __restrict__ g_single,
-    const uint32_t* __restrict__ vals, uint32_t dom_val, const uint32_t* __restrict__ words,
-    uint32_t wbeg, uint32_t wend, bool last_lane, uint32_t state, uint32_t my_count, uint32_t rows,
-    uint32_t min_count, uint8_t* __restrict__ tile, uint8_t* __restrict__ out, size_t row_stride_bytes,
-    uint32_t lane) {
-  using E = typename ElemT<ES>::type;
-  E* trow = reinterpret_cast<E*>(tile);
-  auto load_word = [&](uint32_t i) -> uint32_t { return i < wend ? __ldg(words + i) : 0u; };
-  uint32_t idx = wbeg;
-  uint32_t w0 = load_word(idx), w1 = load_word(idx + 1), w2 = load_word(idx + 2);
-  idx += 3;
-  uint32_t bitpos = 0;
-  uint32_t t = 0;                 // next row this lane decodes
-  bool pending = false;           // a decoded symbol waiting for the next window
-  uint32_t pend_val = 0;
-
-  uint32_t fill = dom_val;
-  if (ES == 1) fill *= 0x01010101u;
-  if (ES == 2) fill *= 0x00010001u;
-  const uint4 fill4 = make_uint4(fill, fill, fill, fill);
-
-  for (uint32_t r0 = 0; r0 < rows; r0 += kTileRows) {
-    const uint32_t rend = min(r0 + kTileRows, rows);
-    for (uint32_t i = lane; i < (kTileRows * 32u * ES) / 16u; i += 32u)
-      reinterpret_cast<uint4*>(tile)[i] = fill4;
-    __syncwarp();
-    if (pending) {                                   // t - 1 is the row it belongs to
-      trow[(t - 1 - r0) * 32u + lane] = static_cast<E>(pend_val);
-      pending = false;
-    }
-    const uint32_t my_end = min(rend, my_count);
-    while (t < my_end) {
-      uint32_t e;
-      if (my_count - t > kMaxRun) e = mtab[state];   // run + 1 <= 16 symbols are still owed
-      else e = __ldg(g_single + state);              // tail: one symbol per look-up
-      t += entry_run(e);
-      const uint32_t val = vals[entry_sym(e)];
-      if (t < rend) trow[(t - r0) * 32u + lane] = static_cast<E>(val);
-      else { pending = true; pend_val = val; }
-      t += 1;
-      const uint32_t nb = entry_nb(e);
-      const uint32_t x = __funnelshift_r(w0, w1, bitpos);
-      state = entry_newx(e) + (x & ((1u << nb) - 1u));
-      bitpos += nb;
-      if (bitpos >= 32u) {
-        w0 = w1; w1 = w2; w2 = load_word(idx); ++idx;
-        bitpos -= 32u;
-      }
-    }
-    __syncwarp();
-    const uint32_t nrows = rend - r0;
-    const bool has_part = (rend == rows) && (min_count < rows);   // last row is ragged
-    const uint32_t full_rows = has_part ? nrows - 1 : nrows;
-    uint32_t part_lanes = 0;
-    if (has_part) part_lanes = __popc(__ballot_sync(kFull, my_count == rows));
-    flush_rows<ES>(tile, out + size_t(r0) * row_stride_bytes, row_stride_bytes, full_rows, part_lanes, lane);
-    __syncwarp();
-  }
-  uint32_t bad = 0;
-  if (state != 0) bad |= ANS_STATUS_BAD_FINAL_STATE;
-  // words used must be exactly the lane's run (the last lane's run is followed by < 16 pad bytes)
-  const uint32_t bits = (idx - 3u - wbeg) * 32u + bitpos;
-  const uint32_t need = (bits + 31u) / 32u;
-  const uint32_t have = wend - wbeg;
-  if (last_lane ? (need > have || have - need >= 4u) : (need != have)) bad |= ANS_STATUS_BAD_LENGTH;
-  return bad;
-}
-
-// ---------------------------------------------------------------------------------------------
-template <int LAYOUT>
-__global__ void __launch_bounds__(kThreads) ans_decode_kernel(const LaunchArgs args) {
+__global__ void __launch_bounds__(kIWarps * 32) ans_decode_interleaved_kernel(const LaunchArgs args) {
   extern __shared__ __align__(16) uint32_t smem[];
   uint32_t* tab = smem;                                   // [table_words]
   uint32_t* vals = smem + args.table_words;               // [256]
-  uint8_t* tiles = reinterpret_cast<uint8_t*>(vals + 256);  // private: kWarps * kTileRows * 128 B
-  __shared__ uint32_t s_dom;
+  constexpr uint32_t kThreads = kIWarps * 32;
 
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   uint64_t cursor = uint64_t(blockIdx.x) * args.items_per_cta;
   const uint64_t cta_end = min(cursor + uint64_t(args.items_per_cta), uint64_t(args.total_work));
   if (cursor >= cta_end) return;
 
-  // layer that holds `cursor`: last layer with work_begin <= cursor
-  int l = 0;
-  {
-    int lo = 0, hi = args.n_layers;
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (layer_at(args, mid).work_begin <= cursor) lo = mid; else hi = mid;
-    }
-    l = lo;
-  }
+  int l = find_layer(args, cursor);
   uint32_t bad = 0;
   for (; cursor < cta_end; ++l) {
     const ans_layer_desc& L = layer_at(args, l);
@@ -226,88 +160,377 @@ __global__ void __launch_bounds__(kThreads) ans_decode_kernel(const LaunchArgs a
     const int R = L.table_log;
     const uint8_t* blob = static_cast<const uint8_t*>(L.d_table);
     const TableHeader* hdr = reinterpret_cast<const TableHeader*>(blob);
-    const uint32_t* g_single = reinterpret_cast<const uint32_t*>(blob + single_offset());
-    const uint32_t* g_tab = LAYOUT == ANS_LAYOUT_PRIVATE
-                                ? reinterpret_cast<const uint32_t*>(blob + multi_offset(R)) : g_single;
+    const uint32_t* g_tab = reinterpret_cast<const uint32_t*>(blob + single_offset());
     const int dtype = args.d_symbols_override ? ANS_U8 : L.out_dtype;
 
     __syncthreads();                                      // previous layer's readers are done
-    {
-      const uint4* src = reinterpret_cast<const uint4*>(g_tab);
-      uint4* dst = reinterpret_cast<uint4*>(tab);
-      const uint32_t n16 = (1u << R) / 4u;
-      for (uint32_t i = threadIdx.x; i < n16; i += kThreads) dst[i] = __ldg(src + i);
-      if (R < 2 && threadIdx.x < (1u << R)) tab[threadIdx.x] = __ldg(g_tab + threadIdx.x);
-      vals[threadIdx.x] = dequant_bits(static_cast<int>(threadIdx.x), L.zero_point, L.scale, dtype);
-      if (threadIdx.x == 0) {
-        s_dom = hdr->dominant;
-        if (hdr->magic != kTableMagic || hdr->table_log != uint32_t(R) ||
-            hdr->alphabet > (1u << L.bitwidth))
-          bad |= ANS_STATUS_BAD_SYMBOL;
+    for (uint32_t i = threadIdx.x; i < (1u << R); i += kThreads) tab[i] = __ldg(g_tab + i);
+    vals[threadIdx.x] = dequant_bits(static_cast<int>(threadIdx.x), L.zero_point, L.scale, dtype);
+    if (threadIdx.x == 0 && (hdr->magic != kTableMagic || hdr->table_log != uint32_t(R) ||
+                             hdr->alphabet > (1u << L.bitwidth)))
+      bad |= ANS_STATUS_BAD_SYMBOL;
+    __syncthreads();
+
+    const uint32_t W = L.lanes;
+    const size_t es = dtype == ANS_U8 ? 1 : dtype == ANS_F32 ? 4 : 2;
+    uint8_t* out_base = args.d_symbols_override ? args.d_symbols_override : static_cast<uint8_t*>(L.d_out);
+    const uint64_t n_sub = uint64_t(L.lanes / 32u) * ((L.n_symbols + L.chunk_symbols - 1) / L.chunk_symbols);
+    for (uint64_t gbase = cursor; gbase < stop; gbase += kIWarps / kGranule) {
+      const uint64_t granule = gbase + warp / kGranule;
+      const uint64_t sub = (granule - lbeg) * kGranule + warp % kGranule;
+      if (granule >= stop || sub >= n_sub) continue;
+      const Item it = make_item(L, sub);
+      const uint32_t lambda = 32u * it.g + lane;
+      const uint32_t my_count = lane_symbols(it.nc, W, lambda);
+      const uint32_t rows = lane_symbols(it.nc, W, 32u * it.g);   // lane 0 owns the most
+      uint8_t* out = out_base + (it.c0 + lambda) * es;
+      const uint32_t state = __ldg(static_cast<const uint16_t*>(L.d_lane_meta) + it.sub * 32 + lane) &
+                             ((1u << R) - 1u);
+      const uint16_t* units = reinterpret_cast<const uint16_t*>(L.d_stream + it.off0);
+      const uint32_t cap = static_cast<uint32_t>(min(it.extent / 2, uint64_t(0xFFFFFFFFu)));
+      uint32_t wbad = it.bad;
+      if (es == 1)
+        wbad |= decode_interleaved<1>(tab, vals, units, cap, state, my_count, rows, out, W, lane);
+      else if (es == 2)
+        wbad |= decode_interleaved<2>(tab, vals, units, cap, state, my_count, rows,
+                                      reinterpret_cast<uint16_t*>(out), W, lane);
+      else
+        wbad |= decode_interleaved<4>(tab, vals, units, cap, state, my_count, rows,
+                                      reinterpret_cast<uint32_t*>(out), W, lane);
+      bad |= wbad;
+    }
+    cursor = stop;
+  }
+  bad = __reduce_or_sync(kFull, bad);
+  if (lane == 0 && bad && args.d_status) atomicOr(args.d_status, bad);
+}
+
+// =============================================================================================
+// Private container: every lane reads its own run of 32-bit words.
+//
+// Look-ups go through the pre-walked table, so one look-up can stand for several symbols: `run`
+// copies of the layer's dominant symbol (its zero-bit states, Section II-A's unlabeled
+// transitions) followed by one more symbol.  Lanes therefore drift apart; each warp keeps a ring
+// of output rows in shared memory, pre-filled with the dominant value, into which lanes drop
+// the other symbols.  A quarter of the ring is written out (16-byte stores) as soon as the
+// slowest lane has left it.  The sub-stream's compressed bytes are brought into shared memory by
+// one bulk asynchronous copy per warp, so a lane's refill is a shared-memory load.
+// =============================================================================================
+constexpr uint32_t kRingBytes = 8192;          // per warp; rows = kRingBytes / (32 * ES)
+constexpr uint32_t kStagePad = 48;             // readable bytes after the staged sub-stream
+constexpr uint32_t kWaitSpins = 1u << 22;
+constexpr uint32_t kPair = 2 * (kMaxRun + 1);  // symbols two look-ups can emit
+
+// shared-memory form of a pre-walked entry: newX*4 [15:0] | sym [23:16] | run [27:24] | nb [31:28]
+__device__ __forceinline__ uint32_t to_smem_entry(uint32_t g) {
+  return (entry_newx(g) << 2) | (entry_sym(g) << 16) | (entry_run(g) << 24) | (entry_nb(g) << 28);
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+
+template <int ES>
+__device__ __forceinline__ void flush_rows(const uint8_t* tile, uint8_t* out_row0, size_t row_stride_bytes,
+                                           uint32_t full_rows, uint32_t part_row_lanes, uint32_t lane) {
+  constexpr uint32_t RB = 32u * ES;                 // bytes per row
+  constexpr uint32_t PPR = RB / 16u;                // 16-byte pieces per row
+  using E = typename ElemT<ES>::type;
+  if ((reinterpret_cast<uintptr_t>(out_row0) & 15u) == 0 && (row_stride_bytes & 15u) == 0) {
+    for (uint32_t idx = lane; idx < full_rows * PPR; idx += 32u) {
+      const uint32_t row = idx / PPR, piece = idx % PPR;
+      const uint4 v = *reinterpret_cast<const uint4*>(tile + size_t(idx) * 16u);
+      *reinterpret_cast<uint4*>(out_row0 + size_t(row) * row_stride_bytes + piece * 16u) = v;
+    }
+  } else {
+    for (uint32_t row = 0; row < full_rows; ++row)
+      reinterpret_cast<E*>(out_row0 + size_t(row) * row_stride_bytes)[lane] =
+          reinterpret_cast<const E*>(tile)[row * 32u + lane];
+  }
+  if (lane < part_row_lanes)
+    reinterpret_cast<E*>(out_row0 + size_t(full_rows) * row_stride_bytes)[lane] =
+        reinterpret_cast<const E*>(tile)[full_rows * 32u + lane];
+}
+
+// Decode one sub-stream.  All shared-memory operands are byte offsets from `sm` (the CTA's
+// dynamic shared memory), so that address arithmetic stays 32-bit; the ring's offset is a
+// multiple of kRingBytes, which lets a row address be formed with one OR.
+// `words` is the sub-stream in global memory; when STAGED its copy sits at sm + stage_off and
+// has kStagePad readable bytes after it.
+template <int ES, bool STAGED>
+__device__ __forceinline__ uint32_t decode_private(
+    uint8_t* __restrict__ sm, uint32_t tab_off, uint32_t vals_off, uint32_t ring_off, uint32_t stage_off,
+    const uint32_t* __restrict__ g_single, uint32_t dom_val, const uint32_t* __restrict__ words,
+    uint32_t ext_words, uint32_t wbeg, uint32_t wend, bool last_lane, uint32_t state, uint32_t my_count,
+    uint32_t rows, uint32_t min_count, uint8_t* __restrict__ out_row0, size_t row_stride_bytes, uint32_t lane) {
+  using E = typename ElemT<ES>::type;
+  constexpr uint32_t RB = 32u * ES;
+  constexpr uint32_t RING = kRingBytes / RB;        // rows in the ring
+  constexpr uint32_t FL = RING / 4;                 // rows written out at a time
+  constexpr uint32_t MASK = kRingBytes - 1u;
+  static_assert(RING - FL >= kPair + FL, "a lane must be able to run ahead of the write-out");
+  uint8_t* ring = sm + ring_off;
+  const uint32_t lane_off = ring_off + lane * ES;
+
+  // bit window: w0/w1 hold the 64 bits being read, w2 is one word ahead.  A staged lane may
+  // look up to word_limit + 4 words into its buffer, which holds ext_words + kStagePad / 4.
+  const uint32_t word_limit = STAGED ? ext_words + 4u : ext_words;
+  auto load_word = [&](uint32_t i) -> uint32_t {
+    if (STAGED) return *reinterpret_cast<const uint32_t*>(sm + stage_off + i * 4u);
+    return i < word_limit ? __ldg(words + i) : 0u;
+  };
+  uint32_t idx = wbeg;
+  uint32_t w0 = load_word(idx), w1 = load_word(idx + 1), w2 = load_word(idx + 2);
+  idx += 3;
+  uint32_t bitpos = 0;
+  bool overran = false;
+
+  uint32_t fill = dom_val;
+  if (ES == 1) fill *= 0x01010101u;
+  if (ES == 2) fill *= 0x00010001u;
+  const uint4 fill4 = make_uint4(fill, fill, fill, fill);
+  for (uint32_t i = lane; i < kRingBytes / 16u; i += 32u) reinterpret_cast<uint4*>(ring)[i] = fill4;
+  __syncwarp();
+
+  // rows [first_row, first_row + n_rows), then `part_lanes` elements of the row after them;
+  // the range may wrap around the ring's end
+  auto write_out = [&](uint32_t first_row, uint32_t n_rows, uint32_t part_lanes) {
+    uint32_t done = 0;
+    while (done < n_rows) {
+      const uint32_t r = first_row + done;
+      const uint32_t ring_row = r % RING;
+      const uint32_t piece = min(n_rows - done, RING - ring_row);
+      flush_rows<ES>(ring + size_t(ring_row) * RB, out_row0 + size_t(r) * row_stride_bytes, row_stride_bytes,
+                     piece, 0u, lane);
+      done += piece;
+    }
+    if (part_lanes) {
+      const uint32_t r = first_row + n_rows;
+      flush_rows<ES>(ring + size_t(r % RING) * RB, out_row0 + size_t(r) * row_stride_bytes, row_stride_bytes,
+                     0u, part_lanes, lane);
+    }
+  };
+
+  uint32_t st4 = state * 4u;                        // byte offset of the state's table entry
+  uint32_t tb = 0;                                  // RB * (next row this lane decodes)
+  // one pre-walked look-up: emits run + 1 symbols, takes its bits from the low end of x
+  auto step = [&](uint32_t x) -> uint32_t {
+    const uint32_t e = *reinterpret_cast<const uint32_t*>(sm + tab_off + st4);
+    const uint32_t nb = e >> 28;
+    st4 = (e & 0xFFFFu) + ((x & ((1u << nb) - 1u)) << 2);
+    const uint32_t val = *reinterpret_cast<const uint32_t*>(sm + vals_off + ((e >> 14) & 0x3FCu));
+    tb += ((e >> 24) & 15u) * RB;
+    *reinterpret_cast<E*>(sm + ((tb & MASK) | lane_off)) = static_cast<E>(val);
+    tb += RB;
+    return nb;
+  };
+  auto refill = [&]() {
+    if (bitpos >= 32u) {
+      w0 = w1; w1 = w2; w2 = load_word(idx); ++idx;
+      bitpos -= 32u;
+    }
+  };
+
+  // main part: two look-ups share one 32-bit extract (2 * 14 bits at most) and one refill check
+  const uint32_t lim2 = (my_count > kPair - 1 ? my_count - (kPair - 1) : 0u) * RB;
+  const uint32_t lim1 = (my_count > kMaxRun ? my_count - kMaxRun : 0u) * RB;
+  uint32_t base = 0;                                // first row not yet written out
+  for (;;) {
+    const uint32_t lim = min(lim2, (base + RING - kPair) * RB);
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (tb < lim) {
+        const uint32_t x = __funnelshift_r(w0, w1, bitpos);
+        const uint32_t nb1 = step(x);
+        const uint32_t nb2 = step(x >> nb1);
+        bitpos += nb1 + nb2;
+        refill();
       }
+    }
+    if (STAGED && idx > word_limit) { overran = true; idx = word_limit; }
+    const uint32_t tmin = __reduce_min_sync(kFull, tb) / RB;
+    while (tmin >= base + FL) {                     // the slowest lane has left these rows
+      __syncwarp();
+      write_out(base, FL, 0u);
+      __syncwarp();
+      uint8_t* part = ring + size_t(base % RING) * RB;
+      for (uint32_t i = lane; i < (FL * RB) / 16u; i += 32u) reinterpret_cast<uint4*>(part)[i] = fill4;
+      base += FL;
+      __syncwarp();
+    }
+    if (__all_sync(kFull, tb >= lim2)) break;
+  }
+  // then single pre-walked look-ups while at least 16 symbols are owed to the lane ...
+  while (tb < lim1) {
+    bitpos += step(__funnelshift_r(w0, w1, bitpos));
+    if (bitpos >= 32u) {
+      w0 = w1; w1 = w2;
+      w2 = (!STAGED || idx < word_limit) ? load_word(idx) : 0u;
+      ++idx;
+      bitpos -= 32u;
+    }
+  }
+  // ... and the last (up to 15) symbols one per look-up through the plain table
+  uint32_t t = tb / RB;
+  state = st4 >> 2;
+  while (t < my_count) {
+    const uint32_t e = __ldg(g_single + state);
+    const uint32_t val = *reinterpret_cast<const uint32_t*>(sm + vals_off + entry_sym(e) * 4u);
+    *reinterpret_cast<E*>(sm + (((t * RB) & MASK) | lane_off)) = static_cast<E>(val);
+    t += 1;
+    const uint32_t nb = entry_nb(e);
+    const uint32_t x = __funnelshift_r(w0, w1, bitpos);
+    state = entry_newx(e) + (x & ((1u << nb) - 1u));
+    bitpos += nb;
+    if (bitpos >= 32u) {
+      w0 = w1; w1 = w2;
+      w2 = (!STAGED || idx < word_limit) ? load_word(idx) : 0u;
+      ++idx;
+      bitpos -= 32u;
+    }
+  }
+  __syncwarp();
+  {
+    const bool has_part = min_count < rows;         // last row is ragged
+    const uint32_t full_rows = (has_part ? rows - 1 : rows) - base;
+    uint32_t part_lanes = 0;
+    if (has_part) part_lanes = __popc(__ballot_sync(kFull, my_count == rows));
+    write_out(base, full_rows, part_lanes);
+  }
+  __syncwarp();
+  uint32_t bad = 0;
+  if (state != 0) bad |= ANS_STATUS_BAD_FINAL_STATE;
+  // words used must be exactly the lane's run (the last lane's run is followed by < 16 pad bytes)
+  const uint32_t bits = (idx - 3u - wbeg) * 32u + bitpos;
+  const uint32_t need = (bits + 31u) / 32u;
+  const uint32_t have = wend - wbeg;
+  if (overran || (last_lane ? (need > have || have - need >= 4u) : (need != have))) bad |= ANS_STATUS_BAD_LENGTH;
+  return bad;
+}
+
+// dynamic shared memory: [rings: NW * kRingBytes][table][vals 256][mbarriers NW][stages NW * stage_bytes]
+__global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const LaunchArgs args) {
+  extern __shared__ __align__(16) uint8_t sm[];
+  const uint32_t NW = blockDim.x >> 5;
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  const uint32_t tab_off = NW * kRingBytes;
+  const uint32_t vals_off = tab_off + args.table_words * 4u;
+  const uint32_t bars_off = vals_off + 1024u;
+  const uint32_t ring_off = warp * kRingBytes;
+  const uint32_t stage_off = bars_off + NW * 8u + warp * args.stage_bytes;
+  uint32_t* tab = reinterpret_cast<uint32_t*>(sm + tab_off);
+  uint32_t* vals = reinterpret_cast<uint32_t*>(sm + vals_off);
+  const uint32_t bar = smem_u32(sm + bars_off + warp * 8u);
+  __shared__ uint32_t s_dom;
+  uint32_t parity = 0;
+
+  uint64_t cursor = uint64_t(blockIdx.x) * args.items_per_cta;
+  const uint64_t cta_end = min(cursor + uint64_t(args.items_per_cta), uint64_t(args.total_work));
+  if (cursor >= cta_end) return;
+  if (lane == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(bar) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+
+  int l = find_layer(args, cursor);
+  uint32_t bad = 0;
+  bool gave_up = false;
+  for (; cursor < cta_end; ++l) {
+    const ans_layer_desc& L = layer_at(args, l);
+    const uint64_t lbeg = L.work_begin, lend = lbeg + L.work_count;
+    if (lend <= cursor) continue;                         // empty layer
+    const uint64_t stop = min(lend, cta_end);
+    const int R = L.table_log;
+    const uint8_t* blob = static_cast<const uint8_t*>(L.d_table);
+    const TableHeader* hdr = reinterpret_cast<const TableHeader*>(blob);
+    const uint32_t* g_single = reinterpret_cast<const uint32_t*>(blob + single_offset());
+    const uint32_t* g_multi = reinterpret_cast<const uint32_t*>(blob + multi_offset(R));
+    const int dtype = args.d_symbols_override ? ANS_U8 : L.out_dtype;
+
+    __syncthreads();                                      // previous layer's readers are done
+    for (uint32_t i = threadIdx.x; i < (1u << R); i += blockDim.x) tab[i] = to_smem_entry(__ldg(g_multi + i));
+    for (uint32_t i = threadIdx.x; i < 256u; i += blockDim.x)
+      vals[i] = dequant_bits(static_cast<int>(i), L.zero_point, L.scale, dtype);
+    if (threadIdx.x == 0) {
+      s_dom = hdr->dominant;
+      if (hdr->magic != kTableMagic || hdr->table_log != uint32_t(R) || hdr->alphabet > (1u << L.bitwidth))
+        bad |= ANS_STATUS_BAD_SYMBOL;
     }
     __syncthreads();
 
-    const uint32_t G = L.lanes / 32u, W = L.lanes, C = L.chunk_symbols;
+    const uint32_t W = L.lanes;
+    const uint64_t n_sub = uint64_t(L.lanes / 32u) * ((L.n_symbols + L.chunk_symbols - 1) / L.chunk_symbols);
     const size_t es = dtype == ANS_U8 ? 1 : dtype == ANS_F32 ? 4 : 2;
     uint8_t* out_base = args.d_symbols_override ? args.d_symbols_override : static_cast<uint8_t*>(L.d_out);
-    for (uint64_t base = cursor; base < stop; base += kWarps) {
-      const uint64_t item = base + warp;
-      if (item >= stop) continue;
-      const uint64_t sub = item - lbeg;
-      const uint64_t chunk = sub / G;
-      const uint32_t g = static_cast<uint32_t>(sub % G);
-      const uint64_t c0 = chunk * C;
-      const uint32_t nc = static_cast<uint32_t>(min(uint64_t(C), L.n_symbols - c0));
-      const uint32_t lambda = 32u * g + lane;
-      const uint32_t my_count = lane_symbols(nc, W, lambda);
-      const uint32_t rows = lane_symbols(nc, W, 32u * g);          // lane 0 owns the most
-      const uint32_t min_count = lane_symbols(nc, W, 32u * g + 31u);
-      const uint64_t off0 = __ldg(L.d_sub_offsets + sub), off1 = __ldg(L.d_sub_offsets + sub + 1);
-      uint32_t wbad = 0;
-      uint64_t extent = off1 - off0;
-      if (off1 < off0 || off1 > L.stream_bytes || (off0 & 15u)) {   // never read outside the stream
-        extent = 0;
-        wbad |= ANS_STATUS_BAD_LENGTH;
+    const uint32_t dom = s_dom < 256u ? vals[s_dom] : 0u;
+    for (uint64_t gbase = cursor; gbase < stop && !gave_up; gbase += NW / kGranule) {
+      const uint64_t granule = gbase + warp / kGranule;
+      const uint64_t sub = (granule - lbeg) * kGranule + warp % kGranule;
+      if (granule >= stop || sub >= n_sub) continue;
+      const Item it = make_item(L, sub);
+      uint32_t wbad = it.bad;
+      const uint32_t lambda = 32u * it.g + lane;
+      const uint32_t my_count = lane_symbols(it.nc, W, lambda);
+      const uint32_t rows = lane_symbols(it.nc, W, 32u * it.g);
+      const uint32_t min_count = lane_symbols(it.nc, W, 32u * it.g + 31u);
+      const uint32_t ext_words = static_cast<uint32_t>(min(it.extent / 4, uint64_t(0x3FFFFFFFu)));
+      const uint8_t* g_bytes = L.d_stream + it.off0;
+
+      // bring the sub-stream into shared memory (one bulk copy), if it fits
+      const bool staged = it.extent > 0 && it.extent + kStagePad <= args.stage_bytes;
+      if (staged) {
+        __syncwarp();                                     // the last item's readers of the stage are done
+        if (lane == 0) {
+          const uint32_t bytes = static_cast<uint32_t>(it.extent);
+          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+          asm volatile(
+              "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+              :: "r"(smem_u32(sm + stage_off)), "l"(g_bytes), "r"(bytes), "r"(bar) : "memory");
+        }
+        if (lane < kStagePad / 4u) reinterpret_cast<uint32_t*>(sm + stage_off + it.extent)[lane] = 0u;
       }
-      uint8_t* out = out_base + (c0 + lambda) * es;
-      const size_t row_stride = W;
-      if (LAYOUT == ANS_LAYOUT_INTERLEAVED) {
-        const uint32_t state = __ldg(static_cast<const uint16_t*>(L.d_lane_meta) + sub * 32 + lane) &
-                               ((1u << R) - 1u);
-        const uint16_t* units = reinterpret_cast<const uint16_t*>(L.d_stream + (extent ? off0 : 0));
-        const uint32_t cap = static_cast<uint32_t>(min(extent / 2, uint64_t(0xFFFFFFFFu)));
-        if (es == 1)
-          wbad |= decode_interleaved<1>(tab, vals, units, cap, state, my_count, rows, out, row_stride, lane);
-        else if (es == 2)
-          wbad |= decode_interleaved<2>(tab, vals, units, cap, state, my_count, rows,
-                                       reinterpret_cast<uint16_t*>(out), row_stride, lane);
-        else
-          wbad |= decode_interleaved<4>(tab, vals, units, cap, state, my_count, rows,
-                                       reinterpret_cast<uint32_t*>(out), row_stride, lane);
+
+      const uint32_t meta = __ldg(static_cast<const uint32_t*>(L.d_lane_meta) + it.sub * 32 + lane);
+      const uint32_t state = meta & ((1u << R) - 1u);
+      uint32_t wbeg = meta >> 16;
+      uint32_t wend = __shfl_down_sync(kFull, wbeg, 1);
+      if (lane == 31) wend = ext_words;
+      if (wend > ext_words) { wend = ext_words; wbad |= ANS_STATUS_BAD_LENGTH; }
+      if (wbeg > wend) { wbeg = wend; wbad |= ANS_STATUS_BAD_LENGTH; }
+      uint8_t* out_row0 = out_base + (it.c0 + 32u * it.g) * es;     // row 0 of this sub-stream
+      const size_t rsb = size_t(W) * es;
+      const uint32_t* words = reinterpret_cast<const uint32_t*>(g_bytes);
+
+      if (staged) {
+        const bool ok = mbar_wait(bar, parity);
+        parity ^= 1u;
+        if (!__all_sync(kFull, ok)) {                     // the copy never landed: stop this warp's work
+          bad |= wbad | kStatusTimeout;
+          gave_up = true;
+          continue;
+        }
+        __syncwarp();
+      }
+#define ANSB_PRIV(ES_, ST_)                                                                              \
+  wbad |= decode_private<ES_, ST_>(sm, tab_off, vals_off, ring_off, stage_off, g_single, dom, words,     \
+                                   ext_words, wbeg, wend, lane == 31, state, my_count, rows, min_count, \
+                                   out_row0, rsb, lane)
+      if (staged) {
+        if (es == 1) ANSB_PRIV(1, true); else if (es == 2) ANSB_PRIV(2, true); else ANSB_PRIV(4, true);
       } else {
-        const uint32_t meta = __ldg(static_cast<const uint32_t*>(L.d_lane_meta) + sub * 32 + lane);
-        const uint32_t state = meta & ((1u << R) - 1u);
-        const uint32_t ext_words = static_cast<uint32_t>(min(extent / 4, uint64_t(0x7FFFFFFFu)));
-        uint32_t wbeg = meta >> 16;
-        uint32_t wend = __shfl_down_sync(kFull, wbeg, 1);
-        if (lane == 31) wend = ext_words;
-        if (wend > ext_words) { wend = ext_words; wbad |= ANS_STATUS_BAD_LENGTH; }
-        if (wbeg > wend) { wbeg = wend; wbad |= ANS_STATUS_BAD_LENGTH; }
-        const uint32_t* words = reinterpret_cast<const uint32_t*>(L.d_stream + (extent ? off0 : 0));
-        uint8_t* tile = tiles + size_t(warp) * (kTileRows * 32u * es);
-        uint8_t* out_row0 = out_base + (c0 + 32u * g) * es;     // row 0 of this sub-stream
-        const uint32_t dom = s_dom < 256u ? vals[s_dom] : 0u;
-        if (es == 1)
-          wbad |= decode_private<1>(tab, g_single, vals, dom, words, wbeg, wend, lane == 31, state, my_count,
-                                    rows, min_count, tile, out_row0, row_stride * es, lane);
-        else if (es == 2)
-          wbad |= decode_private<2>(tab, g_single, vals, dom, words, wbeg, wend, lane == 31, state, my_count,
-                                    rows, min_count, tile, out_row0, row_stride * es, lane);
-        else
-          wbad |= decode_private<4>(tab, g_single, vals, dom, words, wbeg, wend, lane == 31, state, my_count,
-                                    rows, min_count, tile, out_row0, row_stride * es, lane);
+        if (es == 1) ANSB_PRIV(1, false); else if (es == 2) ANSB_PRIV(2, false); else ANSB_PRIV(4, false);
       }
+#undef ANSB_PRIV
       bad |= wbad;
     }
     cursor = stop;
@@ -321,16 +544,19 @@ __global__ void __launch_bounds__(kThreads) ans_decode_kernel(const LaunchArgs a
 // ---------------------------------------------------------------------------------------------
 static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, int n_layers,
                   uint8_t* d_symbols_override, uint32_t* d_status, cudaStream_t st) {
-  int max_log = 1;
-  uint64_t total = 0;
+  int max_log = 1, busy_layers = 0;
+  uint64_t total = 0, stream_total = 0, sub_total = 0;
   const int layout = h_descs[0].layout;
   for (int l = 0; l < n_layers; ++l) {
     const int rc = validate_desc(h_descs[l], d_symbols_override == nullptr);
     if (rc != ANS_OK) return rc;
     if (h_descs[l].layout != layout) return ANS_ERR_UNSUPPORTED;
-    if (h_descs[l].work_begin != total || h_descs[l].work_count != subs_of(h_descs[l]))
+    if (h_descs[l].work_begin != total || h_descs[l].work_count != granules_of(h_descs[l]))
       return ANS_ERR_INVALID_ARG;                         // ans_plan_batch was not run on this array
     total += h_descs[l].work_count;
+    sub_total += subs_of(h_descs[l]);
+    stream_total += h_descs[l].stream_bytes;
+    busy_layers += h_descs[l].work_count != 0;
     if (h_descs[l].table_log > max_log) max_log = h_descs[l].table_log;
   }
   if (total == 0) return ANS_OK;
@@ -344,28 +570,50 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   a.d_status = d_status;
   a.d_symbols_override = d_symbols_override;
   a.table_words = max_log < 2 ? 4u : (1u << max_log);
-  size_t smem = (size_t(a.table_words) + 256) * 4;
-  if (layout == ANS_LAYOUT_PRIVATE) smem += size_t(kWarps) * kTileRows * 32 * 4;
 
-  const void* fn = layout == ANS_LAYOUT_PRIVATE
-                       ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE>)
-                       : reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED>);
-  int dev = 0, sms = 0, per_sm = 0;
+  int dev = 0, sms = 0, per_sm = 0, smem_max = 0;
   ANSB_CUDA(cudaGetDevice(&dev));
   ANSB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  ANSB_CUDA(cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+
+  const bool priv = layout == ANS_LAYOUT_PRIVATE;
+  const void* fn = priv ? reinterpret_cast<const void*>(&ans_decode_private_kernel)
+                        : reinterpret_cast<const void*>(&ans_decode_interleaved_kernel);
+  int warps = kIWarps;
+  size_t smem = (size_t(a.table_words) + 256) * 4;
+  if (priv) {
+    // Layers with many sub-streams share one table among 16 warps; a model of many small layers
+    // runs CTAs of one granule (4 warps) so that each CTA stays inside one layer and several
+    // CTAs, each with its own table, share an SM.
+    const bool big = total / uint64_t(busy_layers) >= 64;
+    // staging buffer per warp: the average sub-stream plus a quarter (a larger one is read from
+    // global memory instead), within what the CTA may hold
+    size_t want = (stream_total / sub_total) * 5 / 4 + kStagePad + 64;
+    want = (want + 127) & ~size_t(127);
+    const size_t table_part = smem + 16 * 8;
+    warps = big ? 16 : 4;
+    while (warps > 4 && table_part + size_t(warps) * (kRingBytes + want) + 1024 > size_t(smem_max)) warps -= 4;
+    const size_t fixed = table_part + size_t(warps) * kRingBytes;
+    const size_t room = size_t(smem_max) > fixed + 1024 ? (size_t(smem_max) - fixed - 1024) / warps : 0;
+    size_t stage = (want < room ? want : room) & ~size_t(15);
+    if (stage < 256) stage = 0;
+    a.stage_bytes = static_cast<uint32_t>(stage);
+    smem = size_t(warps) * kRingBytes + (size_t(a.table_words) + 256) * 4 + size_t(warps) * 8 + size_t(warps) * stage;
+  }
   ANSB_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-  ANSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, smem));
+  ANSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, warps * 32, smem));
   if (per_sm < 1) return ANS_ERR_UNSUPPORTED;
-  const uint64_t want = (total + kWarps - 1) / kWarps;
-  const uint64_t grid = want < uint64_t(sms) * per_sm ? want : uint64_t(sms) * per_sm;
+  const uint64_t step = uint64_t(warps) / kGranule;       // granules a CTA takes at a time
+  const uint64_t want_ctas = (total + step - 1) / step;
+  const uint64_t grid = want_ctas < uint64_t(sms) * per_sm ? want_ctas : uint64_t(sms) * per_sm;
   uint64_t ipc = (total + grid - 1) / grid;
-  ipc = (ipc + kWarps - 1) / kWarps * kWarps;             // whole warps-per-CTA steps
+  ipc = (ipc + step - 1) / step * step;
   a.items_per_cta = static_cast<uint32_t>(ipc);
   const unsigned blocks = static_cast<unsigned>((total + ipc - 1) / ipc);
-  if (layout == ANS_LAYOUT_PRIVATE)
-    ans_decode_kernel<ANS_LAYOUT_PRIVATE><<<blocks, kThreads, smem, st>>>(a);
+  if (priv)
+    ans_decode_private_kernel<<<blocks, warps * 32, smem, st>>>(a);
   else
-    ans_decode_kernel<ANS_LAYOUT_INTERLEAVED><<<blocks, kThreads, smem, st>>>(a);
+    ans_decode_interleaved_kernel<<<blocks, kIWarps * 32, smem, st>>>(a);
   ANSB_CUDA(cudaGetLastError());
   return ANS_OK;
 }
@@ -380,7 +628,7 @@ ANS_EXPORT int ans_plan_batch(ans_layer_desc* h_descs, int n_layers, uint64_t* h
   for (int l = 0; l < n_layers; ++l) {
     ans_layer_desc& d = h_descs[l];
     if (d.chunk_symbols == 0 || d.lanes == 0 || d.lanes % 32) return ANS_ERR_INVALID_ARG;
-    const uint64_t n = subs_of(d);
+    const uint64_t n = granules_of(d);
     if (total + n > 0xFFFFFFFFull) return ANS_ERR_UNSUPPORTED;
     d.work_begin = static_cast<uint32_t>(total);
     d.work_count = static_cast<uint32_t>(n);

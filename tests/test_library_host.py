@@ -57,12 +57,12 @@ def test_host_packer_equals_oracle_encoder(layout, n, C, lanes, R, b):
         assert (o == P.sub_offsets).all() and (m == P.lane_meta).all()
 
 
-def test_plan_batch_counts_sub_streams():
+def test_plan_batch_counts_groups_of_four_sub_streams():
     arr = (ans.ans_layer_desc * 3)()
     for d, (n, C, lanes) in zip(arr, [(36864, 4096, 32), (0, 4096, 64), (10, 4, 128)]):
         d.n_symbols, d.chunk_symbols, d.lanes = n, C, lanes
-    assert ans.ans_plan_batch(arr) == 9 + 0 + 3 * 4
-    assert [d.work_begin for d in arr] == [0, 9, 9] and [d.work_count for d in arr] == [9, 0, 12]
+    assert ans.ans_plan_batch(arr) == 3 + 0 + 3
+    assert [d.work_begin for d in arr] == [0, 3, 3] and [d.work_count for d in arr] == [3, 0, 3]
 
 
 def test_argument_errors_come_back_without_a_gpu():
