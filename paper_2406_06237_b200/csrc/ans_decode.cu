@@ -217,7 +217,7 @@ __global__ void __launch_bounds__(kIWarps * 32) ans_decode_interleaved_kernel(co
 // one bulk asynchronous copy per warp, so a lane's refill is a shared-memory load.
 // =============================================================================================
 constexpr uint32_t kRingBytes = 8192;          // per warp; rows = kRingBytes / (32 * ES)
-constexpr uint32_t kStagePad = 48;             // readable bytes after the staged sub-stream
+constexpr uint32_t kStagePad = 80;             // readable bytes after the staged sub-stream
 constexpr uint32_t kWaitSpins = 1u << 22;
 constexpr uint32_t kPair = 2 * (kMaxRun + 1);  // symbols two look-ups can emit
 
@@ -261,31 +261,110 @@ __device__ __forceinline__ void flush_rows(const uint8_t* tile, uint8_t* out_row
         reinterpret_cast<const E*>(tile)[full_rows * 32u + lane];
 }
 
-// Decode one sub-stream.  All shared-memory operands are byte offsets from `sm` (the CTA's
-// dynamic shared memory), so that address arithmetic stays 32-bit; the ring's offset is a
-// multiple of kRingBytes, which lets a row address be formed with one OR.
-// `words` is the sub-stream in global memory; when STAGED its copy sits at sm + stage_off and
-// has kStagePad readable bytes after it.
+// ---- shared-memory accesses by absolute (shared-window) address --------------------------------
+__device__ __forceinline__ uint32_t lds_u32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+  return v;
+}
+template <int ES>
+__device__ __forceinline__ void sts_elem(uint32_t a, uint32_t v) {
+  if (ES == 1) asm volatile("st.shared.u8 [%0], %1;" :: "r"(a), "r"(v) : "memory");
+  if (ES == 2) asm volatile("st.shared.u16 [%0], %1;" :: "r"(a), "r"(v) : "memory");
+  if (ES == 4) asm volatile("st.shared.u32 [%0], %1;" :: "r"(a), "r"(v) : "memory");
+}
+
+// The hot loop, for a staged sub-stream: kPairsPerCall times, every lane with tb < lim makes two
+// pre-walked look-ups that share one 32-bit extract of its bit window and one refill check.
+// Written as one PTX block so that the loop-carried values stay in registers across iterations.
+//   st  : shared address of the state's table entry      tb : RB * (next row of the lane)
+//   w0,w1,w2 : bit window and the word after it           sp : shared address of the next word
+// Entry: newX*4 [15:0] | sym [23:16] | run [27:24] | nb [31:28].  vals_abs is 1 KB aligned and
+// ring_lane_abs has its low 13 bits (but for lane * ES) clear, so OR forms both addresses.
+constexpr int kPairsPerCall = 8;
+
+#define ANSB_STEP(NB_, STOP_)                                     \
+  "ld.shared.u32 e, [%0];\n\t"                                    \
+  "shr.u32 " NB_ ", e, 28;\n\t"                                   \
+  "bmsk.clamp.b32 m, 0, " NB_ ";\n\t"                             \
+  "and.b32 v, x, m;\n\t"                                          \
+  "and.b32 nx, e, 0xFFFF;\n\t"                                    \
+  "add.u32 nx, nx, %8;\n\t"                                       \
+  "mad.lo.u32 %0, v, 4, nx;\n\t"                                  \
+  "shr.u32 sy, e, 14;\n\t"                                        \
+  "lop3.b32 sy, sy, 0x3FC, %9, 0xEA;\n\t"                         \
+  "ld.shared.u32 val, [sy];\n\t"                                  \
+  "bfe.u32 r, e, 24, 4;\n\t"                                      \
+  "mad.lo.u32 %1, r, %11, %1;\n\t"                                \
+  "lop3.b32 a, %1, %12, %10, 0xEA;\n\t"                           \
+  STOP_ " [a], val;\n\t"                                          \
+  "add.u32 %1, %1, %11;\n\t"
+
+template <int ES>
+__device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tb, uint32_t& bitpos, uint32_t& w0,
+                                           uint32_t& w1, uint32_t& w2, uint32_t& sp, uint32_t lim,
+                                           uint32_t tab_abs, uint32_t vals_abs, uint32_t ring_lane_abs) {
+  constexpr uint32_t RB = 32u * ES;
+  constexpr uint32_t MASK = kRingBytes - 1u;
+#define ANSB_PAIRS(STOP_)                                                                  \
+  asm volatile(                                                                            \
+      "{\n\t"                                                                              \
+      ".reg .pred p, q;\n\t"                                                               \
+      ".reg .u32 x, e, n1, n2, m, v, nx, sy, val, r, a, cnt;\n\t"                         \
+      "mov.u32 cnt, %13;\n"                                                                \
+      "ANSB_LOOP:\n\t"                                                                     \
+      "setp.lt.u32 p, %1, %7;\n\t"                                                         \
+      "@!p bra ANSB_SKIP;\n\t"                                                             \
+      "shf.r.wrap.b32 x, %3, %4, %2;\n\t"                                                  \
+      ANSB_STEP("n1", STOP_)                                                               \
+      "shr.u32 x, x, n1;\n\t"                                                              \
+      ANSB_STEP("n2", STOP_)                                                               \
+      "add.u32 %2, %2, n1;\n\t"                                                            \
+      "add.u32 %2, %2, n2;\n\t"                                                            \
+      "setp.ge.u32 q, %2, 32;\n\t"                                                         \
+      "@q mov.u32 %3, %4;\n\t"                                                             \
+      "@q mov.u32 %4, %5;\n\t"                                                             \
+      "@q ld.shared.u32 %5, [%6];\n\t"                                                     \
+      "@q add.u32 %6, %6, 4;\n\t"                                                          \
+      "@q add.u32 %2, %2, -32;\n"                                                          \
+      "ANSB_SKIP:\n\t"                                                                     \
+      "add.u32 cnt, cnt, -1;\n\t"                                                          \
+      "setp.ne.u32 p, cnt, 0;\n\t"                                                         \
+      "@p bra ANSB_LOOP;\n\t"                                                              \
+      "}"                                                                                  \
+      : "+r"(st), "+r"(tb), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp)           \
+      : "r"(lim), "r"(tab_abs), "r"(vals_abs), "r"(ring_lane_abs), "n"(RB), "n"(MASK),     \
+        "n"(kPairsPerCall)                                                                 \
+      : "memory")
+  if (ES == 1) ANSB_PAIRS("st.shared.u8");
+  if (ES == 2) ANSB_PAIRS("st.shared.u16");
+  if (ES == 4) ANSB_PAIRS("st.shared.u32");
+#undef ANSB_PAIRS
+}
+
+// Decode one sub-stream.  Shared memory is addressed by absolute shared-window addresses:
+// tab_abs (table), vals_abs (dequantised values, 1 KB aligned), ring_abs (this warp's ring,
+// kRingBytes aligned), stage_abs (staged sub-stream when STAGED, with kStagePad readable bytes
+// after it).  `ring` is the generic pointer to the same ring; `words` the sub-stream in
+// global memory, used when it was not staged.
 template <int ES, bool STAGED>
-__device__ __forceinline__ uint32_t decode_private(
-    uint8_t* __restrict__ sm, uint32_t tab_off, uint32_t vals_off, uint32_t ring_off, uint32_t stage_off,
+__device__ __noinline__ uint32_t decode_private(
+    uint32_t tab_abs, uint32_t vals_abs, uint32_t ring_abs, uint32_t stage_abs, uint8_t* __restrict__ ring,
     const uint32_t* __restrict__ g_single, uint32_t dom_val, const uint32_t* __restrict__ words,
     uint32_t ext_words, uint32_t wbeg, uint32_t wend, bool last_lane, uint32_t state, uint32_t my_count,
     uint32_t rows, uint32_t min_count, uint8_t* __restrict__ out_row0, size_t row_stride_bytes, uint32_t lane) {
-  using E = typename ElemT<ES>::type;
   constexpr uint32_t RB = 32u * ES;
   constexpr uint32_t RING = kRingBytes / RB;        // rows in the ring
   constexpr uint32_t FL = RING / 4;                 // rows written out at a time
   constexpr uint32_t MASK = kRingBytes - 1u;
   static_assert(RING - FL >= kPair + FL, "a lane must be able to run ahead of the write-out");
-  uint8_t* ring = sm + ring_off;
-  const uint32_t lane_off = ring_off + lane * ES;
+  const uint32_t ring_lane_abs = ring_abs + lane * ES;
 
   // bit window: w0/w1 hold the 64 bits being read, w2 is one word ahead.  A staged lane may
-  // look up to word_limit + 4 words into its buffer, which holds ext_words + kStagePad / 4.
+  // look up to word_limit + kPairsPerCall + 3 words into its buffer, which holds ext_words + kStagePad / 4.
   const uint32_t word_limit = STAGED ? ext_words + 4u : ext_words;
   auto load_word = [&](uint32_t i) -> uint32_t {
-    if (STAGED) return *reinterpret_cast<const uint32_t*>(sm + stage_off + i * 4u);
+    if (STAGED) return lds_u32(stage_abs + i * 4u);
     return i < word_limit ? __ldg(words + i) : 0u;
   };
   uint32_t idx = wbeg;
@@ -320,22 +399,24 @@ __device__ __forceinline__ uint32_t decode_private(
     }
   };
 
-  uint32_t st4 = state * 4u;                        // byte offset of the state's table entry
+  uint32_t st = tab_abs + state * 4u;               // shared address of the state's table entry
   uint32_t tb = 0;                                  // RB * (next row this lane decodes)
   // one pre-walked look-up: emits run + 1 symbols, takes its bits from the low end of x
   auto step = [&](uint32_t x) -> uint32_t {
-    const uint32_t e = *reinterpret_cast<const uint32_t*>(sm + tab_off + st4);
+    const uint32_t e = lds_u32(st);
     const uint32_t nb = e >> 28;
-    st4 = (e & 0xFFFFu) + ((x & ((1u << nb) - 1u)) << 2);
-    const uint32_t val = *reinterpret_cast<const uint32_t*>(sm + vals_off + ((e >> 14) & 0x3FCu));
+    st = tab_abs + (e & 0xFFFFu) + ((x & ((1u << nb) - 1u)) << 2);
+    const uint32_t val = lds_u32(vals_abs | ((e >> 14) & 0x3FCu));
     tb += ((e >> 24) & 15u) * RB;
-    *reinterpret_cast<E*>(sm + ((tb & MASK) | lane_off)) = static_cast<E>(val);
+    sts_elem<ES>((tb & MASK) | ring_lane_abs, val);
     tb += RB;
     return nb;
   };
-  auto refill = [&]() {
+  auto refill_checked = [&]() {
     if (bitpos >= 32u) {
-      w0 = w1; w1 = w2; w2 = load_word(idx); ++idx;
+      w0 = w1; w1 = w2;
+      w2 = (!STAGED || idx < word_limit) ? load_word(idx) : 0u;
+      ++idx;
       bitpos -= 32u;
     }
   };
@@ -346,17 +427,23 @@ __device__ __forceinline__ uint32_t decode_private(
   uint32_t base = 0;                                // first row not yet written out
   for (;;) {
     const uint32_t lim = min(lim2, (base + RING - kPair) * RB);
+    if (STAGED) {
+      uint32_t sp = stage_abs + idx * 4u;
+      pair_steps<ES>(st, tb, bitpos, w0, w1, w2, sp, lim, tab_abs, vals_abs, ring_lane_abs);
+      idx = (sp - stage_abs) >> 2;
+      if (idx > word_limit) { overran = true; idx = word_limit; }
+    } else {
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      if (tb < lim) {
-        const uint32_t x = __funnelshift_r(w0, w1, bitpos);
-        const uint32_t nb1 = step(x);
-        const uint32_t nb2 = step(x >> nb1);
-        bitpos += nb1 + nb2;
-        refill();
+      for (int u = 0; u < 2; ++u) {
+        if (tb < lim) {
+          const uint32_t x = __funnelshift_r(w0, w1, bitpos);
+          const uint32_t nb1 = step(x);
+          const uint32_t nb2 = step(x >> nb1);
+          bitpos += nb1 + nb2;
+          refill_checked();
+        }
       }
     }
-    if (STAGED && idx > word_limit) { overran = true; idx = word_limit; }
     const uint32_t tmin = __reduce_min_sync(kFull, tb) / RB;
     while (tmin >= base + FL) {                     // the slowest lane has left these rows
       __syncwarp();
@@ -372,31 +459,20 @@ __device__ __forceinline__ uint32_t decode_private(
   // then single pre-walked look-ups while at least 16 symbols are owed to the lane ...
   while (tb < lim1) {
     bitpos += step(__funnelshift_r(w0, w1, bitpos));
-    if (bitpos >= 32u) {
-      w0 = w1; w1 = w2;
-      w2 = (!STAGED || idx < word_limit) ? load_word(idx) : 0u;
-      ++idx;
-      bitpos -= 32u;
-    }
+    refill_checked();
   }
   // ... and the last (up to 15) symbols one per look-up through the plain table
   uint32_t t = tb / RB;
-  state = st4 >> 2;
+  state = (st - tab_abs) >> 2;
   while (t < my_count) {
     const uint32_t e = __ldg(g_single + state);
-    const uint32_t val = *reinterpret_cast<const uint32_t*>(sm + vals_off + entry_sym(e) * 4u);
-    *reinterpret_cast<E*>(sm + (((t * RB) & MASK) | lane_off)) = static_cast<E>(val);
+    sts_elem<ES>(((t * RB) & MASK) | ring_lane_abs, lds_u32(vals_abs + entry_sym(e) * 4u));
     t += 1;
     const uint32_t nb = entry_nb(e);
     const uint32_t x = __funnelshift_r(w0, w1, bitpos);
     state = entry_newx(e) + (x & ((1u << nb) - 1u));
     bitpos += nb;
-    if (bitpos >= 32u) {
-      w0 = w1; w1 = w2;
-      w2 = (!STAGED || idx < word_limit) ? load_word(idx) : 0u;
-      ++idx;
-      bitpos -= 32u;
-    }
+    refill_checked();
   }
   __syncwarp();
   {
@@ -417,19 +493,26 @@ __device__ __forceinline__ uint32_t decode_private(
   return bad;
 }
 
-// dynamic shared memory: [rings: NW * kRingBytes][table][vals 256][mbarriers NW][stages NW * stage_bytes]
+// dynamic shared memory, by absolute shared address: [pad to 8 KB][rings: NW * kRingBytes][table]
+// [pad to 1 KB][vals 256 words][mbarriers NW][stages NW * stage_bytes]
+constexpr uint32_t kPrivPadBytes = kRingBytes + 1024u;   // what the two alignments can cost
+
 __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const LaunchArgs args) {
   extern __shared__ __align__(16) uint8_t sm[];
   const uint32_t NW = blockDim.x >> 5;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-  const uint32_t tab_off = NW * kRingBytes;
-  const uint32_t vals_off = tab_off + args.table_words * 4u;
-  const uint32_t bars_off = vals_off + 1024u;
-  const uint32_t ring_off = warp * kRingBytes;
-  const uint32_t stage_off = bars_off + NW * 8u + warp * args.stage_bytes;
-  uint32_t* tab = reinterpret_cast<uint32_t*>(sm + tab_off);
-  uint32_t* vals = reinterpret_cast<uint32_t*>(sm + vals_off);
-  const uint32_t bar = smem_u32(sm + bars_off + warp * 8u);
+  const uint32_t sm_abs = smem_u32(sm);
+  const uint32_t rings_abs = (sm_abs + kRingBytes - 1u) & ~(kRingBytes - 1u);
+  const uint32_t tab_abs = rings_abs + NW * kRingBytes;
+  const uint32_t vals_abs = (tab_abs + args.table_words * 4u + 1023u) & ~1023u;
+  const uint32_t bars_abs = vals_abs + 1024u;
+  const uint32_t ring_abs = rings_abs + warp * kRingBytes;
+  const uint32_t stage_abs = bars_abs + NW * 8u + warp * args.stage_bytes;
+  uint32_t* tab = reinterpret_cast<uint32_t*>(sm + (tab_abs - sm_abs));
+  uint32_t* vals = reinterpret_cast<uint32_t*>(sm + (vals_abs - sm_abs));
+  uint8_t* ring = sm + (ring_abs - sm_abs);
+  uint8_t* stage = sm + (stage_abs - sm_abs);
+  const uint32_t bar = bars_abs + warp * 8u;
   __shared__ uint32_t s_dom;
   uint32_t parity = 0;
 
@@ -495,9 +578,9 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
           asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
           asm volatile(
               "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-              :: "r"(smem_u32(sm + stage_off)), "l"(g_bytes), "r"(bytes), "r"(bar) : "memory");
+              :: "r"(stage_abs), "l"(g_bytes), "r"(bytes), "r"(bar) : "memory");
         }
-        if (lane < kStagePad / 4u) reinterpret_cast<uint32_t*>(sm + stage_off + it.extent)[lane] = 0u;
+        if (lane < kStagePad / 4u) reinterpret_cast<uint32_t*>(stage + it.extent)[lane] = 0u;
       }
 
       const uint32_t meta = __ldg(static_cast<const uint32_t*>(L.d_lane_meta) + it.sub * 32 + lane);
@@ -522,7 +605,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
         __syncwarp();
       }
 #define ANSB_PRIV(ES_, ST_)                                                                              \
-  wbad |= decode_private<ES_, ST_>(sm, tab_off, vals_off, ring_off, stage_off, g_single, dom, words,     \
+  wbad |= decode_private<ES_, ST_>(tab_abs, vals_abs, ring_abs, stage_abs, ring, g_single, dom, words,  \
                                    ext_words, wbeg, wend, lane == 31, state, my_count, rows, min_count, \
                                    out_row0, rsb, lane)
       if (staged) {
@@ -590,7 +673,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
     // global memory instead), within what the CTA may hold
     size_t want = (stream_total / sub_total) * 5 / 4 + kStagePad + 64;
     want = (want + 127) & ~size_t(127);
-    const size_t table_part = smem + 16 * 8;
+    const size_t table_part = smem + 16 * 8 + kPrivPadBytes;
     warps = big ? 16 : 4;
     while (warps > 4 && table_part + size_t(warps) * (kRingBytes + want) + 1024 > size_t(smem_max)) warps -= 4;
     const size_t fixed = table_part + size_t(warps) * kRingBytes;
@@ -598,7 +681,8 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
     size_t stage = (want < room ? want : room) & ~size_t(15);
     if (stage < 256) stage = 0;
     a.stage_bytes = static_cast<uint32_t>(stage);
-    smem = size_t(warps) * kRingBytes + (size_t(a.table_words) + 256) * 4 + size_t(warps) * 8 + size_t(warps) * stage;
+    smem = kPrivPadBytes + size_t(warps) * kRingBytes + (size_t(a.table_words) + 256) * 4 + size_t(warps) * 8 +
+           size_t(warps) * stage;
   }
   ANSB_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   ANSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, warps * 32, smem));
