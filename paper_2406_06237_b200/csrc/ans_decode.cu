@@ -221,10 +221,14 @@ constexpr uint32_t kStagePad = 80;             // readable bytes after the stage
 constexpr uint32_t kWaitSpins = 1u << 22;
 constexpr uint32_t kPair = 2 * (kMaxRun + 1);  // symbols two look-ups can emit
 
-// shared-memory form of a pre-walked entry: newX*4 [15:0] | sym [23:16] | run [27:24] | nb [31:28]
+// shared-memory form of a pre-walked entry:
+//   nb [3:0] (bit 4 stays 0) | symbols emitted = run + 1 [9:5] | sym [17:10] | newX [31:18]
+// One extra entry after the table (index 2^R, possible while R <= 13) emits nothing, reads
+// nothing and leads to itself: a lane that must wait is parked on it.
 __device__ __forceinline__ uint32_t to_smem_entry(uint32_t g) {
-  return (entry_newx(g) << 2) | (entry_sym(g) << 16) | (entry_run(g) << 24) | (entry_nb(g) << 28);
+  return entry_nb(g) | ((entry_run(g) + 1u) << 5) | (entry_sym(g) << 10) | (entry_newx(g) << 18);
 }
+constexpr int kMaxParkLog = 13;
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
@@ -274,67 +278,69 @@ __device__ __forceinline__ void sts_elem(uint32_t a, uint32_t v) {
   if (ES == 4) asm volatile("st.shared.u32 [%0], %1;" :: "r"(a), "r"(v) : "memory");
 }
 
-// The hot loop, for a staged sub-stream: kPairsPerCall times, every lane with tb < lim makes two
-// pre-walked look-ups that share one 32-bit extract of its bit window and one refill check.
-// Written as one PTX block so that the loop-carried values stay in registers across iterations.
-//   st  : shared address of the state's table entry      tb : RB * (next row of the lane)
-//   w0,w1,w2 : bit window and the word after it           sp : shared address of the next word
-// Entry: newX*4 [15:0] | sym [23:16] | run [27:24] | nb [31:28].  vals_abs is 1 KB aligned and
-// ring_lane_abs has its low 13 bits (but for lane * ES) clear, so OR forms both addresses.
+// The hot loop, for a staged sub-stream: kPairsPerCall times, every lane makes two pre-walked
+// look-ups that share one 32-bit extract of its bit window and one refill check.  A lane whose
+// next row is at or beyond its limit does the same work on the parking entry, which changes
+// nothing, so the loop has no divergent branch.  Written as one PTX block so that the
+// loop-carried values stay in registers across iterations.
+//   st  : shared address of the state's table entry   tbm : RB * (last row the lane wrote), signed
+//   w0,w1,w2 : bit window and the word after it        sp : shared address of the next word
+// vals_abs is 1 KB aligned and ring_lane_abs has its low 13 bits (but for lane * ES) clear, so OR
+// forms both addresses.
 constexpr int kPairsPerCall = 8;
 
 #define ANSB_STEP(NB_, STOP_)                                     \
-  "ld.shared.u32 e, [%0];\n\t"                                    \
-  "shr.u32 " NB_ ", e, 28;\n\t"                                   \
-  "bmsk.clamp.b32 m, 0, " NB_ ";\n\t"                             \
-  "and.b32 v, x, m;\n\t"                                          \
-  "and.b32 nx, e, 0xFFFF;\n\t"                                    \
-  "add.u32 nx, nx, %8;\n\t"                                       \
-  "mad.lo.u32 %0, v, 4, nx;\n\t"                                  \
-  "shr.u32 sy, e, 14;\n\t"                                        \
+  "ld.shared.u32 e, [stx];\n\t"                                   \
+  "shf.l.wrap.b32 m, 0, -1, e;\n\t"                               \
+  "shr.u32 nx, e, 18;\n\t"                                        \
+  "lop3.b32 t, nx, x, m, 0xF4;\n\t"                               \
+  "mad.lo.u32 stx, t, 4, %8;\n\t"                                 \
+  "shr.u32 sy, e, 8;\n\t"                                         \
   "lop3.b32 sy, sy, 0x3FC, %9, 0xEA;\n\t"                         \
   "ld.shared.u32 val, [sy];\n\t"                                  \
-  "bfe.u32 r, e, 24, 4;\n\t"                                      \
+  "bfe.u32 r, e, 5, 5;\n\t"                                       \
   "mad.lo.u32 %1, r, %11, %1;\n\t"                                \
+  "and.b32 " NB_ ", e, 15;\n\t"                                   \
   "lop3.b32 a, %1, %12, %10, 0xEA;\n\t"                           \
-  STOP_ " [a], val;\n\t"                                          \
-  "add.u32 %1, %1, %11;\n\t"
+  "@p " STOP_ " [a], val;\n\t"
 
 template <int ES>
-__device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tb, uint32_t& bitpos, uint32_t& w0,
-                                           uint32_t& w1, uint32_t& w2, uint32_t& sp, uint32_t lim,
-                                           uint32_t tab_abs, uint32_t vals_abs, uint32_t ring_lane_abs) {
+__device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t& bitpos, uint32_t& w0,
+                                           uint32_t& w1, uint32_t& w2, uint32_t& sp, int32_t limm,
+                                           uint32_t tab_abs, uint32_t vals_abs, uint32_t ring_lane_abs,
+                                           uint32_t park_abs) {
   constexpr uint32_t RB = 32u * ES;
   constexpr uint32_t MASK = kRingBytes - 1u;
 #define ANSB_PAIRS(STOP_)                                                                  \
   asm volatile(                                                                            \
       "{\n\t"                                                                              \
       ".reg .pred p, q;\n\t"                                                               \
-      ".reg .u32 x, e, n1, n2, m, v, nx, sy, val, r, a, cnt;\n\t"                         \
+      ".reg .u32 x, e, n1, n2, m, t, nx, sy, val, r, a, cnt, stx;\n\t"                    \
       "mov.u32 cnt, %13;\n"                                                                \
       "ANSB_LOOP:\n\t"                                                                     \
-      "setp.lt.u32 p, %1, %7;\n\t"                                                         \
-      "@!p bra ANSB_SKIP;\n\t"                                                             \
+      "setp.lt.s32 p, %1, %7;\n\t"                                                         \
+      "selp.b32 stx, %0, %14, p;\n\t"                                                      \
       "shf.r.wrap.b32 x, %3, %4, %2;\n\t"                                                  \
       ANSB_STEP("n1", STOP_)                                                               \
       "shr.u32 x, x, n1;\n\t"                                                              \
       ANSB_STEP("n2", STOP_)                                                               \
       "add.u32 %2, %2, n1;\n\t"                                                            \
       "add.u32 %2, %2, n2;\n\t"                                                            \
+      "selp.b32 %0, stx, %0, p;\n\t"                                                       \
       "setp.ge.u32 q, %2, 32;\n\t"                                                         \
       "@q mov.u32 %3, %4;\n\t"                                                             \
       "@q mov.u32 %4, %5;\n\t"                                                             \
       "@q ld.shared.u32 %5, [%6];\n\t"                                                     \
-      "@q add.u32 %6, %6, 4;\n\t"                                                          \
-      "@q add.u32 %2, %2, -32;\n"                                                          \
-      "ANSB_SKIP:\n\t"                                                                     \
+      "shr.u32 t, %2, 5;\n\t"                                                              \
+      "mad.lo.u32 %6, t, 4, %6;\n\t"                                                       \
+      "and.b32 %2, %2, 31;\n\t"                                                            \
       "add.u32 cnt, cnt, -1;\n\t"                                                          \
-      "setp.ne.u32 p, cnt, 0;\n\t"                                                         \
-      "@p bra ANSB_LOOP;\n\t"                                                              \
+      "setp.ne.u32 q, cnt, 0;\n\t"                                                         \
+      "@q bra ANSB_LOOP;\n\t"                                                              \
       "}"                                                                                  \
-      : "+r"(st), "+r"(tb), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp)           \
-      : "r"(lim), "r"(tab_abs), "r"(vals_abs), "r"(ring_lane_abs), "n"(RB), "n"(MASK),     \
-        "n"(kPairsPerCall)                                                                 \
+      : "+r"(st), "+r"(tbm), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp)          \
+      : "r"(limm), "r"(tab_abs), "r"(vals_abs), "r"(ring_lane_abs), "n"(RB), "n"(MASK),    \
+        "n"(kPairsPerCall), "r"(park_abs)                                                  \
       : "memory")
   if (ES == 1) ANSB_PAIRS("st.shared.u8");
   if (ES == 2) ANSB_PAIRS("st.shared.u16");
@@ -349,19 +355,20 @@ __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tb, uint32_t&
 // global memory, used when it was not staged.
 template <int ES, bool STAGED>
 __device__ __noinline__ uint32_t decode_private(
-    uint32_t tab_abs, uint32_t vals_abs, uint32_t ring_abs, uint32_t stage_abs, uint8_t* __restrict__ ring,
-    const uint32_t* __restrict__ g_single, uint32_t dom_val, const uint32_t* __restrict__ words,
-    uint32_t ext_words, uint32_t wbeg, uint32_t wend, bool last_lane, uint32_t state, uint32_t my_count,
-    uint32_t rows, uint32_t min_count, uint8_t* __restrict__ out_row0, size_t row_stride_bytes, uint32_t lane) {
-  constexpr uint32_t RB = 32u * ES;
+    uint32_t tab_abs, uint32_t vals_abs, uint32_t ring_abs, uint32_t stage_abs, uint32_t park_abs,
+    uint8_t* __restrict__ ring, const uint32_t* __restrict__ g_single, uint32_t dom_val,
+    const uint32_t* __restrict__ words, uint32_t ext_words, uint32_t wbeg, uint32_t wend, bool last_lane,
+    uint32_t state, uint32_t my_count, uint32_t rows, uint32_t min_count, uint8_t* __restrict__ out_row0,
+    size_t row_stride_bytes, uint32_t lane) {
+  constexpr int RB = 32 * ES;
   constexpr uint32_t RING = kRingBytes / RB;        // rows in the ring
   constexpr uint32_t FL = RING / 4;                 // rows written out at a time
   constexpr uint32_t MASK = kRingBytes - 1u;
   static_assert(RING - FL >= kPair + FL, "a lane must be able to run ahead of the write-out");
   const uint32_t ring_lane_abs = ring_abs + lane * ES;
 
-  // bit window: w0/w1 hold the 64 bits being read, w2 is one word ahead.  A staged lane may
-  // look up to word_limit + kPairsPerCall + 3 words into its buffer, which holds ext_words + kStagePad / 4.
+  // bit window: w0/w1 hold the 64 bits being read, w2 is one word ahead.  A staged lane may look
+  // up to word_limit + kPairsPerCall + 3 words into its buffer, which holds ext_words + kStagePad / 4.
   const uint32_t word_limit = STAGED ? ext_words + 4u : ext_words;
   auto load_word = [&](uint32_t i) -> uint32_t {
     if (STAGED) return lds_u32(stage_abs + i * 4u);
@@ -400,16 +407,15 @@ __device__ __noinline__ uint32_t decode_private(
   };
 
   uint32_t st = tab_abs + state * 4u;               // shared address of the state's table entry
-  uint32_t tb = 0;                                  // RB * (next row this lane decodes)
+  uint32_t tbm = static_cast<uint32_t>(-RB);        // RB * (last row this lane wrote): none yet
   // one pre-walked look-up: emits run + 1 symbols, takes its bits from the low end of x
   auto step = [&](uint32_t x) -> uint32_t {
     const uint32_t e = lds_u32(st);
-    const uint32_t nb = e >> 28;
-    st = tab_abs + (e & 0xFFFFu) + ((x & ((1u << nb) - 1u)) << 2);
-    const uint32_t val = lds_u32(vals_abs | ((e >> 14) & 0x3FCu));
-    tb += ((e >> 24) & 15u) * RB;
-    sts_elem<ES>((tb & MASK) | ring_lane_abs, val);
-    tb += RB;
+    const uint32_t nb = e & 15u;
+    st = tab_abs + (((e >> 18) | (x & ((1u << nb) - 1u))) << 2);
+    const uint32_t val = lds_u32(vals_abs | ((e >> 8) & 0x3FCu));
+    tbm += ((e >> 5) & 31u) * RB;
+    sts_elem<ES>((tbm & MASK) | ring_lane_abs, val);
     return nb;
   };
   auto refill_checked = [&]() {
@@ -420,22 +426,24 @@ __device__ __noinline__ uint32_t decode_private(
       bitpos -= 32u;
     }
   };
+  auto next_row = [&]() -> int32_t { return (static_cast<int32_t>(tbm) + RB) / RB; };
 
-  // main part: two look-ups share one 32-bit extract (2 * 14 bits at most) and one refill check
-  const uint32_t lim2 = (my_count > kPair - 1 ? my_count - (kPair - 1) : 0u) * RB;
-  const uint32_t lim1 = (my_count > kMaxRun ? my_count - kMaxRun : 0u) * RB;
+  // main part: two look-ups share one 32-bit extract (2 * 14 bits at most) and one refill check;
+  // it stops kPair - 1 symbols short of the lane's end, so a pair can never emit too many
+  const int32_t lim2 = static_cast<int32_t>(my_count > kPair - 1 ? my_count - (kPair - 1) : 0u);
+  const int32_t lim1 = static_cast<int32_t>(my_count > kMaxRun ? my_count - kMaxRun : 0u);
   uint32_t base = 0;                                // first row not yet written out
   for (;;) {
-    const uint32_t lim = min(lim2, (base + RING - kPair) * RB);
-    if (STAGED) {
+    const int32_t lim = min(lim2, static_cast<int32_t>(base + RING - kPair));   // rows
+    if (STAGED && park_abs != 0u) {
       uint32_t sp = stage_abs + idx * 4u;
-      pair_steps<ES>(st, tb, bitpos, w0, w1, w2, sp, lim, tab_abs, vals_abs, ring_lane_abs);
+      pair_steps<ES>(st, tbm, bitpos, w0, w1, w2, sp, (lim - 1) * RB, tab_abs, vals_abs, ring_lane_abs, park_abs);
       idx = (sp - stage_abs) >> 2;
       if (idx > word_limit) { overran = true; idx = word_limit; }
     } else {
 #pragma unroll
       for (int u = 0; u < 2; ++u) {
-        if (tb < lim) {
+        if (next_row() < lim) {
           const uint32_t x = __funnelshift_r(w0, w1, bitpos);
           const uint32_t nb1 = step(x);
           const uint32_t nb2 = step(x >> nb1);
@@ -444,7 +452,7 @@ __device__ __noinline__ uint32_t decode_private(
         }
       }
     }
-    const uint32_t tmin = __reduce_min_sync(kFull, tb) / RB;
+    const uint32_t tmin = static_cast<uint32_t>(__reduce_min_sync(kFull, next_row()));
     while (tmin >= base + FL) {                     // the slowest lane has left these rows
       __syncwarp();
       write_out(base, FL, 0u);
@@ -454,15 +462,15 @@ __device__ __noinline__ uint32_t decode_private(
       base += FL;
       __syncwarp();
     }
-    if (__all_sync(kFull, tb >= lim2)) break;
+    if (__all_sync(kFull, next_row() >= lim2)) break;
   }
   // then single pre-walked look-ups while at least 16 symbols are owed to the lane ...
-  while (tb < lim1) {
+  while (next_row() < lim1) {
     bitpos += step(__funnelshift_r(w0, w1, bitpos));
     refill_checked();
   }
   // ... and the last (up to 15) symbols one per look-up through the plain table
-  uint32_t t = tb / RB;
+  uint32_t t = static_cast<uint32_t>(next_row());
   state = (st - tab_abs) >> 2;
   while (t < my_count) {
     const uint32_t e = __ldg(g_single + state);
@@ -545,7 +553,9 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
     for (uint32_t i = threadIdx.x; i < 256u; i += blockDim.x)
       vals[i] = dequant_bits(static_cast<int>(i), L.zero_point, L.scale, dtype);
     if (threadIdx.x == 0) {
-      s_dom = hdr->dominant;
+      const uint32_t d = hdr->dominant;
+      s_dom = d < 256u ? d : 0u;                          // the ring's fill symbol
+      if (R <= kMaxParkLog) tab[1u << R] = (s_dom << 10) | ((1u << R) << 18);   // parking entry
       if (hdr->magic != kTableMagic || hdr->table_log != uint32_t(R) || hdr->alphabet > (1u << L.bitwidth))
         bad |= ANS_STATUS_BAD_SYMBOL;
     }
@@ -555,7 +565,8 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
     const uint64_t n_sub = uint64_t(L.lanes / 32u) * ((L.n_symbols + L.chunk_symbols - 1) / L.chunk_symbols);
     const size_t es = dtype == ANS_U8 ? 1 : dtype == ANS_F32 ? 4 : 2;
     uint8_t* out_base = args.d_symbols_override ? args.d_symbols_override : static_cast<uint8_t*>(L.d_out);
-    const uint32_t dom = s_dom < 256u ? vals[s_dom] : 0u;
+    const uint32_t dom = vals[s_dom];
+    const uint32_t park_abs = R <= kMaxParkLog ? tab_abs + (4u << R) : 0u;
     for (uint64_t gbase = cursor; gbase < stop && !gave_up; gbase += NW / kGranule) {
       const uint64_t granule = gbase + warp / kGranule;
       const uint64_t sub = (granule - lbeg) * kGranule + warp % kGranule;
@@ -605,7 +616,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
         __syncwarp();
       }
 #define ANSB_PRIV(ES_, ST_)                                                                              \
-  wbad |= decode_private<ES_, ST_>(tab_abs, vals_abs, ring_abs, stage_abs, ring, g_single, dom, words,  \
+  wbad |= decode_private<ES_, ST_>(tab_abs, vals_abs, ring_abs, stage_abs, park_abs, ring, g_single, dom, words, \
                                    ext_words, wbeg, wend, lane == 31, state, my_count, rows, min_count, \
                                    out_row0, rsb, lane)
       if (staged) {
@@ -652,7 +663,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   a.total_work = static_cast<uint32_t>(total);
   a.d_status = d_status;
   a.d_symbols_override = d_symbols_override;
-  a.table_words = max_log < 2 ? 4u : (1u << max_log);
+  a.table_words = (max_log < 2 ? 4u : (1u << max_log)) + 4u;   // + room for the parking entry
 
   int dev = 0, sms = 0, per_sm = 0, smem_max = 0;
   ANSB_CUDA(cudaGetDevice(&dev));
