@@ -217,16 +217,22 @@ __global__ void __launch_bounds__(kIWarps * 32) ans_decode_interleaved_kernel(co
 // one bulk asynchronous copy per warp, so a lane's refill is a shared-memory load.
 // =============================================================================================
 constexpr uint32_t kRingBytes = 8192;          // per warp; rows = kRingBytes / (32 * ES)
-constexpr uint32_t kStagePad = 80;             // readable bytes after the staged sub-stream
+constexpr uint32_t kStagePad = 112;            // readable bytes after the staged sub-stream
 constexpr uint32_t kWaitSpins = 1u << 22;
 constexpr uint32_t kPair = 2 * (kMaxRun + 1);  // symbols two look-ups can emit
 
-// shared-memory form of a pre-walked entry:
-//   nb [3:0] (bit 4 stays 0) | symbols emitted = run + 1 [9:5] | sym [17:10] | newX [31:18]
+// shared-memory form of a pre-walked entry, two words:
+//   a: nb [3:0] (bits 4-5 stay 0) | symbols emitted = run + 1 [10:6] | newX [31:18]
+//   b: 1- and 2-byte outputs: dequantised value [15:0] | row bytes * (run + 1) [31:16]
+//      4-byte outputs:        dequantised value
 // One extra entry after the table (index 2^R, possible while R <= 13) emits nothing, reads
 // nothing and leads to itself: a lane that must wait is parked on it.
-__device__ __forceinline__ uint32_t to_smem_entry(uint32_t g) {
-  return entry_nb(g) | ((entry_run(g) + 1u) << 5) | (entry_sym(g) << 10) | (entry_newx(g) << 18);
+__device__ __forceinline__ uint2 to_smem_entry(uint32_t g, uint32_t val, uint32_t row_bytes) {
+  const uint32_t adv = entry_run(g) + 1u;
+  uint2 e;
+  e.x = entry_nb(g) | (adv << 6) | (entry_newx(g) << 18);
+  e.y = row_bytes == 128u ? val : ((val & 0xFFFFu) | ((adv * row_bytes) << 16));
+  return e;
 }
 constexpr int kMaxParkLog = 13;
 
@@ -284,67 +290,64 @@ __device__ __forceinline__ void sts_elem(uint32_t a, uint32_t v) {
 // nothing, so the loop has no divergent branch.  Written as one PTX block so that the
 // loop-carried values stay in registers across iterations.
 //   st  : shared address of the state's table entry   tbm : RB * (last row the lane wrote), signed
+//   bitpos : bits of w0 already used; only its low 5 bits are kept clean
 //   w0,w1,w2 : bit window and the word after it        sp : shared address of the next word
-// vals_abs is 1 KB aligned and ring_lane_abs has its low 13 bits (but for lane * ES) clear, so OR
-// forms both addresses.
-constexpr int kPairsPerCall = 8;
+// ring_lane_abs has its low 13 bits (but for lane * ES) clear, so OR forms the row address.
+constexpr int kPairsPerCall = 16;
 
-#define ANSB_STEP(NB_, STOP_)                                     \
-  "ld.shared.u32 e, [stx];\n\t"                                   \
-  "shf.l.wrap.b32 m, 0, -1, e;\n\t"                               \
-  "shr.u32 nx, e, 18;\n\t"                                        \
+// ADV_: how tbm advances (from word b for narrow outputs, from word a's field for 4-byte ones)
+#define ANSB_STEP(ADV_, STOP_)                                    \
+  "ld.shared.v2.u32 {ea, eb}, [stx];\n\t"                         \
+  "shf.l.wrap.b32 m, 0, -1, ea;\n\t"                              \
+  "shr.u32 nx, ea, 18;\n\t"                                       \
   "lop3.b32 t, nx, x, m, 0xF4;\n\t"                               \
-  "mad.lo.u32 stx, t, 4, %8;\n\t"                                 \
-  "shr.u32 sy, e, 8;\n\t"                                         \
-  "lop3.b32 sy, sy, 0x3FC, %9, 0xEA;\n\t"                         \
-  "ld.shared.u32 val, [sy];\n\t"                                  \
-  "bfe.u32 r, e, 5, 5;\n\t"                                       \
-  "mad.lo.u32 %1, r, %11, %1;\n\t"                                \
-  "and.b32 " NB_ ", e, 15;\n\t"                                   \
-  "lop3.b32 a, %1, %12, %10, 0xEA;\n\t"                           \
-  "@p " STOP_ " [a], val;\n\t"
+  "mad.lo.u32 stx, t, 8, %8;\n\t"                                 \
+  ADV_                                                            \
+  "lop3.b32 a, %1, %11, %9, 0xEA;\n\t"                            \
+  "@p " STOP_ " [a], eb;\n\t"                                     \
+  "add.u32 %2, %2, ea;\n\t"
+
+#define ANSB_ADV_NARROW "mad.hi.u32 %1, eb, 65536, %1;\n\t"
+#define ANSB_ADV_WIDE "bfe.u32 r, ea, 6, 5;\n\tmad.lo.u32 %1, r, 128, %1;\n\t"
 
 template <int ES>
 __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t& bitpos, uint32_t& w0,
                                            uint32_t& w1, uint32_t& w2, uint32_t& sp, int32_t limm,
-                                           uint32_t tab_abs, uint32_t vals_abs, uint32_t ring_lane_abs,
-                                           uint32_t park_abs) {
-  constexpr uint32_t RB = 32u * ES;
+                                           uint32_t tab_abs, uint32_t ring_lane_abs, uint32_t park_abs) {
   constexpr uint32_t MASK = kRingBytes - 1u;
-#define ANSB_PAIRS(STOP_)                                                                  \
+#define ANSB_PAIRS(ADV_, STOP_)                                                            \
   asm volatile(                                                                            \
       "{\n\t"                                                                              \
       ".reg .pred p, q;\n\t"                                                               \
-      ".reg .u32 x, e, n1, n2, m, t, nx, sy, val, r, a, cnt, stx;\n\t"                    \
-      "mov.u32 cnt, %13;\n"                                                                \
+      ".reg .u32 x, ea, eb, m, t, nx, r, a, cnt, stx;\n\t"                                 \
+      "mov.u32 cnt, %12;\n"                                                                \
       "ANSB_LOOP:\n\t"                                                                     \
       "setp.lt.s32 p, %1, %7;\n\t"                                                         \
-      "selp.b32 stx, %0, %14, p;\n\t"                                                      \
+      "selp.b32 stx, %0, %10, p;\n\t"                                                      \
       "shf.r.wrap.b32 x, %3, %4, %2;\n\t"                                                  \
-      ANSB_STEP("n1", STOP_)                                                               \
-      "shr.u32 x, x, n1;\n\t"                                                              \
-      ANSB_STEP("n2", STOP_)                                                               \
-      "add.u32 %2, %2, n1;\n\t"                                                            \
-      "add.u32 %2, %2, n2;\n\t"                                                            \
+      "and.b32 %2, %2, 31;\n\t"                                                            \
+      ANSB_STEP(ADV_, STOP_)                                                               \
+      "shf.r.wrap.b32 x, x, 0, ea;\n\t"                                                    \
+      ANSB_STEP(ADV_, STOP_)                                                               \
       "selp.b32 %0, stx, %0, p;\n\t"                                                       \
-      "setp.ge.u32 q, %2, 32;\n\t"                                                         \
+      "and.b32 t, %2, 32;\n\t"                                                             \
+      "setp.ne.u32 q, t, 0;\n\t"                                                           \
       "@q mov.u32 %3, %4;\n\t"                                                             \
       "@q mov.u32 %4, %5;\n\t"                                                             \
       "@q ld.shared.u32 %5, [%6];\n\t"                                                     \
-      "shr.u32 t, %2, 5;\n\t"                                                              \
-      "mad.lo.u32 %6, t, 4, %6;\n\t"                                                       \
-      "and.b32 %2, %2, 31;\n\t"                                                            \
+      "mad.hi.u32 %6, t, 0x20000000, %6;\n\t"                                              \
       "add.u32 cnt, cnt, -1;\n\t"                                                          \
       "setp.ne.u32 q, cnt, 0;\n\t"                                                         \
       "@q bra ANSB_LOOP;\n\t"                                                              \
+      "and.b32 %2, %2, 31;\n\t"                                                            \
       "}"                                                                                  \
       : "+r"(st), "+r"(tbm), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp)          \
-      : "r"(limm), "r"(tab_abs), "r"(vals_abs), "r"(ring_lane_abs), "n"(RB), "n"(MASK),    \
-        "n"(kPairsPerCall), "r"(park_abs)                                                  \
+      : "r"(limm), "r"(tab_abs), "r"(ring_lane_abs), "r"(park_abs), "n"(MASK),             \
+        "n"(kPairsPerCall)                                                                 \
       : "memory")
-  if (ES == 1) ANSB_PAIRS("st.shared.u8");
-  if (ES == 2) ANSB_PAIRS("st.shared.u16");
-  if (ES == 4) ANSB_PAIRS("st.shared.u32");
+  if (ES == 1) ANSB_PAIRS(ANSB_ADV_NARROW, "st.shared.u8");
+  if (ES == 2) ANSB_PAIRS(ANSB_ADV_NARROW, "st.shared.u16");
+  if (ES == 4) ANSB_PAIRS(ANSB_ADV_WIDE, "st.shared.u32");
 #undef ANSB_PAIRS
 }
 
@@ -369,6 +372,7 @@ __device__ __noinline__ uint32_t decode_private(
 
   // bit window: w0/w1 hold the 64 bits being read, w2 is one word ahead.  A staged lane may look
   // up to word_limit + kPairsPerCall + 3 words into its buffer, which holds ext_words + kStagePad / 4.
+  static_assert(kStagePad / 4u >= 4u + kPairsPerCall + 4u, "staging pad too small for the look-ahead");
   const uint32_t word_limit = STAGED ? ext_words + 4u : ext_words;
   auto load_word = [&](uint32_t i) -> uint32_t {
     if (STAGED) return lds_u32(stage_abs + i * 4u);
@@ -406,16 +410,15 @@ __device__ __noinline__ uint32_t decode_private(
     }
   };
 
-  uint32_t st = tab_abs + state * 4u;               // shared address of the state's table entry
+  uint32_t st = tab_abs + state * 8u;               // shared address of the state's table entry
   uint32_t tbm = static_cast<uint32_t>(-RB);        // RB * (last row this lane wrote): none yet
   // one pre-walked look-up: emits run + 1 symbols, takes its bits from the low end of x
   auto step = [&](uint32_t x) -> uint32_t {
-    const uint32_t e = lds_u32(st);
-    const uint32_t nb = e & 15u;
-    st = tab_abs + (((e >> 18) | (x & ((1u << nb) - 1u))) << 2);
-    const uint32_t val = lds_u32(vals_abs | ((e >> 8) & 0x3FCu));
-    tbm += ((e >> 5) & 31u) * RB;
-    sts_elem<ES>((tbm & MASK) | ring_lane_abs, val);
+    const uint32_t ea = lds_u32(st), eb = lds_u32(st + 4u);
+    const uint32_t nb = ea & 15u;
+    st = tab_abs + (((ea >> 18) | (x & ((1u << nb) - 1u))) << 3);
+    tbm += ((ea >> 6) & 31u) * RB;
+    sts_elem<ES>((tbm & MASK) | ring_lane_abs, eb);
     return nb;
   };
   auto refill_checked = [&]() {
@@ -437,7 +440,7 @@ __device__ __noinline__ uint32_t decode_private(
     const int32_t lim = min(lim2, static_cast<int32_t>(base + RING - kPair));   // rows
     if (STAGED && park_abs != 0u) {
       uint32_t sp = stage_abs + idx * 4u;
-      pair_steps<ES>(st, tbm, bitpos, w0, w1, w2, sp, (lim - 1) * RB, tab_abs, vals_abs, ring_lane_abs, park_abs);
+      pair_steps<ES>(st, tbm, bitpos, w0, w1, w2, sp, (lim - 1) * RB, tab_abs, ring_lane_abs, park_abs);
       idx = (sp - stage_abs) >> 2;
       if (idx > word_limit) { overran = true; idx = word_limit; }
     } else {
@@ -471,7 +474,7 @@ __device__ __noinline__ uint32_t decode_private(
   }
   // ... and the last (up to 15) symbols one per look-up through the plain table
   uint32_t t = static_cast<uint32_t>(next_row());
-  state = (st - tab_abs) >> 2;
+  state = (st - tab_abs) >> 3;
   while (t < my_count) {
     const uint32_t e = __ldg(g_single + state);
     sts_elem<ES>(((t * RB) & MASK) | ring_lane_abs, lds_u32(vals_abs + entry_sym(e) * 4u));
@@ -516,7 +519,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
   const uint32_t bars_abs = vals_abs + 1024u;
   const uint32_t ring_abs = rings_abs + warp * kRingBytes;
   const uint32_t stage_abs = bars_abs + NW * 8u + warp * args.stage_bytes;
-  uint32_t* tab = reinterpret_cast<uint32_t*>(sm + (tab_abs - sm_abs));
+  uint2* tab = reinterpret_cast<uint2*>(sm + (tab_abs - sm_abs));
   uint32_t* vals = reinterpret_cast<uint32_t*>(sm + (vals_abs - sm_abs));
   uint8_t* ring = sm + (ring_abs - sm_abs);
   uint8_t* stage = sm + (stage_abs - sm_abs);
@@ -549,13 +552,18 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
     const int dtype = args.d_symbols_override ? ANS_U8 : L.out_dtype;
 
     __syncthreads();                                      // previous layer's readers are done
-    for (uint32_t i = threadIdx.x; i < (1u << R); i += blockDim.x) tab[i] = to_smem_entry(__ldg(g_multi + i));
+    const size_t es = dtype == ANS_U8 ? 1 : dtype == ANS_F32 ? 4 : 2;
     for (uint32_t i = threadIdx.x; i < 256u; i += blockDim.x)
       vals[i] = dequant_bits(static_cast<int>(i), L.zero_point, L.scale, dtype);
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < (1u << R); i += blockDim.x) {
+      const uint32_t g = __ldg(g_multi + i);
+      tab[i] = to_smem_entry(g, vals[entry_sym(g)], 32u * static_cast<uint32_t>(es));
+    }
     if (threadIdx.x == 0) {
       const uint32_t d = hdr->dominant;
       s_dom = d < 256u ? d : 0u;                          // the ring's fill symbol
-      if (R <= kMaxParkLog) tab[1u << R] = (s_dom << 10) | ((1u << R) << 18);   // parking entry
+      if (R <= kMaxParkLog) tab[1u << R] = make_uint2((1u << R) << 18, es == 4 ? vals[s_dom] : (vals[s_dom] & 0xFFFFu));
       if (hdr->magic != kTableMagic || hdr->table_log != uint32_t(R) || hdr->alphabet > (1u << L.bitwidth))
         bad |= ANS_STATUS_BAD_SYMBOL;
     }
@@ -563,10 +571,9 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
 
     const uint32_t W = L.lanes;
     const uint64_t n_sub = uint64_t(L.lanes / 32u) * ((L.n_symbols + L.chunk_symbols - 1) / L.chunk_symbols);
-    const size_t es = dtype == ANS_U8 ? 1 : dtype == ANS_F32 ? 4 : 2;
     uint8_t* out_base = args.d_symbols_override ? args.d_symbols_override : static_cast<uint8_t*>(L.d_out);
     const uint32_t dom = vals[s_dom];
-    const uint32_t park_abs = R <= kMaxParkLog ? tab_abs + (4u << R) : 0u;
+    const uint32_t park_abs = R <= kMaxParkLog ? tab_abs + (8u << R) : 0u;
     for (uint64_t gbase = cursor; gbase < stop && !gave_up; gbase += NW / kGranule) {
       const uint64_t granule = gbase + warp / kGranule;
       const uint64_t sub = (granule - lbeg) * kGranule + warp % kGranule;
@@ -663,7 +670,8 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   a.total_work = static_cast<uint32_t>(total);
   a.d_status = d_status;
   a.d_symbols_override = d_symbols_override;
-  a.table_words = (max_log < 2 ? 4u : (1u << max_log)) + 4u;   // + room for the parking entry
+  // interleaved: one word per state; private: two words per state and a parking entry
+  a.table_words = layout == ANS_LAYOUT_PRIVATE ? 2u * ((1u << max_log) + 2u) : (max_log < 2 ? 4u : (1u << max_log));
 
   int dev = 0, sms = 0, per_sm = 0, smem_max = 0;
   ANSB_CUDA(cudaGetDevice(&dev));
