@@ -28,6 +28,7 @@ struct LaunchArgs {
   uint8_t* d_symbols_override;     // ans_decode_layer: write symbols here instead of d_out
   uint32_t table_words;            // shared-memory words reserved for the table
   uint32_t stage_bytes;            // private layout: per-warp staging buffer for compressed bytes
+  uint32_t ring_bytes;             // private layout: per-warp output ring (kRingRows rows of the widest dtype)
 };
 
 __device__ __forceinline__ const ans_layer_desc& layer_at(const LaunchArgs& a, int l) {
@@ -216,7 +217,8 @@ __global__ void __launch_bounds__(kIWarps * 32) ans_decode_interleaved_kernel(co
 // slowest lane has left it.  The sub-stream's compressed bytes are brought into shared memory by
 // one bulk asynchronous copy per warp, so a lane's refill is a shared-memory load.
 // =============================================================================================
-constexpr uint32_t kRingBytes = 8192;          // per warp; rows = kRingBytes / (32 * ES)
+constexpr uint32_t kRingRows = 64;             // rows (of 32 symbols) in a warp's output ring
+constexpr uint32_t kFlushRows = 16;            // rows written out at a time
 constexpr uint32_t kStagePad = 112;            // readable bytes after the staged sub-stream
 constexpr uint32_t kWaitSpins = 1u << 22;
 constexpr uint32_t kPair = 2 * (kMaxRun + 1);  // symbols two look-ups can emit
@@ -285,14 +287,15 @@ __device__ __forceinline__ void sts_elem(uint32_t a, uint32_t v) {
 }
 
 // The hot loop, for a staged sub-stream: kPairsPerCall times, every lane makes two pre-walked
-// look-ups that share one 32-bit extract of its bit window and one refill check.  A lane whose
+// look-ups that share one 32-bit extract of its bit window and one refill check (the loop ends
+// early once no lane has work).  A lane whose
 // next row is at or beyond its limit does the same work on the parking entry, which changes
 // nothing, so the loop has no divergent branch.  Written as one PTX block so that the
 // loop-carried values stay in registers across iterations.
 //   st  : shared address of the state's table entry   tbm : RB * (last row the lane wrote), signed
 //   bitpos : bits of w0 already used; only its low 5 bits are kept clean
 //   w0,w1,w2 : bit window and the word after it        sp : shared address of the next word
-// ring_lane_abs has its low 13 bits (but for lane * ES) clear, so OR forms the row address.
+// ring_lane_abs is the ring's address (a multiple of its size) + lane * ES, so OR forms the row address.
 constexpr int kPairsPerCall = 16;
 
 // ADV_: how tbm advances (from word b for narrow outputs, from word a's field for 4-byte ones)
@@ -314,7 +317,7 @@ template <int ES>
 __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t& bitpos, uint32_t& w0,
                                            uint32_t& w1, uint32_t& w2, uint32_t& sp, int32_t limm,
                                            uint32_t tab_abs, uint32_t ring_lane_abs, uint32_t park_abs) {
-  constexpr uint32_t MASK = kRingBytes - 1u;
+  constexpr uint32_t MASK = kRingRows * 32u * ES - 1u;
 #define ANSB_PAIRS(ADV_, STOP_)                                                            \
   asm volatile(                                                                            \
       "{\n\t"                                                                              \
@@ -323,6 +326,8 @@ __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t
       "mov.u32 cnt, %12;\n"                                                                \
       "ANSB_LOOP:\n\t"                                                                     \
       "setp.lt.s32 p, %1, %7;\n\t"                                                         \
+      "vote.sync.any.pred q, p, 0xffffffff;\n\t"                                           \
+      "@!q bra ANSB_DONE;\n\t"                                                             \
       "selp.b32 stx, %0, %10, p;\n\t"                                                      \
       "shf.r.wrap.b32 x, %3, %4, %2;\n\t"                                                  \
       "and.b32 %2, %2, 31;\n\t"                                                            \
@@ -338,7 +343,8 @@ __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t
       "mad.hi.u32 %6, t, 0x20000000, %6;\n\t"                                              \
       "add.u32 cnt, cnt, -1;\n\t"                                                          \
       "setp.ne.u32 q, cnt, 0;\n\t"                                                         \
-      "@q bra ANSB_LOOP;\n\t"                                                              \
+      "@q bra ANSB_LOOP;\n"                                                                 \
+      "ANSB_DONE:\n\t"                                                                     \
       "and.b32 %2, %2, 31;\n\t"                                                            \
       "}"                                                                                  \
       : "+r"(st), "+r"(tbm), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp)          \
@@ -353,7 +359,7 @@ __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t
 
 // Decode one sub-stream.  Shared memory is addressed by absolute shared-window addresses:
 // tab_abs (table), vals_abs (dequantised values, 1 KB aligned), ring_abs (this warp's ring,
-// kRingBytes aligned), stage_abs (staged sub-stream when STAGED, with kStagePad readable bytes
+// aligned to its size), stage_abs (staged sub-stream when STAGED, with kStagePad readable bytes
 // after it).  `ring` is the generic pointer to the same ring; `words` the sub-stream in
 // global memory, used when it was not staged.
 template <int ES, bool STAGED>
@@ -364,8 +370,9 @@ __device__ __noinline__ uint32_t decode_private(
     uint32_t state, uint32_t my_count, uint32_t rows, uint32_t min_count, uint8_t* __restrict__ out_row0,
     size_t row_stride_bytes, uint32_t lane) {
   constexpr int RB = 32 * ES;
-  constexpr uint32_t RING = kRingBytes / RB;        // rows in the ring
-  constexpr uint32_t FL = RING / 4;                 // rows written out at a time
+  constexpr uint32_t RING = kRingRows;              // rows in the ring
+  constexpr uint32_t FL = kFlushRows;               // rows written out at a time
+  constexpr uint32_t kRingBytes = RING * RB;
   constexpr uint32_t MASK = kRingBytes - 1u;
   static_assert(RING - FL >= kPair + FL, "a lane must be able to run ahead of the write-out");
   const uint32_t ring_lane_abs = ring_abs + lane * ES;
@@ -408,6 +415,36 @@ __device__ __noinline__ uint32_t decode_private(
       flush_rows<ES>(ring + size_t(r % RING) * RB, out_row0 + size_t(r) * row_stride_bytes, row_stride_bytes,
                      0u, part_lanes, lane);
     }
+  };
+  // FL full rows starting at a multiple of FL, then fill them again.  When the output is 16-byte
+  // aligned the rows leave as bulk asynchronous stores straight from the ring: one copy for the
+  // whole block when the sub-stream's rows are contiguous (32 lanes per chunk), else one per row.
+  const bool bulk_ok = ((reinterpret_cast<uintptr_t>(out_row0) | row_stride_bytes) & 15u) == 0;
+  auto write_block = [&](uint32_t first_row) {
+    const uint32_t ring_row = first_row % RING;
+    if (bulk_ok) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ring writes -> visible to the copy engine
+      __syncwarp();
+      const bool contiguous = row_stride_bytes == RB;
+      if (contiguous ? lane == 0 : lane < FL) {
+        const uint32_t row = contiguous ? 0u : lane;
+        const uint32_t bytes = contiguous ? FL * RB : RB;
+        uint8_t* dst = out_row0 + size_t(first_row + row) * row_stride_bytes;
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                     :: "l"(dst), "r"(ring_abs + (ring_row + row) * RB), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the ring rows may be reused
+      }
+      __syncwarp();
+    } else {
+      __syncwarp();
+      flush_rows<ES>(ring + size_t(ring_row) * RB, out_row0 + size_t(first_row) * row_stride_bytes,
+                     row_stride_bytes, FL, 0u, lane);
+      __syncwarp();
+    }
+    uint8_t* part = ring + size_t(ring_row) * RB;
+    for (uint32_t i = lane; i < (FL * RB) / 16u; i += 32u) reinterpret_cast<uint4*>(part)[i] = fill4;
+    __syncwarp();
   };
 
   uint32_t st = tab_abs + state * 8u;               // shared address of the state's table entry
@@ -457,13 +494,8 @@ __device__ __noinline__ uint32_t decode_private(
     }
     const uint32_t tmin = static_cast<uint32_t>(__reduce_min_sync(kFull, next_row()));
     while (tmin >= base + FL) {                     // the slowest lane has left these rows
-      __syncwarp();
-      write_out(base, FL, 0u);
-      __syncwarp();
-      uint8_t* part = ring + size_t(base % RING) * RB;
-      for (uint32_t i = lane; i < (FL * RB) / 16u; i += 32u) reinterpret_cast<uint4*>(part)[i] = fill4;
+      write_block(base);
       base += FL;
-      __syncwarp();
     }
     if (__all_sync(kFull, next_row() >= lim2)) break;
   }
@@ -493,6 +525,7 @@ __device__ __noinline__ uint32_t decode_private(
     if (has_part) part_lanes = __popc(__ballot_sync(kFull, my_count == rows));
     write_out(base, full_rows, part_lanes);
   }
+  if (bulk_ok) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this lane's bulk stores have landed
   __syncwarp();
   uint32_t bad = 0;
   if (state != 0) bad |= ANS_STATUS_BAD_FINAL_STATE;
@@ -504,20 +537,19 @@ __device__ __noinline__ uint32_t decode_private(
   return bad;
 }
 
-// dynamic shared memory, by absolute shared address: [pad to 8 KB][rings: NW * kRingBytes][table]
-// [pad to 1 KB][vals 256 words][mbarriers NW][stages NW * stage_bytes]
-constexpr uint32_t kPrivPadBytes = kRingBytes + 1024u;   // what the two alignments can cost
+// dynamic shared memory, by absolute shared address: [pad to ring_bytes][rings: NW * ring_bytes]
+// [table][pad to 1 KB][vals 256 words][mbarriers NW][stages NW * stage_bytes]
 
 __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const LaunchArgs args) {
   extern __shared__ __align__(16) uint8_t sm[];
   const uint32_t NW = blockDim.x >> 5;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   const uint32_t sm_abs = smem_u32(sm);
-  const uint32_t rings_abs = (sm_abs + kRingBytes - 1u) & ~(kRingBytes - 1u);
-  const uint32_t tab_abs = rings_abs + NW * kRingBytes;
+  const uint32_t rings_abs = (sm_abs + args.ring_bytes - 1u) & ~(args.ring_bytes - 1u);
+  const uint32_t tab_abs = rings_abs + NW * args.ring_bytes;
   const uint32_t vals_abs = (tab_abs + args.table_words * 4u + 1023u) & ~1023u;
   const uint32_t bars_abs = vals_abs + 1024u;
-  const uint32_t ring_abs = rings_abs + warp * kRingBytes;
+  const uint32_t ring_abs = rings_abs + warp * args.ring_bytes;
   const uint32_t stage_abs = bars_abs + NW * 8u + warp * args.stage_bytes;
   uint2* tab = reinterpret_cast<uint2*>(sm + (tab_abs - sm_abs));
   uint32_t* vals = reinterpret_cast<uint32_t*>(sm + (vals_abs - sm_abs));
@@ -646,7 +678,8 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
 static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, int n_layers,
                   uint8_t* d_symbols_override, uint32_t* d_status, cudaStream_t st) {
   int max_log = 1, busy_layers = 0;
-  uint64_t total = 0, stream_total = 0, sub_total = 0;
+  uint64_t total = 0;
+  size_t max_avg_sub = 0, max_es = 1;
   const int layout = h_descs[0].layout;
   for (int l = 0; l < n_layers; ++l) {
     const int rc = validate_desc(h_descs[l], d_symbols_override == nullptr);
@@ -655,9 +688,13 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
     if (h_descs[l].work_begin != total || h_descs[l].work_count != granules_of(h_descs[l]))
       return ANS_ERR_INVALID_ARG;                         // ans_plan_batch was not run on this array
     total += h_descs[l].work_count;
-    sub_total += subs_of(h_descs[l]);
-    stream_total += h_descs[l].stream_bytes;
-    busy_layers += h_descs[l].work_count != 0;
+    if (h_descs[l].work_count != 0) {
+      ++busy_layers;
+      const size_t avg = h_descs[l].stream_bytes / subs_of(h_descs[l]);
+      if (avg > max_avg_sub) max_avg_sub = avg;
+      const size_t es = d_symbols_override ? 1 : elem_size(h_descs[l].out_dtype);
+      if (es > max_es) max_es = es;
+    }
     if (h_descs[l].table_log > max_log) max_log = h_descs[l].table_log;
   }
   if (total == 0) return ANS_OK;
@@ -684,24 +721,25 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   int warps = kIWarps;
   size_t smem = (size_t(a.table_words) + 256) * 4;
   if (priv) {
-    // Layers with many sub-streams share one table among 16 warps; a model of many small layers
-    // runs CTAs of one granule (4 warps) so that each CTA stays inside one layer and several
-    // CTAs, each with its own table, share an SM.
+    // Layers with many sub-streams share one table among up to 16 warps; a model of many small
+    // layers runs CTAs of one granule (4 warps) so that each CTA stays inside one layer and
+    // several CTAs, each with its own table, share an SM.
     const bool big = total / uint64_t(busy_layers) >= 64;
-    // staging buffer per warp: the average sub-stream plus a quarter (a larger one is read from
-    // global memory instead), within what the CTA may hold
-    size_t want = (stream_total / sub_total) * 5 / 4 + kStagePad + 64;
+    // per warp: an output ring of kRingRows rows of the widest dtype, and a staging buffer for
+    // the largest layer-average sub-stream plus a margin (a longer one is read from global memory)
+    const size_t ring = size_t(kRingRows) * 32 * max_es;
+    size_t want = max_avg_sub + max_avg_sub / 16 + 256 + kStagePad;
     want = (want + 127) & ~size_t(127);
-    const size_t table_part = smem + 16 * 8 + kPrivPadBytes;
+    const size_t fixed = ring + 1024 + smem + 16 * 8;     // alignment slack, table, vals, barriers
     warps = big ? 16 : 4;
-    while (warps > 4 && table_part + size_t(warps) * (kRingBytes + want) + 1024 > size_t(smem_max)) warps -= 4;
-    const size_t fixed = table_part + size_t(warps) * kRingBytes;
-    const size_t room = size_t(smem_max) > fixed + 1024 ? (size_t(smem_max) - fixed - 1024) / warps : 0;
+    while (warps > 4 && fixed + size_t(warps) * (ring + want) + 1024 > size_t(smem_max)) warps -= 4;
+    const size_t room = size_t(smem_max) > fixed + size_t(warps) * ring + 1024
+                            ? (size_t(smem_max) - fixed - size_t(warps) * ring - 1024) / warps : 0;
     size_t stage = (want < room ? want : room) & ~size_t(15);
     if (stage < 256) stage = 0;
     a.stage_bytes = static_cast<uint32_t>(stage);
-    smem = kPrivPadBytes + size_t(warps) * kRingBytes + (size_t(a.table_words) + 256) * 4 + size_t(warps) * 8 +
-           size_t(warps) * stage;
+    a.ring_bytes = static_cast<uint32_t>(ring);
+    smem = fixed + size_t(warps) * (ring + stage);
   }
   ANSB_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   ANSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, warps * 32, smem));
