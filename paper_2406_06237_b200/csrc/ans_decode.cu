@@ -318,16 +318,8 @@ __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t
                                            uint32_t& w1, uint32_t& w2, uint32_t& sp, int32_t limm,
                                            uint32_t tab_abs, uint32_t ring_lane_abs, uint32_t park_abs) {
   constexpr uint32_t MASK = kRingRows * 32u * ES - 1u;
-#define ANSB_PAIRS(ADV_, STOP_)                                                            \
-  asm volatile(                                                                            \
-      "{\n\t"                                                                              \
-      ".reg .pred p, q;\n\t"                                                               \
-      ".reg .u32 x, ea, eb, m, t, nx, r, a, cnt, stx;\n\t"                                 \
-      "mov.u32 cnt, %12;\n"                                                                \
-      "ANSB_LOOP:\n\t"                                                                     \
+#define ANSB_ONE_PAIR(ADV_, STOP_)                                                         \
       "setp.lt.s32 p, %1, %7;\n\t"                                                         \
-      "vote.sync.any.pred q, p, 0xffffffff;\n\t"                                           \
-      "@!q bra ANSB_DONE;\n\t"                                                             \
       "selp.b32 stx, %0, %10, p;\n\t"                                                      \
       "shf.r.wrap.b32 x, %3, %4, %2;\n\t"                                                  \
       "and.b32 %2, %2, 31;\n\t"                                                            \
@@ -339,22 +331,36 @@ __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t
       "setp.ne.u32 q, t, 0;\n\t"                                                           \
       "@q mov.u32 %3, %4;\n\t"                                                             \
       "@q mov.u32 %4, %5;\n\t"                                                             \
-      "@q ld.shared.u32 %5, [%6];\n\t"                                                     \
-      "mad.hi.u32 %6, t, 0x20000000, %6;\n\t"                                              \
+      "@q ld.shared.u32 nw, [%6];\n\t"                                                     \
+      "@q mov.u32 %5, nw;\n\t"                                                             \
+      "mad.hi.u32 %6, t, 0x20000000, %6;\n\t"
+#define ANSB_PAIRS(ADV_, STOP_)                                                            \
+  asm volatile(                                                                            \
+      "{\n\t"                                                                              \
+      ".reg .pred p, q;\n\t"                                                               \
+      ".reg .u32 x, ea, eb, m, t, nx, r, a, cnt, stx, nw;\n\t"                             \
+      "mov.u32 cnt, %12;\n"                                                                \
+      "ANSB_LOOP:\n\t"                                                                     \
+      "setp.lt.s32 p, %1, %7;\n\t"                                                         \
+      "vote.sync.any.pred q, p, 0xffffffff;\n\t"                                           \
+      "@!q bra ANSB_DONE;\n\t"                                                             \
+      ANSB_ONE_PAIR(ADV_, STOP_)                                                           \
+      ANSB_ONE_PAIR(ADV_, STOP_)                                                           \
       "add.u32 cnt, cnt, -1;\n\t"                                                          \
       "setp.ne.u32 q, cnt, 0;\n\t"                                                         \
-      "@q bra ANSB_LOOP;\n"                                                                 \
+      "@q bra ANSB_LOOP;\n"                                                                \
       "ANSB_DONE:\n\t"                                                                     \
       "and.b32 %2, %2, 31;\n\t"                                                            \
       "}"                                                                                  \
       : "+r"(st), "+r"(tbm), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp)          \
       : "r"(limm), "r"(tab_abs), "r"(ring_lane_abs), "r"(park_abs), "n"(MASK),             \
-        "n"(kPairsPerCall)                                                                 \
+        "n"(kPairsPerCall / 2)                                                             \
       : "memory")
   if (ES == 1) ANSB_PAIRS(ANSB_ADV_NARROW, "st.shared.u8");
   if (ES == 2) ANSB_PAIRS(ANSB_ADV_NARROW, "st.shared.u16");
   if (ES == 4) ANSB_PAIRS(ANSB_ADV_WIDE, "st.shared.u32");
 #undef ANSB_PAIRS
+#undef ANSB_ONE_PAIR
 }
 
 // Decode one sub-stream.  Shared memory is addressed by absolute shared-window addresses:
