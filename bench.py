@@ -32,6 +32,11 @@ NOMINAL_PEAK_GBS = 8000.0
 FALLBACK_PEAK_GBS = 6650.0
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, scaled from the 2-matrix capture in
+# profiles/ans_decode_private_kernel_large.md to the 8 matrices of a full launch
+NCU_TRAFFIC = {("large", "private", 32, 8, 8192, 0, 0): 933.2e6}
+
+
 def measured_peak():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -74,7 +79,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+                                          "-i", str(self.index), "-lms", "20"], stdout=subprocess.PIPE, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except Exception:
             self.proc = None
@@ -286,9 +291,12 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     kernel_ms = statistics.mean(ms)
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-    kname = "ans_decode_kernel<private>" if args.layout == "private" else "ans_decode_kernel<interleaved>"
+    kname = "ans_decode_private_kernel" if args.layout == "private" else "ans_decode_interleaved_kernel"
+    # DRAM bytes per launch from an ncu capture of this kernel (see profiles/), only for the
+    # configuration that capture covers; None otherwise
+    traffic = NCU_TRAFFIC.get((args.workload, args.layout, args.lanes, args.mats, args.dim, args.chunk, args.table_log))
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "kernel": kname, "peak_kind": f"of {peak_kind}",
+                "traffic": traffic, "kernel": kname, "peak_kind": f"of {peak_kind}",
                 "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms_mean": kernel_ms,
                 "kernel_ms_median": statistics.median(ms), "kernel_ms_min": min(ms),
                 "frac_of_nominal_8TBs": achieved / NOMINAL_PEAK_GBS}
@@ -374,8 +382,8 @@ def run_e2e(ans, db, layers, args, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=list(WORKLOAD_TEXT))
     ap.add_argument("--layout", default="private", choices=["private", "interleaved"])
