@@ -187,6 +187,32 @@ int ans_decode_dequant_host(const ans_layer_desc* h_desc,
                             const uint64_t* h_sub_offsets, const void* h_lane_meta,
                             void* h_out, void* d_scratch, size_t d_scratch_bytes, void* stream);
 
+/*
+ * (No counterpart in the paper: this is a deployment convenience.)
+ * The host-buffer decode call for callers that cannot allocate device memory at all: code that
+ * runs where cudaMalloc is forbidden or unavailable (a plug-in inside a host application that
+ * owns the memory budget, a real-time loop that may not enter the allocator, a process started
+ * with a device memory pool it may not grow).  The call takes ONLY host buffers: the layer's
+ * normalised frequencies, its compressed stream, offsets and lane metadata, and the host
+ * output.  The table is built and everything is staged inside a fixed 8 MiB working area that
+ * belongs to the library image (each GPU that loads the library holds that area until the
+ * process exits; ans_noalloc_max_bytes reports its size).  h_desc's d_* pointers are ignored.
+ *   - A layer whose table + stream + offsets + lane metadata + output (each rounded up to 256
+ *     bytes, plus 256) exceed the area is refused with ANS_ERR_BUFFER_TOO_SMALL.
+ *   - The first call on each device looks up the area's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the one area, which keeps the last call's bytes: two calls
+ *     that overlap on the GPU (different streams or host threads) race.  The call itself is
+ *     synchronous: it returns after h_out is complete.
+ *   - No cudaMalloc / cudaFree or other device allocation is made.
+ * Returns ANS_OK, ANS_ERR_CORRUPT for an unsound stream, or another ANS_ERR_* code.
+ */
+int ans_noalloc_max_bytes(size_t* h_bytes_out);
+int ans_decode_dequant_host_noalloc(const ans_layer_desc* h_desc, const uint32_t* h_norm_freqs,
+                                    int alphabet, const uint8_t* h_stream, uint64_t stream_bytes,
+                                    const uint64_t* h_sub_offsets, const void* h_lane_meta,
+                                    void* h_out, void* stream);
+
 /* ------------------------------------------------------------------------------------
  * Host-side packer: makes the streams the decoder reads.  Runs on the CPU, off the
  * inference path (the paper compresses offline, Section III-A); it is here so that a

@@ -26,6 +26,7 @@ EXPORTS = [
     "ans_plan_batch", "ans_decode_layer", "ans_decode_dequant", "ans_decode_dequant_batch",
     "ans_read_status", "ans_host_scratch_bytes", "ans_decode_dequant_host",
     "ans_host_normalize_freqs", "ans_host_pack_bound", "ans_host_pack_layer",
+    "ans_noalloc_max_bytes", "ans_decode_dequant_host_noalloc",
 ]
 
 
@@ -77,6 +78,8 @@ def lib():
         L.ans_read_status.argtypes = [vp, vp, P(u32)]
         L.ans_host_scratch_bytes.argtypes = [P(ans_layer_desc), u64, P(sz)]
         L.ans_decode_dequant_host.argtypes = [P(ans_layer_desc), vp, u64, vp, vp, vp, vp, sz, vp]
+        L.ans_noalloc_max_bytes.argtypes = [P(sz)]
+        L.ans_decode_dequant_host_noalloc.argtypes = [P(ans_layer_desc), vp, i32, vp, u64, vp, vp, vp, vp]
         L.ans_host_normalize_freqs.argtypes = [vp, i32, i32, vp]
         L.ans_host_pack_bound.argtypes = [u64, u32, u32, i32, P(u64)]
         L.ans_host_pack_layer.argtypes = [vp, u64, vp, i32, i32, u32, u32, i32, vp, u64, P(u64), vp, vp, i32]
@@ -163,6 +166,30 @@ def ans_decode_dequant_host(h_desc, h_stream: np.ndarray, h_sub_offsets: np.ndar
                                        h_out.ctypes.data, d_scratch, d_scratch_bytes, stream)
     if rc not in (ANS_OK, ANS_ERR_CORRUPT):
         raise AnsError(rc, "ans_decode_dequant_host")
+    return rc
+
+
+def ans_noalloc_max_bytes() -> int:
+    out = ctypes.c_size_t()
+    _check(lib().ans_noalloc_max_bytes(ctypes.byref(out)), "ans_noalloc_max_bytes")
+    return out.value
+
+
+def ans_decode_dequant_host_noalloc(h_desc, freqs: np.ndarray, alphabet: int, h_stream: np.ndarray,
+                                    h_sub_offsets: np.ndarray, h_lane_meta: np.ndarray, h_out: np.ndarray,
+                                    stream: int = 0) -> int:
+    """Decode one layer from host buffers to a host buffer without any device allocation by the
+    caller or the library (fixed working area inside the library).  Returns ANS_OK or
+    ANS_ERR_CORRUPT; raises AnsError otherwise (ANS_ERR_BUFFER_TOO_SMALL if the layer does not
+    fit the area)."""
+    f = np.ascontiguousarray(freqs, dtype=np.uint32)
+    assert f.size == 256
+    rc = lib().ans_decode_dequant_host_noalloc(ctypes.byref(h_desc), f.ctypes.data, alphabet,
+                                               h_stream.ctypes.data, h_stream.nbytes,
+                                               h_sub_offsets.ctypes.data, h_lane_meta.ctypes.data,
+                                               h_out.ctypes.data, stream)
+    if rc not in (ANS_OK, ANS_ERR_CORRUPT):
+        raise AnsError(rc, "ans_decode_dequant_host_noalloc")
     return rc
 
 
