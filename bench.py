@@ -291,7 +291,7 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     kernel_ms = statistics.mean(ms)
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-    kname = "ans_decode_private_kernel" if args.layout == "private" else "ans_decode_interleaved_kernel"
+    kname = "ans_decode_kernel<private>" if args.layout == "private" else "ans_decode_kernel<interleaved>"
     # DRAM bytes per launch from an ncu capture of this kernel (see profiles/), only for the
     # configuration that capture covers; None otherwise
     traffic = NCU_TRAFFIC.get((args.workload, args.layout, args.lanes, args.mats, args.dim, args.chunk, args.table_log))

@@ -98,115 +98,6 @@ __device__ __forceinline__ int find_layer(const LaunchArgs& a, uint64_t cursor) 
 }
 
 // =============================================================================================
-// Interleaved container: the warp's 32 lanes share one sequence of 16-bit units; a lane whose
-// buffer holds fewer than 16 bits takes the next unit, its place found by ballot + popcount.
-// =============================================================================================
-constexpr int kIWarps = 8;
-
-template <int ES>
-__device__ __forceinline__ uint32_t decode_interleaved(
-    const uint32_t* __restrict__ tab, const uint32_t* __restrict__ vals,
-    const uint16_t* __restrict__ units, uint32_t unit_cap, uint32_t state, uint32_t my_count,
-    uint32_t rounds, typename ElemT<ES>::type* __restrict__ out, size_t row_stride, uint32_t lane) {
-  using E = typename ElemT<ES>::type;
-  const uint32_t lt = (1u << lane) - 1u;
-  uint32_t buf = 0, pos = 0;
-  int cnt = 0;
-  for (uint32_t r = 0; r < rounds; ++r) {
-    const bool active = r < my_count;               // only the last round can have idle lanes
-    const bool need = active && cnt < 16;
-    const uint32_t b = __ballot_sync(kFull, need);
-    if (need) {
-      const uint32_t idx = pos + __popc(b & lt);
-      const uint32_t u = idx < unit_cap ? static_cast<uint32_t>(__ldg(units + idx)) : 0u;
-      buf |= u << cnt;
-      cnt += 16;
-    }
-    pos += __popc(b);
-    if (active) {
-      const uint32_t e = tab[state];
-      const uint32_t nb = entry_nb(e);
-      const uint32_t v = buf & ((1u << nb) - 1u);
-      buf >>= nb;
-      cnt -= static_cast<int>(nb);
-      state = entry_newx(e) + v;
-      out[size_t(r) * row_stride] = static_cast<E>(vals[entry_sym(e)]);
-    }
-  }
-  uint32_t bad = 0;
-  if (state != 0) bad |= ANS_STATUS_BAD_FINAL_STATE;
-  // the units taken, padded to 16 bytes, must be exactly the sub-stream's extent
-  if (((pos * 2u + 15u) & ~15u) != unit_cap * 2u) bad |= ANS_STATUS_BAD_LENGTH;
-  return bad;
-}
-
-__global__ void __launch_bounds__(kIWarps * 32) ans_decode_interleaved_kernel(const LaunchArgs args) {
-  extern __shared__ __align__(16) uint32_t smem[];
-  uint32_t* tab = smem;                                   // [table_words]
-  uint32_t* vals = smem + args.table_words;               // [256]
-  constexpr uint32_t kThreads = kIWarps * 32;
-
-  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-  uint64_t cursor = uint64_t(blockIdx.x) * args.items_per_cta;
-  const uint64_t cta_end = min(cursor + uint64_t(args.items_per_cta), uint64_t(args.total_work));
-  if (cursor >= cta_end) return;
-
-  int l = find_layer(args, cursor);
-  uint32_t bad = 0;
-  for (; cursor < cta_end; ++l) {
-    const ans_layer_desc& L = layer_at(args, l);
-    const uint64_t lbeg = L.work_begin, lend = lbeg + L.work_count;
-    if (lend <= cursor) continue;                         // empty layer
-    const uint64_t stop = min(lend, cta_end);
-    const int R = L.table_log;
-    const uint8_t* blob = static_cast<const uint8_t*>(L.d_table);
-    const TableHeader* hdr = reinterpret_cast<const TableHeader*>(blob);
-    const uint32_t* g_tab = reinterpret_cast<const uint32_t*>(blob + single_offset());
-    const int dtype = args.d_symbols_override ? ANS_U8 : L.out_dtype;
-
-    __syncthreads();                                      // previous layer's readers are done
-    for (uint32_t i = threadIdx.x; i < (1u << R); i += kThreads) tab[i] = __ldg(g_tab + i);
-    vals[threadIdx.x] = dequant_bits(static_cast<int>(threadIdx.x), L.zero_point, L.scale, dtype);
-    if (threadIdx.x == 0 && (hdr->magic != kTableMagic || hdr->table_log != uint32_t(R) ||
-                             hdr->alphabet > (1u << L.bitwidth)))
-      bad |= ANS_STATUS_BAD_SYMBOL;
-    __syncthreads();
-
-    const uint32_t W = L.lanes;
-    const size_t es = dtype == ANS_U8 ? 1 : dtype == ANS_F32 ? 4 : 2;
-    uint8_t* out_base = args.d_symbols_override ? args.d_symbols_override : static_cast<uint8_t*>(L.d_out);
-    const uint64_t n_sub = uint64_t(L.lanes / 32u) * ((L.n_symbols + L.chunk_symbols - 1) / L.chunk_symbols);
-    for (uint64_t gbase = cursor; gbase < stop; gbase += kIWarps / kGranule) {
-      const uint64_t granule = gbase + warp / kGranule;
-      const uint64_t sub = (granule - lbeg) * kGranule + warp % kGranule;
-      if (granule >= stop || sub >= n_sub) continue;
-      const Item it = make_item(L, sub);
-      const uint32_t lambda = 32u * it.g + lane;
-      const uint32_t my_count = lane_symbols(it.nc, W, lambda);
-      const uint32_t rows = lane_symbols(it.nc, W, 32u * it.g);   // lane 0 owns the most
-      uint8_t* out = out_base + (it.c0 + lambda) * es;
-      const uint32_t state = __ldg(static_cast<const uint16_t*>(L.d_lane_meta) + it.sub * 32 + lane) &
-                             ((1u << R) - 1u);
-      const uint16_t* units = reinterpret_cast<const uint16_t*>(L.d_stream + it.off0);
-      const uint32_t cap = static_cast<uint32_t>(min(it.extent / 2, uint64_t(0xFFFFFFFFu)));
-      uint32_t wbad = it.bad;
-      if (es == 1)
-        wbad |= decode_interleaved<1>(tab, vals, units, cap, state, my_count, rows, out, W, lane);
-      else if (es == 2)
-        wbad |= decode_interleaved<2>(tab, vals, units, cap, state, my_count, rows,
-                                      reinterpret_cast<uint16_t*>(out), W, lane);
-      else
-        wbad |= decode_interleaved<4>(tab, vals, units, cap, state, my_count, rows,
-                                      reinterpret_cast<uint32_t*>(out), W, lane);
-      bad |= wbad;
-    }
-    cursor = stop;
-  }
-  bad = __reduce_or_sync(kFull, bad);
-  if (lane == 0 && bad && args.d_status) atomicOr(args.d_status, bad);
-}
-
-// =============================================================================================
 // Private container: every lane reads its own run of 32-bit words.
 //
 // Look-ups go through the pre-walked table, so one look-up can stand for several symbols: `run`
@@ -543,10 +434,168 @@ __device__ __noinline__ uint32_t decode_private(
   return bad;
 }
 
+// =============================================================================================
+// Interleaved container: the warp's 32 lanes share one sequence of 16-bit units; before each
+// round a lane whose buffer holds fewer than 16 bits takes the next unit, its place found by
+// ballot + popcount; then every lane decodes one symbol.  Same shared-memory table, staging
+// buffer and output ring as above (every look-up emits exactly one symbol, so the ring needs no
+// pre-fill and no parking).
+// =============================================================================================
+template <int ES>
+__device__ __forceinline__ void interleaved_rounds(uint32_t& st, uint32_t& buf, uint32_t& cnt, uint32_t& posaddr,
+                                                   uint32_t& rb, uint32_t n, uint32_t lt, uint32_t limaddr,
+                                                   uint32_t tab_abs, uint32_t ring_lane_abs) {
+  constexpr uint32_t RB = 32u * ES;
+  constexpr uint32_t MASK = kRingRows * RB - 1u;
+#define ANSB_ROUNDS(STOP_)                                                                 \
+  asm volatile(                                                                            \
+      "{\n\t"                                                                              \
+      ".reg .pred p, q;\n\t"                                                               \
+      ".reg .u32 b, t, a, u, inc, ea, eb, m, nx, cntr;\n\t"                                \
+      "mov.u32 cntr, %5;\n"                                                                \
+      "ANSB_RLOOP:\n\t"                                                                    \
+      "setp.lt.u32 p, %2, 16;\n\t"                                                         \
+      "vote.sync.ballot.b32 b, p, 0xffffffff;\n\t"                                         \
+      "and.b32 t, b, %6;\n\t"                                                              \
+      "popc.b32 t, t;\n\t"                                                                 \
+      "mad.lo.u32 a, t, 2, %3;\n\t"                                                        \
+      "min.u32 a, a, %7;\n\t"                                                              \
+      "mov.u32 u, 0;\n\t"                                                                  \
+      "@p ld.shared.u16 u, [a];\n\t"                                                       \
+      "shl.b32 u, u, %2;\n\t"                                                              \
+      "or.b32 %1, %1, u;\n\t"                                                              \
+      "selp.u32 inc, 16, 0, p;\n\t"                                                        \
+      "add.u32 %2, %2, inc;\n\t"                                                           \
+      "popc.b32 t, b;\n\t"                                                                 \
+      "mad.lo.u32 %3, t, 2, %3;\n\t"                                                       \
+      "ld.shared.v2.u32 {ea, eb}, [%0];\n\t"                                               \
+      "shf.l.wrap.b32 m, 0, -1, ea;\n\t"                                                   \
+      "shr.u32 nx, ea, 18;\n\t"                                                            \
+      "lop3.b32 t, nx, %1, m, 0xF4;\n\t"                                                   \
+      "mad.lo.u32 %0, t, 8, %8;\n\t"                                                       \
+      "shf.r.wrap.b32 %1, %1, 0, ea;\n\t"                                                  \
+      "and.b32 t, ea, 15;\n\t"                                                             \
+      "sub.u32 %2, %2, t;\n\t"                                                             \
+      "lop3.b32 a, %4, %11, %9, 0xEA;\n\t"                                                 \
+      STOP_ " [a], eb;\n\t"                                                                \
+      "add.u32 %4, %4, %10;\n\t"                                                           \
+      "add.u32 cntr, cntr, -1;\n\t"                                                        \
+      "setp.ne.u32 q, cntr, 0;\n\t"                                                        \
+      "@q bra ANSB_RLOOP;\n\t"                                                             \
+      "}"                                                                                  \
+      : "+r"(st), "+r"(buf), "+r"(cnt), "+r"(posaddr), "+r"(rb)                            \
+      : "r"(n), "r"(lt), "r"(limaddr), "r"(tab_abs), "r"(ring_lane_abs), "n"(RB), "n"(MASK) \
+      : "memory")
+  if (ES == 1) ANSB_ROUNDS("st.shared.u8");
+  if (ES == 2) ANSB_ROUNDS("st.shared.u16");
+  if (ES == 4) ANSB_ROUNDS("st.shared.u32");
+#undef ANSB_ROUNDS
+}
+
+template <int ES, bool STAGED>
+__device__ __noinline__ uint32_t decode_interleaved(
+    uint32_t tab_abs, uint32_t ring_abs, uint32_t stage_abs, uint8_t* __restrict__ ring,
+    const uint16_t* __restrict__ units, uint32_t unit_cap, uint32_t state, uint32_t my_count, uint32_t rows,
+    uint32_t min_count, uint8_t* __restrict__ out_row0, size_t row_stride_bytes, uint32_t lane) {
+  constexpr uint32_t RB = 32u * ES;
+  constexpr uint32_t RING = kRingRows, FL = kFlushRows;
+  constexpr uint32_t MASK = RING * RB - 1u;
+  const uint32_t ring_lane_abs = ring_abs + lane * ES;
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t st = tab_abs + state * 8u;               // shared address of the state's table entry
+  uint32_t buf = 0, cnt = 0;                        // the lane's bit buffer and how many bits it holds
+  uint32_t pos = 0;                                 // units the warp has taken (same in every lane)
+  uint32_t rb = 0;                                  // RB * round
+
+  // one round in plain code: used when the sub-stream was not staged, and for the ragged round
+  auto round = [&](bool active) {
+    const bool need = active && cnt < 16u;
+    const uint32_t b = __ballot_sync(kFull, need);
+    if (need) {
+      const uint32_t idx = pos + __popc(b & lt);
+      uint32_t u = 0;
+      if (idx < unit_cap) u = STAGED ? (lds_u32(stage_abs + (idx >> 1) * 4u) >> ((idx & 1u) * 16u)) & 0xFFFFu
+                                     : static_cast<uint32_t>(__ldg(units + idx));
+      buf |= u << cnt;
+      cnt += 16u;
+    }
+    pos += __popc(b);
+    if (active) {
+      const uint32_t ea = lds_u32(st), eb = lds_u32(st + 4u);
+      const uint32_t nb = ea & 15u;
+      st = tab_abs + (((ea >> 18) | (buf & ((1u << nb) - 1u))) << 3);
+      buf >>= nb;
+      cnt -= nb;
+      sts_elem<ES>((rb & MASK) | ring_lane_abs, eb);
+    }
+    rb += RB;
+  };
+
+  const bool bulk_ok = ((reinterpret_cast<uintptr_t>(out_row0) | row_stride_bytes) & 15u) == 0;
+  const bool contiguous = row_stride_bytes == RB;
+  const bool issuer = contiguous ? lane == 0 : lane < FL;
+  // FL full rows starting at a multiple of FL leave the ring: bulk asynchronous stores when the
+  // output is 16-byte aligned (a ring slot is written again only four blocks later, by when at
+  // most three newer copies may still be pending), plain 16-byte stores otherwise
+  auto write_block = [&](uint32_t first_row) {
+    const uint32_t ring_row = first_row % RING;
+    if (bulk_ok) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (issuer) {
+        const uint32_t row = contiguous ? 0u : lane;
+        const uint32_t bytes = contiguous ? FL * RB : RB;
+        uint8_t* dst = out_row0 + size_t(first_row + row) * row_stride_bytes;
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                     :: "l"(dst), "r"(ring_abs + (ring_row + row) * RB), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 2;" ::: "memory");
+      }
+      __syncwarp();
+    } else {
+      __syncwarp();
+      flush_rows<ES>(ring + size_t(ring_row) * RB, out_row0 + size_t(first_row) * row_stride_bytes,
+                     row_stride_bytes, FL, 0u, lane);
+      __syncwarp();
+    }
+  };
+
+  uint32_t r = 0;
+  while (r < min_count) {                           // rounds in which all 32 lanes decode
+    const uint32_t n = min(FL - (r % FL), min_count - r);
+    if (STAGED) {
+      uint32_t posaddr = stage_abs + pos * 2u;
+      interleaved_rounds<ES>(st, buf, cnt, posaddr, rb, n, lt, stage_abs + unit_cap * 2u, tab_abs, ring_lane_abs);
+      pos = (posaddr - stage_abs) >> 1;
+    } else {
+      for (uint32_t i = 0; i < n; ++i) round(true);
+    }
+    r += n;
+    if (r % FL == 0) write_block(r - FL);
+  }
+  if (rows > min_count) round(my_count == rows);    // the ragged last round
+  __syncwarp();
+  {
+    const uint32_t base = (min_count / FL) * FL;    // rows before it have left already
+    const uint32_t part_lanes = rows > min_count ? __popc(__ballot_sync(kFull, my_count == rows)) : 0u;
+    flush_rows<ES>(ring + size_t(base % RING) * RB, out_row0 + size_t(base) * row_stride_bytes, row_stride_bytes,
+                   min_count - base, part_lanes, lane);
+  }
+  if (bulk_ok) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  __syncwarp();
+  uint32_t bad = 0;
+  if (st != tab_abs) bad |= ANS_STATUS_BAD_FINAL_STATE;
+  // the units taken, padded to 16 bytes, must be exactly the sub-stream's extent
+  if (((pos * 2u + 15u) & ~15u) != unit_cap * 2u) bad |= ANS_STATUS_BAD_LENGTH;
+  return bad;
+}
+
 // dynamic shared memory, by absolute shared address: [pad to ring_bytes][rings: NW * ring_bytes]
 // [table][pad to 1 KB][vals 256 words][mbarriers NW][stages NW * stage_bytes]
 
-__global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const LaunchArgs args) {
+template <int LAYOUT>
+__global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs args) {
+  constexpr bool kPrivate = LAYOUT == ANS_LAYOUT_PRIVATE;
   extern __shared__ __align__(16) uint8_t sm[];
   const uint32_t NW = blockDim.x >> 5;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
@@ -586,7 +635,8 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
     const uint8_t* blob = static_cast<const uint8_t*>(L.d_table);
     const TableHeader* hdr = reinterpret_cast<const TableHeader*>(blob);
     const uint32_t* g_single = reinterpret_cast<const uint32_t*>(blob + single_offset());
-    const uint32_t* g_multi = reinterpret_cast<const uint32_t*>(blob + multi_offset(R));
+    // private: the pre-walked entries; interleaved: the plain ones (one symbol per look-up)
+    const uint32_t* g_multi = kPrivate ? reinterpret_cast<const uint32_t*>(blob + multi_offset(R)) : g_single;
     const int dtype = args.d_symbols_override ? ANS_U8 : L.out_dtype;
 
     __syncthreads();                                      // previous layer's readers are done
@@ -594,6 +644,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
     for (uint32_t i = threadIdx.x; i < 256u; i += blockDim.x)
       vals[i] = dequant_bits(static_cast<int>(i), L.zero_point, L.scale, dtype);
     __syncthreads();
+#pragma unroll 8
     for (uint32_t i = threadIdx.x; i < (1u << R); i += blockDim.x) {
       const uint32_t g = __ldg(g_multi + i);
       tab[i] = to_smem_entry(g, vals[entry_sym(g)], 32u * static_cast<uint32_t>(es));
@@ -601,7 +652,8 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
     if (threadIdx.x == 0) {
       const uint32_t d = hdr->dominant;
       s_dom = d < 256u ? d : 0u;                          // the ring's fill symbol
-      if (R <= kMaxParkLog) tab[1u << R] = make_uint2((1u << R) << 18, es == 4 ? vals[s_dom] : (vals[s_dom] & 0xFFFFu));
+      if (kPrivate && R <= kMaxParkLog)
+        tab[1u << R] = make_uint2((1u << R) << 18, es == 4 ? vals[s_dom] : (vals[s_dom] & 0xFFFFu));
       if (hdr->magic != kTableMagic || hdr->table_log != uint32_t(R) || hdr->alphabet > (1u << L.bitwidth))
         bad |= ANS_STATUS_BAD_SYMBOL;
     }
@@ -639,16 +691,20 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
         if (lane < kStagePad / 4u) reinterpret_cast<uint32_t*>(stage + it.extent)[lane] = 0u;
       }
 
-      const uint32_t meta = __ldg(static_cast<const uint32_t*>(L.d_lane_meta) + it.sub * 32 + lane);
-      const uint32_t state = meta & ((1u << R) - 1u);
-      uint32_t wbeg = meta >> 16;
-      uint32_t wend = __shfl_down_sync(kFull, wbeg, 1);
-      if (lane == 31) wend = ext_words;
-      if (wend > ext_words) { wend = ext_words; wbad |= ANS_STATUS_BAD_LENGTH; }
-      if (wbeg > wend) { wbeg = wend; wbad |= ANS_STATUS_BAD_LENGTH; }
       uint8_t* out_row0 = out_base + (it.c0 + 32u * it.g) * es;     // row 0 of this sub-stream
       const size_t rsb = size_t(W) * es;
-      const uint32_t* words = reinterpret_cast<const uint32_t*>(g_bytes);
+      uint32_t state, wbeg = 0, wend = 0;
+      if (kPrivate) {
+        const uint32_t meta = __ldg(static_cast<const uint32_t*>(L.d_lane_meta) + it.sub * 32 + lane);
+        state = meta & ((1u << R) - 1u);
+        wbeg = meta >> 16;
+        wend = __shfl_down_sync(kFull, wbeg, 1);
+        if (lane == 31) wend = ext_words;
+        if (wend > ext_words) { wend = ext_words; wbad |= ANS_STATUS_BAD_LENGTH; }
+        if (wbeg > wend) { wbeg = wend; wbad |= ANS_STATUS_BAD_LENGTH; }
+      } else {
+        state = __ldg(static_cast<const uint16_t*>(L.d_lane_meta) + it.sub * 32 + lane) & ((1u << R) - 1u);
+      }
 
       if (staged) {
         const bool ok = mbar_wait(bar, parity);
@@ -660,16 +716,31 @@ __global__ void __launch_bounds__(512, 1) ans_decode_private_kernel(const Launch
         }
         __syncwarp();
       }
-#define ANSB_PRIV(ES_, ST_)                                                                              \
+      if (kPrivate) {
+        const uint32_t* words = reinterpret_cast<const uint32_t*>(g_bytes);
+#define ANSB_CALL(ES_, ST_)                                                                              \
   wbad |= decode_private<ES_, ST_>(tab_abs, vals_abs, ring_abs, stage_abs, park_abs, ring, g_single, dom, words, \
                                    ext_words, wbeg, wend, lane == 31, state, my_count, rows, min_count, \
                                    out_row0, rsb, lane)
-      if (staged) {
-        if (es == 1) ANSB_PRIV(1, true); else if (es == 2) ANSB_PRIV(2, true); else ANSB_PRIV(4, true);
+        if (staged) {
+          if (es == 1) ANSB_CALL(1, true); else if (es == 2) ANSB_CALL(2, true); else ANSB_CALL(4, true);
+        } else {
+          if (es == 1) ANSB_CALL(1, false); else if (es == 2) ANSB_CALL(2, false); else ANSB_CALL(4, false);
+        }
+#undef ANSB_CALL
       } else {
-        if (es == 1) ANSB_PRIV(1, false); else if (es == 2) ANSB_PRIV(2, false); else ANSB_PRIV(4, false);
+        const uint16_t* units = reinterpret_cast<const uint16_t*>(g_bytes);
+        const uint32_t unit_cap = ext_words * 2u;
+#define ANSB_CALL(ES_, ST_)                                                                              \
+  wbad |= decode_interleaved<ES_, ST_>(tab_abs, ring_abs, stage_abs, ring, units, unit_cap, state, my_count, \
+                                       rows, min_count, out_row0, rsb, lane)
+        if (staged) {
+          if (es == 1) ANSB_CALL(1, true); else if (es == 2) ANSB_CALL(2, true); else ANSB_CALL(4, true);
+        } else {
+          if (es == 1) ANSB_CALL(1, false); else if (es == 2) ANSB_CALL(2, false); else ANSB_CALL(4, false);
+        }
+#undef ANSB_CALL
       }
-#undef ANSB_PRIV
       bad |= wbad;
     }
     cursor = stop;
@@ -713,8 +784,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   a.total_work = static_cast<uint32_t>(total);
   a.d_status = d_status;
   a.d_symbols_override = d_symbols_override;
-  // interleaved: one word per state; private: two words per state and a parking entry
-  a.table_words = layout == ANS_LAYOUT_PRIVATE ? 2u * ((1u << max_log) + 2u) : (max_log < 2 ? 4u : (1u << max_log));
+  a.table_words = 2u * ((1u << max_log) + 2u);           // two words per state, and a parking entry
 
   int dev = 0, sms = 0, per_sm = 0, smem_max = 0;
   ANSB_CUDA(cudaGetDevice(&dev));
@@ -722,11 +792,11 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   ANSB_CUDA(cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
 
   const bool priv = layout == ANS_LAYOUT_PRIVATE;
-  const void* fn = priv ? reinterpret_cast<const void*>(&ans_decode_private_kernel)
-                        : reinterpret_cast<const void*>(&ans_decode_interleaved_kernel);
-  int warps = kIWarps;
+  const void* fn = priv ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE>)
+                        : reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED>);
+  int warps = 4;
   size_t smem = (size_t(a.table_words) + 256) * 4;
-  if (priv) {
+  {
     // Layers with many sub-streams share one table among up to 16 warps; a model of many small
     // layers runs CTAs of one granule (4 warps) so that each CTA stays inside one layer and
     // several CTAs, each with its own table, share an SM.
@@ -758,9 +828,9 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   a.items_per_cta = static_cast<uint32_t>(ipc);
   const unsigned blocks = static_cast<unsigned>((total + ipc - 1) / ipc);
   if (priv)
-    ans_decode_private_kernel<<<blocks, warps * 32, smem, st>>>(a);
+    ans_decode_kernel<ANS_LAYOUT_PRIVATE><<<blocks, warps * 32, smem, st>>>(a);
   else
-    ans_decode_interleaved_kernel<<<blocks, kIWarps * 32, smem, st>>>(a);
+    ans_decode_kernel<ANS_LAYOUT_INTERLEAVED><<<blocks, warps * 32, smem, st>>>(a);
   ANSB_CUDA(cudaGetLastError());
   return ANS_OK;
 }
