@@ -18,6 +18,8 @@ namespace ansb {
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr uint32_t kStatusTimeout = 8u;   // a bounded wait on an asynchronous copy ran out
 
+constexpr int kParamLayers = 96;
+
 struct LaunchArgs {
   const ans_layer_desc* d_descs;   // device array, or nullptr when `one` is the only layer
   ans_layer_desc one;
@@ -29,6 +31,8 @@ struct LaunchArgs {
   uint32_t table_words;            // shared-memory words reserved for the table
   uint32_t stage_bytes;            // private layout: per-warp staging buffer for compressed bytes
   uint32_t ring_bytes;             // private layout: per-warp output ring (kRingRows rows of the widest dtype)
+  uint32_t n_begin;                // entries of layer_begin in use (0: search the descriptors instead)
+  uint32_t layer_begin[kParamLayers];   // work_begin of the first layers, searchable without a memory trip
 };
 
 __device__ __forceinline__ const ans_layer_desc& layer_at(const LaunchArgs& a, int l) {
@@ -90,6 +94,13 @@ __device__ __forceinline__ Item make_item(const ans_layer_desc& L, uint64_t sub)
 // layer that holds work item `cursor`: the last layer with work_begin <= cursor
 __device__ __forceinline__ int find_layer(const LaunchArgs& a, uint64_t cursor) {
   int lo = 0, hi = a.n_layers;
+  if (a.n_begin == static_cast<uint32_t>(a.n_layers)) {   // every layer's start is in the parameters
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (a.layer_begin[mid] <= cursor) lo = mid; else hi = mid;
+    }
+    return lo;
+  }
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
     if (layer_at(a, mid).work_begin <= cursor) lo = mid; else hi = mid;
@@ -265,7 +276,7 @@ __device__ __noinline__ uint32_t decode_private(
     uint8_t* __restrict__ ring, const uint32_t* __restrict__ g_single, uint32_t dom_val,
     const uint32_t* __restrict__ words, uint32_t ext_words, uint32_t wbeg, uint32_t wend, bool last_lane,
     uint32_t state, uint32_t my_count, uint32_t rows, uint32_t min_count, uint8_t* __restrict__ out_row0,
-    size_t row_stride_bytes, uint32_t lane) {
+    size_t row_stride_bytes, uint32_t lane, bool allow_bulk) {
   constexpr int RB = 32 * ES;
   constexpr uint32_t RING = kRingRows;              // rows in the ring
   constexpr uint32_t FL = kFlushRows;               // rows written out at a time
@@ -316,7 +327,7 @@ __device__ __noinline__ uint32_t decode_private(
   // FL full rows starting at a multiple of FL, then fill them again.  When the output is 16-byte
   // aligned the rows leave as bulk asynchronous stores straight from the ring: one copy for the
   // whole block when the sub-stream's rows are contiguous (32 lanes per chunk), else one per row.
-  const bool bulk_ok = ((reinterpret_cast<uintptr_t>(out_row0) | row_stride_bytes) & 15u) == 0;
+  const bool bulk_ok = allow_bulk && ((reinterpret_cast<uintptr_t>(out_row0) | row_stride_bytes) & 15u) == 0;
   auto write_block = [&](uint32_t first_row) {
     const uint32_t ring_row = first_row % RING;
     if (bulk_ok) {
@@ -496,7 +507,7 @@ template <int ES, bool STAGED>
 __device__ __noinline__ uint32_t decode_interleaved(
     uint32_t tab_abs, uint32_t ring_abs, uint32_t stage_abs, uint8_t* __restrict__ ring,
     const uint16_t* __restrict__ units, uint32_t unit_cap, uint32_t state, uint32_t my_count, uint32_t rows,
-    uint32_t min_count, uint8_t* __restrict__ out_row0, size_t row_stride_bytes, uint32_t lane) {
+    uint32_t min_count, uint8_t* __restrict__ out_row0, size_t row_stride_bytes, uint32_t lane, bool allow_bulk) {
   constexpr uint32_t RB = 32u * ES;
   constexpr uint32_t RING = kRingRows, FL = kFlushRows;
   constexpr uint32_t MASK = RING * RB - 1u;
@@ -531,7 +542,7 @@ __device__ __noinline__ uint32_t decode_interleaved(
     rb += RB;
   };
 
-  const bool bulk_ok = ((reinterpret_cast<uintptr_t>(out_row0) | row_stride_bytes) & 15u) == 0;
+  const bool bulk_ok = allow_bulk && ((reinterpret_cast<uintptr_t>(out_row0) | row_stride_bytes) & 15u) == 0;
   const bool contiguous = row_stride_bytes == RB;
   const bool issuer = contiguous ? lane == 0 : lane < FL;
   // FL full rows starting at a multiple of FL leave the ring: bulk asynchronous stores when the
@@ -613,6 +624,10 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
   const uint32_t bar = bars_abs + warp * 8u;
   __shared__ uint32_t s_dom;
   uint32_t parity = 0;
+  // Bulk asynchronous stores save instructions but make a warp wait for the copy engine at every
+  // block of rows; that pays when many warps share the SM (large CTAs), not when a few warps run
+  // a short, latency-bound job each.
+  const bool allow_bulk = NW > kGranule;
 
   uint64_t cursor = uint64_t(blockIdx.x) * args.items_per_cta;
   const uint64_t cta_end = min(cursor + uint64_t(args.items_per_cta), uint64_t(args.total_work));
@@ -627,7 +642,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
   uint32_t bad = 0;
   bool gave_up = false;
   for (; cursor < cta_end; ++l) {
-    const ans_layer_desc& L = layer_at(args, l);
+    const ans_layer_desc L = layer_at(args, l);           // one batch of loads, then registers
     const uint64_t lbeg = L.work_begin, lend = lbeg + L.work_count;
     if (lend <= cursor) continue;                         // empty layer
     const uint64_t stop = min(lend, cta_end);
@@ -639,45 +654,18 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
     const uint32_t* g_multi = kPrivate ? reinterpret_cast<const uint32_t*>(blob + multi_offset(R)) : g_single;
     const int dtype = args.d_symbols_override ? ANS_U8 : L.out_dtype;
 
-    __syncthreads();                                      // previous layer's readers are done
     const size_t es = dtype == ANS_U8 ? 1 : dtype == ANS_F32 ? 4 : 2;
-    for (uint32_t i = threadIdx.x; i < 256u; i += blockDim.x)
-      vals[i] = dequant_bits(static_cast<int>(i), L.zero_point, L.scale, dtype);
-    __syncthreads();
-#pragma unroll 8
-    for (uint32_t i = threadIdx.x; i < (1u << R); i += blockDim.x) {
-      const uint32_t g = __ldg(g_multi + i);
-      tab[i] = to_smem_entry(g, vals[entry_sym(g)], 32u * static_cast<uint32_t>(es));
-    }
-    if (threadIdx.x == 0) {
-      const uint32_t d = hdr->dominant;
-      s_dom = d < 256u ? d : 0u;                          // the ring's fill symbol
-      if (kPrivate && R <= kMaxParkLog)
-        tab[1u << R] = make_uint2((1u << R) << 18, es == 4 ? vals[s_dom] : (vals[s_dom] & 0xFFFFu));
-      if (hdr->magic != kTableMagic || hdr->table_log != uint32_t(R) || hdr->alphabet > (1u << L.bitwidth))
-        bad |= ANS_STATUS_BAD_SYMBOL;
-    }
-    __syncthreads();
-
     const uint32_t W = L.lanes;
     const uint64_t n_sub = uint64_t(L.lanes / 32u) * ((L.n_symbols + L.chunk_symbols - 1) / L.chunk_symbols);
-    uint8_t* out_base = args.d_symbols_override ? args.d_symbols_override : static_cast<uint8_t*>(L.d_out);
-    const uint32_t dom = vals[s_dom];
-    const uint32_t park_abs = R <= kMaxParkLog ? tab_abs + (8u << R) : 0u;
-    for (uint64_t gbase = cursor; gbase < stop && !gave_up; gbase += NW / kGranule) {
-      const uint64_t granule = gbase + warp / kGranule;
-      const uint64_t sub = (granule - lbeg) * kGranule + warp % kGranule;
-      if (granule >= stop || sub >= n_sub) continue;
-      const Item it = make_item(L, sub);
-      uint32_t wbad = it.bad;
-      const uint32_t lambda = 32u * it.g + lane;
-      const uint32_t my_count = lane_symbols(it.nc, W, lambda);
-      const uint32_t rows = lane_symbols(it.nc, W, 32u * it.g);
-      const uint32_t min_count = lane_symbols(it.nc, W, 32u * it.g + 31u);
-      const uint32_t ext_words = static_cast<uint32_t>(min(it.extent / 4, uint64_t(0x3FFFFFFFu)));
-      const uint8_t* g_bytes = L.d_stream + it.off0;
 
-      // bring the sub-stream into shared memory (one bulk copy), if it fits
+    // The warp's first sub-stream of this layer: its bulk copy is started now so that it travels
+    // while the table is being staged.
+    auto warp_sub = [&](uint64_t gbase, uint64_t& sub) -> bool {
+      const uint64_t granule = gbase + warp / kGranule;
+      sub = (granule - lbeg) * kGranule + warp % kGranule;
+      return granule < stop && sub < n_sub;
+    };
+    auto start_copy = [&](const Item& it) -> bool {       // true if the sub-stream is being staged
       const bool staged = it.extent > 0 && it.extent + kStagePad <= args.stage_bytes;
       if (staged) {
         __syncwarp();                                     // the last item's readers of the stage are done
@@ -686,10 +674,70 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
           asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
           asm volatile(
               "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-              :: "r"(stage_abs), "l"(g_bytes), "r"(bytes), "r"(bar) : "memory");
+              :: "r"(stage_abs), "l"(L.d_stream + it.off0), "r"(bytes), "r"(bar) : "memory");
         }
         if (lane < kStagePad / 4u) reinterpret_cast<uint32_t*>(stage + it.extent)[lane] = 0u;
       }
+      return staged;
+    };
+    Item first_item;
+    bool first_staged = false;
+    uint64_t first_sub = 0;
+    const bool have_first = warp_sub(cursor, first_sub);
+    if (have_first) {
+      first_item = make_item(L, first_sub);
+      first_staged = start_copy(first_item);
+    }
+
+    __syncthreads();                                      // previous layer's readers of the table are done
+    // Table staging: all of a thread's entries are requested before any is converted, so the
+    // whole table costs about one trip to memory.
+    constexpr uint32_t kStageBatch = 16;
+    const uint32_t n_states = 1u << R;
+    for (uint32_t b0 = 0; b0 < n_states; b0 += blockDim.x * kStageBatch) {
+      uint32_t g[kStageBatch];
+#pragma unroll
+      for (uint32_t k = 0; k < kStageBatch; ++k) {
+        const uint32_t i = b0 + k * blockDim.x + threadIdx.x;
+        g[k] = i < n_states ? __ldg(g_multi + i) : 0u;
+      }
+      if (b0 == 0) {
+        for (uint32_t i = threadIdx.x; i < 256u; i += blockDim.x)
+          vals[i] = dequant_bits(static_cast<int>(i), L.zero_point, L.scale, dtype);
+        if (threadIdx.x == 0) {
+          const uint32_t d = hdr->dominant;
+          s_dom = d < 256u ? d : 0u;                      // the ring's fill symbol
+          if (hdr->magic != kTableMagic || hdr->table_log != uint32_t(R) || hdr->alphabet > (1u << L.bitwidth))
+            bad |= ANS_STATUS_BAD_SYMBOL;
+        }
+        __syncthreads();
+      }
+#pragma unroll
+      for (uint32_t k = 0; k < kStageBatch; ++k) {
+        const uint32_t i = b0 + k * blockDim.x + threadIdx.x;
+        if (i < n_states) tab[i] = to_smem_entry(g[k], vals[entry_sym(g[k])], 32u * static_cast<uint32_t>(es));
+      }
+    }
+    if (threadIdx.x == 0 && kPrivate && R <= kMaxParkLog)
+      tab[n_states] = make_uint2(n_states << 18, es == 4 ? vals[s_dom] : (vals[s_dom] & 0xFFFFu));
+    __syncthreads();
+
+    uint8_t* out_base = args.d_symbols_override ? args.d_symbols_override : static_cast<uint8_t*>(L.d_out);
+    const uint32_t dom = vals[s_dom];
+    const uint32_t park_abs = R <= kMaxParkLog ? tab_abs + (8u << R) : 0u;
+    for (uint64_t gbase = cursor; gbase < stop && !gave_up; gbase += NW / kGranule) {
+      uint64_t sub;
+      if (!warp_sub(gbase, sub)) continue;
+      const bool is_first = gbase == cursor;              // its copy is already under way
+      const Item it = is_first ? first_item : make_item(L, sub);
+      uint32_t wbad = it.bad;
+      const uint32_t lambda = 32u * it.g + lane;
+      const uint32_t my_count = lane_symbols(it.nc, W, lambda);
+      const uint32_t rows = lane_symbols(it.nc, W, 32u * it.g);
+      const uint32_t min_count = lane_symbols(it.nc, W, 32u * it.g + 31u);
+      const uint32_t ext_words = static_cast<uint32_t>(min(it.extent / 4, uint64_t(0x3FFFFFFFu)));
+      const uint8_t* g_bytes = L.d_stream + it.off0;
+      const bool staged = is_first ? first_staged : start_copy(it);
 
       uint8_t* out_row0 = out_base + (it.c0 + 32u * it.g) * es;     // row 0 of this sub-stream
       const size_t rsb = size_t(W) * es;
@@ -721,7 +769,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
 #define ANSB_CALL(ES_, ST_)                                                                              \
   wbad |= decode_private<ES_, ST_>(tab_abs, vals_abs, ring_abs, stage_abs, park_abs, ring, g_single, dom, words, \
                                    ext_words, wbeg, wend, lane == 31, state, my_count, rows, min_count, \
-                                   out_row0, rsb, lane)
+                                   out_row0, rsb, lane, allow_bulk)
         if (staged) {
           if (es == 1) ANSB_CALL(1, true); else if (es == 2) ANSB_CALL(2, true); else ANSB_CALL(4, true);
         } else {
@@ -733,7 +781,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
         const uint32_t unit_cap = ext_words * 2u;
 #define ANSB_CALL(ES_, ST_)                                                                              \
   wbad |= decode_interleaved<ES_, ST_>(tab_abs, ring_abs, stage_abs, ring, units, unit_cap, state, my_count, \
-                                       rows, min_count, out_row0, rsb, lane)
+                                       rows, min_count, out_row0, rsb, lane, allow_bulk)
         if (staged) {
           if (es == 1) ANSB_CALL(1, true); else if (es == 2) ANSB_CALL(2, true); else ANSB_CALL(4, true);
         } else {
@@ -752,6 +800,11 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
+constexpr int kMaxDevices = 64;
+struct LaunchShape { size_t smem = 0; int warps = 0; int per_sm = 0; };
+struct DeviceFacts { int sms = 0; int smem_max = 0; LaunchShape shape[2]; };
+static DeviceFacts g_facts[kMaxDevices];    // remembered per device; racing writers store equal values
+
 static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, int n_layers,
                   uint8_t* d_symbols_override, uint32_t* d_status, cudaStream_t st) {
   int max_log = 1, busy_layers = 0;
@@ -785,11 +838,25 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   a.d_status = d_status;
   a.d_symbols_override = d_symbols_override;
   a.table_words = 2u * ((1u << max_log) + 2u);           // two words per state, and a parking entry
+  if (n_layers <= kParamLayers) {
+    a.n_begin = static_cast<uint32_t>(n_layers);
+    for (int l = 0; l < n_layers; ++l) a.layer_begin[l] = h_descs[l].work_begin;
+  }
 
+  // device facts and per-configuration occupancy are looked up once and remembered (plain values,
+  // no allocation): a launch of a small model should not spend its time in attribute queries
   int dev = 0, sms = 0, per_sm = 0, smem_max = 0;
   ANSB_CUDA(cudaGetDevice(&dev));
-  ANSB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  ANSB_CUDA(cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+  if (dev < 0 || dev >= kMaxDevices) return ANS_ERR_UNSUPPORTED;
+  DeviceFacts& facts = g_facts[dev];
+  if (!facts.sms) {
+    ANSB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    ANSB_CUDA(cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    facts.smem_max = smem_max;
+    facts.sms = sms;
+  }
+  sms = facts.sms;
+  smem_max = facts.smem_max;
 
   const bool priv = layout == ANS_LAYOUT_PRIVATE;
   const void* fn = priv ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE>)
@@ -817,8 +884,17 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
     a.ring_bytes = static_cast<uint32_t>(ring);
     smem = fixed + size_t(warps) * (ring + stage);
   }
-  ANSB_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-  ANSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, warps * 32, smem));
+  {
+    LaunchShape& shape = facts.shape[priv ? 1 : 0];
+    if (shape.smem != smem || shape.warps != warps) {
+      ANSB_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+      ANSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, warps * 32, smem));
+      shape.smem = smem;
+      shape.warps = warps;
+      shape.per_sm = per_sm;
+    }
+    per_sm = shape.per_sm;
+  }
   if (per_sm < 1) return ANS_ERR_UNSUPPORTED;
   const uint64_t step = uint64_t(warps) / kGranule;       // granules a CTA takes at a time
   const uint64_t want_ctas = (total + step - 1) / step;

@@ -55,8 +55,9 @@ def _pad16(n: int) -> int:
 
 class DeviceBatch:
     """All layers of a model resident on the GPU in compressed form, ready to decode in
-    one launch.  Output tensors are allocated once (optionally `n_out_sets` rotating sets,
-    so that repeated timing does not find its working set in L2)."""
+    one launch.  With `n_out_sets` > 1 everything a launch touches (compressed arena, tables,
+    outputs) exists that many times, so that a timing loop which rotates over the sets reads
+    and writes memory that the launches in between have pushed out of L2."""
 
     def __init__(self, layers: list[PackedLayer], device="cuda:0", n_out_sets: int = 1):
         self.layers = layers
@@ -76,7 +77,9 @@ class DeviceBatch:
             for j, a in enumerate((L.stream, L.sub_offsets, L.lane_meta)):
                 s = int(starts[3 * i + j])
                 ah[s:s + a.nbytes] = a.reshape(-1).view(np.uint8)
+        n_sets = max(1, n_out_sets)
         self.arena = arena_h.to(self.device, non_blocking=True)
+        self.arenas = [self.arena] + [self.arena.clone() for _ in range(n_sets - 1)]
         self.arena_host = arena_h
         # tables
         tbytes = sum(B.ans_table_bytes(L.table_log) for L in layers)
@@ -87,21 +90,25 @@ class DeviceBatch:
             self.table_offsets = B.ans_build_decode_tables(
                 freqs, [L.alphabet for L in layers], [L.table_log for L in layers],
                 self.tables.data_ptr(), self.tables.numel(), stream)
+        self.table_sets = [self.tables] + [self.tables.clone() for _ in range(n_sets - 1)]
         # outputs
         self.out_sets = []
-        for _ in range(max(1, n_out_sets)):
+        for _ in range(n_sets):
             self.out_sets.append([torch.empty(max(L.n_symbols, 1), dtype=_TORCH_DTYPE[L.out_dtype],
                                               device=self.device) for L in layers])
         self.status = torch.zeros(64, dtype=torch.int32, device=self.device)
         # descriptors: one host array + device copy per output set
         self.h_descs = []
         self.d_descs = []
-        base = self.arena.data_ptr()
-        for outs in self.out_sets:
+        torch.cuda.synchronize(self.device)                 # tables are built before they are cloned above
+        for k in range(1, n_sets):
+            self.table_sets[k].copy_(self.tables)
+        for k, outs in enumerate(self.out_sets):
+            base = self.arenas[k].data_ptr()
             arr = (B.ans_layer_desc * max(n, 1))()
             for i, L in enumerate(layers):
                 d = arr[i]
-                d.d_table = self.tables.data_ptr() + int(self.table_offsets[i])
+                d.d_table = self.table_sets[k].data_ptr() + int(self.table_offsets[i])
                 d.d_stream = base + int(starts[3 * i])
                 d.d_sub_offsets = base + int(starts[3 * i + 1])
                 d.d_lane_meta = base + int(starts[3 * i + 2])
