@@ -30,6 +30,7 @@ struct LaunchArgs {
   uint8_t* d_symbols_override;     // ans_decode_layer: write symbols here instead of d_out
   uint32_t table_words;            // shared-memory words reserved for the table
   uint32_t stage_bytes;            // private layout: per-warp staging buffer for compressed bytes
+  uint32_t succ_bytes;             // private layout: shared-memory bytes of the successor table
   uint32_t ring_bytes;             // private layout: per-warp output ring (kRingRows rows of the widest dtype)
   uint32_t n_begin;                // entries of layer_begin in use (0: search the descriptors instead)
   uint32_t layer_begin[kParamLayers];   // work_begin of the first layers, searchable without a memory trip
@@ -181,6 +182,11 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t a) {
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
   return v;
 }
+__device__ __forceinline__ uint32_t lds_u16(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+  return v;
+}
 template <int ES>
 __device__ __forceinline__ void sts_elem(uint32_t a, uint32_t v) {
   if (ES == 1) asm volatile("st.shared.u8 [%0], %1;" :: "r"(a), "r"(v) : "memory");
@@ -266,14 +272,14 @@ __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t
 }
 
 // Decode one sub-stream.  Shared memory is addressed by absolute shared-window addresses:
-// tab_abs (table), vals_abs (dequantised values, 1 KB aligned), ring_abs (this warp's ring,
+// tab_abs (table), succ_abs (u16 successor of every zero-bit state), ring_abs (this warp's ring,
 // aligned to its size), stage_abs (staged sub-stream when STAGED, with kStagePad readable bytes
 // after it).  `ring` is the generic pointer to the same ring; `words` the sub-stream in
 // global memory, used when it was not staged.
 template <int ES, bool STAGED>
 __device__ __noinline__ uint32_t decode_private(
-    uint32_t tab_abs, uint32_t vals_abs, uint32_t ring_abs, uint32_t stage_abs, uint32_t park_abs,
-    uint8_t* __restrict__ ring, const uint32_t* __restrict__ g_single, uint32_t dom_val,
+    uint32_t tab_abs, uint32_t succ_abs, uint32_t ring_abs, uint32_t stage_abs, uint32_t park_abs,
+    uint8_t* __restrict__ ring, uint32_t dom_val,
     const uint32_t* __restrict__ words, uint32_t ext_words, uint32_t wbeg, uint32_t wend, bool last_lane,
     uint32_t state, uint32_t my_count, uint32_t rows, uint32_t min_count, uint8_t* __restrict__ out_row0,
     size_t row_stride_bytes, uint32_t lane, bool allow_bulk) {
@@ -344,14 +350,27 @@ __device__ __noinline__ uint32_t decode_private(
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the ring rows may be reused
       }
       __syncwarp();
+      uint8_t* part = ring + size_t(ring_row) * RB;
+      for (uint32_t i = lane; i < (FL * RB) / 16u; i += 32u) reinterpret_cast<uint4*>(part)[i] = fill4;
     } else {
+      // plain stores: each 16-byte piece is read, written out and filled again by the same lane
       __syncwarp();
-      flush_rows<ES>(ring + size_t(ring_row) * RB, out_row0 + size_t(first_row) * row_stride_bytes,
-                     row_stride_bytes, FL, 0u, lane);
-      __syncwarp();
+      uint8_t* part = ring + size_t(ring_row) * RB;
+      uint8_t* dst = out_row0 + size_t(first_row) * row_stride_bytes;
+      constexpr uint32_t PPR = RB / 16u;
+      if (((reinterpret_cast<uintptr_t>(dst) | row_stride_bytes) & 15u) == 0) {
+#pragma unroll
+        for (uint32_t i = lane; i < FL * PPR; i += 32u) {
+          const uint4 v = reinterpret_cast<const uint4*>(part)[i];
+          *reinterpret_cast<uint4*>(dst + size_t(i / PPR) * row_stride_bytes + (i % PPR) * 16u) = v;
+          reinterpret_cast<uint4*>(part)[i] = fill4;
+        }
+      } else {
+        flush_rows<ES>(part, dst, row_stride_bytes, FL, 0u, lane);
+        __syncwarp();
+        for (uint32_t i = lane; i < (FL * RB) / 16u; i += 32u) reinterpret_cast<uint4*>(part)[i] = fill4;
+      }
     }
-    uint8_t* part = ring + size_t(ring_row) * RB;
-    for (uint32_t i = lane; i < (FL * RB) / 16u; i += 32u) reinterpret_cast<uint4*>(part)[i] = fill4;
     __syncwarp();
   };
 
@@ -412,19 +431,20 @@ __device__ __noinline__ uint32_t decode_private(
     bitpos += step(__funnelshift_r(w0, w1, bitpos));
     refill_checked();
   }
-  // ... and the last (up to 15) symbols one per look-up through the plain table
-  uint32_t t = static_cast<uint32_t>(next_row());
-  state = (st - tab_abs) >> 3;
-  while (t < my_count) {
-    const uint32_t e = __ldg(g_single + state);
-    sts_elem<ES>(((t * RB) & MASK) | ring_lane_abs, lds_u32(vals_abs + entry_sym(e) * 4u));
-    t += 1;
-    const uint32_t nb = entry_nb(e);
-    const uint32_t x = __funnelshift_r(w0, w1, bitpos);
-    state = entry_newx(e) + (x & ((1u << nb) - 1u));
-    bitpos += nb;
-    refill_checked();
+  // ... and the last (up to 15) symbols one at a time: a state whose pre-walked entry has no run
+  // is stepped as above; a zero-bit state of the dominant symbol emits that symbol (its value is
+  // already in the ring), reads nothing and goes to its one successor, kept in a side table
+  while (next_row() < static_cast<int32_t>(my_count)) {
+    const uint32_t ea = lds_u32(st);
+    if (((ea >> 6) & 31u) == 1u) {
+      bitpos += step(__funnelshift_r(w0, w1, bitpos));
+      refill_checked();
+    } else {
+      st = tab_abs + lds_u16(succ_abs + ((st - tab_abs) >> 2)) * 8u;
+      tbm += RB;
+    }
   }
+  state = (st - tab_abs) >> 3;
   __syncwarp();
   {
     const bool has_part = min_count < rows;         // last row is ragged
@@ -614,11 +634,13 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
   const uint32_t rings_abs = (sm_abs + args.ring_bytes - 1u) & ~(args.ring_bytes - 1u);
   const uint32_t tab_abs = rings_abs + NW * args.ring_bytes;
   const uint32_t vals_abs = (tab_abs + args.table_words * 4u + 1023u) & ~1023u;
-  const uint32_t bars_abs = vals_abs + 1024u;
+  const uint32_t succ_abs = vals_abs + 1024u;             // private: u16 per state, (2 << max R) bytes
+  const uint32_t bars_abs = succ_abs + args.succ_bytes;
   const uint32_t ring_abs = rings_abs + warp * args.ring_bytes;
   const uint32_t stage_abs = bars_abs + NW * 8u + warp * args.stage_bytes;
   uint2* tab = reinterpret_cast<uint2*>(sm + (tab_abs - sm_abs));
   uint32_t* vals = reinterpret_cast<uint32_t*>(sm + (vals_abs - sm_abs));
+  uint16_t* succ = reinterpret_cast<uint16_t*>(sm + (succ_abs - sm_abs));
   uint8_t* ring = sm + (ring_abs - sm_abs);
   uint8_t* stage = sm + (stage_abs - sm_abs);
   const uint32_t bar = bars_abs + warp * 8u;
@@ -695,11 +717,12 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
     constexpr uint32_t kStageBatch = 16;
     const uint32_t n_states = 1u << R;
     for (uint32_t b0 = 0; b0 < n_states; b0 += blockDim.x * kStageBatch) {
-      uint32_t g[kStageBatch];
+      uint32_t g[kStageBatch], g1[kStageBatch];
 #pragma unroll
       for (uint32_t k = 0; k < kStageBatch; ++k) {
         const uint32_t i = b0 + k * blockDim.x + threadIdx.x;
         g[k] = i < n_states ? __ldg(g_multi + i) : 0u;
+        if (kPrivate) g1[k] = i < n_states ? __ldg(g_single + i) : 0u;
       }
       if (b0 == 0) {
         for (uint32_t i = threadIdx.x; i < 256u; i += blockDim.x)
@@ -715,7 +738,10 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
 #pragma unroll
       for (uint32_t k = 0; k < kStageBatch; ++k) {
         const uint32_t i = b0 + k * blockDim.x + threadIdx.x;
-        if (i < n_states) tab[i] = to_smem_entry(g[k], vals[entry_sym(g[k])], 32u * static_cast<uint32_t>(es));
+        if (i < n_states) {
+          tab[i] = to_smem_entry(g[k], vals[entry_sym(g[k])], 32u * static_cast<uint32_t>(es));
+          if (kPrivate) succ[i] = static_cast<uint16_t>(entry_newx(g1[k]));
+        }
       }
     }
     if (threadIdx.x == 0 && kPrivate && R <= kMaxParkLog)
@@ -767,7 +793,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
       if (kPrivate) {
         const uint32_t* words = reinterpret_cast<const uint32_t*>(g_bytes);
 #define ANSB_CALL(ES_, ST_)                                                                              \
-  wbad |= decode_private<ES_, ST_>(tab_abs, vals_abs, ring_abs, stage_abs, park_abs, ring, g_single, dom, words, \
+  wbad |= decode_private<ES_, ST_>(tab_abs, succ_abs, ring_abs, stage_abs, park_abs, ring, dom, words,     \
                                    ext_words, wbeg, wend, lane == 31, state, my_count, rows, min_count, \
                                    out_row0, rsb, lane, allow_bulk)
         if (staged) {
@@ -862,7 +888,8 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   const void* fn = priv ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE>)
                         : reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED>);
   int warps = 4;
-  size_t smem = (size_t(a.table_words) + 256) * 4;
+  a.succ_bytes = priv ? ((2u << max_log) + 15u) & ~15u : 0u;
+  size_t smem = (size_t(a.table_words) + 256) * 4 + a.succ_bytes;
   {
     // Layers with many sub-streams share one table among up to 16 warps; a model of many small
     // layers runs CTAs of one granule (4 warps) so that each CTA stays inside one layer and
