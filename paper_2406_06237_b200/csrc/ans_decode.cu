@@ -282,7 +282,7 @@ __device__ __noinline__ uint32_t decode_private(
     uint8_t* __restrict__ ring, uint32_t dom_val,
     const uint32_t* __restrict__ words, uint32_t ext_words, uint32_t wbeg, uint32_t wend, bool last_lane,
     uint32_t state, uint32_t my_count, uint32_t rows, uint32_t min_count, uint8_t* __restrict__ out_row0,
-    size_t row_stride_bytes, uint32_t lane, bool allow_bulk) {
+    size_t row_stride_bytes, uint32_t lane) {
   constexpr int RB = 32 * ES;
   constexpr uint32_t RING = kRingRows;              // rows in the ring
   constexpr uint32_t FL = kFlushRows;               // rows written out at a time
@@ -330,46 +330,26 @@ __device__ __noinline__ uint32_t decode_private(
                      0u, part_lanes, lane);
     }
   };
-  // FL full rows starting at a multiple of FL, then fill them again.  When the output is 16-byte
-  // aligned the rows leave as bulk asynchronous stores straight from the ring: one copy for the
-  // whole block when the sub-stream's rows are contiguous (32 lanes per chunk), else one per row.
-  const bool bulk_ok = allow_bulk && ((reinterpret_cast<uintptr_t>(out_row0) | row_stride_bytes) & 15u) == 0;
+  // FL full rows starting at a multiple of FL leave the ring and are filled again: each 16-byte
+  // piece is read, written out and re-filled by the same lane, so one warp barrier on each side
+  // is all the ordering needed.  (Bulk asynchronous stores were measured here too: the wait for
+  // the copy engine before the rows can be re-filled costs more than these few instructions.)
   auto write_block = [&](uint32_t first_row) {
-    const uint32_t ring_row = first_row % RING;
-    if (bulk_ok) {
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ring writes -> visible to the copy engine
-      __syncwarp();
-      const bool contiguous = row_stride_bytes == RB;
-      if (contiguous ? lane == 0 : lane < FL) {
-        const uint32_t row = contiguous ? 0u : lane;
-        const uint32_t bytes = contiguous ? FL * RB : RB;
-        uint8_t* dst = out_row0 + size_t(first_row + row) * row_stride_bytes;
-        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                     :: "l"(dst), "r"(ring_abs + (ring_row + row) * RB), "r"(bytes) : "memory");
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the ring rows may be reused
-      }
-      __syncwarp();
-      uint8_t* part = ring + size_t(ring_row) * RB;
-      for (uint32_t i = lane; i < (FL * RB) / 16u; i += 32u) reinterpret_cast<uint4*>(part)[i] = fill4;
-    } else {
-      // plain stores: each 16-byte piece is read, written out and filled again by the same lane
-      __syncwarp();
-      uint8_t* part = ring + size_t(ring_row) * RB;
-      uint8_t* dst = out_row0 + size_t(first_row) * row_stride_bytes;
-      constexpr uint32_t PPR = RB / 16u;
-      if (((reinterpret_cast<uintptr_t>(dst) | row_stride_bytes) & 15u) == 0) {
+    __syncwarp();
+    uint8_t* part = ring + size_t(first_row % RING) * RB;
+    uint8_t* dst = out_row0 + size_t(first_row) * row_stride_bytes;
+    constexpr uint32_t PPR = RB / 16u;
+    if (((reinterpret_cast<uintptr_t>(dst) | row_stride_bytes) & 15u) == 0) {
 #pragma unroll
-        for (uint32_t i = lane; i < FL * PPR; i += 32u) {
-          const uint4 v = reinterpret_cast<const uint4*>(part)[i];
-          *reinterpret_cast<uint4*>(dst + size_t(i / PPR) * row_stride_bytes + (i % PPR) * 16u) = v;
-          reinterpret_cast<uint4*>(part)[i] = fill4;
-        }
-      } else {
-        flush_rows<ES>(part, dst, row_stride_bytes, FL, 0u, lane);
-        __syncwarp();
-        for (uint32_t i = lane; i < (FL * RB) / 16u; i += 32u) reinterpret_cast<uint4*>(part)[i] = fill4;
+      for (uint32_t i = lane; i < FL * PPR; i += 32u) {
+        const uint4 v = reinterpret_cast<const uint4*>(part)[i];
+        *reinterpret_cast<uint4*>(dst + size_t(i / PPR) * row_stride_bytes + (i % PPR) * 16u) = v;
+        reinterpret_cast<uint4*>(part)[i] = fill4;
       }
+    } else {
+      flush_rows<ES>(part, dst, row_stride_bytes, FL, 0u, lane);
+      __syncwarp();
+      for (uint32_t i = lane; i < (FL * RB) / 16u; i += 32u) reinterpret_cast<uint4*>(part)[i] = fill4;
     }
     __syncwarp();
   };
@@ -453,7 +433,6 @@ __device__ __noinline__ uint32_t decode_private(
     if (has_part) part_lanes = __popc(__ballot_sync(kFull, my_count == rows));
     write_out(base, full_rows, part_lanes);
   }
-  if (bulk_ok) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this lane's bulk stores have landed
   __syncwarp();
   uint32_t bad = 0;
   if (state != 0) bad |= ANS_STATUS_BAD_FINAL_STATE;
@@ -646,9 +625,9 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
   const uint32_t bar = bars_abs + warp * 8u;
   __shared__ uint32_t s_dom;
   uint32_t parity = 0;
-  // Bulk asynchronous stores save instructions but make a warp wait for the copy engine at every
-  // block of rows; that pays when many warps share the SM (large CTAs), not when a few warps run
-  // a short, latency-bound job each.
+  // Interleaved container: bulk asynchronous stores save instructions but make a warp wait for
+  // the copy engine now and then; that pays when many warps share the SM (large CTAs), not when
+  // a few warps run a short, latency-bound job each.
   const bool allow_bulk = NW > kGranule;
 
   uint64_t cursor = uint64_t(blockIdx.x) * args.items_per_cta;
@@ -795,7 +774,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
 #define ANSB_CALL(ES_, ST_)                                                                              \
   wbad |= decode_private<ES_, ST_>(tab_abs, succ_abs, ring_abs, stage_abs, park_abs, ring, dom, words,     \
                                    ext_words, wbeg, wend, lane == 31, state, my_count, rows, min_count, \
-                                   out_row0, rsb, lane, allow_bulk)
+                                   out_row0, rsb, lane)
         if (staged) {
           if (es == 1) ANSB_CALL(1, true); else if (es == 2) ANSB_CALL(2, true); else ANSB_CALL(4, true);
         } else {
