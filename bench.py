@@ -49,7 +49,7 @@ def measured_peak():
 
 def make_specs(args):
     if args.workload == "sweep":
-        return sg.workload_sweep(table_log=args.table_log or 12, chunk=args.chunk or 16384)
+        return sg.workload_sweep(table_log=args.table_log or 12, chunk=args.chunk or 16384, n=args.symbols)
     if args.workload == "large":
         return sg.workload_large(n_mats=args.mats, dim=args.dim, chunk=args.chunk or 32768,
                                  table_log=args.table_log or 12)
@@ -396,6 +396,7 @@ def main():
     ap.add_argument("--table-log", type=int, default=0)
     ap.add_argument("--mats", type=int, default=8, help="large workload: number of matrices (8 = full size)")
     ap.add_argument("--dim", type=int, default=8192, help="large workload: matrix dimension (8192 = full size)")
+    ap.add_argument("--symbols", type=int, default=1 << 28, help="sweep workload: number of symbols (2^28 = full size)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()

@@ -127,19 +127,19 @@ constexpr uint32_t kWaitSpins = 1u << 22;
 constexpr uint32_t kPair = 2 * (kMaxRun + 1);  // symbols two look-ups can emit
 
 // shared-memory form of a pre-walked entry, two words:
-//   a: nb [3:0] (bits 4-5 stay 0) | symbols emitted = run + 1 [10:6] | newX [31:18]
+//   a: nb [3:0] (bits 4-5 stay 0) | symbols emitted = run + 1 [10:6] | newX [31:17]
 //   b: 1- and 2-byte outputs: dequantised value [15:0] | row bytes * (run + 1) [31:16]
 //      4-byte outputs:        dequantised value
-// One extra entry after the table (index 2^R, possible while R <= 13) emits nothing, reads
+// One extra entry after the table (index 2^R, which the 15-bit newX field can hold) emits nothing, reads
 // nothing and leads to itself: a lane that must wait is parked on it.
 __device__ __forceinline__ uint2 to_smem_entry(uint32_t g, uint32_t val, uint32_t row_bytes) {
   const uint32_t adv = entry_run(g) + 1u;
   uint2 e;
-  e.x = entry_nb(g) | (adv << 6) | (entry_newx(g) << 18);
+  e.x = entry_nb(g) | (adv << 6) | (entry_newx(g) << 17);
   e.y = row_bytes == 128u ? val : ((val & 0xFFFFu) | ((adv * row_bytes) << 16));
   return e;
 }
-constexpr int kMaxParkLog = 13;
+constexpr int kMaxParkLog = 14;
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
@@ -210,7 +210,7 @@ constexpr int kPairsPerCall = 16;
 #define ANSB_STEP(ADV_, STOP_)                                    \
   "ld.shared.v2.u32 {ea, eb}, [stx];\n\t"                         \
   "shf.l.wrap.b32 m, 0, -1, ea;\n\t"                              \
-  "shr.u32 nx, ea, 18;\n\t"                                       \
+  "shr.u32 nx, ea, 17;\n\t"                                       \
   "lop3.b32 t, nx, x, m, 0xF4;\n\t"                               \
   "mad.lo.u32 stx, t, 8, %8;\n\t"                                 \
   ADV_                                                            \
@@ -360,7 +360,7 @@ __device__ __noinline__ uint32_t decode_private(
   auto step = [&](uint32_t x) -> uint32_t {
     const uint32_t ea = lds_u32(st), eb = lds_u32(st + 4u);
     const uint32_t nb = ea & 15u;
-    st = tab_abs + (((ea >> 18) | (x & ((1u << nb) - 1u))) << 3);
+    st = tab_abs + (((ea >> 17) | (x & ((1u << nb) - 1u))) << 3);
     tbm += ((ea >> 6) & 31u) * RB;
     sts_elem<ES>((tbm & MASK) | ring_lane_abs, eb);
     return nb;
@@ -480,7 +480,7 @@ __device__ __forceinline__ void interleaved_rounds(uint32_t& st, uint32_t& buf, 
       "mad.lo.u32 %3, t, 2, %3;\n\t"                                                       \
       "ld.shared.v2.u32 {ea, eb}, [%0];\n\t"                                               \
       "shf.l.wrap.b32 m, 0, -1, ea;\n\t"                                                   \
-      "shr.u32 nx, ea, 18;\n\t"                                                            \
+      "shr.u32 nx, ea, 17;\n\t"                                                            \
       "lop3.b32 t, nx, %1, m, 0xF4;\n\t"                                                   \
       "mad.lo.u32 %0, t, 8, %8;\n\t"                                                       \
       "shf.r.wrap.b32 %1, %1, 0, ea;\n\t"                                                  \
@@ -533,7 +533,7 @@ __device__ __noinline__ uint32_t decode_interleaved(
     if (active) {
       const uint32_t ea = lds_u32(st), eb = lds_u32(st + 4u);
       const uint32_t nb = ea & 15u;
-      st = tab_abs + (((ea >> 18) | (buf & ((1u << nb) - 1u))) << 3);
+      st = tab_abs + (((ea >> 17) | (buf & ((1u << nb) - 1u))) << 3);
       buf >>= nb;
       cnt -= nb;
       sts_elem<ES>((rb & MASK) | ring_lane_abs, eb);
@@ -724,7 +724,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
       }
     }
     if (threadIdx.x == 0 && kPrivate && R <= kMaxParkLog)
-      tab[n_states] = make_uint2(n_states << 18, es == 4 ? vals[s_dom] : (vals[s_dom] & 0xFFFFu));
+      tab[n_states] = make_uint2(n_states << 17, es == 4 ? vals[s_dom] : (vals[s_dom] & 0xFFFFu));
     __syncthreads();
 
     uint8_t* out_base = args.d_symbols_override ? args.d_symbols_override : static_cast<uint8_t*>(L.d_out);
