@@ -122,7 +122,7 @@ __device__ __forceinline__ int find_layer(const LaunchArgs& a, uint64_t cursor) 
 // =============================================================================================
 constexpr uint32_t kRingRows = 64;             // rows (of 32 symbols) in a warp's output ring
 constexpr uint32_t kFlushRows = 16;            // rows written out at a time
-constexpr uint32_t kStagePad = 112;            // readable bytes after the staged sub-stream
+constexpr uint32_t kStagePad = 176;            // readable bytes after the staged sub-stream
 constexpr uint32_t kWaitSpins = 1u << 22;
 constexpr uint32_t kPair = 2 * (kMaxRun + 1);  // symbols two look-ups can emit
 
@@ -204,7 +204,7 @@ __device__ __forceinline__ void sts_elem(uint32_t a, uint32_t v) {
 //   bitpos : bits of w0 already used; only its low 5 bits are kept clean
 //   w0,w1,w2 : bit window and the word after it        sp : shared address of the next word
 // ring_lane_abs is the ring's address (a multiple of its size) + lane * ES, so OR forms the row address.
-constexpr int kPairsPerCall = 16;
+constexpr int kPairsPerCall = 32;
 
 // ADV_: how tbm advances (from word b for narrow outputs, from word a's field for 4-byte ones)
 #define ANSB_STEP(ADV_, STOP_)                                    \
@@ -282,7 +282,7 @@ __device__ __noinline__ uint32_t decode_private(
     uint8_t* __restrict__ ring, uint32_t dom_val,
     const uint32_t* __restrict__ words, uint32_t ext_words, uint32_t wbeg, uint32_t wend, bool last_lane,
     uint32_t state, uint32_t my_count, uint32_t rows, uint32_t min_count, uint8_t* __restrict__ out_row0,
-    size_t row_stride_bytes, uint32_t lane) {
+    size_t row_stride_bytes, uint32_t lane, uint32_t max_adv) {
   constexpr int RB = 32 * ES;
   constexpr uint32_t RING = kRingRows;              // rows in the ring
   constexpr uint32_t FL = kFlushRows;               // rows written out at a time
@@ -376,12 +376,14 @@ __device__ __noinline__ uint32_t decode_private(
   auto next_row = [&]() -> int32_t { return (static_cast<int32_t>(tbm) + RB) / RB; };
 
   // main part: two look-ups share one 32-bit extract (2 * 14 bits at most) and one refill check;
-  // it stops kPair - 1 symbols short of the lane's end, so a pair can never emit too many
-  const int32_t lim2 = static_cast<int32_t>(my_count > kPair - 1 ? my_count - (kPair - 1) : 0u);
-  const int32_t lim1 = static_cast<int32_t>(my_count > kMaxRun ? my_count - kMaxRun : 0u);
+  // it stops short of the lane's end by what a pair can emit at most in this layer (2 * max_adv
+  // symbols, max_adv = longest run in the layer's table + 1), so a pair can never emit too many
+  const uint32_t pair_max = 2u * max_adv;
+  const int32_t lim2 = static_cast<int32_t>(my_count > pair_max - 1 ? my_count - (pair_max - 1) : 0u);
+  const int32_t lim1 = static_cast<int32_t>(my_count > max_adv - 1 ? my_count - (max_adv - 1) : 0u);
   uint32_t base = 0;                                // first row not yet written out
   for (;;) {
-    const int32_t lim = min(lim2, static_cast<int32_t>(base + RING - kPair));   // rows
+    const int32_t lim = min(lim2, static_cast<int32_t>(base + RING - pair_max));   // rows
     if (STAGED && park_abs != 0u) {
       uint32_t sp = stage_abs + idx * 4u;
       pair_steps<ES>(st, tbm, bitpos, w0, w1, w2, sp, (lim - 1) * RB, tab_abs, ring_lane_abs, park_abs);
@@ -623,7 +625,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
   uint8_t* ring = sm + (ring_abs - sm_abs);
   uint8_t* stage = sm + (stage_abs - sm_abs);
   const uint32_t bar = bars_abs + warp * 8u;
-  __shared__ uint32_t s_dom;
+  __shared__ uint32_t s_dom, s_maxadv;
   uint32_t parity = 0;
   // Interleaved container: bulk asynchronous stores save instructions but make a warp wait for
   // the copy engine now and then; that pays when many warps share the SM (large CTAs), not when
@@ -677,7 +679,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
               "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
               :: "r"(stage_abs), "l"(L.d_stream + it.off0), "r"(bytes), "r"(bar) : "memory");
         }
-        if (lane < kStagePad / 4u) reinterpret_cast<uint32_t*>(stage + it.extent)[lane] = 0u;
+        for (uint32_t i = lane; i < kStagePad / 4u; i += 32u) reinterpret_cast<uint32_t*>(stage + it.extent)[i] = 0u;
       }
       return staged;
     };
@@ -709,19 +711,24 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
         if (threadIdx.x == 0) {
           const uint32_t d = hdr->dominant;
           s_dom = d < 256u ? d : 0u;                      // the ring's fill symbol
+          s_maxadv = 1u;
           if (hdr->magic != kTableMagic || hdr->table_log != uint32_t(R) || hdr->alphabet > (1u << L.bitwidth))
             bad |= ANS_STATUS_BAD_SYMBOL;
         }
         __syncthreads();
       }
+      uint32_t longest = 0;
 #pragma unroll
       for (uint32_t k = 0; k < kStageBatch; ++k) {
         const uint32_t i = b0 + k * blockDim.x + threadIdx.x;
         if (i < n_states) {
           tab[i] = to_smem_entry(g[k], vals[entry_sym(g[k])], 32u * static_cast<uint32_t>(es));
           if (kPrivate) succ[i] = static_cast<uint16_t>(entry_newx(g1[k]));
+          longest = max(longest, entry_run(g[k]) + 1u);
         }
       }
+      longest = __reduce_max_sync(kFull, longest);
+      if (lane == 0 && longest > 1u) atomicMax(&s_maxadv, longest);
     }
     if (threadIdx.x == 0 && kPrivate && R <= kMaxParkLog)
       tab[n_states] = make_uint2(n_states << 17, es == 4 ? vals[s_dom] : (vals[s_dom] & 0xFFFFu));
@@ -774,7 +781,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
 #define ANSB_CALL(ES_, ST_)                                                                              \
   wbad |= decode_private<ES_, ST_>(tab_abs, succ_abs, ring_abs, stage_abs, park_abs, ring, dom, words,     \
                                    ext_words, wbeg, wend, lane == 31, state, my_count, rows, min_count, \
-                                   out_row0, rsb, lane)
+                                   out_row0, rsb, lane, s_maxadv)
         if (staged) {
           if (es == 1) ANSB_CALL(1, true); else if (es == 2) ANSB_CALL(2, true); else ANSB_CALL(4, true);
         } else {
