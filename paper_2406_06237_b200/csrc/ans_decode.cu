@@ -30,6 +30,7 @@ struct LaunchArgs {
   uint8_t* d_symbols_override;     // ans_decode_layer: write symbols here instead of d_out
   uint32_t table_words;            // shared-memory words reserved for the table
   uint32_t stage_bytes;            // private layout: per-warp staging buffer for compressed bytes
+  uint32_t rep_log;                // log2 of the table copies in shared memory (1, 2, 4, 8 or 16 copies)
   uint32_t succ_bytes;             // private layout: shared-memory bytes of the successor table
   uint32_t ring_bytes;             // private layout: per-warp output ring (kRingRows rows of the widest dtype)
   uint32_t n_begin;                // entries of layer_begin in use (0: search the descriptors instead)
@@ -212,7 +213,7 @@ constexpr int kPairsPerCall = 32;
   "shf.l.wrap.b32 m, 0, -1, ea;\n\t"                              \
   "shr.u32 nx, ea, 17;\n\t"                                       \
   "lop3.b32 t, nx, x, m, 0xF4;\n\t"                               \
-  "mad.lo.u32 stx, t, 8, %8;\n\t"                                 \
+  "mad.lo.u32 stx, t, %13, %8;\n\t"                               \
   ADV_                                                            \
   "lop3.b32 a, %1, %11, %9, 0xEA;\n\t"                            \
   "@p " STOP_ " [a], eb;\n\t"                                     \
@@ -224,7 +225,8 @@ constexpr int kPairsPerCall = 32;
 template <int ES>
 __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t& bitpos, uint32_t& w0,
                                            uint32_t& w1, uint32_t& w2, uint32_t& sp, int32_t limm,
-                                           uint32_t tab_abs, uint32_t ring_lane_abs, uint32_t park_abs) {
+                                           uint32_t tab_abs, uint32_t ring_lane_abs, uint32_t park_abs,
+                                           uint32_t stride) {
   constexpr uint32_t MASK = kRingRows * 32u * ES - 1u;
 #define ANSB_ONE_PAIR(ADV_, STOP_)                                                         \
       "setp.lt.s32 p, %1, %7;\n\t"                                                         \
@@ -262,7 +264,7 @@ __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t
       "}"                                                                                  \
       : "+r"(st), "+r"(tbm), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp)          \
       : "r"(limm), "r"(tab_abs), "r"(ring_lane_abs), "r"(park_abs), "n"(MASK),             \
-        "n"(kPairsPerCall / 2)                                                             \
+        "n"(kPairsPerCall / 2), "r"(stride)                                                \
       : "memory")
   if (ES == 1) ANSB_PAIRS(ANSB_ADV_NARROW, "st.shared.u8");
   if (ES == 2) ANSB_PAIRS(ANSB_ADV_NARROW, "st.shared.u16");
@@ -272,14 +274,15 @@ __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t
 }
 
 // Decode one sub-stream.  Shared memory is addressed by absolute shared-window addresses:
-// tab_abs (table), succ_abs (u16 successor of every zero-bit state), ring_abs (this warp's ring,
+// tab_abs (this lane's copy of the table; entries are 1 << stride_log bytes apart), succ_abs (u16
+// successor of every zero-bit state), ring_abs (this warp's ring,
 // aligned to its size), stage_abs (staged sub-stream when STAGED, with kStagePad readable bytes
 // after it).  `ring` is the generic pointer to the same ring; `words` the sub-stream in
 // global memory, used when it was not staged.
 template <int ES, bool STAGED>
 __device__ __noinline__ uint32_t decode_private(
-    uint32_t tab_abs, uint32_t succ_abs, uint32_t ring_abs, uint32_t stage_abs, uint32_t park_abs,
-    uint8_t* __restrict__ ring, uint32_t dom_val,
+    uint32_t tab_abs, uint32_t stride_log, uint32_t succ_abs, uint32_t ring_abs, uint32_t stage_abs,
+    uint32_t park_abs, uint8_t* __restrict__ ring, uint32_t dom_val,
     const uint32_t* __restrict__ words, uint32_t ext_words, uint32_t wbeg, uint32_t wend, bool last_lane,
     uint32_t state, uint32_t my_count, uint32_t rows, uint32_t min_count, uint8_t* __restrict__ out_row0,
     size_t row_stride_bytes, uint32_t lane, uint32_t max_adv) {
@@ -354,13 +357,13 @@ __device__ __noinline__ uint32_t decode_private(
     __syncwarp();
   };
 
-  uint32_t st = tab_abs + state * 8u;               // shared address of the state's table entry
+  uint32_t st = tab_abs + (state << stride_log);    // shared address of the state's table entry
   uint32_t tbm = static_cast<uint32_t>(-RB);        // RB * (last row this lane wrote): none yet
   // one pre-walked look-up: emits run + 1 symbols, takes its bits from the low end of x
   auto step = [&](uint32_t x) -> uint32_t {
     const uint32_t ea = lds_u32(st), eb = lds_u32(st + 4u);
     const uint32_t nb = ea & 15u;
-    st = tab_abs + (((ea >> 17) | (x & ((1u << nb) - 1u))) << 3);
+    st = tab_abs + (((ea >> 17) | (x & ((1u << nb) - 1u))) << stride_log);
     tbm += ((ea >> 6) & 31u) * RB;
     sts_elem<ES>((tbm & MASK) | ring_lane_abs, eb);
     return nb;
@@ -386,7 +389,8 @@ __device__ __noinline__ uint32_t decode_private(
     const int32_t lim = min(lim2, static_cast<int32_t>(base + RING - pair_max));   // rows
     if (STAGED && park_abs != 0u) {
       uint32_t sp = stage_abs + idx * 4u;
-      pair_steps<ES>(st, tbm, bitpos, w0, w1, w2, sp, (lim - 1) * RB, tab_abs, ring_lane_abs, park_abs);
+      pair_steps<ES>(st, tbm, bitpos, w0, w1, w2, sp, (lim - 1) * RB, tab_abs, ring_lane_abs, park_abs,
+                     1u << stride_log);
       idx = (sp - stage_abs) >> 2;
       if (idx > word_limit) { overran = true; idx = word_limit; }
     } else {
@@ -422,11 +426,11 @@ __device__ __noinline__ uint32_t decode_private(
       bitpos += step(__funnelshift_r(w0, w1, bitpos));
       refill_checked();
     } else {
-      st = tab_abs + lds_u16(succ_abs + ((st - tab_abs) >> 2)) * 8u;
+      st = tab_abs + (lds_u16(succ_abs + (((st - tab_abs) >> stride_log) << 1)) << stride_log);
       tbm += RB;
     }
   }
-  state = (st - tab_abs) >> 3;
+  state = (st - tab_abs) >> stride_log;
   __syncwarp();
   {
     const bool has_part = min_count < rows;         // last row is ragged
@@ -456,7 +460,7 @@ __device__ __noinline__ uint32_t decode_private(
 template <int ES>
 __device__ __forceinline__ void interleaved_rounds(uint32_t& st, uint32_t& buf, uint32_t& cnt, uint32_t& posaddr,
                                                    uint32_t& rb, uint32_t n, uint32_t lt, uint32_t limaddr,
-                                                   uint32_t tab_abs, uint32_t ring_lane_abs) {
+                                                   uint32_t tab_abs, uint32_t ring_lane_abs, uint32_t stride) {
   constexpr uint32_t RB = 32u * ES;
   constexpr uint32_t MASK = kRingRows * RB - 1u;
 #define ANSB_ROUNDS(STOP_)                                                                 \
@@ -484,7 +488,7 @@ __device__ __forceinline__ void interleaved_rounds(uint32_t& st, uint32_t& buf, 
       "shf.l.wrap.b32 m, 0, -1, ea;\n\t"                                                   \
       "shr.u32 nx, ea, 17;\n\t"                                                            \
       "lop3.b32 t, nx, %1, m, 0xF4;\n\t"                                                   \
-      "mad.lo.u32 %0, t, 8, %8;\n\t"                                                       \
+      "mad.lo.u32 %0, t, %12, %8;\n\t"                                                     \
       "shf.r.wrap.b32 %1, %1, 0, ea;\n\t"                                                  \
       "and.b32 t, ea, 15;\n\t"                                                             \
       "sub.u32 %2, %2, t;\n\t"                                                             \
@@ -496,7 +500,8 @@ __device__ __forceinline__ void interleaved_rounds(uint32_t& st, uint32_t& buf, 
       "@q bra ANSB_RLOOP;\n\t"                                                             \
       "}"                                                                                  \
       : "+r"(st), "+r"(buf), "+r"(cnt), "+r"(posaddr), "+r"(rb)                            \
-      : "r"(n), "r"(lt), "r"(limaddr), "r"(tab_abs), "r"(ring_lane_abs), "n"(RB), "n"(MASK) \
+      : "r"(n), "r"(lt), "r"(limaddr), "r"(tab_abs), "r"(ring_lane_abs), "n"(RB), "n"(MASK), \
+        "r"(stride)                                                                        \
       : "memory")
   if (ES == 1) ANSB_ROUNDS("st.shared.u8");
   if (ES == 2) ANSB_ROUNDS("st.shared.u16");
@@ -506,7 +511,7 @@ __device__ __forceinline__ void interleaved_rounds(uint32_t& st, uint32_t& buf, 
 
 template <int ES, bool STAGED>
 __device__ __noinline__ uint32_t decode_interleaved(
-    uint32_t tab_abs, uint32_t ring_abs, uint32_t stage_abs, uint8_t* __restrict__ ring,
+    uint32_t tab_abs, uint32_t stride_log, uint32_t ring_abs, uint32_t stage_abs, uint8_t* __restrict__ ring,
     const uint16_t* __restrict__ units, uint32_t unit_cap, uint32_t state, uint32_t my_count, uint32_t rows,
     uint32_t min_count, uint8_t* __restrict__ out_row0, size_t row_stride_bytes, uint32_t lane, bool allow_bulk) {
   constexpr uint32_t RB = 32u * ES;
@@ -514,7 +519,7 @@ __device__ __noinline__ uint32_t decode_interleaved(
   constexpr uint32_t MASK = RING * RB - 1u;
   const uint32_t ring_lane_abs = ring_abs + lane * ES;
   const uint32_t lt = (1u << lane) - 1u;
-  uint32_t st = tab_abs + state * 8u;               // shared address of the state's table entry
+  uint32_t st = tab_abs + (state << stride_log);    // shared address of the state's table entry
   uint32_t buf = 0, cnt = 0;                        // the lane's bit buffer and how many bits it holds
   uint32_t pos = 0;                                 // units the warp has taken (same in every lane)
   uint32_t rb = 0;                                  // RB * round
@@ -535,7 +540,7 @@ __device__ __noinline__ uint32_t decode_interleaved(
     if (active) {
       const uint32_t ea = lds_u32(st), eb = lds_u32(st + 4u);
       const uint32_t nb = ea & 15u;
-      st = tab_abs + (((ea >> 17) | (buf & ((1u << nb) - 1u))) << 3);
+      st = tab_abs + (((ea >> 17) | (buf & ((1u << nb) - 1u))) << stride_log);
       buf >>= nb;
       cnt -= nb;
       sts_elem<ES>((rb & MASK) | ring_lane_abs, eb);
@@ -577,7 +582,8 @@ __device__ __noinline__ uint32_t decode_interleaved(
     const uint32_t n = min(FL - (r % FL), min_count - r);
     if (STAGED) {
       uint32_t posaddr = stage_abs + pos * 2u;
-      interleaved_rounds<ES>(st, buf, cnt, posaddr, rb, n, lt, stage_abs + unit_cap * 2u, tab_abs, ring_lane_abs);
+      interleaved_rounds<ES>(st, buf, cnt, posaddr, rb, n, lt, stage_abs + unit_cap * 2u, tab_abs, ring_lane_abs,
+                             1u << stride_log);
       pos = (posaddr - stage_abs) >> 1;
     } else {
       for (uint32_t i = 0; i < n; ++i) round(true);
@@ -614,12 +620,18 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
   const uint32_t sm_abs = smem_u32(sm);
   const uint32_t rings_abs = (sm_abs + args.ring_bytes - 1u) & ~(args.ring_bytes - 1u);
   const uint32_t tab_abs = rings_abs + NW * args.ring_bytes;
-  const uint32_t vals_abs = (tab_abs + args.table_words * 4u + 1023u) & ~1023u;
+  const uint32_t vals_abs = (tab_abs + ((args.table_words * 4u) << args.rep_log) + 1023u) & ~1023u;
   const uint32_t succ_abs = vals_abs + 1024u;             // private: u16 per state, (2 << max R) bytes
   const uint32_t bars_abs = succ_abs + args.succ_bytes;
   const uint32_t ring_abs = rings_abs + warp * args.ring_bytes;
   const uint32_t stage_abs = bars_abs + NW * 8u + warp * args.stage_bytes;
   uint2* tab = reinterpret_cast<uint2*>(sm + (tab_abs - sm_abs));
+  // The table may sit in shared memory in several copies, entry i of copy c at slot i * copies + c.
+  // A 64-bit load is served half a warp at a time over 16 bank pairs; with 16 copies every lane
+  // of a half-warp has a bank pair of its own and random look-ups no longer collide.
+  const uint32_t reps = 1u << args.rep_log;
+  const uint32_t stride_log = 3u + args.rep_log;
+  const uint32_t tab_lane = tab_abs + (lane & (reps - 1u)) * 8u;
   uint32_t* vals = reinterpret_cast<uint32_t*>(sm + (vals_abs - sm_abs));
   uint16_t* succ = reinterpret_cast<uint16_t*>(sm + (succ_abs - sm_abs));
   uint8_t* ring = sm + (ring_abs - sm_abs);
@@ -722,7 +734,8 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
       for (uint32_t k = 0; k < kStageBatch; ++k) {
         const uint32_t i = b0 + k * blockDim.x + threadIdx.x;
         if (i < n_states) {
-          tab[i] = to_smem_entry(g[k], vals[entry_sym(g[k])], 32u * static_cast<uint32_t>(es));
+          const uint2 e = to_smem_entry(g[k], vals[entry_sym(g[k])], 32u * static_cast<uint32_t>(es));
+          for (uint32_t c = 0; c < reps; ++c) tab[(i << args.rep_log) + c] = e;
           if (kPrivate) succ[i] = static_cast<uint16_t>(entry_newx(g1[k]));
           longest = max(longest, entry_run(g[k]) + 1u);
         }
@@ -730,13 +743,14 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
       longest = __reduce_max_sync(kFull, longest);
       if (lane == 0 && longest > 1u) atomicMax(&s_maxadv, longest);
     }
-    if (threadIdx.x == 0 && kPrivate && R <= kMaxParkLog)
-      tab[n_states] = make_uint2(n_states << 17, es == 4 ? vals[s_dom] : (vals[s_dom] & 0xFFFFu));
+    if (threadIdx.x < reps && kPrivate && R <= kMaxParkLog)
+      tab[(n_states << args.rep_log) + threadIdx.x] =
+          make_uint2(n_states << 17, es == 4 ? vals[s_dom] : (vals[s_dom] & 0xFFFFu));
     __syncthreads();
 
     uint8_t* out_base = args.d_symbols_override ? args.d_symbols_override : static_cast<uint8_t*>(L.d_out);
     const uint32_t dom = vals[s_dom];
-    const uint32_t park_abs = R <= kMaxParkLog ? tab_abs + (8u << R) : 0u;
+    const uint32_t park_abs = R <= kMaxParkLog ? tab_lane + ((n_states << stride_log)) : 0u;
     for (uint64_t gbase = cursor; gbase < stop && !gave_up; gbase += NW / kGranule) {
       uint64_t sub;
       if (!warp_sub(gbase, sub)) continue;
@@ -779,7 +793,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
       if (kPrivate) {
         const uint32_t* words = reinterpret_cast<const uint32_t*>(g_bytes);
 #define ANSB_CALL(ES_, ST_)                                                                              \
-  wbad |= decode_private<ES_, ST_>(tab_abs, succ_abs, ring_abs, stage_abs, park_abs, ring, dom, words,     \
+  wbad |= decode_private<ES_, ST_>(tab_lane, stride_log, succ_abs, ring_abs, stage_abs, park_abs, ring, dom, words, \
                                    ext_words, wbeg, wend, lane == 31, state, my_count, rows, min_count, \
                                    out_row0, rsb, lane, s_maxadv)
         if (staged) {
@@ -792,7 +806,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
         const uint16_t* units = reinterpret_cast<const uint16_t*>(g_bytes);
         const uint32_t unit_cap = ext_words * 2u;
 #define ANSB_CALL(ES_, ST_)                                                                              \
-  wbad |= decode_interleaved<ES_, ST_>(tab_abs, ring_abs, stage_abs, ring, units, unit_cap, state, my_count, \
+  wbad |= decode_interleaved<ES_, ST_>(tab_lane, stride_log, ring_abs, stage_abs, ring, units, unit_cap, state, my_count, \
                                        rows, min_count, out_row0, rsb, lane, allow_bulk)
         if (staged) {
           if (es == 1) ANSB_CALL(1, true); else if (es == 2) ANSB_CALL(2, true); else ANSB_CALL(4, true);
@@ -849,7 +863,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   a.total_work = static_cast<uint32_t>(total);
   a.d_status = d_status;
   a.d_symbols_override = d_symbols_override;
-  a.table_words = 2u * ((1u << max_log) + 2u);           // two words per state, and a parking entry
+  a.table_words = 2u * ((1u << max_log) + 2u);           // two words per state, and a parking entry (one copy)
   if (n_layers <= kParamLayers) {
     a.n_begin = static_cast<uint32_t>(n_layers);
     for (int l = 0; l < n_layers; ++l) a.layer_begin[l] = h_descs[l].work_begin;
@@ -896,6 +910,15 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
     a.stage_bytes = static_cast<uint32_t>(stage);
     a.ring_bytes = static_cast<uint32_t>(ring);
     smem = fixed + size_t(warps) * (ring + stage);
+    // Shared memory left over goes to extra copies of the table (fewer bank conflicts on the
+    // random look-ups; 16 copies make them conflict-free).  Small CTAs must stay small enough
+    // for three of them to share an SM.
+    const size_t one_table = size_t(a.table_words) * 4;
+    const size_t cap = big ? size_t(smem_max) : size_t(74) << 10;
+    while (a.rep_log < 4 && smem + (one_table << a.rep_log) <= cap) {
+      smem += one_table << a.rep_log;                     // doubling the copies adds as many again
+      ++a.rep_log;
+    }
   }
   {
     LaunchShape& shape = facts.shape[priv ? 1 : 0];
