@@ -34,8 +34,9 @@ FALLBACK_PEAK_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, scaled from the 2-matrix captures in
 # profiles/ans_decode_kernel_*_large.md to the 8 matrices of a full launch
-NCU_TRAFFIC = {("large", "private", 32, 8, 8192, 0, 0): 932.3e6,
-               ("large", "interleaved", 32, 8, 8192, 0, 0): 931.8e6}
+NCU_TRAFFIC = {("large", "private", 32, 8, 8192, 0, 0): 937.0e6,      # 256-state table (the default)
+               ("large", "private", 32, 8, 8192, 0, 12): 932.3e6,
+               ("large", "interleaved", 32, 8, 8192, 0, 12): 931.8e6}
 
 
 def measured_peak():
@@ -53,7 +54,7 @@ def make_specs(args):
         return sg.workload_sweep(table_log=args.table_log or 12, chunk=args.chunk or 16384, n=args.symbols)
     if args.workload == "large":
         return sg.workload_large(n_mats=args.mats, dim=args.dim, chunk=args.chunk or 32768,
-                                 table_log=args.table_log or 12)
+                                 table_log=args.table_log or 8)
     if args.workload in ("resnet18", "resnet50"):
         return sg.WORKLOADS[args.workload](table_log=args.table_log or 12, chunk=args.chunk or 16384)
     return sg.workload_conv3x3()
@@ -64,7 +65,8 @@ WORKLOAD_TEXT = {
     "resnet18": "ResNet-18 conv weights (20 layers, 11.2M), bitwidth {2,3,4,6}, 0.8-1.5 bit/weight, 16K chunks, bf16",
     "resnet50": "ResNet-50 conv weights (53 layers, 23.5M), 1-8 bit mixed precision, P(zp) 0.85-0.95, 16K chunks, bf16",
     "sweep": "256M 8-bit symbols, two-sided geometric (2.5 bit), decode-only to uint8",
-    "large": "large dense layers: 8 matrices of 8192x8192 (537M weights), 3-bit zero-point, P(zp)=0.7, 32K chunks, bf16",
+    "large": "large dense layers: 8 matrices of 8192x8192 (537M weights), 3-bit zero-point, P(zp)=0.7, 32K chunks, bf16 "
+             "(256-state table, the paper's coder size, unless --table-log says otherwise)",
 }
 
 
@@ -291,7 +293,8 @@ def run_ours(args):
     # algorithmic bytes of one launch: everything compressed read once, each layer's table
     # once, every decoded element written once
     table_read = sum(4 << L.table_log for L in layers)
-    algo_bytes = db.compressed_bytes() + table_read + out_bytes
+    comp_bytes = db.compressed_bytes()
+    algo_bytes = comp_bytes + table_read + out_bytes
     peak, peak_kind = measured_peak()
     kernel_ms = statistics.mean(ms)
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
@@ -312,6 +315,25 @@ def run_ours(args):
     if not args.no_e2e:
         e2e = run_e2e(ans, db, layers, args, world)
 
+    # the same workload with the other table size the design notes quote (2^12 states)
+    variants = []
+    if args.workload == "large" and not args.table_log and world == 1 and not args.no_variants:
+        db = None
+        torch.cuda.empty_cache()
+        with ThreadPoolExecutor(4) as ex:
+            layers12 = list(ex.map(lambda sp_sy: pack_layer(sp_sy[1], sp_sy[0].alphabet, 12, sp_sy[0].chunk_symbols,
+                                                            args.lanes, layout, sp_sy[0].bitwidth, sp_sy[0].zero_point,
+                                                            sp_sy[0].scale, ans.DTYPES[sp_sy[0].out_dtype],
+                                                            n_threads=max(1, cores // 2)), zip(specs, syms)))
+        db12 = DeviceBatch(layers12, f"cuda:{local}", n_out_sets=1)
+        ms12, _ = time_workload(db12, min(args.steps, 50), 5, None, 1, 1)
+        bytes12 = db12.compressed_bytes() + sum(4 << 12 for _ in layers12) + out_bytes
+        k12 = statistics.mean(ms12)
+        variants.append({"table_log": 12, "kernel_ms_mean": k12, "value": n_w / (k12 * 1e-3), "unit": "weights/s",
+                         "achieved_gbs": bytes12 / (k12 * 1e-3) / 1e9, "frac": bytes12 / (k12 * 1e-3) / 1e9 / peak,
+                         "coded_bits_per_weight": 8.0 * db12.compressed_bytes() / n_w})
+        del db12
+
     if rank != 0:
         return
     hist = np.zeros(256, dtype=np.float64)
@@ -320,7 +342,7 @@ def run_ours(args):
         c = np.bincount(sym, minlength=256).astype(np.float64)
         p = c[c > 0] / max(1, sym.size)
         ent_bits += float(-(p * np.log2(p)).sum()) * sym.size
-    coded_bits = 8.0 * db.compressed_bytes()
+    coded_bits = 8.0 * comp_bytes
     cpu = cpu_baseline(specs, syms, args.layout) if world == 1 and not args.no_cpu_baseline else None
     out = {
         "metric": METRIC, "value": value, "unit": "weights/s", "n_gpus": world, "steps": args.steps,
@@ -334,9 +356,10 @@ def run_ours(args):
                                  if small else "working set (compressed + output) is larger than L2"),
                    "per_gpu": "every rank decodes its own replica of the workload; no collective on the data path"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "roofline": roofline, "cpu_baseline": cpu,
+        "variants": variants,
         "compression": {"coded_bits_per_weight": coded_bits / max(1, n_w), "entropy_bits_per_weight": ent_bits / max(1, n_w),
                         "gap_bits_per_weight": (coded_bits - ent_bits) / max(1, n_w),
-                        "compressed_bytes": db.compressed_bytes(), "output_bytes": out_bytes},
+                        "compressed_bytes": comp_bytes, "output_bytes": out_bytes},
         "setup_s": setup_s,
     }
     print(json.dumps(out))
@@ -402,6 +425,7 @@ def main():
     ap.add_argument("--symbols", type=int, default=1 << 28, help="sweep workload: number of symbols (2^28 = full size)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-variants", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

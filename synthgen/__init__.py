@@ -255,7 +255,9 @@ def workload_sweep(seed: int = 3, table_log: int = 12, chunk: int = 16384,
 
 
 def workload_large(seed: int = 4, n_mats: int = 8, dim: int = 8192, chunk: int = 32768,
-                   table_log: int = 12) -> list[LayerSpec]:
+                   table_log: int = 8) -> list[LayerSpec]:
+    """8 dense matrices, 7 bins.  The workload's description fixes no table size, so the paper's
+    own 256-state coder (Section III-A) is the default; 2^12 states is the other measured case."""
     A, zp = alphabet_for_bits(3)
     th = theta_for_pzp(A, zp, 0.7)
     return [LayerSpec(f"dense{m}", (dim, dim), 3, A, zp, th, 0.05, table_log, chunk, "bf16",

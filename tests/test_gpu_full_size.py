@@ -45,8 +45,9 @@ def full_size(specs, layout, lanes, sample_chunks=64):
 
 
 @pytest.mark.parametrize("layout", [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE])
-def test_config5_large_layers_full(layout):
-    full_size(sg.workload_large(), layout, 32)
+@pytest.mark.parametrize("table_log", [8, 12])
+def test_config5_large_layers_full(layout, table_log):
+    full_size(sg.workload_large(table_log=table_log), layout, 32)
 
 
 @pytest.mark.parametrize("layout", [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE])
