@@ -19,6 +19,7 @@ constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr uint32_t kStatusTimeout = 8u;   // a bounded wait on an asynchronous copy ran out
 
 constexpr int kParamLayers = 96;
+constexpr int kLockstepMaxLog = 9;        // private container: largest table walked one symbol per look-up
 
 struct LaunchArgs {
   const ans_layer_desc* d_descs;   // device array, or nullptr when `one` is the only layer
@@ -33,6 +34,7 @@ struct LaunchArgs {
   uint32_t rep_log;                // log2 of the table copies in shared memory (1, 2, 4, 8 or 16 copies)
   uint32_t succ_bytes;             // private layout: shared-memory bytes of the successor table
   uint32_t ring_bytes;             // private layout: per-warp output ring (kRingRows rows of the widest dtype)
+  uint32_t unit;                   // the value 1 (a run-time operand keeps a multiply-add a multiply-add)
   uint32_t n_begin;                // entries of layer_begin in use (0: search the descriptors instead)
   uint32_t layer_begin[kParamLayers];   // work_begin of the first layers, searchable without a memory trip
 };
@@ -219,7 +221,7 @@ constexpr int kPairsPerCall = 32;
   "@p " STOP_ " [a], eb;\n\t"                                     \
   "add.u32 %2, %2, ea;\n\t"
 
-#define ANSB_ADV_NARROW "mad.hi.u32 %1, eb, 65536, %1;\n\t"
+#define ANSB_ADV_NARROW "shr.u32 r, eb, 16;\n\tadd.u32 %1, %1, r;\n\t"
 #define ANSB_ADV_WIDE "bfe.u32 r, ea, 6, 5;\n\tmad.lo.u32 %1, r, 128, %1;\n\t"
 
 template <int ES>
@@ -243,7 +245,7 @@ __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t
       "@q mov.u32 %4, %5;\n\t"                                                             \
       "@q ld.shared.u32 nw, [%6];\n\t"                                                     \
       "@q mov.u32 %5, nw;\n\t"                                                             \
-      "mad.hi.u32 %6, t, 0x20000000, %6;\n\t"
+      "@q add.u32 %6, %6, 4;\n\t"
 #define ANSB_PAIRS(ADV_, STOP_)                                                            \
   asm volatile(                                                                            \
       "{\n\t"                                                                              \
@@ -451,6 +453,173 @@ __device__ __noinline__ uint32_t decode_private(
 }
 
 // =============================================================================================
+// Private container, lockstep walk: every look-up emits exactly one symbol (the plain table of
+// Section II-A), so the 32 lanes of a warp stay on the same output row.  A row is complete as
+// soon as it is decoded and each lane stores its element straight to the output: a row is
+// 32 * ES contiguous bytes, whole 32-byte sectors; no ring, no pre-fill, no parking, no tail.
+// The price is one look-up per symbol, which pays when look-ups are cheap (a table small enough
+// for conflict-free copies) or the pre-walked entries would stand for few symbols anyway.
+//
+// kFlushRows rows are decoded by one PTX block (row stores at immediate offsets), K look-ups
+// sharing one 32-bit extract of the bit window and one refill check: K = 4 when a symbol takes
+// at most 8 bits, else 2.  Multiply-high is avoided on purpose (it runs at a fraction of the
+// rate of shifts and adds); the bit count is accumulated on the multiply-add pipe, which is
+// otherwise idle, by a multiplication with a run-time 1.
+// =============================================================================================
+#define ANSB_LS_STEP(STOP_, ADDR_)                                \
+  "ld.shared.v2.u32 {ea, eb}, [%0];\n\t"                          \
+  "shf.l.wrap.b32 m, 0, -1, ea;\n\t"                              \
+  "shr.u32 nx, ea, 17;\n\t"                                       \
+  "lop3.b32 t, nx, x, m, 0xF4;\n\t"                               \
+  "mad.lo.u32 %0, t, %7, %6;\n\t"                                 \
+  "shf.r.wrap.b32 x, x, 0, ea;\n\t"                               \
+  STOP_ " " ADDR_ ", eb;\n\t"                                     \
+  "mad.lo.u32 %1, ea, %9, %1;\n\t"
+#define ANSB_LS_BEGIN "shf.r.wrap.b32 x, %2, %3, %1;\n\t"
+#define ANSB_LS_END                                               \
+  "and.b32 t, %1, 32;\n\t"                                        \
+  "setp.ne.u32 q, t, 0;\n\t"                                      \
+  "@q mov.u32 %2, %3;\n\t"                                        \
+  "@q mov.u32 %3, %4;\n\t"                                        \
+  "@q ld.shared.u32 nw, [%5];\n\t"                                \
+  "@q mov.u32 %4, nw;\n\t"                                        \
+  "@q add.u32 %5, %5, 4;\n\t"                                     \
+  "and.b32 %1, %1, 31;\n\t"
+#define ANSB_LS_G4(S_, A0, A1, A2, A3)                            \
+  ANSB_LS_BEGIN ANSB_LS_STEP(S_, A0) ANSB_LS_STEP(S_, A1) ANSB_LS_STEP(S_, A2) ANSB_LS_STEP(S_, A3) ANSB_LS_END
+#define ANSB_LS_G2(S_, A0, A1) ANSB_LS_BEGIN ANSB_LS_STEP(S_, A0) ANSB_LS_STEP(S_, A1) ANSB_LS_END
+
+// st: shared address of the state's entry; bitpos in [0, 32); w0,w1: bit window, w2 the word after
+// it; sp: shared address of the word after w2; gp: this lane's element of the block's first row
+// in the output (rows are 32 * ES * G bytes apart); one: the value 1, not known at compile time
+template <int ES, int K, int G>
+__device__ __forceinline__ void lockstep_block(uint32_t& st, uint32_t& bitpos, uint32_t& w0, uint32_t& w1,
+                                               uint32_t& w2, uint32_t& sp, uint32_t tab_lane, uint32_t stride,
+                                               uint8_t* gp, uint32_t one) {
+  constexpr uint32_t RS = 32u * ES * G;
+  static_assert(kFlushRows == 16, "the block below is written out for 16 rows");
+#define ANSB_LS_BODY4(S_)                                                                   \
+      ANSB_LS_G4(S_, "[%8]", "[%8+%10]", "[%8+%11]", "[%8+%12]")                            \
+      ANSB_LS_G4(S_, "[%8+%13]", "[%8+%14]", "[%8+%15]", "[%8+%16]")                        \
+      ANSB_LS_G4(S_, "[%8+%17]", "[%8+%18]", "[%8+%19]", "[%8+%20]")                        \
+      ANSB_LS_G4(S_, "[%8+%21]", "[%8+%22]", "[%8+%23]", "[%8+%24]")
+#define ANSB_LS_BODY2(S_)                                                                   \
+      ANSB_LS_G2(S_, "[%8]", "[%8+%10]") ANSB_LS_G2(S_, "[%8+%11]", "[%8+%12]")             \
+      ANSB_LS_G2(S_, "[%8+%13]", "[%8+%14]") ANSB_LS_G2(S_, "[%8+%15]", "[%8+%16]")         \
+      ANSB_LS_G2(S_, "[%8+%17]", "[%8+%18]") ANSB_LS_G2(S_, "[%8+%19]", "[%8+%20]")         \
+      ANSB_LS_G2(S_, "[%8+%21]", "[%8+%22]") ANSB_LS_G2(S_, "[%8+%23]", "[%8+%24]")
+#define ANSB_LS_ASM(BODY_)                                                                  \
+  asm volatile(                                                                             \
+      "{\n\t"                                                                               \
+      ".reg .pred q;\n\t"                                                                   \
+      ".reg .u32 x, ea, eb, m, t, nx, nw;\n\t"                                              \
+      BODY_                                                                                 \
+      "}"                                                                                   \
+      : "+r"(st), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp)                      \
+      : "r"(tab_lane), "r"(stride), "l"(gp), "r"(one), "n"(RS * 1), "n"(RS * 2), "n"(RS * 3), \
+        "n"(RS * 4), "n"(RS * 5), "n"(RS * 6), "n"(RS * 7), "n"(RS * 8), "n"(RS * 9), "n"(RS * 10), \
+        "n"(RS * 11), "n"(RS * 12), "n"(RS * 13), "n"(RS * 14), "n"(RS * 15)                \
+      : "memory")
+  if (K == 4) {
+    if (ES == 1) ANSB_LS_ASM(ANSB_LS_BODY4("st.global.u8"));
+    if (ES == 2) ANSB_LS_ASM(ANSB_LS_BODY4("st.global.u16"));
+    if (ES == 4) ANSB_LS_ASM(ANSB_LS_BODY4("st.global.u32"));
+  } else {
+    if (ES == 1) ANSB_LS_ASM(ANSB_LS_BODY2("st.global.u8"));
+    if (ES == 2) ANSB_LS_ASM(ANSB_LS_BODY2("st.global.u16"));
+    if (ES == 4) ANSB_LS_ASM(ANSB_LS_BODY2("st.global.u32"));
+  }
+#undef ANSB_LS_ASM
+#undef ANSB_LS_BODY2
+#undef ANSB_LS_BODY4
+}
+
+template <int ES>
+__device__ __forceinline__ void stg_elem(uint8_t* p, uint32_t v) {
+  if (ES == 1) *p = static_cast<uint8_t>(v);
+  if (ES == 2) *reinterpret_cast<uint16_t*>(p) = static_cast<uint16_t>(v);
+  if (ES == 4) *reinterpret_cast<uint32_t*>(p) = v;
+}
+
+// Decode one sub-stream in lockstep.  tab_abs: this lane's copy of the plain table; stage_abs: the
+// staged sub-stream when STAGED; words: the sub-stream in global memory otherwise; rows of one
+// sub-stream are `groups` rows of the chunk apart in the output.
+template <int ES, bool STAGED>
+__device__ __noinline__ uint32_t decode_lockstep(
+    uint32_t tab_abs, uint32_t stride_log, uint32_t stage_abs, const uint32_t* __restrict__ words,
+    uint32_t ext_words, uint32_t wbeg, uint32_t wend, bool last_lane, uint32_t state, uint32_t my_count,
+    uint32_t rows, uint32_t min_count, uint8_t* __restrict__ out_row0, uint32_t groups, uint32_t lane,
+    bool wide_steps, uint32_t one) {
+  constexpr uint32_t RB = 32u * ES;
+  constexpr uint32_t FL = kFlushRows;
+  const size_t row_stride_bytes = size_t(RB) * groups;
+  // a staged lane may look up to word_limit + 8 words into its buffer (a block advances it by at
+  // most 8 words), which holds ext_words + kStagePad / 4
+  const uint32_t word_limit = STAGED ? ext_words + 4u : ext_words;
+  auto load_word = [&](uint32_t i) -> uint32_t {
+    if (STAGED) return lds_u32(stage_abs + i * 4u);
+    return i < word_limit ? __ldg(words + i) : 0u;
+  };
+  uint32_t idx = wbeg;
+  uint32_t w0 = load_word(idx), w1 = load_word(idx + 1), w2 = load_word(idx + 2);
+  idx += 3;
+  uint32_t bitpos = 0;
+  bool overran = false;
+  uint32_t st = tab_abs + (state << stride_log);
+  uint8_t* gp = out_row0 + size_t(lane) * ES;       // this lane's element of the next row
+
+  // one look-up in plain code: rows outside whole blocks, and sub-streams that were not staged
+  auto step = [&]() {
+    const uint32_t ea = lds_u32(st), eb = lds_u32(st + 4u);
+    const uint32_t nb = ea & 15u;
+    const uint32_t x = __funnelshift_r(w0, w1, bitpos);
+    st = tab_abs + (((ea >> 17) | (x & ((1u << nb) - 1u))) << stride_log);
+    stg_elem<ES>(gp, eb);
+    gp += row_stride_bytes;
+    bitpos += nb;
+    if (bitpos >= 32u) {
+      w0 = w1; w1 = w2;
+      w2 = (!STAGED || idx < word_limit) ? load_word(idx) : 0u;
+      ++idx;
+      bitpos -= 32u;
+    }
+  };
+
+  uint32_t r = 0;
+  if (STAGED) {
+    uint32_t sp = stage_abs + idx * 4u;
+    const uint32_t sp_limit = stage_abs + word_limit * 4u;
+    const uint32_t stride = 1u << stride_log;
+#define ANSB_LS_LOOP(K_, G_)                                                                \
+    while (r + FL <= min_count) {                                                           \
+      lockstep_block<ES, K_, G_>(st, bitpos, w0, w1, w2, sp, tab_abs, stride, gp, one);     \
+      if (sp > sp_limit) { overran = true; sp = sp_limit; }                                 \
+      gp += FL * RB * G_;                                                                   \
+      r += FL;                                                                              \
+    }
+    if (wide_steps) {
+      if (groups == 1) { ANSB_LS_LOOP(4, 1) } else if (groups == 2) { ANSB_LS_LOOP(4, 2) }
+      else if (groups == 4) { ANSB_LS_LOOP(4, 4) } else if (groups == 8) { ANSB_LS_LOOP(4, 8) }
+    } else {
+      if (groups == 1) { ANSB_LS_LOOP(2, 1) } else if (groups == 2) { ANSB_LS_LOOP(2, 2) }
+      else if (groups == 4) { ANSB_LS_LOOP(2, 4) } else if (groups == 8) { ANSB_LS_LOOP(2, 8) }
+    }
+#undef ANSB_LS_LOOP
+    idx = (sp - stage_abs) >> 2;
+  }
+  for (; r < min_count; ++r) step();
+  if (rows > min_count && my_count == rows) step();   // the ragged last row
+  uint32_t bad = 0;
+  if (st != tab_abs) bad |= ANS_STATUS_BAD_FINAL_STATE;
+  // words used must be exactly the lane's run (the last lane's run is followed by < 16 pad bytes)
+  const uint32_t bits = (idx - 3u - wbeg) * 32u + bitpos;
+  const uint32_t need = (bits + 31u) / 32u;
+  const uint32_t have = wend - wbeg;
+  if (overran || (last_lane ? (need > have || have - need >= 4u) : (need != have))) bad |= ANS_STATUS_BAD_LENGTH;
+  return bad;
+}
+
+// =============================================================================================
 // Interleaved container: the warp's 32 lanes share one sequence of 16-bit units; before each
 // round a lane whose buffer holds fewer than 16 bits takes the next unit, its place found by
 // ballot + popcount; then every lane decodes one symbol.  Same shared-memory table, staging
@@ -611,14 +780,16 @@ __device__ __noinline__ uint32_t decode_interleaved(
 // dynamic shared memory, by absolute shared address: [pad to ring_bytes][rings: NW * ring_bytes]
 // [table][pad to 1 KB][vals 256 words][mbarriers NW][stages NW * stage_bytes]
 
-template <int LAYOUT>
-__global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs args) {
+template <int LAYOUT, bool LOCK>
+__global__ void __launch_bounds__(LOCK ? 1024 : 512, 1) ans_decode_kernel(const LaunchArgs args) {
   constexpr bool kPrivate = LAYOUT == ANS_LAYOUT_PRIVATE;
+  constexpr bool lock = kPrivate && LOCK;           // private container walked one symbol per look-up
   extern __shared__ __align__(16) uint8_t sm[];
   const uint32_t NW = blockDim.x >> 5;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   const uint32_t sm_abs = smem_u32(sm);
-  const uint32_t rings_abs = (sm_abs + args.ring_bytes - 1u) & ~(args.ring_bytes - 1u);
+  const uint32_t ring_align = args.ring_bytes ? args.ring_bytes : 16u;
+  const uint32_t rings_abs = (sm_abs + ring_align - 1u) & ~(ring_align - 1u);
   const uint32_t tab_abs = rings_abs + NW * args.ring_bytes;
   const uint32_t vals_abs = (tab_abs + ((args.table_words * 4u) << args.rep_log) + 1023u) & ~1023u;
   const uint32_t succ_abs = vals_abs + 1024u;             // private: u16 per state, (2 << max R) bytes
@@ -666,7 +837,8 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
     const TableHeader* hdr = reinterpret_cast<const TableHeader*>(blob);
     const uint32_t* g_single = reinterpret_cast<const uint32_t*>(blob + single_offset());
     // private: the pre-walked entries; interleaved: the plain ones (one symbol per look-up)
-    const uint32_t* g_multi = kPrivate ? reinterpret_cast<const uint32_t*>(blob + multi_offset(R)) : g_single;
+    const uint32_t* g_multi =
+        (kPrivate && !lock) ? reinterpret_cast<const uint32_t*>(blob + multi_offset(R)) : g_single;
     const int dtype = args.d_symbols_override ? ANS_U8 : L.out_dtype;
 
     const size_t es = dtype == ANS_U8 ? 1 : dtype == ANS_F32 ? 4 : 2;
@@ -715,7 +887,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
       for (uint32_t k = 0; k < kStageBatch; ++k) {
         const uint32_t i = b0 + k * blockDim.x + threadIdx.x;
         g[k] = i < n_states ? __ldg(g_multi + i) : 0u;
-        if (kPrivate) g1[k] = i < n_states ? __ldg(g_single + i) : 0u;
+        if (kPrivate && !lock) g1[k] = i < n_states ? __ldg(g_single + i) : 0u;
       }
       if (b0 == 0) {
         for (uint32_t i = threadIdx.x; i < 256u; i += blockDim.x)
@@ -736,14 +908,14 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
         if (i < n_states) {
           const uint2 e = to_smem_entry(g[k], vals[entry_sym(g[k])], 32u * static_cast<uint32_t>(es));
           for (uint32_t c = 0; c < reps; ++c) tab[(i << args.rep_log) + c] = e;
-          if (kPrivate) succ[i] = static_cast<uint16_t>(entry_newx(g1[k]));
+          if (kPrivate && !lock) succ[i] = static_cast<uint16_t>(entry_newx(g1[k]));
           longest = max(longest, entry_run(g[k]) + 1u);
         }
       }
       longest = __reduce_max_sync(kFull, longest);
       if (lane == 0 && longest > 1u) atomicMax(&s_maxadv, longest);
     }
-    if (threadIdx.x < reps && kPrivate && R <= kMaxParkLog)
+    if (threadIdx.x < reps && kPrivate && !lock && R <= kMaxParkLog)
       tab[(n_states << args.rep_log) + threadIdx.x] =
           make_uint2(n_states << 17, es == 4 ? vals[s_dom] : (vals[s_dom] & 0xFFFFu));
     __syncthreads();
@@ -796,11 +968,23 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
   wbad |= decode_private<ES_, ST_>(tab_lane, stride_log, succ_abs, ring_abs, stage_abs, park_abs, ring, dom, words, \
                                    ext_words, wbeg, wend, lane == 31, state, my_count, rows, min_count, \
                                    out_row0, rsb, lane, s_maxadv)
-        if (staged) {
-          if (es == 1) ANSB_CALL(1, true); else if (es == 2) ANSB_CALL(2, true); else ANSB_CALL(4, true);
+#define ANSB_LCALL(ES_, ST_)                                                                             \
+  wbad |= decode_lockstep<ES_, ST_>(tab_lane, stride_log, stage_abs, words, ext_words, wbeg, wend, lane == 31, \
+                                    state, my_count, rows, min_count, out_row0, W / 32u, lane, R <= 8, args.unit)
+        if constexpr (lock) {
+          if (staged) {
+            if (es == 1) ANSB_LCALL(1, true); else if (es == 2) ANSB_LCALL(2, true); else ANSB_LCALL(4, true);
+          } else {
+            if (es == 1) ANSB_LCALL(1, false); else if (es == 2) ANSB_LCALL(2, false); else ANSB_LCALL(4, false);
+          }
         } else {
-          if (es == 1) ANSB_CALL(1, false); else if (es == 2) ANSB_CALL(2, false); else ANSB_CALL(4, false);
+          if (staged) {
+            if (es == 1) ANSB_CALL(1, true); else if (es == 2) ANSB_CALL(2, true); else ANSB_CALL(4, true);
+          } else {
+            if (es == 1) ANSB_CALL(1, false); else if (es == 2) ANSB_CALL(2, false); else ANSB_CALL(4, false);
+          }
         }
+#undef ANSB_LCALL
 #undef ANSB_CALL
       } else {
         const uint16_t* units = reinterpret_cast<const uint16_t*>(g_bytes);
@@ -828,7 +1012,7 @@ __global__ void __launch_bounds__(512, 1) ans_decode_kernel(const LaunchArgs arg
 // ---------------------------------------------------------------------------------------------
 constexpr int kMaxDevices = 64;
 struct LaunchShape { size_t smem = 0; int warps = 0; int per_sm = 0; };
-struct DeviceFacts { int sms = 0; int smem_max = 0; LaunchShape shape[2]; };
+struct DeviceFacts { int sms = 0; int smem_max = 0; LaunchShape shape[3]; };
 static DeviceFacts g_facts[kMaxDevices];    // remembered per device; racing writers store equal values
 
 static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, int n_layers,
@@ -863,6 +1047,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   a.total_work = static_cast<uint32_t>(total);
   a.d_status = d_status;
   a.d_symbols_override = d_symbols_override;
+  a.unit = 1u;
   a.table_words = 2u * ((1u << max_log) + 2u);           // two words per state, and a parking entry (one copy)
   if (n_layers <= kParamLayers) {
     a.n_begin = static_cast<uint32_t>(n_layers);
@@ -885,23 +1070,32 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   smem_max = facts.smem_max;
 
   const bool priv = layout == ANS_LAYOUT_PRIVATE;
-  const void* fn = priv ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE>)
-                        : reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED>);
+  // Layers with many sub-streams share one table among many warps; a model of many small
+  // layers runs CTAs of one granule (4 warps) so that each CTA stays inside one layer and
+  // several CTAs, each with its own table, share an SM.
+  const bool big = total / uint64_t(busy_layers) >= 64;
+  // Private container, large layers: tables of up to 512 states (the paper's coder has 256) fit
+  // shared memory in many conflict-free copies beside 28 warps' staging buffers, which makes
+  // the one-symbol-per-look-up walk the faster one (measured); larger tables, and models of
+  // small layers, are walked through the pre-walked entries.
+  const bool lock = priv && big && max_log <= kLockstepMaxLog;
+  const void* fn = lock   ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, true>)
+                   : priv ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, false>)
+                          : reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, false>);
   int warps = 4;
-  a.succ_bytes = priv ? ((2u << max_log) + 15u) & ~15u : 0u;
+  a.succ_bytes = (priv && !lock) ? ((2u << max_log) + 15u) & ~15u : 0u;
   size_t smem = (size_t(a.table_words) + 256) * 4 + a.succ_bytes;
   {
-    // Layers with many sub-streams share one table among up to 16 warps; a model of many small
-    // layers runs CTAs of one granule (4 warps) so that each CTA stays inside one layer and
-    // several CTAs, each with its own table, share an SM.
-    const bool big = total / uint64_t(busy_layers) >= 64;
     // per warp: an output ring of kRingRows rows of the widest dtype, and a staging buffer for
     // the largest layer-average sub-stream plus a margin (a longer one is read from global memory)
-    const size_t ring = size_t(kRingRows) * 32 * max_es;
+    const size_t ring = lock ? 0 : size_t(kRingRows) * 32 * max_es;   // lockstep rows go straight to the output
     size_t want = max_avg_sub + max_avg_sub / 16 + 256 + kStagePad;
     want = (want + 127) & ~size_t(127);
-    const size_t fixed = ring + 1024 + smem + 16 * 8;     // alignment slack, table, vals, barriers
-    warps = big ? 16 : 4;
+    const size_t fixed = ring + 1024 + smem + 32 * 8;     // alignment slack, table, vals, barriers
+    // lockstep warps need few registers and no ring: up to 28 of them, leaving room for the copies
+    const size_t copies_room = lock ? (size_t(a.table_words) * 4) * 15 : 0;
+    warps = big ? (lock ? 28 : 16) : 4;
+    while (warps > 4 && fixed + copies_room + size_t(warps) * (ring + want) + 1024 > size_t(smem_max)) warps -= 4;
     while (warps > 4 && fixed + size_t(warps) * (ring + want) + 1024 > size_t(smem_max)) warps -= 4;
     const size_t room = size_t(smem_max) > fixed + size_t(warps) * ring + 1024
                             ? (size_t(smem_max) - fixed - size_t(warps) * ring - 1024) / warps : 0;
@@ -921,7 +1115,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
     }
   }
   {
-    LaunchShape& shape = facts.shape[priv ? 1 : 0];
+    LaunchShape& shape = facts.shape[lock ? 2 : priv ? 1 : 0];
     if (shape.smem != smem || shape.warps != warps) {
       ANSB_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
       ANSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, warps * 32, smem));
@@ -939,10 +1133,12 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   ipc = (ipc + step - 1) / step * step;
   a.items_per_cta = static_cast<uint32_t>(ipc);
   const unsigned blocks = static_cast<unsigned>((total + ipc - 1) / ipc);
-  if (priv)
-    ans_decode_kernel<ANS_LAYOUT_PRIVATE><<<blocks, warps * 32, smem, st>>>(a);
+  if (lock)
+    ans_decode_kernel<ANS_LAYOUT_PRIVATE, true><<<blocks, warps * 32, smem, st>>>(a);
+  else if (priv)
+    ans_decode_kernel<ANS_LAYOUT_PRIVATE, false><<<blocks, warps * 32, smem, st>>>(a);
   else
-    ans_decode_kernel<ANS_LAYOUT_INTERLEAVED><<<blocks, warps * 32, smem, st>>>(a);
+    ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, false><<<blocks, warps * 32, smem, st>>>(a);
   ANSB_CUDA(cudaGetLastError());
   return ANS_OK;
 }

@@ -111,6 +111,55 @@ def test_config5_reduced(layout):
     run_and_compare(sg.workload_large(n_mats=2, dim=2048), layout, 32)
 
 
+@pytest.mark.parametrize("lanes", [32, 64, 128, 256])
+@pytest.mark.parametrize("R", [1, 5, 8, 9])
+def test_private_layers_of_many_substreams(lanes, R):
+    """Private layers that average 64 or more work items and have at most 512 states are walked
+    one symbol per look-up, every lane storing straight to the output: whole 16-row blocks, the
+    rows after them, a ragged last row, every output type and every lane count."""
+    b = 1 if R == 1 else min(5, R)
+    g = lanes // 32
+    specs = [tiny_spec(300_017 // g * g + 5, b, 0.6, R, 999, "u8", index=0),
+             tiny_spec(400_001, b, 0.75, R, 1001 * g, "bf16", index=1),
+             tiny_spec(270_000 * g, b, 0.9, R, 777 * g, "f32", index=2),
+             tiny_spec(1_100_000, b, 0.5, R, 4096, "bf16", index=3)]
+    db, prepared = run_and_compare(specs, ans.ANS_LAYOUT_PRIVATE, lanes)
+    assert (db.decode_symbols(1).cpu().numpy() == prepared[1][1]).all()
+    assert db.read_status() == 0
+    run_and_compare(specs[:2], ans.ANS_LAYOUT_PRIVATE, lanes, per_layer=True)
+
+
+def test_private_many_long_substreams_read_from_global_memory():
+    """Sub-streams too long for the shared-memory staging buffer are read word by word from
+    global memory; with many of them the layer still takes the one-symbol-per-look-up walk."""
+    run_and_compare([tiny_spec(260 * 65536 + 321, 5, 0.15, 8, 65536, "u8")], ans.ANS_LAYOUT_PRIVATE, 32)
+
+
+def test_private_many_substreams_corruption_is_flagged():
+    spec = tiny_spec(600_000, 3, 0.7, 8, 2048, "bf16")
+    sym = sg.draw_symbols(spec)
+    T, P, f256 = oracle_pack_spec(spec, sym, ans.ANS_LAYOUT_PRIVATE, 32)
+    rng = np.random.default_rng(1)
+    flagged = 0
+    for trial in range(4):
+        s = P.stream.copy()
+        pos = rng.integers(0, s.size, size=8)
+        s[pos] ^= rng.integers(1, 256, size=8).astype(np.uint8)
+        P2 = oracle.Packed(P.layout, s, P.sub_offsets, P.lane_meta, P.n, P.chunk, P.groups)
+        db = DeviceBatch([to_packed_layer(spec, P2, f256)])
+        db.decode()
+        st = db.read_status()
+        _, orc = oracle.unpack(T, P2)
+        assert (st != 0) == (orc != oracle.OK)
+        flagged += st != 0
+    assert flagged > 0
+    m = P.lane_meta.copy(); m[5, 7] += 1 << 16            # a lane's first word moved
+    db = DeviceBatch([to_packed_layer(spec, oracle.Packed(P.layout, P.stream, P.sub_offsets, m, P.n, P.chunk,
+                                                          P.groups), f256)])
+    db.decode()
+    assert db.read_status() != 0
+
+
 @pytest.mark.parametrize("layout", LAYOUTS)
 def test_corrupt_streams_are_flagged_not_fatal(layout):
     """Corruption is planted on the host.  Reads are clamped to the stream and every loop is
