@@ -55,6 +55,9 @@ def _lib():
         L.anso_pack_private.argtypes = [vp, vp, i64, i64, i32, vp, u64, vp, vp]
         L.anso_pack_private.restype = i64
         L.anso_unpack_private.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, i64, vp]
+        L.anso_pack_quads.argtypes = [vp, vp, i64, i64, i32, vp, u64, vp, vp]
+        L.anso_pack_quads.restype = i64
+        L.anso_unpack_quads.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, i64, vp]
         L.anso_dequant_f32.argtypes = [vp, i64, i32, ctypes.c_float, vp]
         L.anso_dequant_f32.restype = None
         L.anso_dequant_bf16.argtypes = [vp, i64, i32, ctypes.c_float, vp]
@@ -70,7 +73,7 @@ def _p(a: np.ndarray):
     return a.ctypes.data
 
 
-INTERLEAVED, PRIVATE = 0, 1
+INTERLEAVED, PRIVATE, QUADS = 0, 1, 2
 
 
 class Table:
@@ -184,7 +187,8 @@ def pack(T: Table, symbols, chunk: int, groups: int = 1, layout: int = INTERLEAV
         total = lib.anso_pack_interleaved(T.ptr, _p(symbols), n, chunk, groups, _p(stream), cap, _p(offs), _p(meta))
     else:
         meta = np.zeros((n_sub, 32), dtype=np.uint32)
-        total = lib.anso_pack_private(T.ptr, _p(symbols), n, chunk, groups, _p(stream), cap, _p(offs), _p(meta))
+        fn = lib.anso_pack_private if layout == PRIVATE else lib.anso_pack_quads
+        total = fn(T.ptr, _p(symbols), n, chunk, groups, _p(stream), cap, _p(offs), _p(meta))
     if total < 0:
         raise OracleError(total, "pack")
     return Packed(layout, stream[:total].copy(), offs, meta, n, chunk, groups)
@@ -194,7 +198,8 @@ def unpack(T: Table, P: Packed, threads: int = 1, chunk_range=None):
     """Decode a packed layer to symbols.  Returns (symbols, rc)."""
     out = np.zeros(max(P.n, 1), dtype=np.uint8)
     lib = _lib()
-    fn = lib.anso_unpack_interleaved if P.layout == INTERLEAVED else lib.anso_unpack_private
+    fn = {INTERLEAVED: lib.anso_unpack_interleaved, PRIVATE: lib.anso_unpack_private,
+          QUADS: lib.anso_unpack_quads}[P.layout]
     lo, hi = chunk_range if chunk_range is not None else (0, P.n_chunks)
 
     def work(rng):

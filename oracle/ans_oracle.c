@@ -27,7 +27,9 @@
  *   - two containers that carry many lanes:
  *       "interleaved": 32 lanes share one sequence of 16-bit units, ordered by
  *                      the decoder's refill schedule;
- *       "private":     each lane owns a contiguous run of 32-bit words.
+ *       "private":     each lane owns a contiguous run of 32-bit words;
+ *       "quads":       private lanes that take four consecutive symbols per
+ *                      turn and fill their words most significant bit first.
  *   - frequency normalisation (largest-remainder, every present symbol >= 1).
  *
  * Pins (see tests): hand-enumerated state traces, table tiling invariants,
@@ -424,6 +426,134 @@ int anso_unpack_private(const anso_table* T, const uint8_t* stream, const uint64
         }
         if (i != 0) rc = ANSO_ERR_CORRUPT;
         /* the lane's words must be exactly what its bits need (last lane: up to the pad) */
+        const uint64_t need = ((pos + 31) / 32) * 4;
+        if (k < 31 ? (need != end - begin) : (need > end - begin || end - begin - need >= 16)) rc = ANSO_ERR_CORRUPT;
+      }
+    }
+  }
+  return rc;
+}
+
+/*
+ * Quads container: private lanes as above, with two differences that the paper
+ * leaves open just the same (Section II-A fixes neither the order of bits in a
+ * stream word nor which symbols a stream owns):
+ *   - lanes take the chunk's symbols FOUR AT A TIME: chunk-relative symbol q
+ *     sits in quad j = q div 4; quad j belongs to lane j mod W, as that lane's
+ *     (j div W)-th quad; inside the lane the quad's symbols keep their order.
+ *     (A chunk's last quad may hold fewer than four symbols.)
+ *   - a lane's bit string fills its 32-bit words from the MOST significant bit
+ *     down, and a field's most significant bit comes first.  Words are stored
+ *     little-endian, zero-padded as in the private container.
+ * lane_meta and the sub-stream order are those of the private container.
+ */
+static int64_t quad_lane_count(int64_t n_chunk, int W, int lambda) {
+  /* symbols lane lambda owns: 4 per full quad, plus the short last quad if it is the lane's */
+  const int64_t full = n_chunk / 4, rem = n_chunk % 4;
+  int64_t cnt = 4 * (full > lambda ? (full - lambda + W - 1) / W : 0);
+  if (rem && full % W == lambda) cnt += rem;
+  return cnt;
+}
+
+/* chunk-relative position of lane lambda's t-th symbol */
+static int64_t quad_position(int W, int lambda, int64_t t) {
+  return ((t / 4) * W + lambda) * 4 + t % 4;
+}
+
+/* Append `nb` bits of `val`, most significant first; bit position p of the string is bit
+ * 31 - p%32 of 32-bit little-endian word p/32. */
+static void put_bits_msb(uint8_t* bytes, uint64_t* pos, uint32_t val, int nb) {
+  for (int b = nb - 1; b >= 0; --b, ++*pos) {
+    const int bit_in_word = 31 - (int)(*pos % 32);
+    if (val & (1u << b)) bytes[(*pos / 32) * 4 + bit_in_word / 8] |= (uint8_t)(1u << (bit_in_word % 8));
+  }
+}
+
+static uint32_t get_bits_msb(const uint8_t* bytes, uint64_t nbytes, uint64_t pos, int nb) {
+  uint32_t v = 0;
+  for (int b = 0; b < nb; ++b, ++pos) {
+    const int bit_in_word = 31 - (int)(pos % 32);
+    const uint64_t byte = (pos / 32) * 4 + (uint64_t)(bit_in_word / 8);
+    v <<= 1;
+    if (byte < nbytes && (bytes[byte] >> (bit_in_word % 8)) & 1) v |= 1u;
+  }
+  return v;
+}
+
+int64_t anso_pack_quads(const anso_table* T, const uint8_t* symbols, int64_t n,
+                        int64_t C, int G, uint8_t* stream, uint64_t cap_bytes,
+                        uint64_t* sub_offsets, uint32_t* lane_meta) {
+  if (!T || C < 1 || G < 1 || n < 0) return ANSO_ERR_ARG;
+  const int W = 32 * G;
+  const int64_t n_chunks = (n + C - 1) / C;
+  const int64_t max_lane = 4 * ((C / 4 + W - 1) / W) + 4;
+  uint8_t* mine = (uint8_t*)malloc((size_t)max_lane);
+  uint8_t* fnb = (uint8_t*)malloc((size_t)max_lane);
+  uint16_t* fval = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)max_lane);
+  uint64_t off = 0;
+  int64_t rc = ANSO_OK;
+  for (int64_t c = 0; c < n_chunks && rc >= 0; ++c) {
+    const uint8_t* cs = symbols + c * C;
+    const int64_t nc = (n - c * C) < C ? (n - c * C) : C;
+    for (int g = 0; g < G && rc >= 0; ++g) {
+      const int64_t sub = c * G + g;
+      sub_offsets[sub] = off;
+      const uint64_t base = off;
+      for (int k = 0; k < 32; ++k) {
+        const int lambda = 32 * g + k;
+        const int64_t cnt = quad_lane_count(nc, W, lambda);
+        for (int64_t t = 0; t < cnt; ++t) mine[t] = cs[quad_position(W, lambda, t)];
+        int init = anso_encode_lane(T, mine, cnt, 1, fnb, fval);
+        if (init < 0) { rc = init; break; }
+        uint64_t nbits = 0;
+        for (int64_t t = 0; t < cnt; ++t) nbits += fnb[t];
+        const uint64_t nbytes = ((nbits + 31) / 32) * 4;
+        const uint64_t word0 = (off - base) / 4;
+        if (word0 > 0xFFFF) { rc = ANSO_ERR_ARG; break; }
+        if (off + nbytes > cap_bytes) { rc = ANSO_ERR_SPACE; break; }
+        lane_meta[sub * 32 + k] = (uint32_t)init | ((uint32_t)word0 << 16);
+        memset(stream + off, 0, (size_t)nbytes);
+        uint64_t pos = 0;
+        for (int64_t t = 0; t < cnt; ++t) put_bits_msb(stream + off, &pos, fval[t], fnb[t]);
+        off += nbytes;
+      }
+      while (rc >= 0 && off % 16) { if (off >= cap_bytes) { rc = ANSO_ERR_SPACE; break; } stream[off++] = 0; }
+    }
+  }
+  if (rc >= 0) sub_offsets[n_chunks * G] = off;
+  free(mine); free(fnb); free(fval);
+  return rc < 0 ? rc : (int64_t)off;
+}
+
+int anso_unpack_quads(const anso_table* T, const uint8_t* stream, const uint64_t* sub_offsets,
+                      const uint32_t* lane_meta, int64_t n, int64_t C, int G,
+                      int64_t chunk_begin, int64_t chunk_end, uint8_t* out) {
+  const int W = 32 * G;
+  int rc = ANSO_OK;
+  for (int64_t c = chunk_begin; c < chunk_end; ++c) {
+    uint8_t* co = out + c * C;
+    const int64_t nc = (n - c * C) < C ? (n - c * C) : C;
+    for (int g = 0; g < G; ++g) {
+      const int64_t sub = c * G + g;
+      const uint8_t* p = stream + sub_offsets[sub];
+      const uint64_t extent = sub_offsets[sub + 1] - sub_offsets[sub];
+      for (int k = 0; k < 32; ++k) {
+        const int lambda = 32 * g + k;
+        const int64_t cnt = quad_lane_count(nc, W, lambda);
+        const uint32_t meta = lane_meta[sub * 32 + k];
+        const uint64_t begin = (uint64_t)(meta >> 16) * 4;
+        const uint64_t end = (k < 31) ? (uint64_t)(lane_meta[sub * 32 + k + 1] >> 16) * 4 : extent;
+        if (begin > end || end > extent) { rc = ANSO_ERR_CORRUPT; continue; }
+        uint32_t i = meta & 0xFFFF;
+        uint64_t pos = 0;
+        for (int64_t t = 0; t < cnt; ++t) {
+          co[quad_position(W, lambda, t)] = T->sym[i];
+          const int nb = T->nb[i];
+          const uint32_t v = get_bits_msb(p + begin, end - begin, pos, nb);
+          pos += (uint64_t)nb;
+          i = T->newx[i] + v;
+        }
+        if (i != 0) rc = ANSO_ERR_CORRUPT;
         const uint64_t need = ((pos + 31) / 32) * 4;
         if (k < 31 ? (need != end - begin) : (need > end - begin || end - begin - need >= 16)) rc = ANSO_ERR_CORRUPT;
       }
