@@ -5,7 +5,7 @@ One step = one pass of the whole hot path (stage tables, read compressed streams
 dequantise, store) over one synthetic workload, as ONE batched kernel launch.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload large|resnet50|resnet18|conv3x3|sweep]
-                  [--layout private|interleaved] [--lanes 32|64|128|256] [--impl ours|reference]
+                  [--layout private|interleaved|quads] [--lanes 32|64|128|256] [--impl ours|reference]
 
 Prints one JSON line (rank 0).  With --impl reference the CPU oracle is timed instead.
 """
@@ -115,7 +115,7 @@ def cpu_baseline(specs, syms, layout_name, budget_s=12.0):
     """The CPU oracle, as it stands, decoding + dequantising a bounded sample of the same
     workload on this host's cores: single thread and all cores."""
     import oracle
-    layout = oracle.PRIVATE if layout_name == "private" else oracle.INTERLEAVED
+    layout = {"private": oracle.PRIVATE, "interleaved": oracle.INTERLEAVED, "quads": oracle.QUADS}[layout_name]
     cores = os.cpu_count() or 1
     target = 48_000_000                         # symbols in the sample (about 10-30 s of CPU work in all)
     sample, total = [], 0
@@ -156,7 +156,7 @@ def run_reference(args):
     if rank != 0:
         return
     specs = make_specs(args)
-    layout = oracle.PRIVATE if args.layout == "private" else oracle.INTERLEAVED
+    layout = {"private": oracle.PRIVATE, "interleaved": oracle.INTERLEAVED, "quads": oracle.QUADS}[args.layout]
     cores = os.cpu_count() or 1
     target = 24_000_000
     sample, total = [], 0
@@ -253,7 +253,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     ans.lib()                                           # fail loudly if the library is missing
 
-    layout = ans.ANS_LAYOUT_PRIVATE if args.layout == "private" else ans.ANS_LAYOUT_INTERLEAVED
+    layout = {"private": ans.ANS_LAYOUT_PRIVATE, "interleaved": ans.ANS_LAYOUT_INTERLEAVED,
+              "quads": ans.ANS_LAYOUT_QUADS}[args.layout]
     specs = make_specs(args)
     t_setup = time.perf_counter()
     from concurrent.futures import ThreadPoolExecutor
@@ -298,7 +299,7 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     kernel_ms = statistics.mean(ms)
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-    kname = "ans_decode_kernel<private>" if args.layout == "private" else "ans_decode_kernel<interleaved>"
+    kname = f"ans_decode_kernel<{args.layout}>"
     # DRAM bytes per launch from an ncu capture of this kernel (see profiles/), only for the
     # configuration that capture covers; None otherwise
     traffic = NCU_TRAFFIC.get((args.workload, args.layout, args.lanes, args.mats, args.dim, args.chunk, args.table_log))
@@ -416,7 +417,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=list(WORKLOAD_TEXT))
-    ap.add_argument("--layout", default="private", choices=["private", "interleaved"])
+    ap.add_argument("--layout", default="private", choices=["private", "interleaved", "quads"])
     ap.add_argument("--lanes", type=int, default=32)
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--table-log", type=int, default=0)

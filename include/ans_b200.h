@@ -42,6 +42,12 @@
  *       words inside its sub-stream, lanes in ascending order.
  *       d_lane_meta is uint32_t[n_sub][32]: initial state | (first word, counted from
  *       the sub-stream's start) << 16.
+ *     ANS_LAYOUT_QUADS: private lanes with two differences.  Lanes take the chunk's symbols
+ *       four at a time: chunk-relative symbol q sits in quad j = q / 4, quad j is the
+ *       (j / lanes)-th quad of lane j % lanes (the chunk's last quad may be short), so a
+ *       lane writes 4 adjacent outputs per turn.  And a lane's bits fill its 32-bit words
+ *       from the most significant bit down, each field most significant bit first (the
+ *       words themselves are stored little-endian).  d_lane_meta as for ANS_LAYOUT_PRIVATE.
  */
 #ifndef ANS_B200_H
 #define ANS_B200_H
@@ -67,6 +73,7 @@ extern "C" {
 
 #define ANS_LAYOUT_INTERLEAVED 0
 #define ANS_LAYOUT_PRIVATE     1
+#define ANS_LAYOUT_QUADS       2
 
 #define ANS_MAX_TABLE_LOG 14
 #define ANS_MAX_ALPHABET  256
@@ -235,7 +242,7 @@ int ans_host_pack_bound(uint64_t n_symbols, uint32_t chunk_symbols, uint32_t lan
  * append its label bits) into the chosen container.
  *   h_symbols[n_symbols]; h_freqs[256] as given to ans_build_decode_tables
  *   h_stream_out (capacity stream_cap), h_sub_offsets_out[n_sub + 1],
- *   h_lane_meta_out: uint16_t[n_sub][32] (interleaved) or uint32_t[n_sub][32] (private)
+ *   h_lane_meta_out: uint16_t[n_sub][32] (interleaved) or uint32_t[n_sub][32] (private, quads)
  *   n_threads: host threads to use (<= 0: all)
  * *h_stream_bytes_out receives the bytes written.
  */

@@ -13,7 +13,8 @@ void set_last_cuda_error(cudaError_t e) { g_last_cuda_error.store(static_cast<in
 int validate_desc(const ans_layer_desc& d, bool need_out) {
   if (d.table_log < 1 || d.table_log > ANS_MAX_TABLE_LOG) return ANS_ERR_UNSUPPORTED;
   if (d.lanes != 32 && d.lanes != 64 && d.lanes != 128 && d.lanes != 256) return ANS_ERR_UNSUPPORTED;
-  if (d.layout != ANS_LAYOUT_INTERLEAVED && d.layout != ANS_LAYOUT_PRIVATE) return ANS_ERR_UNSUPPORTED;
+  if (d.layout != ANS_LAYOUT_INTERLEAVED && d.layout != ANS_LAYOUT_PRIVATE && d.layout != ANS_LAYOUT_QUADS)
+    return ANS_ERR_UNSUPPORTED;
   if (d.out_dtype != ANS_U8 && d.out_dtype != ANS_F32 && d.out_dtype != ANS_BF16) return ANS_ERR_UNSUPPORTED;
   if (d.chunk_symbols == 0) return ANS_ERR_INVALID_ARG;
   if (d.bitwidth < 1 || d.bitwidth > 8) return ANS_ERR_INVALID_ARG;
@@ -71,7 +72,7 @@ ANS_EXPORT int ans_host_scratch_bytes(const ans_layer_desc* h_desc, uint64_t str
   if (!h_desc || !h_bytes_out) return ANS_ERR_INVALID_ARG;
   if (h_desc->chunk_symbols == 0 || h_desc->lanes == 0 || h_desc->lanes % 32) return ANS_ERR_INVALID_ARG;
   const uint64_t n_sub = subs_of(*h_desc);
-  const size_t meta = n_sub * 32 * (h_desc->layout == ANS_LAYOUT_PRIVATE ? 4 : 2);
+  const size_t meta = n_sub * 32 * (h_desc->layout == ANS_LAYOUT_INTERLEAVED ? 2 : 4);
   *h_bytes_out = 256 + up256(stream_bytes) + up256((n_sub + 1) * 8) + up256(meta) +
                  up256(h_desc->n_symbols * elem_size(h_desc->out_dtype));
   return ANS_OK;
@@ -92,7 +93,7 @@ ANS_EXPORT int ans_decode_dequant_host(const ans_layer_desc* h_desc, const uint8
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
   const uint64_t n_sub = subs_of(*h_desc);
-  const size_t meta_bytes = n_sub * 32 * (h_desc->layout == ANS_LAYOUT_PRIVATE ? 4 : 2);
+  const size_t meta_bytes = n_sub * 32 * (h_desc->layout == ANS_LAYOUT_INTERLEAVED ? 2 : 4);
   const size_t out_bytes = h_desc->n_symbols * elem_size(h_desc->out_dtype);
   uint8_t* p = static_cast<uint8_t*>(d_scratch);
   uint32_t* d_status = reinterpret_cast<uint32_t*>(p); p += 256;

@@ -620,6 +620,157 @@ __device__ __noinline__ uint32_t decode_lockstep(
 }
 
 // =============================================================================================
+// Quads container: the lockstep walk with two changes that the container makes possible.
+// A lane owns four adjacent output elements per turn, so the four values of a turn leave in one
+// vector store (8 bytes of bf16 per lane, 256 contiguous bytes per warp) instead of four.  And
+// the bit window is kept top-aligned (bits are taken from the most significant end), so that
+// one funnel shift builds the next state: with q = newX >> nb_bits kept in the entry,
+// (q << nb) | (window >> (32 - nb)) needs no mask; a second one drops the bits taken.
+//
+// shared-memory entry, two words:
+//   1- and 2-byte outputs:  a = nb [4:0] | dequantised value [31:16]      b = q
+//   4-byte outputs:         a = nb [4:0] | q [31:8]                       b = dequantised value
+// =============================================================================================
+__device__ __forceinline__ uint2 to_quads_entry(uint32_t g, uint32_t val, bool narrow) {
+  const uint32_t nb = entry_nb(g), q = entry_newx(g) >> nb;
+  return narrow ? make_uint2(nb | (val << 16), q) : make_uint2(nb | (q << 8), val);
+}
+
+#define ANSB_QD_STEP_N(I_)                                        \
+  "ld.shared.v2.u32 {ea" I_ ", eb" I_ "}, [%0];\n\t"              \
+  "shf.l.wrap.b32 t, x, eb" I_ ", ea" I_ ";\n\t"                  \
+  "shf.l.wrap.b32 x, 0, x, ea" I_ ";\n\t"                         \
+  "mad.lo.u32 %0, t, %7, %6;\n\t"                                 \
+  "mad.lo.u32 %1, ea" I_ ", %9, %1;\n\t"
+#define ANSB_QD_STEP_W(I_)                                        \
+  "ld.shared.v2.u32 {ea" I_ ", eb" I_ "}, [%0];\n\t"              \
+  "shr.u32 nx, ea" I_ ", 8;\n\t"                                  \
+  "shf.l.wrap.b32 t, x, nx, ea" I_ ";\n\t"                        \
+  "shf.l.wrap.b32 x, 0, x, ea" I_ ";\n\t"                         \
+  "mad.lo.u32 %0, t, %7, %6;\n\t"                                 \
+  "mad.lo.u32 %1, ea" I_ ", %9, %1;\n\t"
+#define ANSB_QD_BEGIN "shf.l.wrap.b32 x, %3, %2, %1;\n\t"
+// four look-ups of one turn: one refill check when a symbol takes at most 8 bits, else two
+#define ANSB_QD_TURN4(ST_) ANSB_QD_BEGIN ST_("0") ST_("1") ST_("2") ST_("3") ANSB_LS_END
+#define ANSB_QD_TURN2(ST_) ANSB_QD_BEGIN ST_("0") ST_("1") ANSB_LS_END ANSB_QD_BEGIN ST_("2") ST_("3") ANSB_LS_END
+#define ANSB_QD_OUT1(A_)                                          \
+  "prmt.b32 v0, ea0, ea1, 0x0062;\n\t"                            \
+  "prmt.b32 v1, ea2, ea3, 0x0062;\n\t"                            \
+  "prmt.b32 v0, v0, v1, 0x5410;\n\t"                              \
+  "st.global.u32 " A_ ", v0;\n\t"
+#define ANSB_QD_OUT2(A_)                                          \
+  "prmt.b32 v0, ea0, ea1, 0x7632;\n\t"                            \
+  "prmt.b32 v1, ea2, ea3, 0x7632;\n\t"                            \
+  "st.global.v2.u32 " A_ ", {v0, v1};\n\t"
+#define ANSB_QD_OUT4(A_) "st.global.v4.u32 " A_ ", {eb0, eb1, eb2, eb3};\n\t"
+
+constexpr uint32_t kQuadTurns = 4;     // turns (of four symbols per lane) decoded by one PTX block
+
+// Same operands as lockstep_block; gp: this lane's four elements of the block's first turn
+// (turns are 128 * ES * G bytes apart).
+template <int ES, int K, int G>
+__device__ __forceinline__ void quads_block(uint32_t& st, uint32_t& bitpos, uint32_t& w0, uint32_t& w1,
+                                            uint32_t& w2, uint32_t& sp, uint32_t tab_lane, uint32_t stride,
+                                            uint8_t* gp, uint32_t unit) {
+  constexpr uint32_t RS = 128u * ES * G;
+#define ANSB_QD_ASM(TURN_, ST_, OUT_)                                                       \
+  asm volatile(                                                                             \
+      "{\n\t"                                                                               \
+      ".reg .pred q;\n\t"                                                                   \
+      ".reg .u32 x, t, nx, nw, v0, v1, ea0, ea1, ea2, ea3, eb0, eb1, eb2, eb3;\n\t"          \
+      TURN_(ST_) OUT_("[%8]") TURN_(ST_) OUT_("[%8+%10]")                                   \
+      TURN_(ST_) OUT_("[%8+%11]") TURN_(ST_) OUT_("[%8+%12]")                               \
+      "}"                                                                                   \
+      : "+r"(st), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp)                      \
+      : "r"(tab_lane), "r"(stride), "l"(gp), "r"(unit), "n"(RS * 1), "n"(RS * 2), "n"(RS * 3) \
+      : "memory")
+  if (K == 4) {
+    if (ES == 1) ANSB_QD_ASM(ANSB_QD_TURN4, ANSB_QD_STEP_N, ANSB_QD_OUT1);
+    if (ES == 2) ANSB_QD_ASM(ANSB_QD_TURN4, ANSB_QD_STEP_N, ANSB_QD_OUT2);
+    if (ES == 4) ANSB_QD_ASM(ANSB_QD_TURN4, ANSB_QD_STEP_W, ANSB_QD_OUT4);
+  } else {
+    if (ES == 1) ANSB_QD_ASM(ANSB_QD_TURN2, ANSB_QD_STEP_N, ANSB_QD_OUT1);
+    if (ES == 2) ANSB_QD_ASM(ANSB_QD_TURN2, ANSB_QD_STEP_N, ANSB_QD_OUT2);
+    if (ES == 4) ANSB_QD_ASM(ANSB_QD_TURN2, ANSB_QD_STEP_W, ANSB_QD_OUT4);
+  }
+#undef ANSB_QD_ASM
+}
+
+// Decode one sub-stream of the quads container.  full_turns: turns in which every lane of the
+// sub-stream owns a whole quad; out_lane: this lane's first output element; a lane's turns are
+// 128 * ES * groups bytes apart.
+template <int ES, bool STAGED>
+__device__ __noinline__ uint32_t decode_quads(
+    uint32_t tab_abs, uint32_t stride_log, uint32_t stage_abs, const uint32_t* __restrict__ words,
+    uint32_t ext_words, uint32_t wbeg, uint32_t wend, bool last_lane, uint32_t state, uint32_t my_count,
+    uint32_t full_turns, uint8_t* __restrict__ out_lane, uint32_t groups, bool wide_steps, uint32_t unit) {
+  constexpr bool NARROW = ES != 4;
+  constexpr uint32_t QB = 4u * ES;                  // bytes of a quad
+  const size_t turn_stride = size_t(128u * ES) * groups;
+  const uint32_t word_limit = STAGED ? ext_words + 4u : ext_words;
+  auto load_word = [&](uint32_t i) -> uint32_t {
+    if (STAGED) return lds_u32(stage_abs + i * 4u);
+    return i < word_limit ? __ldg(words + i) : 0u;
+  };
+  uint32_t idx = wbeg;
+  uint32_t w0 = load_word(idx), w1 = load_word(idx + 1), w2 = load_word(idx + 2);
+  idx += 3;
+  uint32_t bitpos = 0;
+  bool overran = false;
+  uint32_t st = tab_abs + (state << stride_log);
+  uint32_t k = 0;                                   // symbols this lane has decoded
+
+  uint32_t turn = 0;
+  // whole blocks: needs the staged copy, and quads that may leave as one vector store
+  if (STAGED && (reinterpret_cast<uintptr_t>(out_lane) & (QB - 1u)) == 0) {
+    uint32_t sp = stage_abs + idx * 4u;
+    const uint32_t sp_limit = stage_abs + word_limit * 4u;
+    const uint32_t stride = 1u << stride_log;
+    uint8_t* gp = out_lane;
+#define ANSB_QD_LOOP(K_, G_)                                                                \
+    while (turn + kQuadTurns <= full_turns) {                                               \
+      quads_block<ES, K_, G_>(st, bitpos, w0, w1, w2, sp, tab_abs, stride, gp, unit);       \
+      if (sp > sp_limit) { overran = true; sp = sp_limit; }                                 \
+      gp += kQuadTurns * 128u * ES * G_;                                                    \
+      turn += kQuadTurns;                                                                   \
+    }
+    if (wide_steps) {
+      if (groups == 1) { ANSB_QD_LOOP(4, 1) } else if (groups == 2) { ANSB_QD_LOOP(4, 2) }
+      else if (groups == 4) { ANSB_QD_LOOP(4, 4) } else if (groups == 8) { ANSB_QD_LOOP(4, 8) }
+    } else {
+      if (groups == 1) { ANSB_QD_LOOP(2, 1) } else if (groups == 2) { ANSB_QD_LOOP(2, 2) }
+      else if (groups == 4) { ANSB_QD_LOOP(2, 4) } else if (groups == 8) { ANSB_QD_LOOP(2, 8) }
+    }
+#undef ANSB_QD_LOOP
+    idx = (sp - stage_abs) >> 2;
+    k = 4u * turn;
+  }
+  // the rest in plain code, one symbol and one element store at a time
+  for (; k < my_count; ++k) {
+    const uint32_t ea = lds_u32(st), eb = lds_u32(st + 4u);
+    const uint32_t nb = ea & 31u;
+    const uint32_t q = NARROW ? eb : ea >> 8, val = NARROW ? ea >> 16 : eb;
+    const uint32_t x = __funnelshift_l(w1, w0, bitpos);
+    st = tab_abs + (__funnelshift_l(x, q, nb) << stride_log);
+    stg_elem<ES>(out_lane + size_t(k >> 2) * turn_stride + (k & 3u) * ES, val);
+    bitpos += nb;
+    if (bitpos >= 32u) {
+      w0 = w1; w1 = w2;
+      w2 = (!STAGED || idx < word_limit) ? load_word(idx) : 0u;
+      ++idx;
+      bitpos -= 32u;
+    }
+  }
+  uint32_t bad = 0;
+  if (st != tab_abs) bad |= ANS_STATUS_BAD_FINAL_STATE;
+  const uint32_t bits = (idx - 3u - wbeg) * 32u + bitpos;
+  const uint32_t need = (bits + 31u) / 32u;
+  const uint32_t have = wend - wbeg;
+  if (overran || (last_lane ? (need > have || have - need >= 4u) : (need != have))) bad |= ANS_STATUS_BAD_LENGTH;
+  return bad;
+}
+
+// =============================================================================================
 // Interleaved container: the warp's 32 lanes share one sequence of 16-bit units; before each
 // round a lane whose buffer holds fewer than 16 bits takes the next unit, its place found by
 // ballot + popcount; then every lane decodes one symbol.  Same shared-memory table, staging
@@ -782,8 +933,9 @@ __device__ __noinline__ uint32_t decode_interleaved(
 
 template <int LAYOUT, bool LOCK>
 __global__ void __launch_bounds__(LOCK ? 1024 : 512, 1) ans_decode_kernel(const LaunchArgs args) {
-  constexpr bool kPrivate = LAYOUT == ANS_LAYOUT_PRIVATE;
-  constexpr bool lock = kPrivate && LOCK;           // private container walked one symbol per look-up
+  constexpr bool kQuads = LAYOUT == ANS_LAYOUT_QUADS;
+  constexpr bool kPrivate = LAYOUT != ANS_LAYOUT_INTERLEAVED;   // lanes own their words
+  constexpr bool lock = kPrivate && LOCK;           // walked one symbol per look-up (quads always are)
   extern __shared__ __align__(16) uint8_t sm[];
   const uint32_t NW = blockDim.x >> 5;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
@@ -906,7 +1058,8 @@ __global__ void __launch_bounds__(LOCK ? 1024 : 512, 1) ans_decode_kernel(const 
       for (uint32_t k = 0; k < kStageBatch; ++k) {
         const uint32_t i = b0 + k * blockDim.x + threadIdx.x;
         if (i < n_states) {
-          const uint2 e = to_smem_entry(g[k], vals[entry_sym(g[k])], 32u * static_cast<uint32_t>(es));
+          const uint2 e = kQuads ? to_quads_entry(g[k], vals[entry_sym(g[k])], es != 4)
+                                 : to_smem_entry(g[k], vals[entry_sym(g[k])], 32u * static_cast<uint32_t>(es));
           for (uint32_t c = 0; c < reps; ++c) tab[(i << args.rep_log) + c] = e;
           if (kPrivate && !lock) succ[i] = static_cast<uint16_t>(entry_newx(g1[k]));
           longest = max(longest, entry_run(g[k]) + 1u);
@@ -930,14 +1083,25 @@ __global__ void __launch_bounds__(LOCK ? 1024 : 512, 1) ans_decode_kernel(const 
       const Item it = is_first ? first_item : make_item(L, sub);
       uint32_t wbad = it.bad;
       const uint32_t lambda = 32u * it.g + lane;
-      const uint32_t my_count = lane_symbols(it.nc, W, lambda);
-      const uint32_t rows = lane_symbols(it.nc, W, 32u * it.g);
-      const uint32_t min_count = lane_symbols(it.nc, W, 32u * it.g + 31u);
+      // round-robin containers: symbols of this lane, rows of the sub-stream, rows all 32 lanes have.
+      // quads: symbols of this lane; rows / min_count count the turns some / all lanes own a whole quad in
+      uint32_t my_count, rows, min_count;
+      if (kQuads) {
+        const uint32_t full = it.nc >> 2, rem = it.nc & 3u;
+        my_count = 4u * lane_symbols(full, W, lambda) + ((rem && full % W == lambda) ? rem : 0u);
+        rows = lane_symbols(full, W, 32u * it.g);
+        min_count = lane_symbols(full, W, 32u * it.g + 31u);
+      } else {
+        my_count = lane_symbols(it.nc, W, lambda);
+        rows = lane_symbols(it.nc, W, 32u * it.g);
+        min_count = lane_symbols(it.nc, W, 32u * it.g + 31u);
+      }
       const uint32_t ext_words = static_cast<uint32_t>(min(it.extent / 4, uint64_t(0x3FFFFFFFu)));
       const uint8_t* g_bytes = L.d_stream + it.off0;
       const bool staged = is_first ? first_staged : start_copy(it);
 
-      uint8_t* out_row0 = out_base + (it.c0 + 32u * it.g) * es;     // row 0 of this sub-stream
+      // row 0 of this sub-stream (quads: a row holds four elements per lane)
+      uint8_t* out_row0 = out_base + (it.c0 + (kQuads ? 128u : 32u) * it.g) * es;
       const size_t rsb = size_t(W) * es;
       uint32_t state, wbeg = 0, wend = 0;
       if (kPrivate) {
@@ -971,7 +1135,16 @@ __global__ void __launch_bounds__(LOCK ? 1024 : 512, 1) ans_decode_kernel(const 
 #define ANSB_LCALL(ES_, ST_)                                                                             \
   wbad |= decode_lockstep<ES_, ST_>(tab_lane, stride_log, stage_abs, words, ext_words, wbeg, wend, lane == 31, \
                                     state, my_count, rows, min_count, out_row0, W / 32u, lane, R <= 8, args.unit)
-        if constexpr (lock) {
+#define ANSB_QCALL(ES_, ST_)                                                                             \
+  wbad |= decode_quads<ES_, ST_>(tab_lane, stride_log, stage_abs, words, ext_words, wbeg, wend, lane == 31, state, \
+                                 my_count, min_count, out_row0 + size_t(lane) * 4u * ES_, W / 32u, R <= 8, args.unit)
+        if constexpr (kQuads) {
+          if (staged) {
+            if (es == 1) ANSB_QCALL(1, true); else if (es == 2) ANSB_QCALL(2, true); else ANSB_QCALL(4, true);
+          } else {
+            if (es == 1) ANSB_QCALL(1, false); else if (es == 2) ANSB_QCALL(2, false); else ANSB_QCALL(4, false);
+          }
+        } else if constexpr (lock) {
           if (staged) {
             if (es == 1) ANSB_LCALL(1, true); else if (es == 2) ANSB_LCALL(2, true); else ANSB_LCALL(4, true);
           } else {
@@ -984,6 +1157,7 @@ __global__ void __launch_bounds__(LOCK ? 1024 : 512, 1) ans_decode_kernel(const 
             if (es == 1) ANSB_CALL(1, false); else if (es == 2) ANSB_CALL(2, false); else ANSB_CALL(4, false);
           }
         }
+#undef ANSB_QCALL
 #undef ANSB_LCALL
 #undef ANSB_CALL
       } else {
@@ -1012,7 +1186,7 @@ __global__ void __launch_bounds__(LOCK ? 1024 : 512, 1) ans_decode_kernel(const 
 // ---------------------------------------------------------------------------------------------
 constexpr int kMaxDevices = 64;
 struct LaunchShape { size_t smem = 0; int warps = 0; int per_sm = 0; };
-struct DeviceFacts { int sms = 0; int smem_max = 0; LaunchShape shape[3]; };
+struct DeviceFacts { int sms = 0; int smem_max = 0; LaunchShape shape[4]; };
 static DeviceFacts g_facts[kMaxDevices];    // remembered per device; racing writers store equal values
 
 static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, int n_layers,
@@ -1069,7 +1243,8 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   sms = facts.sms;
   smem_max = facts.smem_max;
 
-  const bool priv = layout == ANS_LAYOUT_PRIVATE;
+  const bool quads = layout == ANS_LAYOUT_QUADS;
+  const bool priv = layout != ANS_LAYOUT_INTERLEAVED;
   // Layers with many sub-streams share one table among many warps; a model of many small
   // layers runs CTAs of one granule (4 warps) so that each CTA stays inside one layer and
   // several CTAs, each with its own table, share an SM.
@@ -1078,8 +1253,9 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   // shared memory in many conflict-free copies beside 28 warps' staging buffers, which makes
   // the one-symbol-per-look-up walk the faster one (measured); larger tables, and models of
   // small layers, are walked through the pre-walked entries.
-  const bool lock = priv && big && max_log <= kLockstepMaxLog;
-  const void* fn = lock   ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, true>)
+  const bool lock = quads || (priv && big && max_log <= kLockstepMaxLog);
+  const void* fn = quads  ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_QUADS, true>)
+                   : lock ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, true>)
                    : priv ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, false>)
                           : reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, false>);
   int warps = 4;
@@ -1115,7 +1291,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
     }
   }
   {
-    LaunchShape& shape = facts.shape[lock ? 2 : priv ? 1 : 0];
+    LaunchShape& shape = facts.shape[quads ? 3 : lock ? 2 : priv ? 1 : 0];
     if (shape.smem != smem || shape.warps != warps) {
       ANSB_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
       ANSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, warps * 32, smem));
@@ -1133,7 +1309,9 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   ipc = (ipc + step - 1) / step * step;
   a.items_per_cta = static_cast<uint32_t>(ipc);
   const unsigned blocks = static_cast<unsigned>((total + ipc - 1) / ipc);
-  if (lock)
+  if (quads)
+    ans_decode_kernel<ANS_LAYOUT_QUADS, true><<<blocks, warps * 32, smem, st>>>(a);
+  else if (lock)
     ans_decode_kernel<ANS_LAYOUT_PRIVATE, true><<<blocks, warps * 32, smem, st>>>(a);
   else if (priv)
     ans_decode_kernel<ANS_LAYOUT_PRIVATE, false><<<blocks, warps * 32, smem, st>>>(a);

@@ -1,4 +1,4 @@
-// Host-side packer: histogram normalisation and tANS encoding into the two containers the
+// Host-side packer: histogram normalisation and tANS encoding into the containers the
 // decode kernels read.  CPU only, off the inference path (the paper compresses offline,
 // Section III-A).  The encoder is table driven: per symbol a threshold decides how many bits a
 // state sheds (Section II-A: "following a state transition ... and concatenating the binary
@@ -102,22 +102,64 @@ struct BitWriter {
 
 inline size_t lane_count(size_t nc, size_t W, size_t lambda) { return nc > lambda ? (nc - lambda + W - 1) / W : 0; }
 
+// Bits from the top of 32-bit words down, a field's high bit first; words go out little-endian.
+struct TopBitWriter {
+  std::vector<uint8_t>& out;
+  uint64_t acc = 0;      // pending bits, left-aligned in the low `fill` positions counted from bit 63
+  int fill = 0;
+  explicit TopBitWriter(std::vector<uint8_t>& o) : out(o) {}
+  void word(uint32_t w) { for (int b = 0; b < 4; ++b) out.push_back(static_cast<uint8_t>(w >> (8 * b))); }
+  void put(uint32_t v, int n) {
+    if (n == 0) return;
+    acc |= static_cast<uint64_t>(v) << (64 - fill - n);
+    fill += n;
+    if (fill >= 32) { word(static_cast<uint32_t>(acc >> 32)); acc <<= 32; fill -= 32; }
+  }
+  void finish() { if (fill > 0) { word(static_cast<uint32_t>(acc >> 32)); acc = 0; fill = 0; } }
+};
+
+// quads container: symbols a lane owns, and where its t-th symbol sits in the chunk
+inline size_t quad_lane_count(size_t nc, size_t W, size_t lambda) {
+  const size_t full = nc / 4, rem = nc % 4;
+  return 4 * (full > lambda ? (full - lambda + W - 1) / W : 0) + ((rem && full % W == lambda) ? rem : 0);
+}
+inline size_t quad_position(size_t W, size_t lambda, size_t t) { return ((t / 4) * W + lambda) * 4 + t % 4; }
+
 // One sub-stream (32 lanes) into `bytes` (appended) and meta (32 entries).
 bool pack_sub(const EncTable& T, const uint8_t* chunk, size_t nc, size_t W, size_t g, int layout,
               std::vector<uint8_t>& bytes, void* meta32, std::vector<uint8_t>& nb, std::vector<uint16_t>& val,
               std::vector<uint8_t>& lane_bytes) {
-  const size_t max_lane = lane_count(nc, W, 32 * g);
+  const bool quads = layout == ANS_LAYOUT_QUADS;
+  const size_t max_lane = quads ? 4 * ((nc / 4 + W - 1) / W) + 4 : lane_count(nc, W, 32 * g);
   nb.resize(32 * max_lane + 1);
   val.resize(32 * max_lane + 1);
   size_t cnt[32];
   int init[32];
   for (size_t k = 0; k < 32; ++k) {
-    cnt[k] = lane_count(nc, W, 32 * g + k);
-    init[k] = encode_lane(T, chunk + 32 * g + k, cnt[k], W, nb.data() + k * max_lane, val.data() + k * max_lane);
+    const size_t lambda = 32 * g + k;
+    if (quads) {
+      cnt[k] = quad_lane_count(nc, W, lambda);
+      lane_bytes.resize(max_lane);                    // the lane's symbols, gathered
+      for (size_t t = 0; t < cnt[k]; ++t) lane_bytes[t] = chunk[quad_position(W, lambda, t)];
+      init[k] = encode_lane(T, lane_bytes.data(), cnt[k], 1, nb.data() + k * max_lane, val.data() + k * max_lane);
+    } else {
+      cnt[k] = lane_count(nc, W, lambda);
+      init[k] = encode_lane(T, chunk + lambda, cnt[k], W, nb.data() + k * max_lane, val.data() + k * max_lane);
+    }
     if (init[k] < 0) return false;
   }
   const size_t base = bytes.size();
-  if (layout == ANS_LAYOUT_PRIVATE) {
+  if (quads) {
+    uint32_t* meta = static_cast<uint32_t*>(meta32);
+    for (size_t k = 0; k < 32; ++k) {
+      const size_t word0 = (bytes.size() - base) / 4;
+      if (word0 > 0xFFFF) return false;
+      meta[k] = static_cast<uint32_t>(init[k]) | (static_cast<uint32_t>(word0) << 16);
+      TopBitWriter bw(bytes);
+      for (size_t t = 0; t < cnt[k]; ++t) bw.put(val[k * max_lane + t], nb[k * max_lane + t]);
+      bw.finish();
+    }
+  } else if (layout == ANS_LAYOUT_PRIVATE) {
     uint32_t* meta = static_cast<uint32_t*>(meta32);
     for (size_t k = 0; k < 32; ++k) {
       const size_t word0 = (bytes.size() - base) / 4;
@@ -206,7 +248,8 @@ ANS_EXPORT int ans_host_normalize_freqs(const uint64_t* h_counts, int alphabet, 
 ANS_EXPORT int ans_host_pack_bound(uint64_t n_symbols, uint32_t chunk_symbols, uint32_t lanes, int layout,
                                    uint64_t* h_bytes_out) {
   if (!h_bytes_out || chunk_symbols == 0 || lanes == 0 || lanes % 32) return ANS_ERR_INVALID_ARG;
-  if (layout != ANS_LAYOUT_INTERLEAVED && layout != ANS_LAYOUT_PRIVATE) return ANS_ERR_UNSUPPORTED;
+  if (layout != ANS_LAYOUT_INTERLEAVED && layout != ANS_LAYOUT_PRIVATE && layout != ANS_LAYOUT_QUADS)
+    return ANS_ERR_UNSUPPORTED;
   const uint64_t chunks = n_symbols ? (n_symbols + chunk_symbols - 1) / chunk_symbols : 0;
   const uint64_t subs = chunks * (lanes / 32);
   // <= 14 bits per symbol, plus per lane a last unit/word, plus per sub-stream 16 bytes of pad
@@ -223,14 +266,15 @@ ANS_EXPORT int ans_host_pack_layer(const uint8_t* h_symbols, uint64_t n_symbols,
   if (alphabet < 1 || alphabet > ANS_MAX_ALPHABET || chunk_symbols == 0) return ANS_ERR_INVALID_ARG;
   if (table_log < 1 || table_log > ANS_MAX_TABLE_LOG) return ANS_ERR_UNSUPPORTED;
   if (lanes != 32 && lanes != 64 && lanes != 128 && lanes != 256) return ANS_ERR_UNSUPPORTED;
-  if (layout != ANS_LAYOUT_INTERLEAVED && layout != ANS_LAYOUT_PRIVATE) return ANS_ERR_UNSUPPORTED;
+  if (layout != ANS_LAYOUT_INTERLEAVED && layout != ANS_LAYOUT_PRIVATE && layout != ANS_LAYOUT_QUADS)
+    return ANS_ERR_UNSUPPORTED;
   if (n_symbols && (!h_symbols || !h_stream_out || !h_lane_meta_out)) return ANS_ERR_INVALID_ARG;
   EncTable T;
   if (!make_enc_table(h_freqs, alphabet, table_log, T)) return ANS_ERR_BAD_FREQS;
 
   const size_t C = chunk_symbols, W = lanes, G = lanes / 32;
   const size_t chunks = n_symbols ? (n_symbols + C - 1) / C : 0;
-  const size_t meta_es = layout == ANS_LAYOUT_PRIVATE ? 4 : 2;
+  const size_t meta_es = layout == ANS_LAYOUT_INTERLEAVED ? 2 : 4;
   unsigned nt = n_threads > 0 ? static_cast<unsigned>(n_threads) : std::thread::hardware_concurrency();
   nt = std::max(1u, std::min<unsigned>(nt, static_cast<unsigned>(std::max<size_t>(chunks, 1))));
 

@@ -58,7 +58,7 @@ ANS_EXPORT int ans_decode_dequant_host_noalloc(const ans_layer_desc* h_desc, con
   if (rc != ANS_OK) return rc;
   const uint64_t n_sub = subs_of(*h_desc);
   const size_t offs_bytes = (n_sub + 1) * 8;
-  const size_t meta_bytes = n_sub * 32 * (h_desc->layout == ANS_LAYOUT_PRIVATE ? 4 : 2);
+  const size_t meta_bytes = n_sub * 32 * (h_desc->layout == ANS_LAYOUT_INTERLEAVED ? 2 : 4);
   const size_t out_bytes = h_desc->n_symbols * elem_size(h_desc->out_dtype);
   const size_t need = 256 + up256(table_bytes) + up256(stream_bytes) + up256(offs_bytes) + up256(meta_bytes) +
                       up256(out_bytes);

@@ -44,13 +44,13 @@ def full_size(specs, layout, lanes, sample_chunks=64):
             assert np.array_equal(got[a:b], expected_bits(want)[a:b])
 
 
-@pytest.mark.parametrize("layout", [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE])
+@pytest.mark.parametrize("layout", [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE, ans.ANS_LAYOUT_QUADS])
 @pytest.mark.parametrize("table_log", [8, 12])
 def test_config5_large_layers_full(layout, table_log):
     full_size(sg.workload_large(table_log=table_log), layout, 32)
 
 
-@pytest.mark.parametrize("layout", [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE])
+@pytest.mark.parametrize("layout", [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE, ans.ANS_LAYOUT_QUADS])
 @pytest.mark.parametrize("chunk,R", [(1024, 11), (65536, 14), (16384, 12)])
 def test_config4_sweep_full(layout, chunk, R):
     full_size(sg.workload_sweep(table_log=R, chunk=chunk), layout, 32)

@@ -14,7 +14,8 @@ from helpers import (bits_view, expected_bits, oracle_expected, oracle_pack_spec
                      to_packed_layer)
 
 pytestmark = pytest.mark.gpu
-LAYOUTS = [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE]
+LAYOUTS = [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE, ans.ANS_LAYOUT_QUADS]
+OWN_WORDS = [ans.ANS_LAYOUT_PRIVATE, ans.ANS_LAYOUT_QUADS]
 
 
 def run_and_compare(specs, layout, lanes=32, per_layer=False, threads=8, chunk=None, table_log=None):
@@ -111,34 +112,38 @@ def test_config5_reduced(layout):
     run_and_compare(sg.workload_large(n_mats=2, dim=2048), layout, 32)
 
 
+@pytest.mark.parametrize("layout", OWN_WORDS)
 @pytest.mark.parametrize("lanes", [32, 64, 128, 256])
-@pytest.mark.parametrize("R", [1, 5, 8, 9])
-def test_private_layers_of_many_substreams(lanes, R):
-    """Private layers that average 64 or more work items and have at most 512 states are walked
-    one symbol per look-up, every lane storing straight to the output: whole 16-row blocks, the
-    rows after them, a ragged last row, every output type and every lane count."""
+@pytest.mark.parametrize("R", [1, 5, 8, 9, 12])
+def test_private_layers_of_many_substreams(layout, lanes, R):
+    """Private layers that average 64 or more work items and have at most 512 states, and quads
+    layers of any kind, are walked one symbol per look-up, every lane storing straight to the
+    output: whole blocks, the rows after them, a ragged end, chunks that start off a quad's
+    alignment, every output type and every lane count."""
     b = 1 if R == 1 else min(5, R)
     g = lanes // 32
     specs = [tiny_spec(300_017 // g * g + 5, b, 0.6, R, 999, "u8", index=0),
              tiny_spec(400_001, b, 0.75, R, 1001 * g, "bf16", index=1),
              tiny_spec(270_000 * g, b, 0.9, R, 777 * g, "f32", index=2),
              tiny_spec(1_100_000, b, 0.5, R, 4096, "bf16", index=3)]
-    db, prepared = run_and_compare(specs, ans.ANS_LAYOUT_PRIVATE, lanes)
+    db, prepared = run_and_compare(specs, layout, lanes)
     assert (db.decode_symbols(1).cpu().numpy() == prepared[1][1]).all()
     assert db.read_status() == 0
-    run_and_compare(specs[:2], ans.ANS_LAYOUT_PRIVATE, lanes, per_layer=True)
+    run_and_compare(specs[:2], layout, lanes, per_layer=True)
 
 
-def test_private_many_long_substreams_read_from_global_memory():
+@pytest.mark.parametrize("layout", OWN_WORDS)
+def test_private_many_long_substreams_read_from_global_memory(layout):
     """Sub-streams too long for the shared-memory staging buffer are read word by word from
     global memory; with many of them the layer still takes the one-symbol-per-look-up walk."""
-    run_and_compare([tiny_spec(260 * 65536 + 321, 5, 0.15, 8, 65536, "u8")], ans.ANS_LAYOUT_PRIVATE, 32)
+    run_and_compare([tiny_spec(260 * 65536 + 321, 5, 0.15, 8, 65536, "u8")], layout, 32)
 
 
-def test_private_many_substreams_corruption_is_flagged():
+@pytest.mark.parametrize("layout", OWN_WORDS)
+def test_private_many_substreams_corruption_is_flagged(layout):
     spec = tiny_spec(600_000, 3, 0.7, 8, 2048, "bf16")
     sym = sg.draw_symbols(spec)
-    T, P, f256 = oracle_pack_spec(spec, sym, ans.ANS_LAYOUT_PRIVATE, 32)
+    T, P, f256 = oracle_pack_spec(spec, sym, layout, 32)
     rng = np.random.default_rng(1)
     flagged = 0
     for trial in range(4):
