@@ -664,36 +664,76 @@ __device__ __forceinline__ uint2 to_quads_entry(uint32_t g, uint32_t val, bool n
   "st.global.v2.u32 " A_ ", {v0, v1};\n\t"
 #define ANSB_QD_OUT4(A_) "st.global.v4.u32 " A_ ", {eb0, eb1, eb2, eb3};\n\t"
 
-constexpr uint32_t kQuadTurns = 4;     // turns (of four symbols per lane) decoded by one PTX block
+constexpr uint32_t kQuadTurns = 4;     // turns (of four symbols per lane) per trip of the PTX loop
 
-// Same operands as lockstep_block; gp: this lane's four elements of the block's first turn
-// (turns are 128 * ES * G bytes apart).
-template <int ES, int K, int G>
-__device__ __forceinline__ void quads_block(uint32_t& st, uint32_t& bitpos, uint32_t& w0, uint32_t& w1,
-                                            uint32_t& w2, uint32_t& sp, uint32_t tab_lane, uint32_t stride,
-                                            uint8_t* gp, uint32_t unit) {
-  constexpr uint32_t RS = 128u * ES * G;
-#define ANSB_QD_ASM(TURN_, ST_, OUT_)                                                       \
+// The hot loop of the quads container: `blocks` times kQuadTurns turns, entirely in PTX (loop
+// included, so that nothing is carried through the compiler between trips).  Operands as in
+// lockstep_block; gp: this lane's four elements of the first turn; turns are 128 * ES * groups
+// bytes apart (immediate offsets when groups == 1); sp is held at sp_limit if a corrupt stream
+// drives it that far.
+template <int ES, int K>
+__device__ __forceinline__ void quads_loop(uint32_t& st, uint32_t& bitpos, uint32_t& w0, uint32_t& w1,
+                                           uint32_t& w2, uint32_t& sp, uint32_t tab_lane, uint32_t stride,
+                                           uint8_t* gp, uint32_t unit, uint32_t groups, uint32_t blocks,
+                                           uint32_t sp_limit) {
+  constexpr uint32_t RS = 128u * ES;
+#define ANSB_QD_ASM1(LBL_, TURN_, ST_, OUT_)                                                \
   asm volatile(                                                                             \
       "{\n\t"                                                                               \
       ".reg .pred q;\n\t"                                                                   \
-      ".reg .u32 x, t, nx, nw, v0, v1, ea0, ea1, ea2, ea3, eb0, eb1, eb2, eb3;\n\t"          \
-      TURN_(ST_) OUT_("[%8]") TURN_(ST_) OUT_("[%8+%10]")                                   \
-      TURN_(ST_) OUT_("[%8+%11]") TURN_(ST_) OUT_("[%8+%12]")                               \
+      ".reg .u32 x, t, nx, nw, v0, v1, cnt, ea0, ea1, ea2, ea3, eb0, eb1, eb2, eb3;\n\t"     \
+      ".reg .u64 gpp;\n\t"                                                                  \
+      "mov.u64 gpp, %8;\n\t"                                                                \
+      "mov.u32 cnt, %10;\n"                                                                 \
+      LBL_ ":\n\t"                                                                          \
+      TURN_(ST_) OUT_("[gpp]") TURN_(ST_) OUT_("[gpp+%12]")                                 \
+      TURN_(ST_) OUT_("[gpp+%13]") TURN_(ST_) OUT_("[gpp+%14]")                             \
+      "add.u64 gpp, gpp, %15;\n\t"                                                          \
+      "min.u32 %5, %5, %11;\n\t"                                                            \
+      "add.u32 cnt, cnt, -1;\n\t"                                                           \
+      "setp.ne.u32 q, cnt, 0;\n\t"                                                          \
+      "@q bra " LBL_ ";\n\t"                                                                \
       "}"                                                                                   \
       : "+r"(st), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp)                      \
-      : "r"(tab_lane), "r"(stride), "l"(gp), "r"(unit), "n"(RS * 1), "n"(RS * 2), "n"(RS * 3) \
+      : "r"(tab_lane), "r"(stride), "l"(gp), "r"(unit), "r"(blocks), "r"(sp_limit),         \
+        "n"(RS * 1), "n"(RS * 2), "n"(RS * 3), "n"(RS * 4)                                  \
       : "memory")
+#define ANSB_QD_ASMG(LBL_, TURN_, ST_, OUT_)                                                \
+  asm volatile(                                                                             \
+      "{\n\t"                                                                               \
+      ".reg .pred q;\n\t"                                                                   \
+      ".reg .u32 x, t, nx, nw, v0, v1, cnt, ea0, ea1, ea2, ea3, eb0, eb1, eb2, eb3;\n\t"     \
+      ".reg .u64 gpp;\n\t"                                                                  \
+      "mov.u64 gpp, %8;\n\t"                                                                \
+      "mov.u32 cnt, %10;\n"                                                                 \
+      LBL_ ":\n\t"                                                                          \
+      TURN_(ST_) OUT_("[gpp]") "add.u64 gpp, gpp, %12;\n\t"                                 \
+      TURN_(ST_) OUT_("[gpp]") "add.u64 gpp, gpp, %12;\n\t"                                 \
+      TURN_(ST_) OUT_("[gpp]") "add.u64 gpp, gpp, %12;\n\t"                                 \
+      TURN_(ST_) OUT_("[gpp]") "add.u64 gpp, gpp, %12;\n\t"                                 \
+      "min.u32 %5, %5, %11;\n\t"                                                            \
+      "add.u32 cnt, cnt, -1;\n\t"                                                           \
+      "setp.ne.u32 q, cnt, 0;\n\t"                                                          \
+      "@q bra " LBL_ ";\n\t"                                                                \
+      "}"                                                                                   \
+      : "+r"(st), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp)                      \
+      : "r"(tab_lane), "r"(stride), "l"(gp), "r"(unit), "r"(blocks), "r"(sp_limit),         \
+        "l"(static_cast<unsigned long long>(RS) * groups)                                   \
+      : "memory")
+#define ANSB_QD_BOTH(L1_, LG_, TURN_, ST_, OUT_)                                            \
+  if (groups == 1) ANSB_QD_ASM1(L1_, TURN_, ST_, OUT_); else ANSB_QD_ASMG(LG_, TURN_, ST_, OUT_)
   if (K == 4) {
-    if (ES == 1) ANSB_QD_ASM(ANSB_QD_TURN4, ANSB_QD_STEP_N, ANSB_QD_OUT1);
-    if (ES == 2) ANSB_QD_ASM(ANSB_QD_TURN4, ANSB_QD_STEP_N, ANSB_QD_OUT2);
-    if (ES == 4) ANSB_QD_ASM(ANSB_QD_TURN4, ANSB_QD_STEP_W, ANSB_QD_OUT4);
+    if (ES == 1) { ANSB_QD_BOTH("ANSB_Q41", "ANSB_Q4G", ANSB_QD_TURN4, ANSB_QD_STEP_N, ANSB_QD_OUT1); }
+    if (ES == 2) { ANSB_QD_BOTH("ANSB_Q41", "ANSB_Q4G", ANSB_QD_TURN4, ANSB_QD_STEP_N, ANSB_QD_OUT2); }
+    if (ES == 4) { ANSB_QD_BOTH("ANSB_Q41", "ANSB_Q4G", ANSB_QD_TURN4, ANSB_QD_STEP_W, ANSB_QD_OUT4); }
   } else {
-    if (ES == 1) ANSB_QD_ASM(ANSB_QD_TURN2, ANSB_QD_STEP_N, ANSB_QD_OUT1);
-    if (ES == 2) ANSB_QD_ASM(ANSB_QD_TURN2, ANSB_QD_STEP_N, ANSB_QD_OUT2);
-    if (ES == 4) ANSB_QD_ASM(ANSB_QD_TURN2, ANSB_QD_STEP_W, ANSB_QD_OUT4);
+    if (ES == 1) { ANSB_QD_BOTH("ANSB_Q21", "ANSB_Q2G", ANSB_QD_TURN2, ANSB_QD_STEP_N, ANSB_QD_OUT1); }
+    if (ES == 2) { ANSB_QD_BOTH("ANSB_Q21", "ANSB_Q2G", ANSB_QD_TURN2, ANSB_QD_STEP_N, ANSB_QD_OUT2); }
+    if (ES == 4) { ANSB_QD_BOTH("ANSB_Q21", "ANSB_Q2G", ANSB_QD_TURN2, ANSB_QD_STEP_W, ANSB_QD_OUT4); }
   }
-#undef ANSB_QD_ASM
+#undef ANSB_QD_BOTH
+#undef ANSB_QD_ASMG
+#undef ANSB_QD_ASM1
 }
 
 // Decode one sub-stream of the quads container.  full_turns: turns in which every lane of the
@@ -724,24 +764,16 @@ __device__ __noinline__ uint32_t decode_quads(
   // whole blocks: needs the staged copy, and quads that may leave as one vector store
   if (STAGED && (reinterpret_cast<uintptr_t>(out_lane) & (QB - 1u)) == 0) {
     uint32_t sp = stage_abs + idx * 4u;
-    const uint32_t sp_limit = stage_abs + word_limit * 4u;
-    const uint32_t stride = 1u << stride_log;
-    uint8_t* gp = out_lane;
-#define ANSB_QD_LOOP(K_, G_)                                                                \
-    while (turn + kQuadTurns <= full_turns) {                                               \
-      quads_block<ES, K_, G_>(st, bitpos, w0, w1, w2, sp, tab_abs, stride, gp, unit);       \
-      if (sp > sp_limit) { overran = true; sp = sp_limit; }                                 \
-      gp += kQuadTurns * 128u * ES * G_;                                                    \
-      turn += kQuadTurns;                                                                   \
+    const uint32_t sp_limit = stage_abs + word_limit * 4u;   // a sound lane stays below it
+    const uint32_t blocks = full_turns / kQuadTurns;
+    if (blocks) {
+      if (wide_steps) quads_loop<ES, 4>(st, bitpos, w0, w1, w2, sp, tab_abs, 1u << stride_log, out_lane, unit, groups,
+                                        blocks, sp_limit);
+      else quads_loop<ES, 2>(st, bitpos, w0, w1, w2, sp, tab_abs, 1u << stride_log, out_lane, unit, groups, blocks,
+                             sp_limit);
+      if (sp >= sp_limit) overran = true;
+      turn = blocks * kQuadTurns;
     }
-    if (wide_steps) {
-      if (groups == 1) { ANSB_QD_LOOP(4, 1) } else if (groups == 2) { ANSB_QD_LOOP(4, 2) }
-      else if (groups == 4) { ANSB_QD_LOOP(4, 4) } else if (groups == 8) { ANSB_QD_LOOP(4, 8) }
-    } else {
-      if (groups == 1) { ANSB_QD_LOOP(2, 1) } else if (groups == 2) { ANSB_QD_LOOP(2, 2) }
-      else if (groups == 4) { ANSB_QD_LOOP(2, 4) } else if (groups == 8) { ANSB_QD_LOOP(2, 8) }
-    }
-#undef ANSB_QD_LOOP
     idx = (sp - stage_abs) >> 2;
     k = 4u * turn;
   }
@@ -932,7 +964,7 @@ __device__ __noinline__ uint32_t decode_interleaved(
 // [table][pad to 1 KB][vals 256 words][mbarriers NW][stages NW * stage_bytes]
 
 template <int LAYOUT, bool LOCK>
-__global__ void __launch_bounds__(LOCK ? 1024 : 512, 1) ans_decode_kernel(const LaunchArgs args) {
+__global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const LaunchArgs args) {
   constexpr bool kQuads = LAYOUT == ANS_LAYOUT_QUADS;
   constexpr bool kPrivate = LAYOUT != ANS_LAYOUT_INTERLEAVED;   // lanes own their words
   constexpr bool lock = kPrivate && LOCK;           // walked one symbol per look-up (quads always are)
