@@ -75,7 +75,9 @@ struct Item {
   uint32_t bad;
 };
 
-__device__ __forceinline__ Item make_item(const ans_layer_desc& L, uint64_t sub) {
+// off0 / off1: d_sub_offsets[sub] and [sub + 1], loaded by the caller (so that it can request
+// them together with whatever else it needs from memory)
+__device__ __forceinline__ Item make_item(const ans_layer_desc& L, uint64_t sub, uint64_t off0, uint64_t off1) {
   Item it;
   const uint32_t G = L.lanes / 32u;
   it.sub = sub;
@@ -83,8 +85,7 @@ __device__ __forceinline__ Item make_item(const ans_layer_desc& L, uint64_t sub)
   it.g = static_cast<uint32_t>(sub % G);
   it.c0 = chunk * L.chunk_symbols;
   it.nc = static_cast<uint32_t>(min(uint64_t(L.chunk_symbols), L.n_symbols - it.c0));
-  it.off0 = __ldg(L.d_sub_offsets + sub);
-  const uint64_t off1 = __ldg(L.d_sub_offsets + sub + 1);
+  it.off0 = off0;
   it.extent = off1 - it.off0;
   it.bad = 0;
   if (off1 < it.off0 || off1 > L.stream_bytes || (it.off0 & 15u)) {   // never read outside the stream
@@ -1029,8 +1030,6 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
     const uint32_t W = L.lanes;
     const uint64_t n_sub = uint64_t(L.lanes / 32u) * ((L.n_symbols + L.chunk_symbols - 1) / L.chunk_symbols);
 
-    // The warp's first sub-stream of this layer: its bulk copy is started now so that it travels
-    // while the table is being staged.
     auto warp_sub = [&](uint64_t gbase, uint64_t& sub) -> bool {
       const uint64_t granule = gbase + warp / kGranule;
       sub = (granule - lbeg) * kGranule + warp % kGranule;
@@ -1051,36 +1050,55 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
       }
       return staged;
     };
-    Item first_item;
-    bool first_staged = false;
-    uint64_t first_sub = 0;
-    const bool have_first = warp_sub(cursor, first_sub);
-    if (have_first) {
-      first_item = make_item(L, first_sub);
-      first_staged = start_copy(first_item);
-    }
-
-    __syncthreads();                                      // previous layer's readers of the table are done
-    // Table staging: all of a thread's entries are requested before any is converted, so the
-    // whole table costs about one trip to memory.
+    // Everything the layer's start needs from memory is requested here, before any of it is
+    // used, so that it costs one trip and not one per item: the offsets and lane states of the
+    // warp's first sub-stream, the table's header, the first batch of table entries.
     constexpr uint32_t kStageBatch = 16;
     const uint32_t n_states = 1u << R;
-    for (uint32_t b0 = 0; b0 < n_states; b0 += blockDim.x * kStageBatch) {
-      uint32_t g[kStageBatch], g1[kStageBatch];
+    auto load_meta = [&](uint64_t sub) -> uint32_t {
+      if (kPrivate) return __ldg(static_cast<const uint32_t*>(L.d_lane_meta) + sub * 32 + lane);
+      return __ldg(static_cast<const uint16_t*>(L.d_lane_meta) + sub * 32 + lane);
+    };
+    uint64_t first_sub = 0, first_off0 = 0, first_off1 = 0;
+    uint32_t first_meta = 0;
+    const bool have_first = warp_sub(cursor, first_sub);
+    if (have_first) {
+      first_off0 = __ldg(L.d_sub_offsets + first_sub);
+      first_off1 = __ldg(L.d_sub_offsets + first_sub + 1);
+      first_meta = load_meta(first_sub);
+    }
+    const uint32_t h_magic = __ldg(&hdr->magic), h_log = __ldg(&hdr->table_log), h_alphabet = __ldg(&hdr->alphabet),
+                   h_dominant = __ldg(&hdr->dominant);
+    uint32_t g[kStageBatch], g1[kStageBatch];
+    auto request_entries = [&](uint32_t b0) {
 #pragma unroll
       for (uint32_t k = 0; k < kStageBatch; ++k) {
         const uint32_t i = b0 + k * blockDim.x + threadIdx.x;
         g[k] = i < n_states ? __ldg(g_multi + i) : 0u;
         if (kPrivate && !lock) g1[k] = i < n_states ? __ldg(g_single + i) : 0u;
       }
+    };
+    request_entries(0);
+
+    // The warp's first sub-stream of this layer: its bulk copy is started now so that it travels
+    // while the table is being staged.
+    Item first_item;
+    bool first_staged = false;
+    if (have_first) {
+      first_item = make_item(L, first_sub, first_off0, first_off1);
+      first_staged = start_copy(first_item);
+    }
+
+    __syncthreads();                                      // previous layer's readers of the table are done
+    for (uint32_t b0 = 0; b0 < n_states; b0 += blockDim.x * kStageBatch) {
+      if (b0 != 0) request_entries(b0);                   // a batch is requested whole before any entry is converted
       if (b0 == 0) {
         for (uint32_t i = threadIdx.x; i < 256u; i += blockDim.x)
           vals[i] = dequant_bits(static_cast<int>(i), L.zero_point, L.scale, dtype);
         if (threadIdx.x == 0) {
-          const uint32_t d = hdr->dominant;
-          s_dom = d < 256u ? d : 0u;                      // the ring's fill symbol
+          s_dom = h_dominant < 256u ? h_dominant : 0u;    // the ring's fill symbol
           s_maxadv = 1u;
-          if (hdr->magic != kTableMagic || hdr->table_log != uint32_t(R) || hdr->alphabet > (1u << L.bitwidth))
+          if (h_magic != kTableMagic || h_log != uint32_t(R) || h_alphabet > (1u << L.bitwidth))
             bad |= ANS_STATUS_BAD_SYMBOL;
         }
         __syncthreads();
@@ -1112,7 +1130,14 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
       uint64_t sub;
       if (!warp_sub(gbase, sub)) continue;
       const bool is_first = gbase == cursor;              // its copy is already under way
-      const Item it = is_first ? first_item : make_item(L, sub);
+      uint64_t off0 = 0, off1 = 0;
+      uint32_t meta = first_meta;
+      if (!is_first) {                                    // offsets and lane states in one trip
+        off0 = __ldg(L.d_sub_offsets + sub);
+        off1 = __ldg(L.d_sub_offsets + sub + 1);
+        meta = load_meta(sub);
+      }
+      const Item it = is_first ? first_item : make_item(L, sub, off0, off1);
       uint32_t wbad = it.bad;
       const uint32_t lambda = 32u * it.g + lane;
       // round-robin containers: symbols of this lane, rows of the sub-stream, rows all 32 lanes have.
@@ -1137,7 +1162,6 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
       const size_t rsb = size_t(W) * es;
       uint32_t state, wbeg = 0, wend = 0;
       if (kPrivate) {
-        const uint32_t meta = __ldg(static_cast<const uint32_t*>(L.d_lane_meta) + it.sub * 32 + lane);
         state = meta & ((1u << R) - 1u);
         wbeg = meta >> 16;
         wend = __shfl_down_sync(kFull, wbeg, 1);
@@ -1145,7 +1169,7 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
         if (wend > ext_words) { wend = ext_words; wbad |= ANS_STATUS_BAD_LENGTH; }
         if (wbeg > wend) { wbeg = wend; wbad |= ANS_STATUS_BAD_LENGTH; }
       } else {
-        state = __ldg(static_cast<const uint16_t*>(L.d_lane_meta) + it.sub * 32 + lane) & ((1u << R) - 1u);
+        state = meta & ((1u << R) - 1u);
       }
 
       if (staged) {
