@@ -31,7 +31,8 @@ struct LaunchArgs {
   uint8_t* d_symbols_override;     // ans_decode_layer: write symbols here instead of d_out
   uint32_t table_words;            // shared-memory words reserved for the table
   uint32_t stage_bytes;            // private layout: per-warp staging buffer for compressed bytes
-  uint32_t rep_log;                // log2 of the table copies in shared memory (1, 2, 4, 8 or 16 copies)
+  uint32_t rep_log;                // log2 of the copies of a largest table in shared memory (1 .. 16 copies)
+  uint32_t max_log;                // largest table_log of the launch
   uint32_t succ_bytes;             // private layout: shared-memory bytes of the successor table
   uint32_t ring_bytes;             // private layout: per-warp output ring (kRingRows rows of the widest dtype)
   uint32_t unit;                   // the value 1 (a run-time operand keeps a multiply-add a multiply-add)
@@ -985,9 +986,6 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
   // The table may sit in shared memory in several copies, entry i of copy c at slot i * copies + c.
   // A 64-bit load is served half a warp at a time over 16 bank pairs; with 16 copies every lane
   // of a half-warp has a bank pair of its own and random look-ups no longer collide.
-  const uint32_t reps = 1u << args.rep_log;
-  const uint32_t stride_log = 3u + args.rep_log;
-  const uint32_t tab_lane = tab_abs + (lane & (reps - 1u)) * 8u;
   uint32_t* vals = reinterpret_cast<uint32_t*>(sm + (vals_abs - sm_abs));
   uint16_t* succ = reinterpret_cast<uint16_t*>(sm + (succ_abs - sm_abs));
   uint8_t* ring = sm + (ring_abs - sm_abs);
@@ -1018,6 +1016,13 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
     if (lend <= cursor) continue;                         // empty layer
     const uint64_t stop = min(lend, cta_end);
     const int R = L.table_log;
+    // copies of this layer's table: a table smaller than the launch's largest uses the room for
+    // more of them (the pre-walked walk keeps an extra entry after the table, so it does not)
+    const uint32_t rep_log = (kPrivate && !lock) ? args.rep_log
+                                                 : min(4u, args.rep_log + (args.max_log - static_cast<uint32_t>(R)));
+    const uint32_t reps = 1u << rep_log;
+    const uint32_t stride_log = 3u + rep_log;
+    const uint32_t tab_lane = tab_abs + (lane & (reps - 1u)) * 8u;
     const uint8_t* blob = static_cast<const uint8_t*>(L.d_table);
     const TableHeader* hdr = reinterpret_cast<const TableHeader*>(blob);
     const uint32_t* g_single = reinterpret_cast<const uint32_t*>(blob + single_offset());
@@ -1110,7 +1115,8 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
         if (i < n_states) {
           const uint2 e = kQuads ? to_quads_entry(g[k], vals[entry_sym(g[k])], es != 4)
                                  : to_smem_entry(g[k], vals[entry_sym(g[k])], 32u * static_cast<uint32_t>(es));
-          for (uint32_t c = 0; c < reps; ++c) tab[(i << args.rep_log) + c] = e;
+          // every lane starts at another copy: the stores of a warp spread over the banks
+          for (uint32_t c = 0; c < reps; ++c) tab[(i << rep_log) + ((c + lane) & (reps - 1u))] = e;
           if (kPrivate && !lock) succ[i] = static_cast<uint16_t>(entry_newx(g1[k]));
           longest = max(longest, entry_run(g[k]) + 1u);
         }
@@ -1119,7 +1125,7 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
       if (lane == 0 && longest > 1u) atomicMax(&s_maxadv, longest);
     }
     if (threadIdx.x < reps && kPrivate && !lock && R <= kMaxParkLog)
-      tab[(n_states << args.rep_log) + threadIdx.x] =
+      tab[(n_states << rep_log) + threadIdx.x] =
           make_uint2(n_states << 17, es == 4 ? vals[s_dom] : (vals[s_dom] & 0xFFFFu));
     __syncthreads();
 
@@ -1278,6 +1284,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   a.d_status = d_status;
   a.d_symbols_override = d_symbols_override;
   a.unit = 1u;
+  a.max_log = static_cast<uint32_t>(max_log);
   a.table_words = 2u * ((1u << max_log) + 2u);           // two words per state, and a parking entry (one copy)
   if (n_layers <= kParamLayers) {
     a.n_begin = static_cast<uint32_t>(n_layers);
@@ -1327,6 +1334,9 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
     // lockstep warps need few registers and no ring: up to 28 of them, leaving room for the copies
     const size_t copies_room = lock ? (size_t(a.table_words) * 4) * 15 : 0;
     warps = big ? (lock ? 28 : 16) : 4;
+    // a model of small layers that would not fit one wave of 4-warp CTAs (three per SM): the
+    // lockstep kernels, light on registers, take two granules side by side rather than in turn
+    if (!big && lock && total > uint64_t(3) * sms) warps = 8;
     while (warps > 4 && fixed + copies_room + size_t(warps) * (ring + want) + 1024 > size_t(smem_max)) warps -= 4;
     while (warps > 4 && fixed + size_t(warps) * (ring + want) + 1024 > size_t(smem_max)) warps -= 4;
     const size_t room = size_t(smem_max) > fixed + size_t(warps) * ring + 1024
