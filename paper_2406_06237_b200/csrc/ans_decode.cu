@@ -37,7 +37,11 @@ struct LaunchArgs {
   uint32_t ring_bytes;             // private layout: per-warp output ring (kRingRows rows of the widest dtype)
   uint32_t unit;                   // the value 1 (a run-time operand keeps a multiply-add a multiply-add)
   uint32_t n_begin;                // entries of layer_begin in use (0: search the descriptors instead)
-  uint32_t layer_begin[kParamLayers];   // work_begin of the first layers, searchable without a memory trip
+  // Where each layer's work items start in the numbering the CTAs walk.  When the launch's layers
+  // all fit here, every layer's count is rounded up to the items a CTA takes at a time, so that
+  // a CTA's rounds line up with the start of every layer it meets (the padding items are empty);
+  // otherwise the numbering is the plan's (work_begin) and the descriptors are searched.
+  uint32_t layer_begin[kParamLayers];
 };
 
 __device__ __forceinline__ const ans_layer_desc& layer_at(const LaunchArgs& a, int l) {
@@ -1010,10 +1014,13 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
   int l = find_layer(args, cursor);
   uint32_t bad = 0;
   bool gave_up = false;
-  for (; cursor < cta_end; ++l) {
+  const bool begins_in_params = args.n_begin == static_cast<uint32_t>(args.n_layers);
+  for (; cursor < cta_end && l < args.n_layers; ++l) {
     const ans_layer_desc L = layer_at(args, l);           // one batch of loads, then registers
-    const uint64_t lbeg = L.work_begin, lend = lbeg + L.work_count;
-    if (lend <= cursor) continue;                         // empty layer
+    const uint64_t lbeg = begins_in_params ? args.layer_begin[l] : L.work_begin, lend = lbeg + L.work_count;
+    if (lend <= cursor) continue;                         // empty layer, or only its padding is left
+    if (cursor < lbeg) cursor = lbeg;                     // past the padding after the layer before
+    if (cursor >= cta_end) break;
     const uint64_t stop = min(lend, cta_end);
     const int R = L.table_log;
     // copies of this layer's table: a table smaller than the launch's largest uses the room for
@@ -1286,10 +1293,6 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   a.unit = 1u;
   a.max_log = static_cast<uint32_t>(max_log);
   a.table_words = 2u * ((1u << max_log) + 2u);           // two words per state, and a parking entry (one copy)
-  if (n_layers <= kParamLayers) {
-    a.n_begin = static_cast<uint32_t>(n_layers);
-    for (int l = 0; l < n_layers; ++l) a.layer_begin[l] = h_descs[l].work_begin;
-  }
 
   // device facts and per-configuration occupancy are looked up once and remembered (plain values,
   // no allocation): a launch of a small model should not spend its time in attribute queries
@@ -1369,6 +1372,19 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   }
   if (per_sm < 1) return ANS_ERR_UNSUPPORTED;
   const uint64_t step = uint64_t(warps) / kGranule;       // granules a CTA takes at a time
+  if (n_layers <= kParamLayers) {
+    // every layer starts on a multiple of `step` in the numbering the CTAs walk: a CTA that meets
+    // a new layer starts it with a full round of warps instead of finishing a ragged one first
+    a.n_begin = static_cast<uint32_t>(n_layers);
+    uint64_t padded = 0;
+    for (int l = 0; l < n_layers; ++l) {
+      a.layer_begin[l] = static_cast<uint32_t>(padded);
+      padded += (uint64_t(h_descs[l].work_count) + step - 1) / step * step;
+    }
+    if (padded > 0xFFFFFFFFull) return ANS_ERR_UNSUPPORTED;
+    total = padded;
+    a.total_work = static_cast<uint32_t>(total);
+  }
   const uint64_t want_ctas = (total + step - 1) / step;
   const uint64_t grid = want_ctas < uint64_t(sms) * per_sm ? want_ctas : uint64_t(sms) * per_sm;
   uint64_t ipc = (total + grid - 1) / grid;
