@@ -32,9 +32,9 @@ NOMINAL_PEAK_GBS = 8000.0
 FALLBACK_PEAK_GBS = 6650.0
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, scaled from the 2-matrix captures in
-# profiles/ans_decode_kernel_*_large.md to the 8 matrices of a full launch
-NCU_TRAFFIC = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, scaled from the 2-matrix capture in
+# profiles/ans_decode_kernel_quads_large.md to the 8 matrices of a full launch
+NCU_TRAFFIC = {("large", "quads", 32, 8, 8192, 0, 0): 1014.3e6}      # 256-state table (the default)
 
 
 def measured_peak():
@@ -71,7 +71,8 @@ WORKLOAD_TEXT = {
 
 
 # the container each workload is timed on unless --layout says otherwise: the fastest measured
-DEFAULT_LAYOUT = {"large": "quads", "resnet18": "quads", "resnet50": "quads", "sweep": "private", "conv3x3": "private"}
+DEFAULT_LAYOUT = {"large": "quads", "resnet18": "quads", "resnet50": "private", "sweep": "private",
+                  "conv3x3": "private"}
 
 
 class ClockSampler:
@@ -82,12 +83,16 @@ class ClockSampler:
 
     def __init__(self, index):
         self.index, self.rows, self.proc = index, [], None
+        self.first, self.last, self.in_timed = 0, None, None     # rows taken under the timed load
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
                                           "-i", str(self.index), "-lms", "20"], stdout=subprocess.PIPE, text=True)
             threading.Thread(target=self._read, daemon=True).start()
+            t_end = time.perf_counter() + 5.0               # be sampling before the warm-up starts
+            while not self.rows and time.perf_counter() < t_end:
+                time.sleep(0.01)
         except Exception:
             self.proc = None
 
@@ -102,17 +107,23 @@ class ClockSampler:
                 self.proc.wait(timeout=5)
             except Exception:
                 pass
-        sm = [float(r[1]) for r in self.rows if len(r) >= 9 and r[1].replace(".", "").isdigit()]
-        mx = [float(r[2]) for r in self.rows if len(r) >= 9 and r[2].replace(".", "").isdigit()]
+        rows = self.rows[self.first:self.last]
+        sm = [float(r[1]) for r in rows if len(r) >= 9 and r[1].replace(".", "").isdigit()]
+        mx = [float(r[2]) for r in rows if len(r) >= 9 and r[2].replace(".", "").isdigit()]
         reasons = set()
-        for r in self.rows:
+        for r in rows:
             if len(r) < 9:
                 continue
             for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        out = {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+               "reasons": sorted(reasons), "samples": len(sm)}
+        if self.in_timed is not None and self.in_timed < len(sm):
+            out["samples_in_timed_region"] = self.in_timed
+            out["note"] = ("the timed region is shorter than a few sampling periods (20 ms): the same launches "
+                           "were kept running right after it until 5 samples were in")
+        return out
 
 
 def cpu_baseline(specs, syms, layout_name, budget_s=12.0):
@@ -210,7 +221,7 @@ def reduce_max(x: float, world: int) -> float:
     return float(t.item())
 
 
-def time_workload(db, steps, warmup, flush, n_sets, world):
+def time_workload(db, steps, warmup, flush, n_sets, world, sampler=None):
     """K timed steps, each bracketed by CUDA events on the launching stream; the L2 flush (if
     any) sits outside the brackets.  Returns per-step milliseconds (max over ranks of the sum)."""
     import torch
@@ -225,6 +236,8 @@ def time_workload(db, steps, warmup, flush, n_sets, world):
         dist.barrier()
     torch.cuda.synchronize()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    if sampler is not None:
+        sampler.first = len(sampler.rows)
     for i in range(steps):
         if flush is not None:
             flush.add_(1)
@@ -232,6 +245,16 @@ def time_workload(db, steps, warmup, flush, n_sets, world):
         db.decode(i % n_sets)
         ev[i][1].record(st)
     torch.cuda.synchronize()
+    if sampler is not None and sampler.proc is not None:
+        # a clock reading needs a few sampling periods of load: keep the same launches going
+        # (outside every timing bracket) until they are in
+        sampler.in_timed = len(sampler.rows) - sampler.first
+        t_end = time.perf_counter() + 2.0
+        while len(sampler.rows) - sampler.first < 5 and time.perf_counter() < t_end:
+            for i in range(steps):
+                db.decode(i % n_sets)
+            torch.cuda.synchronize()
+        sampler.last = len(sampler.rows)
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
@@ -288,7 +311,7 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ms, span = time_workload(db, args.steps, args.warmup, flush, n_sets, world)
+    ms, span = time_workload(db, args.steps, args.warmup, flush, n_sets, world, sampler if rank == 0 else None)
     clocks = sampler.stop() if rank == 0 else None
     total_ms = reduce_max(span, world)
     ms_per_step = total_ms / args.steps
@@ -320,21 +343,22 @@ def run_ours(args):
     if not args.no_e2e:
         e2e = run_e2e(ans, db, layers, args, world)
 
-    # the same workload with the other table size the design notes quote (2^12 states)
+    # the same workload with the other table size the design notes quote (2^12 states), in the
+    # container that is fastest there (private lanes walked through the pre-walked entries)
     variants = []
     if args.workload == "large" and not args.table_log and world == 1 and not args.no_variants:
         db = None
         torch.cuda.empty_cache()
         with ThreadPoolExecutor(4) as ex:
             layers12 = list(ex.map(lambda sp_sy: pack_layer(sp_sy[1], sp_sy[0].alphabet, 12, sp_sy[0].chunk_symbols,
-                                                            args.lanes, layout, sp_sy[0].bitwidth, sp_sy[0].zero_point,
+                                                            args.lanes, ans.ANS_LAYOUT_PRIVATE, sp_sy[0].bitwidth, sp_sy[0].zero_point,
                                                             sp_sy[0].scale, ans.DTYPES[sp_sy[0].out_dtype],
                                                             n_threads=max(1, cores // 2)), zip(specs, syms)))
         db12 = DeviceBatch(layers12, f"cuda:{local}", n_out_sets=1)
         ms12, _ = time_workload(db12, min(args.steps, 50), 5, None, 1, 1)
         bytes12 = db12.compressed_bytes() + sum(4 << 12 for _ in layers12) + out_bytes
         k12 = statistics.mean(ms12)
-        variants.append({"table_log": 12, "kernel_ms_mean": k12, "value": n_w / (k12 * 1e-3), "unit": "weights/s",
+        variants.append({"table_log": 12, "layout": "private", "kernel_ms_mean": k12, "value": n_w / (k12 * 1e-3), "unit": "weights/s",
                          "achieved_gbs": bytes12 / (k12 * 1e-3) / 1e9, "frac": bytes12 / (k12 * 1e-3) / 1e9 / peak,
                          "coded_bits_per_weight": 8.0 * db12.compressed_bytes() / n_w})
         del db12

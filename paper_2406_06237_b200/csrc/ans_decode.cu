@@ -3,12 +3,15 @@
 // Paper Section II-A / Fig. 2: state -> (symbol, nb_bits, newX); take nb_bits from the stream;
 // next state = newX + bits.  Section III-B: one table per layer, a vector of states, one state per
 // stream.  Here a warp holds 32 of those states (one per thread) and walks them together; the
-// layer's table sits in shared memory; the decoded symbol goes through a 256-entry table of
-// already dequantised values (Section II-B: w = scale * (q - zero_point)) on its way out.
+// layer's table sits in shared memory, its entries already carrying the dequantised value
+// (Section II-B: w = scale * (q - zero_point)) in the output's bit pattern.
 //
 // One sub-stream (32 lanes) is decoded by one warp.  The work list counts granules of up to
 // kGranule consecutive sub-streams of a layer; a CTA owns a contiguous range of granules, walks
 // it one sub-stream per warp at a time and restages the table only when the layer changes.
+// Four walks share that skeleton: the interleaved container; the private container through its
+// pre-walked entries (a look-up may emit a run of the dominant symbol plus one symbol) or one
+// symbol per look-up with the lanes in lockstep; the quads container (always lockstep).
 #include <cuda_bf16.h>
 
 #include "ans_common.cuh"
@@ -967,7 +970,7 @@ __device__ __noinline__ uint32_t decode_interleaved(
 }
 
 // dynamic shared memory, by absolute shared address: [pad to ring_bytes][rings: NW * ring_bytes]
-// [table][pad to 1 KB][vals 256 words][mbarriers NW][stages NW * stage_bytes]
+// [table, in copies][pad to 1 KB][vals 256 words][successor table][mbarriers NW][stages NW * stage_bytes]
 
 template <int LAYOUT, bool LOCK>
 __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const LaunchArgs args) {

@@ -89,6 +89,18 @@ def test_batch_with_mixed_layers_one_launch(layout):
 
 
 @pytest.mark.parametrize("layout", LAYOUTS)
+def test_batch_of_more_layers_than_the_kernel_parameters_hold(layout):
+    """Beyond 96 layers the CTAs search the descriptors for their layer instead of the launch
+    parameters, and walk the plan's own numbering; empty layers and one-chunk layers mixed in."""
+    dts = ("bf16", "u8", "f32")
+    specs = [tiny_spec(0 if i % 17 == 5 else 900 + 611 * (i % 13) + (40_000 if i % 29 == 0 else 0),
+                       1 + i % 6, 0.55 + 0.04 * (i % 10), 6 + i % 7, 1024 << (i % 3), dts[i % 3], index=i)
+             for i in range(131)]
+    run_and_compare(specs, layout, 32)
+    run_and_compare(specs[:100], layout, 64)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
 def test_config2_resnet18_bf16(layout):
     run_and_compare(sg.workload_resnet18(), layout, 32)
 
