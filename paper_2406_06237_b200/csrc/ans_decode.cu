@@ -814,16 +814,14 @@ __device__ __noinline__ uint32_t decode_quads(
 // =============================================================================================
 // Interleaved container: the warp's 32 lanes share one sequence of 16-bit units; before each
 // round a lane whose buffer holds fewer than 16 bits takes the next unit, its place found by
-// ballot + popcount; then every lane decodes one symbol.  Same shared-memory table, staging
-// buffer and output ring as above (every look-up emits exactly one symbol, so the ring needs no
-// pre-fill and no parking).
+// ballot + popcount; then every lane decodes one symbol.  Same shared-memory table and staging
+// buffer as above.  Every look-up emits exactly one symbol, so a round completes a row of the
+// output and every lane stores its element straight to it (32 * ES contiguous bytes per row).
 // =============================================================================================
 template <int ES>
 __device__ __forceinline__ void interleaved_rounds(uint32_t& st, uint32_t& buf, uint32_t& cnt, uint32_t& posaddr,
-                                                   uint32_t& rb, uint32_t n, uint32_t lt, uint32_t limaddr,
-                                                   uint32_t tab_abs, uint32_t ring_lane_abs, uint32_t stride) {
-  constexpr uint32_t RB = 32u * ES;
-  constexpr uint32_t MASK = kRingRows * RB - 1u;
+                                                   uint8_t*& gp, uint32_t n, uint32_t lt, uint32_t limaddr,
+                                                   uint32_t tab_abs, uint32_t stride, unsigned long long row_stride) {
 #define ANSB_ROUNDS(STOP_)                                                                 \
   asm volatile(                                                                            \
       "{\n\t"                                                                              \
@@ -849,41 +847,35 @@ __device__ __forceinline__ void interleaved_rounds(uint32_t& st, uint32_t& buf, 
       "shf.l.wrap.b32 m, 0, -1, ea;\n\t"                                                   \
       "shr.u32 nx, ea, 17;\n\t"                                                            \
       "lop3.b32 t, nx, %1, m, 0xF4;\n\t"                                                   \
-      "mad.lo.u32 %0, t, %12, %8;\n\t"                                                     \
+      "mad.lo.u32 %0, t, %9, %8;\n\t"                                                      \
       "shf.r.wrap.b32 %1, %1, 0, ea;\n\t"                                                  \
       "and.b32 t, ea, 15;\n\t"                                                             \
       "sub.u32 %2, %2, t;\n\t"                                                             \
-      "lop3.b32 a, %4, %11, %9, 0xEA;\n\t"                                                 \
-      STOP_ " [a], eb;\n\t"                                                                \
-      "add.u32 %4, %4, %10;\n\t"                                                           \
+      STOP_ " [%4], eb;\n\t"                                                               \
+      "add.u64 %4, %4, %10;\n\t"                                                           \
       "add.u32 cntr, cntr, -1;\n\t"                                                        \
       "setp.ne.u32 q, cntr, 0;\n\t"                                                        \
       "@q bra ANSB_RLOOP;\n\t"                                                             \
       "}"                                                                                  \
-      : "+r"(st), "+r"(buf), "+r"(cnt), "+r"(posaddr), "+r"(rb)                            \
-      : "r"(n), "r"(lt), "r"(limaddr), "r"(tab_abs), "r"(ring_lane_abs), "n"(RB), "n"(MASK), \
-        "r"(stride)                                                                        \
+      : "+r"(st), "+r"(buf), "+r"(cnt), "+r"(posaddr), "+l"(gp)                            \
+      : "r"(n), "r"(lt), "r"(limaddr), "r"(tab_abs), "r"(stride), "l"(row_stride)          \
       : "memory")
-  if (ES == 1) ANSB_ROUNDS("st.shared.u8");
-  if (ES == 2) ANSB_ROUNDS("st.shared.u16");
-  if (ES == 4) ANSB_ROUNDS("st.shared.u32");
+  if (ES == 1) ANSB_ROUNDS("st.global.u8");
+  if (ES == 2) ANSB_ROUNDS("st.global.u16");
+  if (ES == 4) ANSB_ROUNDS("st.global.u32");
 #undef ANSB_ROUNDS
 }
 
 template <int ES, bool STAGED>
 __device__ __noinline__ uint32_t decode_interleaved(
-    uint32_t tab_abs, uint32_t stride_log, uint32_t ring_abs, uint32_t stage_abs, uint8_t* __restrict__ ring,
-    const uint16_t* __restrict__ units, uint32_t unit_cap, uint32_t state, uint32_t my_count, uint32_t rows,
-    uint32_t min_count, uint8_t* __restrict__ out_row0, size_t row_stride_bytes, uint32_t lane, bool allow_bulk) {
-  constexpr uint32_t RB = 32u * ES;
-  constexpr uint32_t RING = kRingRows, FL = kFlushRows;
-  constexpr uint32_t MASK = RING * RB - 1u;
-  const uint32_t ring_lane_abs = ring_abs + lane * ES;
+    uint32_t tab_abs, uint32_t stride_log, uint32_t stage_abs, const uint16_t* __restrict__ units, uint32_t unit_cap,
+    uint32_t state, uint32_t my_count, uint32_t rows, uint32_t min_count, uint8_t* __restrict__ out_row0,
+    size_t row_stride_bytes, uint32_t lane) {
   const uint32_t lt = (1u << lane) - 1u;
   uint32_t st = tab_abs + (state << stride_log);    // shared address of the state's table entry
   uint32_t buf = 0, cnt = 0;                        // the lane's bit buffer and how many bits it holds
   uint32_t pos = 0;                                 // units the warp has taken (same in every lane)
-  uint32_t rb = 0;                                  // RB * round
+  uint8_t* gp = out_row0 + size_t(lane) * ES;       // this lane's element of the next row
 
   // one round in plain code: used when the sub-stream was not staged, and for the ragged round
   auto round = [&](bool active) {
@@ -904,64 +896,20 @@ __device__ __noinline__ uint32_t decode_interleaved(
       st = tab_abs + (((ea >> 17) | (buf & ((1u << nb) - 1u))) << stride_log);
       buf >>= nb;
       cnt -= nb;
-      sts_elem<ES>((rb & MASK) | ring_lane_abs, eb);
+      stg_elem<ES>(gp, eb);
     }
-    rb += RB;
+    gp += row_stride_bytes;
   };
 
-  const bool bulk_ok = allow_bulk && ((reinterpret_cast<uintptr_t>(out_row0) | row_stride_bytes) & 15u) == 0;
-  const bool contiguous = row_stride_bytes == RB;
-  const bool issuer = contiguous ? lane == 0 : lane < FL;
-  // FL full rows starting at a multiple of FL leave the ring: bulk asynchronous stores when the
-  // output is 16-byte aligned (a ring slot is written again only four blocks later, by when at
-  // most three newer copies may still be pending), plain 16-byte stores otherwise
-  auto write_block = [&](uint32_t first_row) {
-    const uint32_t ring_row = first_row % RING;
-    if (bulk_ok) {
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      __syncwarp();
-      if (issuer) {
-        const uint32_t row = contiguous ? 0u : lane;
-        const uint32_t bytes = contiguous ? FL * RB : RB;
-        uint8_t* dst = out_row0 + size_t(first_row + row) * row_stride_bytes;
-        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                     :: "l"(dst), "r"(ring_abs + (ring_row + row) * RB), "r"(bytes) : "memory");
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        asm volatile("cp.async.bulk.wait_group.read 2;" ::: "memory");
-      }
-      __syncwarp();
-    } else {
-      __syncwarp();
-      flush_rows<ES>(ring + size_t(ring_row) * RB, out_row0 + size_t(first_row) * row_stride_bytes,
-                     row_stride_bytes, FL, 0u, lane);
-      __syncwarp();
-    }
-  };
-
-  uint32_t r = 0;
-  while (r < min_count) {                           // rounds in which all 32 lanes decode
-    const uint32_t n = min(FL - (r % FL), min_count - r);
-    if (STAGED) {
-      uint32_t posaddr = stage_abs + pos * 2u;
-      interleaved_rounds<ES>(st, buf, cnt, posaddr, rb, n, lt, stage_abs + unit_cap * 2u, tab_abs, ring_lane_abs,
-                             1u << stride_log);
-      pos = (posaddr - stage_abs) >> 1;
-    } else {
-      for (uint32_t i = 0; i < n; ++i) round(true);
-    }
-    r += n;
-    if (r % FL == 0) write_block(r - FL);
+  if (STAGED && min_count) {                        // rounds in which all 32 lanes decode
+    uint32_t posaddr = stage_abs + pos * 2u;
+    interleaved_rounds<ES>(st, buf, cnt, posaddr, gp, min_count, lt, stage_abs + unit_cap * 2u, tab_abs,
+                           1u << stride_log, static_cast<unsigned long long>(row_stride_bytes));
+    pos = (posaddr - stage_abs) >> 1;
+  } else {
+    for (uint32_t i = 0; i < min_count; ++i) round(true);
   }
   if (rows > min_count) round(my_count == rows);    // the ragged last round
-  __syncwarp();
-  {
-    const uint32_t base = (min_count / FL) * FL;    // rows before it have left already
-    const uint32_t part_lanes = rows > min_count ? __popc(__ballot_sync(kFull, my_count == rows)) : 0u;
-    flush_rows<ES>(ring + size_t(base % RING) * RB, out_row0 + size_t(base) * row_stride_bytes, row_stride_bytes,
-                   min_count - base, part_lanes, lane);
-  }
-  if (bulk_ok) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-  __syncwarp();
   uint32_t bad = 0;
   if (st != tab_abs) bad |= ANS_STATUS_BAD_FINAL_STATE;
   // the units taken, padded to 16 bytes, must be exactly the sub-stream's extent
@@ -974,6 +922,8 @@ __device__ __noinline__ uint32_t decode_interleaved(
 
 template <int LAYOUT, bool LOCK>
 __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const LaunchArgs args) {
+  // LOCK: the walks that store rows straight to the output (interleaved, private lockstep, quads);
+  // they run up to 28 warps per CTA.  Not LOCK: the private container's pre-walked walk.
   constexpr bool kQuads = LAYOUT == ANS_LAYOUT_QUADS;
   constexpr bool kPrivate = LAYOUT != ANS_LAYOUT_INTERLEAVED;   // lanes own their words
   constexpr bool lock = kPrivate && LOCK;           // walked one symbol per look-up (quads always are)
@@ -1000,10 +950,6 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
   const uint32_t bar = bars_abs + warp * 8u;
   __shared__ uint32_t s_dom, s_maxadv;
   uint32_t parity = 0;
-  // Interleaved container: bulk asynchronous stores save instructions but make a warp wait for
-  // the copy engine now and then; that pays when many warps share the SM (large CTAs), not when
-  // a few warps run a short, latency-bound job each.
-  const bool allow_bulk = NW > kGranule;
 
   uint64_t cursor = uint64_t(blockIdx.x) * args.items_per_cta;
   const uint64_t cta_end = min(cursor + uint64_t(args.items_per_cta), uint64_t(args.total_work));
@@ -1236,8 +1182,8 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
         const uint16_t* units = reinterpret_cast<const uint16_t*>(g_bytes);
         const uint32_t unit_cap = ext_words * 2u;
 #define ANSB_CALL(ES_, ST_)                                                                              \
-  wbad |= decode_interleaved<ES_, ST_>(tab_lane, stride_log, ring_abs, stage_abs, ring, units, unit_cap, state, my_count, \
-                                       rows, min_count, out_row0, rsb, lane, allow_bulk)
+  wbad |= decode_interleaved<ES_, ST_>(tab_lane, stride_log, stage_abs, units, unit_cap, state, my_count, rows, \
+                                       min_count, out_row0, rsb, lane)
         if (staged) {
           if (es == 1) ANSB_CALL(1, true); else if (es == 2) ANSB_CALL(2, true); else ANSB_CALL(4, true);
         } else {
@@ -1326,20 +1272,27 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   const void* fn = quads  ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_QUADS, true>)
                    : lock ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, true>)
                    : priv ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, false>)
-                          : reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, false>);
+                          : reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, true>);
   int warps = 4;
   a.succ_bytes = (priv && !lock) ? ((2u << max_log) + 15u) & ~15u : 0u;
   size_t smem = (size_t(a.table_words) + 256) * 4 + a.succ_bytes;
   {
     // per warp: an output ring of kRingRows rows of the widest dtype, and a staging buffer for
     // the largest layer-average sub-stream plus a margin (a longer one is read from global memory)
-    const size_t ring = lock ? 0 : size_t(kRingRows) * 32 * max_es;   // lockstep rows go straight to the output
+    // only the pre-walked walk buffers its output; the others store rows straight to it
+    const bool direct = lock || !priv;
+    const size_t ring = direct ? 0 : size_t(kRingRows) * 32 * max_es;
     size_t want = max_avg_sub + max_avg_sub / 16 + 256 + kStagePad;
     want = (want + 127) & ~size_t(127);
     const size_t fixed = ring + 1024 + smem + 32 * 8;     // alignment slack, table, vals, barriers
-    // lockstep warps need few registers and no ring: up to 28 of them, leaving room for the copies
-    const size_t copies_room = lock ? (size_t(a.table_words) * 4) * 15 : 0;
-    warps = big ? (lock ? 28 : 16) : 4;
+    // warps that store straight to the output need few registers and no ring: up to 28 of them,
+    // leaving room for the copies
+    // (tables of up to 512 states get all 16 copies, which pays for the warps they displace;
+    // larger ones about 33 KB in all: 4 copies of 1024 states, ..., 1 from 4096 up; measured)
+    const size_t one = size_t(a.table_words) * 4;
+    const size_t copies_room = !direct ? 0 : max_log <= 9 ? one * 15
+                               : one < (size_t(33) << 10) ? (size_t(33) << 10) - one : 0;
+    warps = big ? (direct ? 28 : 16) : 4;
     // a model of small layers that would not fit one wave of 4-warp CTAs (three per SM): the
     // lockstep kernels, light on registers, take two granules side by side rather than in turn
     if (!big && lock && total > uint64_t(3) * sms) warps = 8;
@@ -1401,7 +1354,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   else if (priv)
     ans_decode_kernel<ANS_LAYOUT_PRIVATE, false><<<blocks, warps * 32, smem, st>>>(a);
   else
-    ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, false><<<blocks, warps * 32, smem, st>>>(a);
+    ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, true><<<blocks, warps * 32, smem, st>>>(a);
   ANSB_CUDA(cudaGetLastError());
   return ANS_OK;
 }
