@@ -71,8 +71,7 @@ WORKLOAD_TEXT = {
 
 
 # the container each workload is timed on unless --layout says otherwise: the fastest measured
-DEFAULT_LAYOUT = {"large": "quads", "resnet18": "quads", "resnet50": "private", "sweep": "quads",
-                  "conv3x3": "private"}
+DEFAULT_LAYOUT = {"large": "quads", "resnet18": "quads", "resnet50": "quads", "sweep": "quads", "conv3x3": "quads"}
 
 
 class ClockSampler:

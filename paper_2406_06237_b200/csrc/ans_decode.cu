@@ -920,10 +920,13 @@ __device__ __noinline__ uint32_t decode_interleaved(
 // dynamic shared memory, by absolute shared address: [pad to ring_bytes][rings: NW * ring_bytes]
 // [table, in copies][pad to 1 KB][vals 256 words][successor table][mbarriers NW][stages NW * stage_bytes]
 
-template <int LAYOUT, bool LOCK>
-__global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const LaunchArgs args) {
-  // LOCK: the walks that store rows straight to the output (interleaved, private lockstep, quads);
-  // they run up to 28 warps per CTA.  Not LOCK: the private container's pre-walked walk.
+template <int LAYOUT, bool LOCK, bool MANY>
+__global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const LaunchArgs args) {
+  // LOCK: the walks that store rows straight to the output (interleaved, private lockstep, quads).
+  // Not LOCK: the private container's pre-walked walk.  MANY: up to 28 warps per CTA on 72
+  // registers (the LOCK walks on large layers); otherwise up to 16 warps and no register
+  // pressure, which the small CTAs of small-layer models want: a spill there is a cold trip to
+  // memory on a path that is all latency.
   constexpr bool kQuads = LAYOUT == ANS_LAYOUT_QUADS;
   constexpr bool kPrivate = LAYOUT != ANS_LAYOUT_INTERLEAVED;   // lanes own their words
   constexpr bool lock = kPrivate && LOCK;           // walked one symbol per look-up (quads always are)
@@ -1204,7 +1207,7 @@ __global__ void __launch_bounds__(LOCK ? 896 : 512, 1) ans_decode_kernel(const L
 // ---------------------------------------------------------------------------------------------
 constexpr int kMaxDevices = 64;
 struct LaunchShape { size_t smem = 0; int warps = 0; int per_sm = 0; };
-struct DeviceFacts { int sms = 0; int smem_max = 0; LaunchShape shape[4]; };
+struct DeviceFacts { int sms = 0; int smem_max = 0; LaunchShape shape[8]; };
 static DeviceFacts g_facts[kMaxDevices];    // remembered per device; racing writers store equal values
 
 static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, int n_layers,
@@ -1269,11 +1272,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   // the one-symbol-per-look-up walk the faster one (measured); larger tables, and models of
   // small layers, are walked through the pre-walked entries.
   const bool lock = quads || (priv && big && max_log <= kLockstepMaxLog);
-  const void* fn = quads  ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_QUADS, true>)
-                   : lock ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, true>)
-                   : priv ? reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, false>)
-                          : reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, true>);
-  int warps = 4;
+  int warps = 4, launch_which = 0;
   a.succ_bytes = (priv && !lock) ? ((2u << max_log) + 15u) & ~15u : 0u;
   size_t smem = (size_t(a.table_words) + 256) * 4 + a.succ_bytes;
   {
@@ -1316,7 +1315,21 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
     }
   }
   {
-    LaunchShape& shape = facts.shape[quads ? 3 : lock ? 2 : priv ? 1 : 0];
+    // which instantiation: the walk, and whether the CTA is one of many warps
+    const bool many = warps > 16;
+    const int which = (quads ? 0 : lock ? 1 : priv ? 2 : 3) * 2 + (many ? 1 : 0);
+    const void* fn = nullptr;
+    switch (which) {
+      case 0: fn = reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_QUADS, true, false>); break;
+      case 1: fn = reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_QUADS, true, true>); break;
+      case 2: fn = reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, true, false>); break;
+      case 3: fn = reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, true, true>); break;
+      case 4: case 5: fn = reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, false, false>); break;
+      case 6: fn = reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, true, false>); break;
+      default: fn = reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, true, true>); break;
+    }
+    launch_which = which;
+    LaunchShape& shape = facts.shape[which];
     if (shape.smem != smem || shape.warps != warps) {
       ANSB_CUDA(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
       ANSB_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, warps * 32, smem));
@@ -1347,14 +1360,16 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   ipc = (ipc + step - 1) / step * step;
   a.items_per_cta = static_cast<uint32_t>(ipc);
   const unsigned blocks = static_cast<unsigned>((total + ipc - 1) / ipc);
-  if (quads)
-    ans_decode_kernel<ANS_LAYOUT_QUADS, true><<<blocks, warps * 32, smem, st>>>(a);
-  else if (lock)
-    ans_decode_kernel<ANS_LAYOUT_PRIVATE, true><<<blocks, warps * 32, smem, st>>>(a);
-  else if (priv)
-    ans_decode_kernel<ANS_LAYOUT_PRIVATE, false><<<blocks, warps * 32, smem, st>>>(a);
-  else
-    ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, true><<<blocks, warps * 32, smem, st>>>(a);
+  const dim3 grid_dim(blocks), block_dim(static_cast<unsigned>(warps) * 32u);
+  switch (launch_which) {
+    case 0: ans_decode_kernel<ANS_LAYOUT_QUADS, true, false><<<grid_dim, block_dim, smem, st>>>(a); break;
+    case 1: ans_decode_kernel<ANS_LAYOUT_QUADS, true, true><<<grid_dim, block_dim, smem, st>>>(a); break;
+    case 2: ans_decode_kernel<ANS_LAYOUT_PRIVATE, true, false><<<grid_dim, block_dim, smem, st>>>(a); break;
+    case 3: ans_decode_kernel<ANS_LAYOUT_PRIVATE, true, true><<<grid_dim, block_dim, smem, st>>>(a); break;
+    case 4: case 5: ans_decode_kernel<ANS_LAYOUT_PRIVATE, false, false><<<grid_dim, block_dim, smem, st>>>(a); break;
+    case 6: ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, true, false><<<grid_dim, block_dim, smem, st>>>(a); break;
+    default: ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, true, true><<<grid_dim, block_dim, smem, st>>>(a); break;
+  }
   ANSB_CUDA(cudaGetLastError());
   return ANS_OK;
 }
