@@ -101,6 +101,25 @@ def test_batch_of_more_layers_than_the_kernel_parameters_hold(layout):
 
 
 @pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("shift", [1, 2, 3, 5])
+def test_symbols_into_a_buffer_of_any_alignment(layout, shift):
+    """ans_decode_layer asks no alignment of the symbol buffer: the vector stores of the fast
+    paths must give way to byte stores, and nothing outside the buffer may be touched."""
+    for n, chunk, lanes in [(70_001, 4096, 32), (1_200_000, 2048, 64)]:
+        spec = tiny_spec(n, 3, 0.7, 8, chunk, "u8", index=shift)
+        sym = sg.draw_symbols(spec)
+        T, P, f256 = oracle_pack_spec(spec, sym, layout, lanes)
+        db = DeviceBatch([to_packed_layer(spec, P, f256)])
+        buf = torch.full((n + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+        ans.ans_decode_layer(db.h_descs[0][0], buf.data_ptr() + shift, db.status.data_ptr(),
+                             torch.cuda.current_stream().cuda_stream)
+        assert db.read_status() == 0
+        got = buf.cpu().numpy()
+        assert (got[shift:shift + n] == sym).all()
+        assert (got[:shift] == 0xA5).all() and (got[shift + n:] == 0xA5).all()
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
 def test_config2_resnet18_bf16(layout):
     run_and_compare(sg.workload_resnet18(), layout, 32)
 
