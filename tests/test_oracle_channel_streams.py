@@ -18,7 +18,7 @@ import synthgen as sg
 
 
 def _study_layers():
-    """Every second ResNet-50 conv (27 layers, 11.6 M weights keep the test short): 31 bins in the
+    """Every second ResNet-50 conv (27 layers, 12.9 M weights keep the test short): 31 bins in the
     first half of the network, 15 then 7 bins later (the paper's training ends between 31 and 13
     bins), entropy 0.85 bit per weight."""
     shapes = sg.resnet50_conv_shapes()[::2]
