@@ -286,9 +286,23 @@ def run_ours(args):
     from concurrent.futures import ThreadPoolExecutor
     cores = os.cpu_count() or 1
 
+    by_channel = args.grouping == "channel"
+    if by_channel:
+        # the paper's own grouping (Section III-B): one chunk per layer, one lane per input channel,
+        # weights stored channels-last so that lane c carries input channel c; layers whose input
+        # channels are no multiple of 32 (the first conv, which the paper leaves uncompressed) are left out
+        import dataclasses
+        specs = [dataclasses.replace(sp, chunk_symbols=sp.n) for sp in specs
+                 if len(sp.shape) == 4 and sp.shape[1] % 32 == 0 and sp.shape[1] <= 2048]
+        args.no_cpu_baseline = args.no_e2e = True
+
     def prep(spec):
         sym = sg.draw_symbols(spec, threads=max(1, cores // 4))
-        pl = pack_layer(sym, spec.alphabet, spec.table_log, spec.chunk_symbols, args.lanes, layout, spec.bitwidth,
+        lanes = args.lanes
+        if by_channel:
+            sym = np.ascontiguousarray(sym.reshape(spec.shape).transpose(0, 2, 3, 1)).ravel()
+            lanes = spec.shape[1]
+        pl = pack_layer(sym, spec.alphabet, spec.table_log, spec.chunk_symbols, lanes, layout, spec.bitwidth,
                         spec.zero_point, spec.scale, ans.DTYPES[spec.out_dtype], n_threads=max(1, cores // 2))
         return sym, pl
 
@@ -376,7 +390,8 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": WORKLOAD_TEXT[args.workload], "name": args.workload, "layout": args.layout,
-                   "lanes": args.lanes, "table_log": layers[0].table_log, "chunk_symbols": layers[0].chunk_symbols,
+                   "lanes": "one per input channel" if args.grouping == "channel" else args.lanes,
+                   "grouping": args.grouping, "table_log": layers[0].table_log, "chunk_symbols": layers[0].chunk_symbols,
                    "layers": len(layers), "weights": n_w, "out_dtype": specs[0].out_dtype,
                    "l2_policy": (f"inputs larger than L2: launches rotate over {n_sets} full copies of the workload "
                                  f"({n_sets * ws / 2**20:.0f} MB in all)"
@@ -446,6 +461,8 @@ def main():
     ap.add_argument("--layout", default=None, choices=["private", "interleaved", "quads"],
                     help="container; default: the fastest measured for the workload")
     ap.add_argument("--lanes", type=int, default=32)
+    ap.add_argument("--grouping", default="chunks", choices=["chunks", "channel"],
+                    help="channel (ResNet workloads): one stream per input channel of every conv, as in the paper")
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--table-log", type=int, default=0)
     ap.add_argument("--mats", type=int, default=8, help="large workload: number of matrices (8 = full size)")

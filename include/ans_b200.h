@@ -31,6 +31,9 @@
  *   layer share the layer's table.  Lane 32*g + k is lane k of sub-stream g; sub-streams
  *   are numbered chunk-major: sub = chunk*G + g.  Every sub-stream's bytes start at a
  *   16-byte aligned offset of d_stream, given by d_sub_offsets[sub] (n_sub + 1 entries).
+ *   (With one chunk per layer and as many lanes as a conv layer has input channels, over
+ *   weights stored channels-last, lane c is the stream of input channel c: the paper's own
+ *   grouping, Section III-B.)
  *   Bits are packed least-significant first; a lane's encoder starts from state index 0,
  *   so a sound stream makes its decoder END in state index 0.
  *     ANS_LAYOUT_INTERLEAVED: the 32 lanes of a sub-stream share ONE sequence of
@@ -76,6 +79,7 @@ extern "C" {
 #define ANS_LAYOUT_QUADS       2
 
 #define ANS_MAX_TABLE_LOG 14
+#define ANS_MAX_LANES     2048   /* lanes per chunk: any multiple of 32 up to this */
 #define ANS_MAX_ALPHABET  256
 
 /* bits of the device status word (0 = every stream sound) */
@@ -96,7 +100,7 @@ typedef struct ans_layer_desc {
   uint64_t        stream_bytes;   /* bytes readable at d_stream (offsets beyond it are flagged) */
   uint64_t        n_symbols;      /* weights in the layer; may be 0                          */
   uint32_t        chunk_symbols;  /* symbols per chunk (last chunk may be shorter), >= 1    */
-  uint32_t        lanes;          /* 32*G, G in {1,2,4,8}                                    */
+  uint32_t        lanes;          /* 32*G, G in 1..64 (the kernels' fast paths: G in {1,2,4,8}) */
   int32_t         table_log;      /* R: the table has 2^R states (paper: l = 64..256; here 1..14) */
   int32_t         bitwidth;       /* b in [1,8]: symbols must be < 2^b (checked on the device) */
   int32_t         zero_point;     /* symbol that dequantises to 0 (Section II-B)            */

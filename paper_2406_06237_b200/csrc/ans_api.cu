@@ -12,7 +12,7 @@ void set_last_cuda_error(cudaError_t e) { g_last_cuda_error.store(static_cast<in
 
 int validate_desc(const ans_layer_desc& d, bool need_out) {
   if (d.table_log < 1 || d.table_log > ANS_MAX_TABLE_LOG) return ANS_ERR_UNSUPPORTED;
-  if (d.lanes != 32 && d.lanes != 64 && d.lanes != 128 && d.lanes != 256) return ANS_ERR_UNSUPPORTED;
+  if (d.lanes < 32 || d.lanes > ANS_MAX_LANES || d.lanes % 32) return ANS_ERR_UNSUPPORTED;
   if (d.layout != ANS_LAYOUT_INTERLEAVED && d.layout != ANS_LAYOUT_PRIVATE && d.layout != ANS_LAYOUT_QUADS)
     return ANS_ERR_UNSUPPORTED;
   if (d.out_dtype != ANS_U8 && d.out_dtype != ANS_F32 && d.out_dtype != ANS_BF16) return ANS_ERR_UNSUPPORTED;

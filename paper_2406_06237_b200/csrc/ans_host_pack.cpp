@@ -265,7 +265,7 @@ ANS_EXPORT int ans_host_pack_layer(const uint8_t* h_symbols, uint64_t n_symbols,
   if (!h_freqs || !h_stream_bytes_out || !h_sub_offsets_out) return ANS_ERR_INVALID_ARG;
   if (alphabet < 1 || alphabet > ANS_MAX_ALPHABET || chunk_symbols == 0) return ANS_ERR_INVALID_ARG;
   if (table_log < 1 || table_log > ANS_MAX_TABLE_LOG) return ANS_ERR_UNSUPPORTED;
-  if (lanes != 32 && lanes != 64 && lanes != 128 && lanes != 256) return ANS_ERR_UNSUPPORTED;
+  if (lanes < 32 || lanes > ANS_MAX_LANES || lanes % 32) return ANS_ERR_UNSUPPORTED;
   if (layout != ANS_LAYOUT_INTERLEAVED && layout != ANS_LAYOUT_PRIVATE && layout != ANS_LAYOUT_QUADS)
     return ANS_ERR_UNSUPPORTED;
   if (n_symbols && (!h_symbols || !h_stream_out || !h_lane_meta_out)) return ANS_ERR_INVALID_ARG;

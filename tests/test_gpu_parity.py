@@ -119,6 +119,36 @@ def test_symbols_into_a_buffer_of_any_alignment(layout, shift):
         assert (got[:shift] == 0xA5).all() and (got[shift + n:] == 0xA5).all()
 
 
+def _channels_last(sym, shape):
+    """The OHWI flattening of symbols drawn for an OIHW tensor: a permutation of the input."""
+    return np.ascontiguousarray(sym.reshape(shape).transpose(0, 2, 3, 1)).ravel()
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_streams_grouped_by_input_channel(layout):
+    """The paper's own grouping (Section III-B): one chunk per layer, as many lanes as the conv has
+    input channels, weights stored channels-last, so that lane c carries input channel c.  Lane
+    counts that are no power of two and up to the largest allowed ride along."""
+    shapes = [(64, 64, 1, 1), (64, 64, 3, 3), (256, 96, 1, 1), (128, 512, 1, 1), (96, 2048, 1, 1), (32, 160, 3, 3)]
+    prepared = []
+    for i, shape in enumerate(shapes):
+        spec = tiny_spec(int(np.prod(shape)), 3 + i % 3, 0.8, 8, int(np.prod(shape)), ("bf16", "f32", "u8")[i % 3],
+                         index=i)
+        sym = _channels_last(sg.draw_symbols(spec), shape)
+        if layout == ans.ANS_LAYOUT_PRIVATE:             # lane c holds exactly input channel c
+            per_channel = sym.reshape(-1, shape[1])
+            assert (per_channel[:, 5] == sym[5::shape[1]]).all()
+        T, P, f256 = oracle_pack_spec(spec, sym, layout, shape[1])
+        want_sym, want = oracle_expected(spec, T, P)
+        assert (want_sym == sym).all()
+        prepared.append((to_packed_layer(spec, P, f256), want))
+    db = DeviceBatch([p[0] for p in prepared])
+    db.decode()
+    assert db.read_status() == 0
+    for i, (pl, want) in enumerate(prepared):
+        assert np.array_equal(bits_view(db.output(i)), expected_bits(want)), f"layer {i}"
+
+
 @pytest.mark.parametrize("layout", LAYOUTS)
 def test_config2_resnet18_bf16(layout):
     run_and_compare(sg.workload_resnet18(), layout, 32)

@@ -44,7 +44,8 @@ def test_table_bytes():
 @pytest.mark.parametrize("layout", [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE, ans.ANS_LAYOUT_QUADS])
 @pytest.mark.parametrize("n,C,lanes,R,b", [(36864, 4096, 32, 12, 4), (5000, 1024, 64, 8, 3), (100_003, 16384, 128, 11, 6),
                                            (33, 64, 32, 6, 2), (70_000, 65536, 256, 14, 8), (4097, 4096, 32, 12, 1),
-                                           (10_007, 1001, 32, 9, 4), (130, 130, 32, 5, 3)])
+                                           (10_007, 1001, 32, 9, 4), (130, 130, 32, 5, 3),
+                                           (50_000, 50_000, 96, 8, 3), (300_000, 300_000, 2048, 8, 4)])
 def test_host_packer_equals_oracle_encoder(layout, n, C, lanes, R, b):
     spec = tiny_spec(n, bitwidth=b, pzp=0.7, table_log=R, chunk=C)
     sym = sg.draw_symbols(spec)
