@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
   uint8_t* ring = sm + (ring_abs - sm_abs);
   uint8_t* stage = sm + (stage_abs - sm_abs);
   const uint32_t bar = bars_abs + warp * 8u;
-  __shared__ uint32_t s_dom, s_maxadv;
+  __shared__ uint32_t s_dom, s_maxadv, s_maxnb;
   uint32_t parity = 0;
 
   uint64_t cursor = uint64_t(blockIdx.x) * args.items_per_cta;
@@ -165,12 +165,13 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
         if (threadIdx.x == 0) {
           s_dom = h_dominant < 256u ? h_dominant : 0u;    // the ring's fill symbol
           s_maxadv = 1u;
+          s_maxnb = 0u;
           if (h_magic != kTableMagic || h_log != uint32_t(R) || h_alphabet > (1u << L.bitwidth))
             bad |= ANS_STATUS_BAD_SYMBOL;
         }
         __syncthreads();
       }
-      uint32_t longest = 0;
+      uint32_t longest = 0, most_bits = 0;
 #pragma unroll
       for (uint32_t k = 0; k < kStageBatch; ++k) {
         const uint32_t i = b0 + k * blockDim.x + threadIdx.x;
@@ -181,10 +182,15 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
           for (uint32_t c = 0; c < reps; ++c) tab[(i << rep_log) + ((c + lane) & (reps - 1u))] = e;
           if (kPrivate && !lock) succ[i] = static_cast<uint16_t>(entry_newx(g1[k]));
           longest = max(longest, entry_run(g[k]) + 1u);
+          most_bits = max(most_bits, entry_nb(g[k]));
         }
       }
       longest = __reduce_max_sync(kFull, longest);
       if (lane == 0 && longest > 1u) atomicMax(&s_maxadv, longest);
+      // the lockstep walks share one 32-bit extract among four look-ups when no state of this
+      // table takes more than 8 bits (a table of 2^12 states over a handful of symbols does not)
+      most_bits = __reduce_max_sync(kFull, most_bits);
+      if (lane == 0) atomicMax(&s_maxnb, most_bits);
     }
     if (threadIdx.x < reps && kPrivate && !lock && R <= kMaxParkLog)
       tab[(n_states << rep_log) + threadIdx.x] =
@@ -258,10 +264,10 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
                                    out_row0, rsb, lane, s_maxadv)
 #define ANSB_LCALL(ES_, ST_)                                                                             \
   wbad |= decode_lockstep<ES_, ST_>(tab_lane, stride_log, stage_abs, words, ext_words, wbeg, wend, lane == 31, \
-                                    state, my_count, rows, min_count, out_row0, W / 32u, lane, R <= 8, args.unit)
+                                    state, my_count, rows, min_count, out_row0, W / 32u, lane, s_maxnb <= 8u, args.unit)
 #define ANSB_QCALL(ES_, ST_)                                                                             \
   wbad |= decode_quads<ES_, ST_>(tab_lane, stride_log, stage_abs, words, ext_words, wbeg, wend, lane == 31, state, \
-                                 my_count, min_count, out_row0 + size_t(lane) * 4u * ES_, W / 32u, R <= 8, args.unit)
+                                 my_count, min_count, out_row0 + size_t(lane) * 4u * ES_, W / 32u, s_maxnb <= 8u, args.unit)
         if constexpr (kQuads) {
           if (staged) {
             if (es == 1) ANSB_QCALL(1, true); else if (es == 2) ANSB_QCALL(2, true); else ANSB_QCALL(4, true);

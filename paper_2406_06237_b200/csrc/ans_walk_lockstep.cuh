@@ -14,8 +14,8 @@ namespace ansb {
 // for conflict-free copies) or the pre-walked entries would stand for few symbols anyway.
 //
 // kFlushRows rows are decoded by one PTX block (row stores at immediate offsets), K look-ups
-// sharing one 32-bit extract of the bit window and one refill check: K = 4 when a symbol takes
-// at most 8 bits, else 2.  Multiply-high is avoided on purpose (it runs at a fraction of the
+// sharing one 32-bit extract of the bit window and one refill check: K = 4 when no state of the
+// table takes more than 8 bits, else 2.  Multiply-high is avoided on purpose (it runs at a fraction of the
 // rate of shifts and adds); the bit count is accumulated on the multiply-add pipe, which is
 // otherwise idle, by a multiplication with a run-time 1.
 // =============================================================================================
