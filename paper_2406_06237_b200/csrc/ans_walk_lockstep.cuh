@@ -15,9 +15,9 @@ namespace ansb {
 //
 // kFlushRows rows are decoded by one PTX block (row stores at immediate offsets), K look-ups
 // sharing one 32-bit extract of the bit window and one refill check: K = 4 when no state of the
-// table takes more than 8 bits, else 2.  Multiply-high is avoided on purpose (it runs at a fraction of the
-// rate of shifts and adds); the bit count is accumulated on the multiply-add pipe, which is
-// otherwise idle, by a multiplication with a run-time 1.
+// table takes more than 8 bits, else 2.  Multiply-high is avoided on purpose (it runs at a
+// fraction of the rate of shifts and adds); the bit count is accumulated on the multiply-add
+// pipe, which is otherwise idle, by a multiplication with a run-time 1.
 // =============================================================================================
 #define ANSB_LS_STEP(STOP_, ADDR_)                                \
   "ld.shared.v2.u32 {ea, eb}, [%0];\n\t"                          \
