@@ -80,11 +80,13 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
     const int R = L.table_log;
     // copies of this layer's table: a table smaller than the launch's largest uses the room for
     // more of them (the pre-walked walk keeps an extra entry after the table, so it does not)
-    const uint32_t rep_log = (kPrivate && !lock) ? args.rep_log
-                                                 : min(4u, args.rep_log + (args.max_log - static_cast<uint32_t>(R)));
+    // quads with 1-byte outputs: one-word entries, so twice the copies (up to 32) in the same room
+    const bool short_entries = kQuads && (args.d_symbols_override || L.out_dtype == ANS_U8);
+    const uint32_t rep_two = min(4u, args.rep_log + (args.max_log - static_cast<uint32_t>(R)));
+    const uint32_t rep_log = (kPrivate && !lock) ? args.rep_log : short_entries ? rep_two + 1u : rep_two;
     const uint32_t reps = 1u << rep_log;
-    const uint32_t stride_log = 3u + rep_log;
-    const uint32_t tab_lane = tab_abs + (lane & (reps - 1u)) * 8u;
+    const uint32_t stride_log = (short_entries ? 2u : 3u) + rep_log;
+    const uint32_t tab_lane = tab_abs + (lane & (reps - 1u)) * (short_entries ? 4u : 8u);
     const uint8_t* blob = static_cast<const uint8_t*>(L.d_table);
     const TableHeader* hdr = reinterpret_cast<const TableHeader*>(blob);
     const uint32_t* g_single = reinterpret_cast<const uint32_t*>(blob + single_offset());
@@ -179,7 +181,14 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
           const uint2 e = kQuads ? to_quads_entry(g[k], vals[entry_sym(g[k])], es != 4)
                                  : to_smem_entry(g[k], vals[entry_sym(g[k])], 32u * static_cast<uint32_t>(es));
           // every lane starts at another copy: the stores of a warp spread over the banks
-          for (uint32_t c = 0; c < reps; ++c) tab[(i << rep_log) + ((c + lane) & (reps - 1u))] = e;
+          if (short_entries) {
+            const uint32_t e1 = entry_nb(g[k]) | ((entry_newx(g[k]) >> entry_nb(g[k])) << 8) |
+                                (vals[entry_sym(g[k])] << 24);
+            for (uint32_t c = 0; c < reps; ++c)
+              reinterpret_cast<uint32_t*>(tab)[(i << rep_log) + ((c + lane) & (reps - 1u))] = e1;
+          } else {
+            for (uint32_t c = 0; c < reps; ++c) tab[(i << rep_log) + ((c + lane) & (reps - 1u))] = e;
+          }
           if (kPrivate && !lock) succ[i] = static_cast<uint16_t>(entry_newx(g1[k]));
           longest = max(longest, entry_run(g[k]) + 1u);
           most_bits = max(most_bits, entry_nb(g[k]));
@@ -265,14 +274,17 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
 #define ANSB_LCALL(ES_, ST_)                                                                             \
   wbad |= decode_lockstep<ES_, ST_>(tab_lane, stride_log, stage_abs, words, ext_words, wbeg, wend, lane == 31, \
                                     state, my_count, rows, min_count, out_row0, W / 32u, lane, s_maxnb <= 8u, args.unit)
-#define ANSB_QCALL(ES_, ST_)                                                                             \
-  wbad |= decode_quads<ES_, ST_>(tab_lane, stride_log, stage_abs, words, ext_words, wbeg, wend, lane == 31, state, \
-                                 my_count, min_count, out_row0 + size_t(lane) * 4u * ES_, W / 32u, s_maxnb <= 8u, args.unit)
-        if constexpr (kQuads) {
+#define ANSB_QCALL(ES_, ST_, SH_)                                                                        \
+  wbad |= decode_quads<ES_, ST_, SH_>(tab_lane, stride_log, stage_abs, words, ext_words, wbeg, wend, lane == 31, \
+                                      state, my_count, min_count, out_row0 + size_t(lane) * 4u * ES_, W / 32u, \
+                                      s_maxnb <= 8u, args.unit)
+        if constexpr (kQuads) {                           // (1-byte outputs: one-word entries, see above)
           if (staged) {
-            if (es == 1) ANSB_QCALL(1, true); else if (es == 2) ANSB_QCALL(2, true); else ANSB_QCALL(4, true);
+            if (es == 1) ANSB_QCALL(1, true, true); else if (es == 2) ANSB_QCALL(2, true, false);
+            else ANSB_QCALL(4, true, false);
           } else {
-            if (es == 1) ANSB_QCALL(1, false); else if (es == 2) ANSB_QCALL(2, false); else ANSB_QCALL(4, false);
+            if (es == 1) ANSB_QCALL(1, false, true); else if (es == 2) ANSB_QCALL(2, false, false);
+            else ANSB_QCALL(4, false, false);
           }
         } else if constexpr (lock) {
           if (staged) {

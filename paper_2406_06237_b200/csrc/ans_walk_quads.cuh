@@ -16,6 +16,9 @@ namespace ansb {
 // shared-memory entry, two words:
 //   1- and 2-byte outputs:  a = nb [4:0] | dequantised value [31:16]      b = q
 //   4-byte outputs:         a = nb [4:0] | q [31:8]                       b = dequantised value
+// or, for 1-byte outputs, ONE word: nb [4:0] | q [21:8] | value [31:24].  Half the bytes per
+// table, so twice the copies fit: it pays where copies are short (tables of 2^11 states and up,
+// whose random look-ups collide), at the price of one more instruction per look-up.
 // =============================================================================================
 __device__ __forceinline__ uint2 to_quads_entry(uint32_t g, uint32_t val, bool narrow) {
   const uint32_t nb = entry_nb(g), q = entry_newx(g) >> nb;
@@ -25,6 +28,13 @@ __device__ __forceinline__ uint2 to_quads_entry(uint32_t g, uint32_t val, bool n
 #define ANSB_QD_STEP_N(I_)                                        \
   "ld.shared.v2.u32 {ea" I_ ", eb" I_ "}, [%0];\n\t"              \
   "shf.l.wrap.b32 t, x, eb" I_ ", ea" I_ ";\n\t"                  \
+  "shf.l.wrap.b32 x, 0, x, ea" I_ ";\n\t"                         \
+  "mad.lo.u32 %0, t, %7, %6;\n\t"                                 \
+  "mad.lo.u32 %1, ea" I_ ", %9, %1;\n\t"
+#define ANSB_QD_STEP_S(I_)                                        \
+  "ld.shared.u32 ea" I_ ", [%0];\n\t"                             \
+  "bfe.u32 nx, ea" I_ ", 8, 14;\n\t"                              \
+  "shf.l.wrap.b32 t, x, nx, ea" I_ ";\n\t"                        \
   "shf.l.wrap.b32 x, 0, x, ea" I_ ";\n\t"                         \
   "mad.lo.u32 %0, t, %7, %6;\n\t"                                 \
   "mad.lo.u32 %1, ea" I_ ", %9, %1;\n\t"
@@ -44,6 +54,11 @@ __device__ __forceinline__ uint2 to_quads_entry(uint32_t g, uint32_t val, bool n
   "prmt.b32 v1, ea2, ea3, 0x0062;\n\t"                            \
   "prmt.b32 v0, v0, v1, 0x5410;\n\t"                              \
   "st.global.u32 " A_ ", v0;\n\t"
+#define ANSB_QD_OUT1S(A_)                                         \
+  "prmt.b32 v0, ea0, ea1, 0x0073;\n\t"                            \
+  "prmt.b32 v1, ea2, ea3, 0x0073;\n\t"                            \
+  "prmt.b32 v0, v0, v1, 0x5410;\n\t"                              \
+  "st.global.u32 " A_ ", v0;\n\t"
 #define ANSB_QD_OUT2(A_)                                          \
   "prmt.b32 v0, ea0, ea1, 0x7632;\n\t"                            \
   "prmt.b32 v1, ea2, ea3, 0x7632;\n\t"                            \
@@ -57,7 +72,7 @@ constexpr uint32_t kQuadTurns = 4;     // turns (of four symbols per lane) per t
 // lockstep_block; gp: this lane's four elements of the first turn; turns are 128 * ES * groups
 // bytes apart (immediate offsets when groups == 1); sp is held at sp_limit if a corrupt stream
 // drives it that far.
-template <int ES, int K>
+template <int ES, int K, bool SHORT = false>
 __device__ __forceinline__ void quads_loop(uint32_t& st, uint32_t& bitpos, uint32_t& w0, uint32_t& w1,
                                            uint32_t& w2, uint32_t& sp, uint32_t tab_lane, uint32_t stride,
                                            uint8_t* gp, uint32_t unit, uint32_t groups, uint32_t blocks,
@@ -108,7 +123,10 @@ __device__ __forceinline__ void quads_loop(uint32_t& st, uint32_t& bitpos, uint3
       : "memory")
 #define ANSB_QD_BOTH(L1_, LG_, TURN_, ST_, OUT_)                                            \
   if (groups == 1) ANSB_QD_ASM1(L1_, TURN_, ST_, OUT_); else ANSB_QD_ASMG(LG_, TURN_, ST_, OUT_)
-  if (K == 4) {
+  if (SHORT) {     // one-word entries (1-byte outputs)
+    if (K == 4) { ANSB_QD_BOTH("ANSB_QS41", "ANSB_QS4G", ANSB_QD_TURN4, ANSB_QD_STEP_S, ANSB_QD_OUT1S); }
+    else { ANSB_QD_BOTH("ANSB_QS21", "ANSB_QS2G", ANSB_QD_TURN2, ANSB_QD_STEP_S, ANSB_QD_OUT1S); }
+  } else if (K == 4) {
     if (ES == 1) { ANSB_QD_BOTH("ANSB_Q41", "ANSB_Q4G", ANSB_QD_TURN4, ANSB_QD_STEP_N, ANSB_QD_OUT1); }
     if (ES == 2) { ANSB_QD_BOTH("ANSB_Q41", "ANSB_Q4G", ANSB_QD_TURN4, ANSB_QD_STEP_N, ANSB_QD_OUT2); }
     if (ES == 4) { ANSB_QD_BOTH("ANSB_Q41", "ANSB_Q4G", ANSB_QD_TURN4, ANSB_QD_STEP_W, ANSB_QD_OUT4); }
@@ -125,7 +143,7 @@ __device__ __forceinline__ void quads_loop(uint32_t& st, uint32_t& bitpos, uint3
 // Decode one sub-stream of the quads container.  full_turns: turns in which every lane of the
 // sub-stream owns a whole quad; out_lane: this lane's first output element; a lane's turns are
 // 128 * ES * groups bytes apart.
-template <int ES, bool STAGED>
+template <int ES, bool STAGED, bool SHORT = false>
 __device__ __noinline__ uint32_t decode_quads(
     uint32_t tab_abs, uint32_t stride_log, uint32_t stage_abs, const uint32_t* __restrict__ words,
     uint32_t ext_words, uint32_t wbeg, uint32_t wend, bool last_lane, uint32_t state, uint32_t my_count,
@@ -153,10 +171,10 @@ __device__ __noinline__ uint32_t decode_quads(
     const uint32_t sp_limit = stage_abs + word_limit * 4u;   // a sound lane stays below it
     const uint32_t blocks = full_turns / kQuadTurns;
     if (blocks) {
-      if (wide_steps) quads_loop<ES, 4>(st, bitpos, w0, w1, w2, sp, tab_abs, 1u << stride_log, out_lane, unit, groups,
-                                        blocks, sp_limit);
-      else quads_loop<ES, 2>(st, bitpos, w0, w1, w2, sp, tab_abs, 1u << stride_log, out_lane, unit, groups, blocks,
-                             sp_limit);
+      if (wide_steps) quads_loop<ES, 4, SHORT>(st, bitpos, w0, w1, w2, sp, tab_abs, 1u << stride_log, out_lane, unit,
+                                               groups, blocks, sp_limit);
+      else quads_loop<ES, 2, SHORT>(st, bitpos, w0, w1, w2, sp, tab_abs, 1u << stride_log, out_lane, unit, groups,
+                                    blocks, sp_limit);
       if (sp >= sp_limit) overran = true;
       turn = blocks * kQuadTurns;
     }
@@ -165,9 +183,10 @@ __device__ __noinline__ uint32_t decode_quads(
   }
   // the rest in plain code, one symbol and one element store at a time
   for (; k < my_count; ++k) {
-    const uint32_t ea = lds_u32(st), eb = lds_u32(st + 4u);
+    const uint32_t ea = lds_u32(st), eb = SHORT ? 0u : lds_u32(st + 4u);
     const uint32_t nb = ea & 31u;
-    const uint32_t q = NARROW ? eb : ea >> 8, val = NARROW ? ea >> 16 : eb;
+    const uint32_t q = SHORT ? (ea >> 8) & 0x3FFFu : NARROW ? eb : ea >> 8;
+    const uint32_t val = SHORT ? ea >> 24 : NARROW ? ea >> 16 : eb;
     const uint32_t x = __funnelshift_l(w1, w0, bitpos);
     st = tab_abs + (__funnelshift_l(x, q, nb) << stride_log);
     stg_elem<ES>(out_lane + size_t(k >> 2) * turn_stride + (k & 3u) * ES, val);
