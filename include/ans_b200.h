@@ -30,7 +30,9 @@
  *   q % lanes); every lane is its own tANS stream with its own state, all lanes of a
  *   layer share the layer's table.  Lane 32*g + k is lane k of sub-stream g; sub-streams
  *   are numbered chunk-major: sub = chunk*G + g.  Every sub-stream's bytes start at a
- *   16-byte aligned offset of d_stream, given by d_sub_offsets[sub] (n_sub + 1 entries).
+ *   16-byte aligned offset of d_stream, given by d_sub_offsets[sub] (n_sub + 1 entries, each
+ *   a multiple of 16; a sub-stream whose begin or end is not, or lies outside the stream, is
+ *   flagged ANS_STATUS_BAD_LENGTH and not read).
  *   (With one chunk per layer and as many lanes as a conv layer has input channels, over
  *   weights stored channels-last, lane c is the stream of input channel c: the paper's own
  *   grouping, Section III-B.)
@@ -86,6 +88,9 @@ extern "C" {
 #define ANS_STATUS_BAD_FINAL_STATE 1u   /* a lane did not end in state index 0          */
 #define ANS_STATUS_BAD_LENGTH      2u   /* a sub-stream consumed more or fewer bytes than it holds */
 #define ANS_STATUS_BAD_SYMBOL      4u   /* a decoded symbol does not fit `bitwidth` bits  */
+#define ANS_STATUS_COPY_TIMEOUT    8u   /* an asynchronous copy of compressed bytes into shared memory
+                                           did not complete within the kernel's bounded wait; the
+                                           warp that waited decoded nothing further            */
 
 /*
  * One layer of a decode call.  For the *_batch call an array of these lives in device

@@ -71,7 +71,11 @@ static size_t up256(size_t x) { return (x + 255) & ~size_t(255); }
 ANS_EXPORT int ans_host_scratch_bytes(const ans_layer_desc* h_desc, uint64_t stream_bytes, size_t* h_bytes_out) {
   if (!h_desc || !h_bytes_out) return ANS_ERR_INVALID_ARG;
   if (h_desc->chunk_symbols == 0 || h_desc->lanes == 0 || h_desc->lanes % 32) return ANS_ERR_INVALID_ARG;
+  // sizes that cannot be those of a real layer are refused before they can wrap a sum
+  constexpr uint64_t kMaxBytes = uint64_t(1) << 46;
+  if (h_desc->n_symbols > kMaxBytes / 4 || stream_bytes > kMaxBytes) return ANS_ERR_INVALID_ARG;
   const uint64_t n_sub = subs_of(*h_desc);
+  if (n_sub > kMaxBytes / 128) return ANS_ERR_INVALID_ARG;
   const size_t meta = n_sub * 32 * (h_desc->layout == ANS_LAYOUT_INTERLEAVED ? 2 : 4);
   *h_bytes_out = 256 + up256(stream_bytes) + up256((n_sub + 1) * 8) + up256(meta) +
                  up256(h_desc->n_symbols * elem_size(h_desc->out_dtype));

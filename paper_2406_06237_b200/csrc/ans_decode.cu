@@ -130,7 +130,9 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
     };
     uint64_t first_sub = 0, first_off0 = 0, first_off1 = 0;
     uint32_t first_meta = 0;
-    const bool have_first = warp_sub(cursor, first_sub);
+    // (a warp whose wait on a copy ran out takes no further work: it only keeps the CTA's
+    // barriers company, so that nothing is issued on a barrier whose phase never completed)
+    const bool have_first = !gave_up && warp_sub(cursor, first_sub);
     if (have_first) {
       first_off0 = __ldg(L.d_sub_offsets + first_sub);
       first_off1 = __ldg(L.d_sub_offsets + first_sub + 1);
@@ -257,12 +259,12 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
 
       if (staged) {
         const bool ok = mbar_wait(bar, parity);
-        parity ^= 1u;
         if (!__all_sync(kFull, ok)) {                     // the copy never landed: stop this warp's work
           bad |= wbad | kStatusTimeout;
           gave_up = true;
           continue;
         }
+        parity ^= 1u;
         __syncwarp();
       }
       if (kPrivate) {

@@ -9,7 +9,7 @@
 namespace ansb {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
-constexpr uint32_t kStatusTimeout = 8u;   // a bounded wait on an asynchronous copy ran out
+constexpr uint32_t kStatusTimeout = ANS_STATUS_COPY_TIMEOUT;   // a bounded wait on an asynchronous copy ran out
 
 constexpr int kParamLayers = 96;
 constexpr int kLockstepMaxLog = 9;        // private container: largest table walked one symbol per look-up
@@ -86,7 +86,9 @@ __device__ __forceinline__ Item make_item(const ans_layer_desc& L, uint64_t sub,
   it.off0 = off0;
   it.extent = off1 - it.off0;
   it.bad = 0;
-  if (off1 < it.off0 || off1 > L.stream_bytes || (it.off0 & 15u)) {   // never read outside the stream
+  // never read outside the stream; both ends on 16-byte boundaries, as the bulk copy and the
+  // zero fill after the staged bytes need
+  if (off1 < it.off0 || off1 > L.stream_bytes || ((it.off0 | off1) & 15u)) {
     it.extent = 0;
     it.off0 = 0;
     it.bad = ANS_STATUS_BAD_LENGTH;

@@ -49,14 +49,17 @@ ANS_EXPORT int ans_decode_dequant_host_noalloc(const ans_layer_desc* h_desc, con
                                                void* h_out, void* stream) {
   if (!h_desc || !h_norm_freqs) return ANS_ERR_INVALID_ARG;
   if (h_desc->chunk_symbols == 0 || h_desc->lanes == 0 || h_desc->lanes % 32) return ANS_ERR_INVALID_ARG;
-  if (h_desc->n_symbols == 0) return ANS_OK;
+  if (h_desc->n_symbols == 0) return validate_desc(*h_desc, false);   // nothing to decode, but still a sound layer?
   if (!h_stream || !h_sub_offsets || !h_lane_meta || !h_out) return ANS_ERR_INVALID_ARG;
 
-  // lay the call out in the fixed area and refuse what does not fit
+  // lay the call out in the fixed area and refuse what does not fit.  Every term is bounded by
+  // the area before it enters a sum, so that no size, however absurd, can wrap around and pass.
   size_t table_bytes = 0;
   int rc = ans_table_bytes(h_desc->table_log, &table_bytes);
   if (rc != ANS_OK) return rc;
-  const uint64_t n_sub = subs_of(*h_desc);
+  if (h_desc->n_symbols > kNoAllocBytes || stream_bytes > kNoAllocBytes) return ANS_ERR_BUFFER_TOO_SMALL;
+  const uint64_t n_sub = subs_of(*h_desc);               // <= n_symbols * 64 groups: no overflow
+  if (n_sub > kNoAllocBytes / 128) return ANS_ERR_BUFFER_TOO_SMALL;
   const size_t offs_bytes = (n_sub + 1) * 8;
   const size_t meta_bytes = n_sub * 32 * (h_desc->layout == ANS_LAYOUT_INTERLEAVED ? 2 : 4);
   const size_t out_bytes = h_desc->n_symbols * elem_size(h_desc->out_dtype);

@@ -50,7 +50,15 @@ def test_config5_large_layers_full(layout, table_log):
     full_size(sg.workload_large(table_log=table_log), layout, 32)
 
 
-@pytest.mark.parametrize("layout", [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE, ans.ANS_LAYOUT_QUADS])
+@pytest.mark.parametrize("layout", [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE])
 @pytest.mark.parametrize("chunk,R", [(1024, 11), (65536, 14), (16384, 12)])
 def test_config4_sweep_full(layout, chunk, R):
     full_size(sg.workload_sweep(table_log=R, chunk=chunk), layout, 32)
+
+
+@pytest.mark.parametrize("chunk", [1024, 4096, 16384, 65536])
+@pytest.mark.parametrize("R", [11, 12, 14])
+def test_config4_sweep_full_every_cell_on_the_benchmark_container(chunk, R):
+    """All twelve (chunk, table size) cells of the granularity sweep at 2^28 symbols on the quads
+    container, the one the benchmark times."""
+    full_size(sg.workload_sweep(table_log=R, chunk=chunk), ans.ANS_LAYOUT_QUADS, 32)

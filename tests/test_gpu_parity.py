@@ -164,8 +164,11 @@ def test_config3_resnet50_bf16(layout, lanes):
 @pytest.mark.parametrize("chunk", [1024, 4096, 16384, 65536])
 @pytest.mark.parametrize("R", [11, 12, 14])
 def test_config4_sweep_reduced(layout, chunk, R):
-    """The granularity sweep at 2^22 symbols (the full 2^28 runs in test_gpu_full_size)."""
-    run_and_compare(sg.workload_sweep(table_log=R, chunk=chunk, n=(1 << 22) + 12345), layout, 32)
+    """The granularity sweep at reduced size (the full 2^28 runs in test_gpu_full_size): 2^22
+    symbols, and 2^24 for the 64 K-symbol chunks, so that every cell has the 256 sub-streams and
+    more from which a launch takes the many-warp shape the full size runs in."""
+    n = (1 << 24) + 12345 if chunk == 65536 else (1 << 22) + 12345
+    run_and_compare(sg.workload_sweep(table_log=R, chunk=chunk, n=n), layout, 32)
 
 
 @pytest.mark.parametrize("layout", LAYOUTS)
@@ -264,6 +267,69 @@ def test_corrupt_streams_are_flagged_not_fatal(layout):
     short = P.stream[:P.stream.size - 16].copy()         # truncated stream
     st, _ = decode(oracle.Packed(P.layout, short, P.sub_offsets, P.lane_meta, P.n, P.chunk, P.groups))
     assert st & 2
+
+
+DEQUANT_EDGES = [(0, 1.0), (7, 0.02), (127, 0.1 / 256), (3, 0.05), (15, 1.0 / 3.0), (31, 3.0e-39),
+                 (1, 257.0 / 65536.0), (127, 1.0 + 2.0 ** -8), (0, 1.0 + 3 * 2.0 ** -8), (255, 1.0 + 2.0 ** -8),
+                 (0, -0.75), (200, 1.0e30), (128, 2.0 ** -140)]
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("out_dtype", ["f32", "bf16"])
+def test_dequantiser_edge_cases_reach_the_kernel(layout, out_dtype):
+    """Every one of the 256 symbols goes through a layer for each (zero_point, scale) pair that
+    pins the oracle's dequantiser (Section II-B): scales whose products are exact bf16 ties with
+    an even and with an odd kept mantissa, subnormal products (no flush to zero), products that
+    are not representable (1/3), the extreme zero-points.  One batched launch holds all pairs; the
+    output must equal the oracle's, bit for bit."""
+    rng = np.random.default_rng(7)
+    base = np.concatenate([np.arange(256, dtype=np.uint8), rng.integers(0, 256, size=5000, dtype=np.uint8)])
+    prepared = []
+    for i, (zp, scale) in enumerate(DEQUANT_EDGES):
+        sym = np.roll(base, 17 * i)
+        spec = sg.LayerSpec(f"edge{i}", (sym.size,), 8, 256, zp, 0.5, scale, 10 + i % 3, 1024, out_dtype,
+                            sg.stream_key(11, i))
+        T, P, f256 = oracle_pack_spec(spec, sym, layout, 32)
+        want_sym, want = oracle_expected(spec, T, P)
+        assert (want_sym == sym).all()
+        prepared.append((to_packed_layer(spec, P, f256), want))
+    # the oracle's values are themselves what the test expects them to be: ties and subnormals
+    b = oracle.dequant(np.array([1, 2, 3], np.uint8), 0, 1.0 + 2.0 ** -8, "bf16")
+    assert b.tolist() == [0x3F80, 0x4000, 0x4041]
+    tiny = oracle.dequant(np.array([32, 33], np.uint8), 31, 3.0e-39, "f32")
+    assert tiny[0] != 0.0 and tiny[0] < 1.2e-38 and tiny[1] == np.float32(2) * np.float32(3.0e-39)
+    db = DeviceBatch([p[0] for p in prepared])
+    for o in db.out_sets[0]:
+        o.view(torch.uint8).fill_(0xA5)
+    db.decode()
+    assert db.read_status() == 0
+    for i, (pl, want) in enumerate(prepared):
+        assert np.array_equal(bits_view(db.output(i)), expected_bits(want)), f"pair {DEQUANT_EDGES[i]}"
+    db.decode_per_layer()                                # the single-layer entry point takes the same values
+    assert db.read_status() == 0
+    for i, (pl, want) in enumerate(prepared):
+        assert np.array_equal(bits_view(db.output(i)), expected_bits(want)), f"pair {DEQUANT_EDGES[i]}"
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_substream_ends_off_a_16_byte_boundary_are_flagged(layout):
+    """An offsets table whose entries are not multiples of 16 (planted on the host) must be
+    flagged as a bad length; the sub-streams it touches are not read at all."""
+    spec = tiny_spec(40_000, 4, 0.6, 12, 4096, "bf16")
+    sym = sg.draw_symbols(spec)
+    T, P, f256 = oracle_pack_spec(spec, sym, layout, 32)
+    for which, delta in [(3, 4), (len(P.sub_offsets) - 1, -1), (1, 8), (2, -12)]:
+        o = P.sub_offsets.copy()
+        o[which] = np.uint64(int(o[which]) + delta)
+        db = DeviceBatch([to_packed_layer(spec, oracle.Packed(P.layout, P.stream, o, P.lane_meta, P.n, P.chunk,
+                                                              P.groups), f256)])
+        guard = torch.full((1 << 16,), 0x5A, dtype=torch.uint8, device="cuda")
+        db.decode()
+        assert db.read_status() & 2
+        assert (guard == 0x5A).all()
+    db = DeviceBatch([to_packed_layer(spec, P, f256)])   # and the context is still good
+    db.decode()
+    assert db.read_status() == 0
 
 
 def test_bitwidth_check():

@@ -35,3 +35,14 @@ def test_known_small_cases():
         oracle.normalize_freqs([1, 1, 1, 1, 1], 5, 2)
     with pytest.raises(oracle.OracleError):
         oracle.normalize_freqs([0, 0], 2, 4)
+
+
+def test_histogram_is_a_plain_count():
+    rng = np.random.default_rng(3)
+    for n in (0, 1, 255, 100_003):
+        sym = rng.integers(0, 256, size=n, dtype=np.uint8)
+        if n > 10:
+            sym[::3] = 7                                   # a peak, as in weight symbols
+        h = oracle.histogram(sym)
+        assert h.shape == (256,) and int(h.sum()) == n
+        assert (h == np.bincount(sym, minlength=256)).all()
