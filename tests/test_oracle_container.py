@@ -221,3 +221,137 @@ def test_quads_word_of_the_hand_trace(name):
     assert bytes(P.stream[:4]) == bytes.fromhex(g["quads_word_hex"].replace(" ", ""))
     out, rc = oracle.unpack(T, P)
     assert rc == oracle.OK and out[pos].tolist() == msg and (out == sym).all()
+
+
+# ---- segments container -------------------------------------------------------------------
+SEG_CASES = [(0, 512, 1), (1, 512, 1), (6, 512, 1), (511, 512, 1), (512, 512, 1), (513, 512, 1),
+             (5000, 1024, 2), (4096, 1024, 1), (777, 4096, 4), (65536 + 17, 16384, 2), (3000, 2048, 2),
+             (100, 32, 1), (1000, 64, 2)]
+
+
+@pytest.mark.parametrize("n,C,G", SEG_CASES)
+def test_segments_round_trip(n, C, G):
+    rng = np.random.default_rng(n + C + G)
+    msg = _source(rng, max(n, 1))
+    T = _table(msg, 15, 12)
+    msg = msg[:n]
+    P = oracle.pack(T, msg, C, G, oracle.SEGMENTS)
+    assert P.sub_offsets.size == P.n_sub + 1 and P.sub_offsets[-1] == P.stream.size
+    assert all(int(o) % 16 == 0 for o in P.sub_offsets) and P.lane_meta.size == 0
+    out, rc = oracle.unpack(T, P)
+    assert rc == oracle.OK and (out == msg).all()
+
+
+def test_segments_chunk_must_be_a_multiple_of_the_lanes():
+    T = oracle.Table([3, 1], 2)
+    with pytest.raises(oracle.OracleError):
+        oracle.pack(T, np.zeros(10, dtype=np.uint8), 1000, 1, oracle.SEGMENTS)
+
+
+@pytest.mark.parametrize("n,C,G", [(3000, 2048, 2), (1000, 1024, 1), (517, 256, 4), (130, 4096, 1), (40000, 16384, 2)])
+def test_segments_equal_plain_single_lane_coding(n, C, G):
+    """Independent build of every sub-stream in Python: lane lambda owns the contiguous run
+    [lambda*S, (lambda+1)*S) of its chunk; its string is the plain one-lane coder's initial state
+    in R bits followed by that coder's fields, most significant bit first; a sub-stream is the 32
+    lengths as little-endian uint16, then the strings back to back in 32-bit little-endian words
+    filled from the top bit, zero-padded to 16 bytes."""
+    rng = np.random.default_rng(n)
+    W, R = 32 * G, 10
+    S = C // W
+    msg = _source(rng, n)
+    T = _table(msg, 15, R)
+    P = oracle.pack(T, msg, C, G, oracle.SEGMENTS)
+    for c in range(P.n_chunks):
+        chunk = msg[c * C:(c + 1) * C]
+        for g in range(G):
+            sub = c * G + g
+            lens, bits = [], ""
+            for k in range(32):
+                mine = chunk[(32 * g + k) * S:(32 * g + k + 1) * S]
+                s = ""
+                if mine.size:
+                    init, nb, val = oracle.encode_lane_fields(T, mine)
+                    s = format(init, "b").zfill(R)
+                    s += "".join(format(int(v), "b").zfill(int(b)) if b else "" for b, v in zip(nb, val))
+                lens.append(len(s))
+                bits += s
+            words = (len(bits) + 31) // 32
+            bits = bits.ljust(32 * words, "0")
+            want = b"".join(int(x).to_bytes(2, "little") for x in lens)
+            want += b"".join(int(bits[32 * i:32 * i + 32], 2).to_bytes(4, "little") for i in range(words))
+            want += bytes(-len(want) % 16)
+            b0, b1 = int(P.sub_offsets[sub]), int(P.sub_offsets[sub + 1])
+            assert bytes(P.stream[b0:b1]) == want
+
+
+@pytest.mark.parametrize("name", ["trace_T1.txt", "trace_T2.txt"])
+def test_segments_bytes_of_the_hand_trace(name):
+    """A layer that is the hand trace's message alone: lane 0 owns all of it, the other lanes
+    are empty; lengths, first word and size are the ones worked out by hand in the fixture."""
+    g = read_golden(name)
+    T = oracle.Table(_ints(g["freqs"]), int(g["table_log"]))
+    msg = np.array(_ints(g["message"]), dtype=np.uint8)
+    P = oracle.pack(T, msg, 512, 1, oracle.SEGMENTS)
+    lens = np.frombuffer(bytes(P.stream[:64]), dtype="<u2")
+    assert int(lens[0]) == len(g["segments_lane_bits"]) and not lens[1:].any()
+    assert bytes(P.stream[64:68]) == bytes.fromhex(g["segments_first_word_hex"].replace(" ", ""))
+    assert P.stream.size == int(g["segments_sub_stream_bytes"]) and not P.stream[68:].any()
+    out, rc = oracle.unpack(T, P)
+    assert rc == oracle.OK and out.tolist() == msg.tolist()
+
+
+def test_segments_same_symbols_for_every_chunking_and_threads():
+    rng = np.random.default_rng(21)
+    msg = _source(rng, 50000)
+    T = _table(msg, 15, 11)
+    for C, G in [(1024, 1), (4096, 1), (4096, 4), (16384, 2), (65536, 8), (32, 1), (131072, 1)]:
+        P = oracle.pack(T, msg, C, G, oracle.SEGMENTS)
+        for th in (1, 4):
+            out, rc = oracle.unpack(T, P, threads=th)
+            assert rc == oracle.OK and (out == msg).all()
+
+
+def test_segments_corruption_is_reported():
+    rng = np.random.default_rng(16)
+    msg = _source(rng, 8192)
+    T = _table(msg, 15, 12)
+    P = oracle.pack(T, msg, 4096, 1, oracle.SEGMENTS)
+    flagged = 0
+    positions = list(range(3, P.stream.size, 97))
+    for pos in positions:
+        Q = oracle.Packed(P.layout, P.stream.copy(), P.sub_offsets, P.lane_meta, P.n, P.chunk, P.groups)
+        Q.stream[pos] ^= 0x5A
+        flagged += (oracle.unpack(T, Q)[1] == oracle.ERR_CORRUPT)
+    assert flagged > len(positions) // 2
+    for k in (0, 7, 31):                                   # a wrong length is always caught
+        Q = oracle.Packed(P.layout, P.stream.copy(), P.sub_offsets, P.lane_meta, P.n, P.chunk, P.groups)
+        Q.stream[2 * k] ^= 1
+        assert oracle.unpack(T, Q)[1] == oracle.ERR_CORRUPT
+    Q = oracle.Packed(P.layout, P.stream, P.sub_offsets.copy(), P.lane_meta, P.n, P.chunk, P.groups)
+    Q.sub_offsets[1] -= 16                                 # truncated sub-stream
+    Q.sub_offsets[2:] -= 16
+    Q.stream = np.delete(P.stream, np.s_[int(P.sub_offsets[1]) - 16:int(P.sub_offsets[1])])
+    assert oracle.unpack(T, Q)[1] == oracle.ERR_CORRUPT
+
+
+def test_segments_overhead_per_lane_is_the_state_and_a_length():
+    """Coded size = the plain coder's bits of every lane + (R + 16) bits per lane that owns
+    symbols + 16 bits per empty lane + word/16-byte padding + 8 bytes of offset per sub-stream."""
+    rng = np.random.default_rng(19)
+    n, C, G, R = 1 << 17, 16384, 2, 8
+    msg = _source(rng, n, A=7, zp=3, th=0.1)
+    T = _table(msg, 7, R)
+    P = oracle.pack(T, msg, C, G, oracle.SEGMENTS)
+    S = C // (32 * G)
+    bits = 0
+    for lam in range(n // S):
+        bits += oracle.encode_plain(T, msg[lam * S:(lam + 1) * S])[2] + R
+    pad = 0
+    for sub in range(P.n_sub):
+        lens = np.frombuffer(bytes(P.stream[int(P.sub_offsets[sub]):int(P.sub_offsets[sub]) + 64]), dtype="<u2")
+        body = int(lens.sum())
+        pad += (int(P.sub_offsets[sub + 1]) - int(P.sub_offsets[sub]) - 64) * 8 - body
+        assert 0 <= (int(P.sub_offsets[sub + 1]) - int(P.sub_offsets[sub]) - 64) * 8 - body < 128 + 32
+    assert P.stream.size * 8 == bits + 16 * (n // S) + pad
+    # and it is slimmer than the quads container at the same number of lanes
+    assert P.total_bytes() < oracle.pack(T, msg, C, G, oracle.QUADS).total_bytes()
