@@ -58,9 +58,9 @@ def _lib():
         L.anso_pack_quads.argtypes = [vp, vp, i64, i64, i32, vp, u64, vp, vp]
         L.anso_pack_quads.restype = i64
         L.anso_unpack_quads.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, i64, vp]
-        L.anso_pack_segments.argtypes = [vp, vp, i64, i64, i32, vp, u64, vp]
-        L.anso_pack_segments.restype = i64
-        L.anso_unpack_segments.argtypes = [vp, vp, vp, i64, i64, i32, i64, i64, vp]
+        L.anso_pack_strips.argtypes = [vp, vp, i64, i64, i32, vp, u64, vp]
+        L.anso_pack_strips.restype = i64
+        L.anso_unpack_strips.argtypes = [vp, vp, vp, i64, i64, i32, i64, i64, vp]
         L.anso_dequant_f32.argtypes = [vp, i64, i32, ctypes.c_float, vp]
         L.anso_dequant_f32.restype = None
         L.anso_dequant_bf16.argtypes = [vp, i64, i32, ctypes.c_float, vp]
@@ -76,7 +76,7 @@ def _p(a: np.ndarray):
     return a.ctypes.data
 
 
-INTERLEAVED, PRIVATE, QUADS, SEGMENTS = 0, 1, 2, 3
+INTERLEAVED, PRIVATE, QUADS, STRIPS = 0, 1, 2, 3
 
 
 class Table:
@@ -182,16 +182,16 @@ def pack(T: Table, symbols, chunk: int, groups: int = 1, layout: int = INTERLEAV
     n_chunks = (n + chunk - 1) // chunk
     n_sub = n_chunks * groups
     cap = n * 2 + n_sub * (32 * 8 + 32) + 64
-    if layout == SEGMENTS:                 # per sub-stream: lengths, 32 states, worst-case fields, padding
-        if chunk % (32 * groups):
-            raise OracleError(ERR_ARG, "pack (segments: chunk must be a multiple of the lanes)")
+    if layout == STRIPS:                   # per sub-stream: lengths, 32 states, worst-case fields, padding
+        if chunk % (128 * groups):
+            raise OracleError(ERR_ARG, "pack (strips: chunk must be a multiple of 4 * lanes)")
         cap = n_sub * (64 + 4 * (chunk // (32 * groups) + 1) * T.R + 36) + 64
     stream = np.zeros(cap, dtype=np.uint8)
     offs = np.zeros(n_sub + 1, dtype=np.uint64)
     lib = _lib()
-    if layout == SEGMENTS:
+    if layout == STRIPS:
         meta = np.zeros((n_sub, 0), dtype=np.uint32)       # this container has no per-lane array
-        total = lib.anso_pack_segments(T.ptr, _p(symbols), n, chunk, groups, _p(stream), cap, _p(offs))
+        total = lib.anso_pack_strips(T.ptr, _p(symbols), n, chunk, groups, _p(stream), cap, _p(offs))
     elif layout == INTERLEAVED:
         meta = np.zeros((n_sub, 32), dtype=np.uint16)
         total = lib.anso_pack_interleaved(T.ptr, _p(symbols), n, chunk, groups, _p(stream), cap, _p(offs), _p(meta))
@@ -209,9 +209,9 @@ def unpack(T: Table, P: Packed, threads: int = 1, chunk_range=None):
     out = np.zeros(max(P.n, 1), dtype=np.uint8)
     lib = _lib()
     lo, hi = chunk_range if chunk_range is not None else (0, P.n_chunks)
-    if P.layout == SEGMENTS:
+    if P.layout == STRIPS:
         def work(rng):
-            return lib.anso_unpack_segments(T.ptr, _p(P.stream), _p(P.sub_offsets), P.n, P.chunk, P.groups,
+            return lib.anso_unpack_strips(T.ptr, _p(P.stream), _p(P.sub_offsets), P.n, P.chunk, P.groups,
                                             rng[0], rng[1], _p(out))
     else:
         fn = {INTERLEAVED: lib.anso_unpack_interleaved, PRIVATE: lib.anso_unpack_private,

@@ -30,9 +30,10 @@
  *       "private":     each lane owns a contiguous run of 32-bit words;
  *       "quads":       private lanes that take four consecutive symbols per
  *                      turn and fill their words most significant bit first.
- *       "segments":    every lane owns a contiguous run of the chunk; a lane's
- *                      bits begin with its initial state; a sub-stream carries
- *                      its lanes' bit lengths and their strings back to back.
+ *       "strips":      a sub-stream owns a contiguous strip of the chunk, dealt
+ *                      to its lanes four symbols at a time; a lane's bits begin
+ *                      with its initial state; a sub-stream carries its lanes'
+ *                      bit lengths and their strings back to back.
  *   - frequency normalisation (largest-remainder, every present symbol >= 1).
  *
  * Pins (see tests): hand-enumerated state traces, table tiling invariants,
@@ -566,60 +567,73 @@ int anso_unpack_quads(const anso_table* T, const uint8_t* stream, const uint64_t
 }
 
 /*
- * Segments container.  The paper leaves open which symbols a stream owns and
- * how a stream is laid out (Section III-B only fixes one state per stream and a
- * shared table); this container gives every lane a CONTIGUOUS run of the chunk
- * and keeps the per-lane overhead to the state and one 16-bit length:
- *   - C must be a multiple of W = 32*G; S = C / W <= 4096.  Lane lambda owns the
- *     chunk-relative symbols [lambda*S, min((lambda+1)*S, n_chunk)): a run that
- *     may be short or empty in the layer's last chunk.
+ * Strips container.  The paper leaves open which symbols a stream owns and how
+ * a stream is laid out (Section III-B only fixes one state per stream and a
+ * shared table); this container keeps a sub-stream's symbols in one contiguous
+ * strip of the chunk and the per-lane overhead down to the state and one
+ * 16-bit length:
+ *   - C must be a multiple of 4*W, W = 32*G; S = C / W <= 4096 is the number
+ *     of symbols a lane owns in a full chunk.
+ *   - Sub-stream g of a chunk owns the chunk-relative symbols
+ *     [g*32*S, min((g+1)*32*S, n_chunk)): its strip, which may be short or
+ *     empty in the layer's last chunk.
+ *   - Inside the strip the 32 lanes take the symbols four at a time, as in the
+ *     quads container with 32 lanes: strip-relative symbol q sits in quad
+ *     j = q div 4, quad j is the (j div 32)-th quad of lane j mod 32; the
+ *     strip's last quad may be short.
  *   - A lane that owns at least one symbol has the bit string
  *         initial decode state index (R bits), field_0, field_1, ...
  *     every item most significant bit first; a lane without symbols has the
  *     empty string.
- *   - A sub-stream (32 lanes) is: 32 little-endian uint16 = the bit lengths of
+ *   - The sub-stream's bytes: 32 little-endian uint16 = the bit lengths of
  *     its lanes' strings; then the 32 strings back to back, without gaps, in
  *     lane order, filling 32-bit little-endian words from the most significant
  *     bit down (as in the quads container); zero-padded to a multiple of 16
  *     bytes.  There is no lane_meta array.
  * Sub-streams are numbered chunk-major as in the other containers.
  */
-#define ANSO_SEG_HEADER 64   /* bytes: 32 lanes x uint16 bit length */
-#define ANSO_SEG_MAX_S 4096
+#define ANSO_STRIP_HEADER 64   /* bytes: 32 lanes x uint16 bit length */
+#define ANSO_STRIP_MAX_S 4096
 
-int64_t anso_pack_segments(const anso_table* T, const uint8_t* symbols, int64_t n,
-                           int64_t C, int G, uint8_t* stream, uint64_t cap_bytes,
-                           uint64_t* sub_offsets) {
+static int64_t strip_symbols(int64_t n_chunk, int64_t S, int g) {
+  int64_t ns = n_chunk - (int64_t)g * 32 * S;
+  if (ns > 32 * S) ns = 32 * S;
+  return ns < 0 ? 0 : ns;
+}
+
+int64_t anso_pack_strips(const anso_table* T, const uint8_t* symbols, int64_t n,
+                         int64_t C, int G, uint8_t* stream, uint64_t cap_bytes,
+                         uint64_t* sub_offsets) {
   if (!T || C < 1 || G < 1 || n < 0) return ANSO_ERR_ARG;
   const int W = 32 * G;
-  if (C % W) return ANSO_ERR_ARG;
+  if (C % (4 * W)) return ANSO_ERR_ARG;
   const int64_t S = C / W;
-  if (S > ANSO_SEG_MAX_S) return ANSO_ERR_ARG;
+  if (S > ANSO_STRIP_MAX_S) return ANSO_ERR_ARG;
   const int64_t n_chunks = (n + C - 1) / C;
+  uint8_t* mine = (uint8_t*)malloc((size_t)S);
   uint8_t* fnb = (uint8_t*)malloc((size_t)S);
   uint16_t* fval = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)S);
   uint64_t off = 0;
   int64_t rc = ANSO_OK;
   for (int64_t c = 0; c < n_chunks && rc >= 0; ++c) {
-    const uint8_t* cs = symbols + c * C;
     const int64_t nc = (n - c * C) < C ? (n - c * C) : C;
     for (int g = 0; g < G && rc >= 0; ++g) {
       const int64_t sub = c * G + g;
+      const uint8_t* strip = symbols + c * C + (int64_t)g * 32 * S;
+      const int64_t ns = strip_symbols(nc, S, g);
       sub_offsets[sub] = off;
       /* worst case: header + 32 lanes of R + S*R bits, + padding */
-      const uint64_t worst = ANSO_SEG_HEADER + (uint64_t)(32 * (S + 1) * T->R + 7) / 8 + 20;
+      const uint64_t worst = ANSO_STRIP_HEADER + (uint64_t)(32 * (S + 1) * T->R + 7) / 8 + 20;
       if (off + worst > cap_bytes) { rc = ANSO_ERR_SPACE; break; }
       memset(stream + off, 0, (size_t)worst);
-      uint8_t* body = stream + off + ANSO_SEG_HEADER;
+      uint8_t* body = stream + off + ANSO_STRIP_HEADER;
       uint64_t pos = 0;                                /* bit position in the body */
       for (int k = 0; k < 32; ++k) {
-        const int64_t first = (int64_t)(32 * g + k) * S;
-        int64_t cnt = nc - first;
-        if (cnt > S) cnt = S;
-        if (cnt < 0) cnt = 0;
+        const int64_t cnt = quad_lane_count(ns, 32, k);
         const uint64_t pos0 = pos;
         if (cnt > 0) {
-          int init = anso_encode_lane(T, cs + first, cnt, 1, fnb, fval);
+          for (int64_t t = 0; t < cnt; ++t) mine[t] = strip[quad_position(32, k, t)];
+          int init = anso_encode_lane(T, mine, cnt, 1, fnb, fval);
           if (init < 0) { rc = init; break; }
           put_bits_msb(body, &pos, (uint32_t)init, T->R);
           for (int64_t t = 0; t < cnt; ++t) put_bits_msb(body, &pos, fval[t], fnb[t]);
@@ -629,45 +643,43 @@ int64_t anso_pack_segments(const anso_table* T, const uint8_t* symbols, int64_t 
         stream[off + 2 * k + 1] = (uint8_t)(len >> 8);
       }
       if (rc < 0) break;
-      off += ANSO_SEG_HEADER + ((pos + 31) / 32) * 4;
+      off += ANSO_STRIP_HEADER + ((pos + 31) / 32) * 4;
       while (off % 16) ++off;                          /* already zero */
     }
   }
   if (rc >= 0) sub_offsets[n_chunks * G] = off;
-  free(fnb); free(fval);
+  free(mine); free(fnb); free(fval);
   return rc < 0 ? rc : (int64_t)off;
 }
 
-int anso_unpack_segments(const anso_table* T, const uint8_t* stream, const uint64_t* sub_offsets,
-                         int64_t n, int64_t C, int G,
-                         int64_t chunk_begin, int64_t chunk_end, uint8_t* out) {
+int anso_unpack_strips(const anso_table* T, const uint8_t* stream, const uint64_t* sub_offsets,
+                       int64_t n, int64_t C, int G,
+                       int64_t chunk_begin, int64_t chunk_end, uint8_t* out) {
   const int W = 32 * G;
-  if (C % W) return ANSO_ERR_ARG;
+  if (C % (4 * W)) return ANSO_ERR_ARG;
   const int64_t S = C / W;
   int rc = ANSO_OK;
   for (int64_t c = chunk_begin; c < chunk_end; ++c) {
-    uint8_t* co = out + c * C;
     const int64_t nc = (n - c * C) < C ? (n - c * C) : C;
     for (int g = 0; g < G; ++g) {
       const int64_t sub = c * G + g;
+      uint8_t* so = out + c * C + (int64_t)g * 32 * S;      /* the strip's place in the output */
+      const int64_t ns = strip_symbols(nc, S, g);
       const uint8_t* p = stream + sub_offsets[sub];
       const uint64_t extent = sub_offsets[sub + 1] - sub_offsets[sub];
-      if (extent < ANSO_SEG_HEADER) { rc = ANSO_ERR_CORRUPT; continue; }
-      const uint8_t* body = p + ANSO_SEG_HEADER;
-      const uint64_t body_bytes = extent - ANSO_SEG_HEADER;
+      if (extent < ANSO_STRIP_HEADER) { rc = ANSO_ERR_CORRUPT; continue; }
+      const uint8_t* body = p + ANSO_STRIP_HEADER;
+      const uint64_t body_bytes = extent - ANSO_STRIP_HEADER;
       uint64_t start = 0;                              /* bit position of lane k's string */
       for (int k = 0; k < 32; ++k) {
-        const int64_t first = (int64_t)(32 * g + k) * S;
-        int64_t cnt = nc - first;
-        if (cnt > S) cnt = S;
-        if (cnt < 0) cnt = 0;
+        const int64_t cnt = quad_lane_count(ns, 32, k);
         const uint64_t len = (uint64_t)p[2 * k] | ((uint64_t)p[2 * k + 1] << 8);
         uint64_t pos = start;
         if (cnt > 0) {
           uint32_t i = get_bits_msb(body, body_bytes, pos, T->R);
           pos += (uint64_t)T->R;
           for (int64_t t = 0; t < cnt; ++t) {
-            co[first + t] = T->sym[i];
+            so[quad_position(32, k, t)] = T->sym[i];
             const int nb = T->nb[i];
             const uint32_t v = get_bits_msb(body, body_bytes, pos, nb);
             pos += (uint64_t)nb;
@@ -679,7 +691,7 @@ int anso_unpack_segments(const anso_table* T, const uint8_t* stream, const uint6
         start += len;
       }
       /* the sub-stream holds exactly the header, the words its bits need, and the pad */
-      uint64_t want = ANSO_SEG_HEADER + ((start + 31) / 32) * 4;
+      uint64_t want = ANSO_STRIP_HEADER + ((start + 31) / 32) * 4;
       want = (want + 15) / 16 * 16;
       if (want != extent) rc = ANSO_ERR_CORRUPT;
     }

@@ -223,51 +223,56 @@ def test_quads_word_of_the_hand_trace(name):
     assert rc == oracle.OK and out[pos].tolist() == msg and (out == sym).all()
 
 
-# ---- segments container -------------------------------------------------------------------
-SEG_CASES = [(0, 512, 1), (1, 512, 1), (6, 512, 1), (511, 512, 1), (512, 512, 1), (513, 512, 1),
-             (5000, 1024, 2), (4096, 1024, 1), (777, 4096, 4), (65536 + 17, 16384, 2), (3000, 2048, 2),
-             (100, 32, 1), (1000, 64, 2)]
+# ---- strips container -----------------------------------------------------------------------
+STRIP_CASES = [(0, 512, 1), (1, 512, 1), (6, 512, 1), (130, 512, 1), (511, 512, 1), (512, 512, 1), (513, 512, 1),
+               (5000, 1024, 2), (4096, 1024, 1), (777, 4096, 4), (65536 + 17, 16384, 2), (3000, 2048, 2),
+               (1000, 128, 1), (1000, 256, 2), (40001, 16384, 4)]
 
 
-@pytest.mark.parametrize("n,C,G", SEG_CASES)
-def test_segments_round_trip(n, C, G):
+@pytest.mark.parametrize("n,C,G", STRIP_CASES)
+def test_strips_round_trip(n, C, G):
     rng = np.random.default_rng(n + C + G)
     msg = _source(rng, max(n, 1))
     T = _table(msg, 15, 12)
     msg = msg[:n]
-    P = oracle.pack(T, msg, C, G, oracle.SEGMENTS)
+    P = oracle.pack(T, msg, C, G, oracle.STRIPS)
     assert P.sub_offsets.size == P.n_sub + 1 and P.sub_offsets[-1] == P.stream.size
     assert all(int(o) % 16 == 0 for o in P.sub_offsets) and P.lane_meta.size == 0
     out, rc = oracle.unpack(T, P)
     assert rc == oracle.OK and (out == msg).all()
 
 
-def test_segments_chunk_must_be_a_multiple_of_the_lanes():
+def test_strips_chunk_must_be_a_multiple_of_four_times_the_lanes():
     T = oracle.Table([3, 1], 2)
-    with pytest.raises(oracle.OracleError):
-        oracle.pack(T, np.zeros(10, dtype=np.uint8), 1000, 1, oracle.SEGMENTS)
+    for C, G in ((1000, 1), (64, 1), (384, 2)):
+        with pytest.raises(oracle.OracleError):
+            oracle.pack(T, np.zeros(10, dtype=np.uint8), C, G, oracle.STRIPS)
 
 
-@pytest.mark.parametrize("n,C,G", [(3000, 2048, 2), (1000, 1024, 1), (517, 256, 4), (130, 4096, 1), (40000, 16384, 2)])
-def test_segments_equal_plain_single_lane_coding(n, C, G):
-    """Independent build of every sub-stream in Python: lane lambda owns the contiguous run
-    [lambda*S, (lambda+1)*S) of its chunk; its string is the plain one-lane coder's initial state
-    in R bits followed by that coder's fields, most significant bit first; a sub-stream is the 32
-    lengths as little-endian uint16, then the strings back to back in 32-bit little-endian words
-    filled from the top bit, zero-padded to 16 bytes."""
+@pytest.mark.parametrize("n,C,G", [(3000, 2048, 2), (1000, 1024, 1), (517, 512, 4), (130, 4096, 1), (40000, 16384, 2)])
+def test_strips_equal_plain_single_lane_coding(n, C, G):
+    """Independent build of every sub-stream in Python.  Sub-stream g owns the strip
+    [g*32*S, (g+1)*32*S) of its chunk; the strip is dealt to 32 lanes four symbols at a time;
+    a lane's string is the plain one-lane coder's initial state in R bits followed by that
+    coder's fields, most significant bit first; the sub-stream is the 32 lengths as
+    little-endian uint16, then the strings back to back in 32-bit little-endian words filled
+    from the top bit, zero-padded to 16 bytes."""
     rng = np.random.default_rng(n)
     W, R = 32 * G, 10
     S = C // W
     msg = _source(rng, n)
     T = _table(msg, 15, R)
-    P = oracle.pack(T, msg, C, G, oracle.SEGMENTS)
+    P = oracle.pack(T, msg, C, G, oracle.STRIPS)
     for c in range(P.n_chunks):
         chunk = msg[c * C:(c + 1) * C]
         for g in range(G):
             sub = c * G + g
+            strip = chunk[g * 32 * S:(g + 1) * 32 * S]
+            owned = _quads_lanes(strip.size, 32)
+            assert sorted(q for l in owned for q in l) == list(range(strip.size))
             lens, bits = [], ""
             for k in range(32):
-                mine = chunk[(32 * g + k) * S:(32 * g + k + 1) * S]
+                mine = strip[owned[k]]
                 s = ""
                 if mine.size:
                     init, nb, val = oracle.encode_lane_fields(T, mine)
@@ -284,38 +289,79 @@ def test_segments_equal_plain_single_lane_coding(n, C, G):
             assert bytes(P.stream[b0:b1]) == want
 
 
+def _body_bits(stream, nbits):
+    words = np.frombuffer(bytes(stream[64:64 + 4 * ((nbits + 31) // 32)]), dtype="<u4")
+    return "".join(format(int(w), "032b") for w in words)[:nbits]
+
+
 @pytest.mark.parametrize("name", ["trace_T1.txt", "trace_T2.txt"])
-def test_segments_bytes_of_the_hand_trace(name):
-    """A layer that is the hand trace's message alone: lane 0 owns all of it, the other lanes
-    are empty; lengths, first word and size are the ones worked out by hand in the fixture."""
+def test_strips_bytes_of_the_hand_trace(name):
+    """Lane 0 of a one-strip layer carrying the hand trace's message (positions 0..3, 128..131,
+    ...; the other positions hold the first symbol): its length and bits are the ones worked
+    out by hand in the fixture; for T1 so are the other lanes' and the first word."""
     g = read_golden(name)
-    T = oracle.Table(_ints(g["freqs"]), int(g["table_log"]))
-    msg = np.array(_ints(g["message"]), dtype=np.uint8)
-    P = oracle.pack(T, msg, 512, 1, oracle.SEGMENTS)
-    lens = np.frombuffer(bytes(P.stream[:64]), dtype="<u2")
-    assert int(lens[0]) == len(g["segments_lane_bits"]) and not lens[1:].any()
-    assert bytes(P.stream[64:68]) == bytes.fromhex(g["segments_first_word_hex"].replace(" ", ""))
-    assert P.stream.size == int(g["segments_sub_stream_bytes"]) and not P.stream[68:].any()
+    R = int(g["table_log"])
+    T = oracle.Table(_ints(g["freqs"]), R)
+    msg = _ints(g["message"])
+    pos = [(t // 4) * 128 + t % 4 for t in range(len(msg))]
+    sym = np.full(pos[-1] + 1, msg[0], dtype=np.uint8)
+    sym[pos] = msg
+    P = oracle.pack(T, sym, 512, 1, oracle.STRIPS)
+    lens = np.frombuffer(bytes(P.stream[:64]), dtype="<u2").astype(int)
+    want = g["strips_lane_bits"]
+    assert lens[0] == len(want) and _body_bits(P.stream, len(want)) == want
+    if "strips_other_lane_bits" in g:
+        other = g["strips_other_lane_bits"]
+        assert (lens[1:] == len(other)).all()
+        assert _body_bits(P.stream, int(lens.sum())) == want + other * 31
+        assert bytes(P.stream[64:68]) == bytes.fromhex(g["strips_first_word_hex"].replace(" ", ""))
+        assert P.stream.size == int(g["strips_sub_stream_bytes"])
     out, rc = oracle.unpack(T, P)
-    assert rc == oracle.OK and out.tolist() == msg.tolist()
+    assert rc == oracle.OK and out[pos].tolist() == msg and (out == sym).all()
 
 
-def test_segments_same_symbols_for_every_chunking_and_threads():
+def test_strips_same_symbols_for_every_chunking_and_threads():
     rng = np.random.default_rng(21)
     msg = _source(rng, 50000)
     T = _table(msg, 15, 11)
-    for C, G in [(1024, 1), (4096, 1), (4096, 4), (16384, 2), (65536, 8), (32, 1), (131072, 1)]:
-        P = oracle.pack(T, msg, C, G, oracle.SEGMENTS)
+    for C, G in [(1024, 1), (4096, 1), (4096, 4), (16384, 2), (65536, 8), (128, 1), (131072, 1)]:
+        P = oracle.pack(T, msg, C, G, oracle.STRIPS)
         for th in (1, 4):
             out, rc = oracle.unpack(T, P, threads=th)
             assert rc == oracle.OK and (out == msg).all()
 
 
-def test_segments_corruption_is_reported():
+def test_strips_with_one_group_own_the_symbols_of_quads():
+    """With 32 lanes per chunk the strip is the whole chunk, so lane k owns the very symbols it
+    owns in the quads container: same initial states, same fields."""
+    rng = np.random.default_rng(23)
+    msg = _source(rng, 9000)
+    T = _table(msg, 15, 9)
+    Pq = oracle.pack(T, msg, 4096, 1, oracle.QUADS)
+    Ps = oracle.pack(T, msg, 4096, 1, oracle.STRIPS)
+    for sub in range(Pq.n_sub):
+        b0 = int(Ps.sub_offsets[sub])
+        lens = np.frombuffer(bytes(Ps.stream[b0:b0 + 64]), dtype="<u2").astype(int)
+        body = _body_bits(Ps.stream[b0:], int(lens.sum()))
+        start = 0
+        for k in range(32):
+            meta = int(Pq.lane_meta[sub, k])
+            mine = body[start:start + lens[k]]
+            start += lens[k]
+            if not lens[k]:
+                continue
+            assert int(mine[:9], 2) == (meta & 0xFFFF)
+            q0 = int(Pq.sub_offsets[sub]) + 4 * (meta >> 16)
+            nw = (lens[k] - 9 + 31) // 32
+            qbits = "".join(format(int(w), "032b") for w in np.frombuffer(bytes(Pq.stream[q0:q0 + 4 * nw]), dtype="<u4"))
+            assert qbits[:lens[k] - 9] == mine[9:]
+
+
+def test_strips_corruption_is_reported():
     rng = np.random.default_rng(16)
     msg = _source(rng, 8192)
     T = _table(msg, 15, 12)
-    P = oracle.pack(T, msg, 4096, 1, oracle.SEGMENTS)
+    P = oracle.pack(T, msg, 4096, 1, oracle.STRIPS)
     flagged = 0
     positions = list(range(3, P.stream.size, 97))
     for pos in positions:
@@ -334,24 +380,25 @@ def test_segments_corruption_is_reported():
     assert oracle.unpack(T, Q)[1] == oracle.ERR_CORRUPT
 
 
-def test_segments_overhead_per_lane_is_the_state_and_a_length():
-    """Coded size = the plain coder's bits of every lane + (R + 16) bits per lane that owns
-    symbols + 16 bits per empty lane + word/16-byte padding + 8 bytes of offset per sub-stream."""
+def test_strips_overhead_per_lane_is_the_state_and_a_length():
+    """Coded size = the plain coder's bits of every lane + (R + 16) bits per lane + word and
+    16-byte padding per sub-stream; slimmer than the quads container at the same lanes."""
     rng = np.random.default_rng(19)
     n, C, G, R = 1 << 17, 16384, 2, 8
     msg = _source(rng, n, A=7, zp=3, th=0.1)
     T = _table(msg, 7, R)
-    P = oracle.pack(T, msg, C, G, oracle.SEGMENTS)
+    P = oracle.pack(T, msg, C, G, oracle.STRIPS)
     S = C // (32 * G)
     bits = 0
-    for lam in range(n // S):
-        bits += oracle.encode_plain(T, msg[lam * S:(lam + 1) * S])[2] + R
+    for sub in range(P.n_sub):
+        strip = msg[sub * 32 * S:(sub + 1) * 32 * S]
+        for mine in _quads_lanes(strip.size, 32):
+            bits += oracle.encode_plain(T, strip[mine])[2] + R + 16
     pad = 0
     for sub in range(P.n_sub):
-        lens = np.frombuffer(bytes(P.stream[int(P.sub_offsets[sub]):int(P.sub_offsets[sub]) + 64]), dtype="<u2")
-        body = int(lens.sum())
-        pad += (int(P.sub_offsets[sub + 1]) - int(P.sub_offsets[sub]) - 64) * 8 - body
-        assert 0 <= (int(P.sub_offsets[sub + 1]) - int(P.sub_offsets[sub]) - 64) * 8 - body < 128 + 32
-    assert P.stream.size * 8 == bits + 16 * (n // S) + pad
-    # and it is slimmer than the quads container at the same number of lanes
+        b0, b1 = int(P.sub_offsets[sub]), int(P.sub_offsets[sub + 1])
+        body = int(np.frombuffer(bytes(P.stream[b0:b0 + 64]), dtype="<u2").astype(int).sum())
+        assert 0 <= (b1 - b0 - 64) * 8 - body < 128 + 32
+        pad += (b1 - b0 - 64) * 8 - body
+    assert P.stream.size * 8 == bits + pad
     assert P.total_bytes() < oracle.pack(T, msg, C, G, oracle.QUADS).total_bytes()
