@@ -53,6 +53,18 @@
  *       lane writes 4 adjacent outputs per turn.  And a lane's bits fill its 32-bit words
  *       from the most significant bit down, each field most significant bit first (the
  *       words themselves are stored little-endian).  d_lane_meta as for ANS_LAYOUT_PRIVATE.
+ *     ANS_LAYOUT_STRIPS: made for layers in which one symbol owns most of the states, so that
+ *       many transitions take no bits (Section II-A) and a look-up can stand for a run of that
+ *       symbol plus one more.  chunk_symbols must be a multiple of lanes, with
+ *       S = chunk_symbols / lanes <= 4096.  Sub-stream g of a chunk owns the chunk's symbols
+ *       [g * 32 * S, (g + 1) * 32 * S): a contiguous strip (short or empty at the layer's end).
+ *       Inside the strip its 32 lanes take the symbols round-robin (strip-relative symbol q is
+ *       the (q / 32)-th symbol of lane q % 32).  A lane that owns symbols has the bit string: initial state (table_log
+ *       bits), then its fields, every item most significant bit first.  The sub-stream's bytes
+ *       are 32 little-endian uint16 (the lanes' bit lengths), then the 32 strings back to back
+ *       without gaps, filling 32-bit little-endian words from the most significant bit down,
+ *       zero-padded to a multiple of 16 bytes.  There is no per-lane array: d_lane_meta is
+ *       ignored and may be NULL.
  */
 #ifndef ANS_B200_H
 #define ANS_B200_H
@@ -79,10 +91,12 @@ extern "C" {
 #define ANS_LAYOUT_INTERLEAVED 0
 #define ANS_LAYOUT_PRIVATE     1
 #define ANS_LAYOUT_QUADS       2
+#define ANS_LAYOUT_STRIPS      3
 
 #define ANS_MAX_TABLE_LOG 14
 #define ANS_MAX_LANES     2048   /* lanes per chunk: any multiple of 32 up to this */
 #define ANS_MAX_ALPHABET  256
+#define ANS_MAX_STRIP_LANE_SYMBOLS 4096   /* ANS_LAYOUT_STRIPS: chunk_symbols / lanes at most */
 
 /* bits of the device status word (0 = every stream sound) */
 #define ANS_STATUS_BAD_FINAL_STATE 1u   /* a lane did not end in state index 0          */
@@ -100,7 +114,8 @@ typedef struct ans_layer_desc {
   const void*     d_table;        /* this layer's table, written by ans_build_decode_tables  */
   const uint8_t*  d_stream;       /* compressed bytes of all the layer's sub-streams, 16-byte aligned */
   const uint64_t* d_sub_offsets;  /* [n_sub + 1] byte offsets into d_stream, each a multiple of 16 */
-  const void*     d_lane_meta;    /* per-lane initial state (and first word): see the layouts above */
+  const void*     d_lane_meta;    /* per-lane initial state (and first word): see the layouts above;
+                                     unused (may be NULL) for ANS_LAYOUT_STRIPS                */
   void*           d_out;          /* n_symbols elements of out_dtype, 16-byte aligned       */
   uint64_t        stream_bytes;   /* bytes readable at d_stream (offsets beyond it are flagged) */
   uint64_t        n_symbols;      /* weights in the layer; may be 0                          */
@@ -251,7 +266,8 @@ int ans_host_pack_bound(uint64_t n_symbols, uint32_t chunk_symbols, uint32_t lan
  * append its label bits) into the chosen container.
  *   h_symbols[n_symbols]; h_freqs[256] as given to ans_build_decode_tables
  *   h_stream_out (capacity stream_cap), h_sub_offsets_out[n_sub + 1],
- *   h_lane_meta_out: uint16_t[n_sub][32] (interleaved) or uint32_t[n_sub][32] (private, quads)
+ *   h_lane_meta_out: uint16_t[n_sub][32] (interleaved) or uint32_t[n_sub][32] (private, quads);
+ *                    unused (may be NULL) for the strips layout
  *   n_threads: host threads to use (<= 0: all)
  * *h_stream_bytes_out receives the bytes written.
  */

@@ -183,8 +183,8 @@ def pack(T: Table, symbols, chunk: int, groups: int = 1, layout: int = INTERLEAV
     n_sub = n_chunks * groups
     cap = n * 2 + n_sub * (32 * 8 + 32) + 64
     if layout == STRIPS:                   # per sub-stream: lengths, 32 states, worst-case fields, padding
-        if chunk % (128 * groups):
-            raise OracleError(ERR_ARG, "pack (strips: chunk must be a multiple of 4 * lanes)")
+        if chunk % (32 * groups):
+            raise OracleError(ERR_ARG, "pack (strips: chunk must be a multiple of the lanes)")
         cap = n_sub * (64 + 4 * (chunk // (32 * groups) + 1) * T.R + 36) + 64
     stream = np.zeros(cap, dtype=np.uint8)
     offs = np.zeros(n_sub + 1, dtype=np.uint64)

@@ -31,9 +31,9 @@
  *       "quads":       private lanes that take four consecutive symbols per
  *                      turn and fill their words most significant bit first.
  *       "strips":      a sub-stream owns a contiguous strip of the chunk, dealt
- *                      to its lanes four symbols at a time; a lane's bits begin
- *                      with its initial state; a sub-stream carries its lanes'
- *                      bit lengths and their strings back to back.
+ *                      round-robin to its lanes; a lane's bits begin with its
+ *                      initial state; a sub-stream carries its lanes' bit
+ *                      lengths and their strings back to back.
  *   - frequency normalisation (largest-remainder, every present symbol >= 1).
  *
  * Pins (see tests): hand-enumerated state traces, table tiling invariants,
@@ -572,15 +572,13 @@ int anso_unpack_quads(const anso_table* T, const uint8_t* stream, const uint64_t
  * shared table); this container keeps a sub-stream's symbols in one contiguous
  * strip of the chunk and the per-lane overhead down to the state and one
  * 16-bit length:
- *   - C must be a multiple of 4*W, W = 32*G; S = C / W <= 4096 is the number
- *     of symbols a lane owns in a full chunk.
+ *   - C must be a multiple of W = 32*G; S = C / W <= 4096 is the number of
+ *     symbols a lane owns in a full chunk.
  *   - Sub-stream g of a chunk owns the chunk-relative symbols
  *     [g*32*S, min((g+1)*32*S, n_chunk)): its strip, which may be short or
  *     empty in the layer's last chunk.
- *   - Inside the strip the 32 lanes take the symbols four at a time, as in the
- *     quads container with 32 lanes: strip-relative symbol q sits in quad
- *     j = q div 4, quad j is the (j div 32)-th quad of lane j mod 32; the
- *     strip's last quad may be short.
+ *   - Inside the strip the 32 lanes take the symbols round-robin: strip-relative
+ *     symbol q is the (q div 32)-th symbol of lane q mod 32.
  *   - A lane that owns at least one symbol has the bit string
  *         initial decode state index (R bits), field_0, field_1, ...
  *     every item most significant bit first; a lane without symbols has the
@@ -588,8 +586,8 @@ int anso_unpack_quads(const anso_table* T, const uint8_t* stream, const uint64_t
  *   - The sub-stream's bytes: 32 little-endian uint16 = the bit lengths of
  *     its lanes' strings; then the 32 strings back to back, without gaps, in
  *     lane order, filling 32-bit little-endian words from the most significant
- *     bit down (as in the quads container); zero-padded to a multiple of 16
- *     bytes.  There is no lane_meta array.
+ *     bit down (the bit order of the quads container); zero-padded to a
+ *     multiple of 16 bytes.  There is no lane_meta array.
  * Sub-streams are numbered chunk-major as in the other containers.
  */
 #define ANSO_STRIP_HEADER 64   /* bytes: 32 lanes x uint16 bit length */
@@ -606,11 +604,10 @@ int64_t anso_pack_strips(const anso_table* T, const uint8_t* symbols, int64_t n,
                          uint64_t* sub_offsets) {
   if (!T || C < 1 || G < 1 || n < 0) return ANSO_ERR_ARG;
   const int W = 32 * G;
-  if (C % (4 * W)) return ANSO_ERR_ARG;
+  if (C % W) return ANSO_ERR_ARG;
   const int64_t S = C / W;
   if (S > ANSO_STRIP_MAX_S) return ANSO_ERR_ARG;
   const int64_t n_chunks = (n + C - 1) / C;
-  uint8_t* mine = (uint8_t*)malloc((size_t)S);
   uint8_t* fnb = (uint8_t*)malloc((size_t)S);
   uint16_t* fval = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)S);
   uint64_t off = 0;
@@ -629,11 +626,10 @@ int64_t anso_pack_strips(const anso_table* T, const uint8_t* symbols, int64_t n,
       uint8_t* body = stream + off + ANSO_STRIP_HEADER;
       uint64_t pos = 0;                                /* bit position in the body */
       for (int k = 0; k < 32; ++k) {
-        const int64_t cnt = quad_lane_count(ns, 32, k);
+        const int64_t cnt = lane_count(ns, 32, k);
         const uint64_t pos0 = pos;
         if (cnt > 0) {
-          for (int64_t t = 0; t < cnt; ++t) mine[t] = strip[quad_position(32, k, t)];
-          int init = anso_encode_lane(T, mine, cnt, 1, fnb, fval);
+          int init = anso_encode_lane(T, strip + k, cnt, 32, fnb, fval);
           if (init < 0) { rc = init; break; }
           put_bits_msb(body, &pos, (uint32_t)init, T->R);
           for (int64_t t = 0; t < cnt; ++t) put_bits_msb(body, &pos, fval[t], fnb[t]);
@@ -648,7 +644,7 @@ int64_t anso_pack_strips(const anso_table* T, const uint8_t* symbols, int64_t n,
     }
   }
   if (rc >= 0) sub_offsets[n_chunks * G] = off;
-  free(mine); free(fnb); free(fval);
+  free(fnb); free(fval);
   return rc < 0 ? rc : (int64_t)off;
 }
 
@@ -656,7 +652,7 @@ int anso_unpack_strips(const anso_table* T, const uint8_t* stream, const uint64_
                        int64_t n, int64_t C, int G,
                        int64_t chunk_begin, int64_t chunk_end, uint8_t* out) {
   const int W = 32 * G;
-  if (C % (4 * W)) return ANSO_ERR_ARG;
+  if (C % W) return ANSO_ERR_ARG;
   const int64_t S = C / W;
   int rc = ANSO_OK;
   for (int64_t c = chunk_begin; c < chunk_end; ++c) {
@@ -672,14 +668,14 @@ int anso_unpack_strips(const anso_table* T, const uint8_t* stream, const uint64_
       const uint64_t body_bytes = extent - ANSO_STRIP_HEADER;
       uint64_t start = 0;                              /* bit position of lane k's string */
       for (int k = 0; k < 32; ++k) {
-        const int64_t cnt = quad_lane_count(ns, 32, k);
+        const int64_t cnt = lane_count(ns, 32, k);
         const uint64_t len = (uint64_t)p[2 * k] | ((uint64_t)p[2 * k + 1] << 8);
         uint64_t pos = start;
         if (cnt > 0) {
           uint32_t i = get_bits_msb(body, body_bytes, pos, T->R);
           pos += (uint64_t)T->R;
           for (int64_t t = 0; t < cnt; ++t) {
-            so[quad_position(32, k, t)] = T->sym[i];
+            so[t * 32 + k] = T->sym[i];
             const int nb = T->nb[i];
             const uint32_t v = get_bits_msb(body, body_bytes, pos, nb);
             pos += (uint64_t)nb;

@@ -17,7 +17,7 @@ ANS_OK = 0
 ANS_ERR_INVALID_ARG, ANS_ERR_BAD_FREQS, ANS_ERR_UNSUPPORTED = -1, -2, -3
 ANS_ERR_BUFFER_TOO_SMALL, ANS_ERR_CUDA, ANS_ERR_CORRUPT = -4, -5, -6
 ANS_U8, ANS_F32, ANS_BF16 = 0, 1, 2
-ANS_LAYOUT_INTERLEAVED, ANS_LAYOUT_PRIVATE, ANS_LAYOUT_QUADS = 0, 1, 2
+ANS_LAYOUT_INTERLEAVED, ANS_LAYOUT_PRIVATE, ANS_LAYOUT_QUADS, ANS_LAYOUT_STRIPS = 0, 1, 2, 3
 DTYPES = {"u8": ANS_U8, "f32": ANS_F32, "bf16": ANS_BF16}
 ELEM_SIZE = {ANS_U8: 1, ANS_F32: 4, ANS_BF16: 2}
 
@@ -214,7 +214,8 @@ def ans_host_pack_layer(symbols: np.ndarray, freqs: np.ndarray, alphabet: int, t
     n_sub = n_chunks * (lanes // 32)
     stream = np.empty(cap.value, dtype=np.uint8)
     offs = np.zeros(n_sub + 1, dtype=np.uint64)
-    meta = np.zeros((n_sub, 32), dtype=np.uint16 if layout == ANS_LAYOUT_INTERLEAVED else np.uint32)
+    meta = np.zeros((n_sub, 0 if layout == ANS_LAYOUT_STRIPS else 32),
+                    dtype=np.uint16 if layout == ANS_LAYOUT_INTERLEAVED else np.uint32)
     used = ctypes.c_uint64()
     _check(lib().ans_host_pack_layer(sym.ctypes.data, sym.size, f.ctypes.data, alphabet, table_log,
                                      chunk_symbols, lanes, layout, stream.ctypes.data, cap.value,

@@ -13,15 +13,18 @@ void set_last_cuda_error(cudaError_t e) { g_last_cuda_error.store(static_cast<in
 int validate_desc(const ans_layer_desc& d, bool need_out) {
   if (d.table_log < 1 || d.table_log > ANS_MAX_TABLE_LOG) return ANS_ERR_UNSUPPORTED;
   if (d.lanes < 32 || d.lanes > ANS_MAX_LANES || d.lanes % 32) return ANS_ERR_UNSUPPORTED;
-  if (d.layout != ANS_LAYOUT_INTERLEAVED && d.layout != ANS_LAYOUT_PRIVATE && d.layout != ANS_LAYOUT_QUADS)
-    return ANS_ERR_UNSUPPORTED;
+  if (!known_layout(d.layout)) return ANS_ERR_UNSUPPORTED;
   if (d.out_dtype != ANS_U8 && d.out_dtype != ANS_F32 && d.out_dtype != ANS_BF16) return ANS_ERR_UNSUPPORTED;
   if (d.chunk_symbols == 0) return ANS_ERR_INVALID_ARG;
+  if (d.layout == ANS_LAYOUT_STRIPS &&
+      (d.chunk_symbols % d.lanes || d.chunk_symbols / d.lanes > ANS_MAX_STRIP_LANE_SYMBOLS))
+    return ANS_ERR_UNSUPPORTED;
   if (d.bitwidth < 1 || d.bitwidth > 8) return ANS_ERR_INVALID_ARG;
   if (d.zero_point < 0 || d.zero_point >= (1 << d.bitwidth)) return ANS_ERR_INVALID_ARG;
   if (!std::isfinite(d.scale)) return ANS_ERR_INVALID_ARG;
   if (d.n_symbols == 0) return ANS_OK;
-  if (!d.d_table || !d.d_stream || !d.d_sub_offsets || !d.d_lane_meta) return ANS_ERR_INVALID_ARG;
+  if (!d.d_table || !d.d_stream || !d.d_sub_offsets) return ANS_ERR_INVALID_ARG;
+  if (!d.d_lane_meta && lane_meta_size(d.layout)) return ANS_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(d.d_table) & 15) return ANS_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(d.d_stream) & 15) return ANS_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(d.d_sub_offsets) & 7) return ANS_ERR_INVALID_ARG;
@@ -46,7 +49,7 @@ ANS_EXPORT const char* ans_strerror(int code) {
     case ANS_OK: return "ok";
     case ANS_ERR_INVALID_ARG: return "invalid argument";
     case ANS_ERR_BAD_FREQS: return "frequencies do not describe a table of 2^table_log states";
-    case ANS_ERR_UNSUPPORTED: return "unsupported table_log, lanes, layout or dtype";
+    case ANS_ERR_UNSUPPORTED: return "unsupported table_log, lanes, chunk size, layout or dtype";
     case ANS_ERR_BUFFER_TOO_SMALL: return "buffer too small";
     case ANS_ERR_CUDA: return "CUDA call failed (see ans_last_cuda_error)";
     case ANS_ERR_CORRUPT: return "a compressed stream did not decode soundly";
@@ -76,7 +79,7 @@ ANS_EXPORT int ans_host_scratch_bytes(const ans_layer_desc* h_desc, uint64_t str
   if (h_desc->n_symbols > kMaxBytes / 4 || stream_bytes > kMaxBytes) return ANS_ERR_INVALID_ARG;
   const uint64_t n_sub = subs_of(*h_desc);
   if (n_sub > kMaxBytes / 128) return ANS_ERR_INVALID_ARG;
-  const size_t meta = n_sub * 32 * (h_desc->layout == ANS_LAYOUT_INTERLEAVED ? 2 : 4);
+  const size_t meta = n_sub * 32 * lane_meta_size(h_desc->layout);
   *h_bytes_out = 256 + up256(stream_bytes) + up256((n_sub + 1) * 8) + up256(meta) +
                  up256(h_desc->n_symbols * elem_size(h_desc->out_dtype));
   return ANS_OK;
@@ -91,13 +94,14 @@ ANS_EXPORT int ans_decode_dequant_host(const ans_layer_desc* h_desc, const uint8
   int rc = ans_host_scratch_bytes(h_desc, stream_bytes, &need);
   if (rc != ANS_OK) return rc;
   if (h_desc->n_symbols == 0) return validate_desc(*h_desc, false);
-  if (!h_stream || !h_sub_offsets || !h_lane_meta || !h_out || !d_scratch) return ANS_ERR_INVALID_ARG;
+  if (!h_stream || !h_sub_offsets || !h_out || !d_scratch) return ANS_ERR_INVALID_ARG;
+  if (!h_lane_meta && lane_meta_size(h_desc->layout)) return ANS_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(d_scratch) & 255) return ANS_ERR_INVALID_ARG;
   if (d_scratch_bytes < need) return ANS_ERR_BUFFER_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
   const uint64_t n_sub = subs_of(*h_desc);
-  const size_t meta_bytes = n_sub * 32 * (h_desc->layout == ANS_LAYOUT_INTERLEAVED ? 2 : 4);
+  const size_t meta_bytes = n_sub * 32 * lane_meta_size(h_desc->layout);
   const size_t out_bytes = h_desc->n_symbols * elem_size(h_desc->out_dtype);
   uint8_t* p = static_cast<uint8_t*>(d_scratch);
   uint32_t* d_status = reinterpret_cast<uint32_t*>(p); p += 256;
@@ -109,7 +113,7 @@ ANS_EXPORT int ans_decode_dequant_host(const ans_layer_desc* h_desc, const uint8
   ANSB_CUDA(cudaMemsetAsync(d_status, 0, 4, st));
   ANSB_CUDA(cudaMemcpyAsync(d_stream, h_stream, stream_bytes, cudaMemcpyHostToDevice, st));
   ANSB_CUDA(cudaMemcpyAsync(d_offs, h_sub_offsets, (n_sub + 1) * 8, cudaMemcpyHostToDevice, st));
-  ANSB_CUDA(cudaMemcpyAsync(d_meta, h_lane_meta, meta_bytes, cudaMemcpyHostToDevice, st));
+  if (meta_bytes) ANSB_CUDA(cudaMemcpyAsync(d_meta, h_lane_meta, meta_bytes, cudaMemcpyHostToDevice, st));
   ans_layer_desc d = *h_desc;
   d.stream_bytes = stream_bytes;
   d.d_stream = d_stream; d.d_sub_offsets = d_offs; d.d_lane_meta = d_meta; d.d_out = d_out;

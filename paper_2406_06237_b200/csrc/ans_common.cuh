@@ -64,5 +64,10 @@ inline uint64_t subs_of(const ans_layer_desc& d) { return chunks_of(d) * groups_
 constexpr uint32_t kGranule = 4;   // sub-streams per work item of the batch plan
 inline uint64_t granules_of(const ans_layer_desc& d) { return (subs_of(d) + kGranule - 1) / kGranule; }
 inline size_t elem_size(int dtype) { return dtype == ANS_U8 ? 1 : dtype == ANS_F32 ? 4 : 2; }
+// bytes of d_lane_meta per lane (the strips layout has no such array)
+inline size_t lane_meta_size(int layout) {
+  return layout == ANS_LAYOUT_INTERLEAVED ? 2 : layout == ANS_LAYOUT_STRIPS ? 0 : 4;
+}
+inline bool known_layout(int layout) { return layout >= ANS_LAYOUT_INTERLEAVED && layout <= ANS_LAYOUT_STRIPS; }
 
 }  // namespace ansb

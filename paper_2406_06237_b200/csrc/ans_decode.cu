@@ -333,6 +333,9 @@ struct LaunchShape { size_t smem = 0; int warps = 0; int per_sm = 0; };
 struct DeviceFacts { int sms = 0; int smem_max = 0; LaunchShape shape[8]; };
 static DeviceFacts g_facts[kMaxDevices];    // remembered per device; racing writers store equal values
 
+int launch_strips(const ans_layer_desc* h_descs, int n_layers, uint8_t* d_symbols_override, uint32_t* d_status,
+                  cudaStream_t st);                       // ans_decode_strips.cu
+
 static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, int n_layers,
                   uint8_t* d_symbols_override, uint32_t* d_status, cudaStream_t st) {
   int max_log = 1, busy_layers = 0;
@@ -357,6 +360,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   }
   if (total == 0) return ANS_OK;
   if (total > 0xFFFFFFFFull) return ANS_ERR_UNSUPPORTED;
+  if (layout == ANS_LAYOUT_STRIPS) return launch_strips(h_descs, n_layers, d_symbols_override, d_status, st);
 
   LaunchArgs a{};
   a.d_descs = d_descs;
@@ -540,6 +544,6 @@ ANS_EXPORT int ans_decode_dequant_batch(const ans_layer_desc* d_descs, const ans
                                         int n_layers, uint32_t* d_status, void* stream) {
   if (n_layers < 0 || !d_status) return ANS_ERR_INVALID_ARG;
   if (n_layers == 0) return ANS_OK;
-  if (!d_descs || !h_descs) return ANS_ERR_INVALID_ARG;
+  if (!h_descs || (!d_descs && h_descs[0].layout != ANS_LAYOUT_STRIPS)) return ANS_ERR_INVALID_ARG;
   return launch(d_descs, h_descs, n_layers, nullptr, d_status, static_cast<cudaStream_t>(stream));
 }

@@ -1,0 +1,616 @@
+// Decode (+ dequantise) kernel of the strips container, for sm_100a.
+//
+// Paper Section II-A: some transitions of the automaton take no bits; they belong to the one
+// symbol that owns more than half of the states and are what carries the rate under one bit per
+// weight.  The pre-walked table folds such chains into the entry that starts them: one look-up
+// stands for `run` copies of the dominant symbol followed by one more symbol (state -> symbol,
+// nb_bits, newX as in Fig. 2, after `run` unlabeled transitions).  Section III-B: one table per
+// layer, a vector of states; here a warp holds the 32 states of a sub-stream.
+//
+// The container keeps a sub-stream's symbols in one contiguous strip of the layer, dealt to the
+// 32 lanes round-robin, so a look-up that emits several symbols only moves a lane's own
+// position: nothing has to be kept in step.  A warp collects a window of its strip in shared
+// memory, pre-filled with the dominant symbol's value; a lane only writes the symbol that ends a
+// run; a full window is contiguous in the output and leaves in 16-byte stores.
+//
+// One CTA = one work item of the batch plan (up to four consecutive sub-streams of ONE layer,
+// a warp each).  Up to kStripParamLayers layer records travel in the kernel parameters, so a
+// CTA reaches its layer without a trip to memory; the trips that remain are the sub-stream's
+// offsets (then its bytes, one bulk copy) and, beside them, the layer's table.
+#include "ans_decode_common.cuh"
+
+namespace ansb {
+
+constexpr int kStripWarps = static_cast<int>(kGranule);   // sub-streams (warps) per CTA
+constexpr int kStripParamLayers = 64;                     // layers of one launch
+constexpr uint32_t kStripHeader = 64;                     // bytes: 32 lanes x 16-bit length
+constexpr uint32_t kStripWindow = 4096;                   // bytes of output a warp collects before writing them out
+constexpr uint32_t kStripBatch = 8;                       // table entries a thread requests at a time
+constexpr uint32_t kStripCtaTable = 2048;                 // launches of up to this many CTAs carry a CTA -> layer table
+constexpr uint32_t kStripPad = 256;                       // readable bytes after a staged sub-stream: more than a lane
+                                                          // can advance while it walks one window (128 symbols of 14 bits)
+static_assert(kStripWindow / 32 * 14 / 8 + 32 <= kStripPad, "a window's walk must stay inside the padding");
+
+struct StripLayer {                // what the kernel needs of one layer, 64 bytes
+  const uint8_t* blob;             // table blob
+  const uint8_t* stream;
+  const uint64_t* sub_offsets;
+  uint8_t* out;
+  uint64_t stream_bytes;
+  uint64_t n_symbols;
+  uint32_t chunk_symbols;
+  uint32_t n_sub;
+  float scale;
+  uint32_t packed;                 // zero_point [7:0] | table_log [11:8] | bitwidth [15:12] | dtype [17:16] | lanes / 32 [24:18]
+};
+
+struct StripArgs {
+  StripLayer layer[kStripParamLayers];
+  uint32_t cta_begin[kStripParamLayers + 1];   // first CTA of each layer
+  int n_layers;
+  uint32_t* d_status;
+  uint32_t table_bytes;            // shared-memory bytes reserved for the table copies
+  uint32_t max_log;
+  uint32_t succ_bytes;             // shared-memory bytes of the successor table (2 << max_log, at least 16)
+  uint32_t stage_bytes;            // per-warp staging buffer for the sub-stream's bytes
+  uint32_t unit;                   // the value 1 (keeps a multiply-add a multiply-add)
+  uint32_t ctas;                   // CTAs of the launch
+  uint8_t cta_layer[kStripCtaTable];   // layer of every CTA when ctas <= kStripCtaTable: one look-up instead of a search
+};
+
+// shared-memory form of a pre-walked entry.  Two words:
+//   1- and 2-byte outputs:  a = nb [4:0] | run [11:8] | value [31:16]    b = q
+//   4-byte outputs:         a = nb [4:0] | run [11:8] | q [31:16]        b = value
+// q = newX >> nb, so that the next state is (q << nb) | bits: one funnel shift on a bit window
+// that is kept top-aligned.  Bits 5-7 of a stay zero: the walk adds all of a to its bit count.
+// Or ONE word, for tables of up to 256 states (the paper's sizes) and 1- or 2-byte outputs:
+//   value [15:0] | nb [19:16] | run [23:20] | q [31:24]
+// Half the bytes, so twice the copies fit and a look-up takes fewer shared-memory wavefronts,
+// for one more instruction (the fields have to be cut out; the value is stored as it lies).
+__device__ __forceinline__ uint2 to_strip_entry(uint32_t g, uint32_t val, bool narrow) {
+  const uint32_t nb = entry_nb(g), q = entry_newx(g) >> nb, run = entry_run(g);
+  return narrow ? make_uint2(nb | (run << 8) | (val << 16), q) : make_uint2(nb | (run << 8) | (q << 16), val);
+}
+__device__ __forceinline__ uint32_t to_strip_entry_short(uint32_t g, uint32_t val) {
+  const uint32_t nb = entry_nb(g);
+  return (val & 0xFFFFu) | (nb << 16) | (entry_run(g) << 20) | ((entry_newx(g) >> nb) << 24);
+}
+
+#define ANSB_SP_BEGIN "shf.l.wrap.b32 x, %3, %2, %1;\n\t"
+#define ANSB_SP_END                                               \
+  "and.b32 tt, %1, 32;\n\t"                                       \
+  "setp.ne.u32 pq, tt, 0;\n\t"                                    \
+  "@pq mov.u32 %2, %3;\n\t"                                       \
+  "@pq mov.u32 %3, %4;\n\t"                                       \
+  "@pq ld.shared.u32 nw, [%5];\n\t"                               \
+  "@pq mov.u32 %4, nw;\n\t"                                       \
+  "@pq add.u32 %5, %5, 4;\n\t"                                    \
+  "and.b32 %1, %1, 31;\n\t"
+// One look-up.  %6: the lane's next position; zn: the position of the symbol that ends the run;
+// the lane takes the step only if that position is inside the window (and the lane), else it
+// keeps its state and waits.
+#define ANSB_SP_STEP_N(STS_)                                      \
+  "ld.shared.v2.u32 {ea, eb}, [%0];\n\t"                          \
+  "bfe.u32 av, ea, 8, 4;\n\t"                                     \
+  "add.u32 zn, %6, av;\n\t"                                       \
+  "setp.lt.u32 act, zn, %10;\n\t"                                 \
+  "mad.lo.u32 ad, zn, %13, %9;\n\t"                               \
+  "shr.u32 vv, ea, 16;\n\t"                                       \
+  "@act " STS_ " [ad], vv;\n\t"                                   \
+  "@act shf.l.wrap.b32 tt, x, eb, ea;\n\t"                        \
+  "@act shf.l.wrap.b32 x, 0, x, ea;\n\t"                          \
+  "@act mad.lo.u32 %0, tt, %8, %7;\n\t"                           \
+  "@act mad.lo.u32 %1, ea, %11, %1;\n\t"                          \
+  "@act add.u32 %6, zn, 1;\n\t"
+#define ANSB_SP_STEP_S(STS_)                                      \
+  "ld.shared.u32 ea, [%0];\n\t"                                   \
+  "bfe.u32 av, ea, 20, 4;\n\t"                                    \
+  "add.u32 zn, %6, av;\n\t"                                       \
+  "setp.lt.u32 act, zn, %10;\n\t"                                 \
+  "mad.lo.u32 ad, zn, %13, %9;\n\t"                               \
+  "@act " STS_ " [ad], ea;\n\t"                                   \
+  "bfe.u32 eb, ea, 16, 4;\n\t"                                    \
+  "shr.u32 av, ea, 24;\n\t"                                       \
+  "@act shf.l.wrap.b32 tt, x, av, eb;\n\t"                        \
+  "@act shf.l.wrap.b32 x, 0, x, eb;\n\t"                          \
+  "@act mad.lo.u32 %0, tt, %8, %7;\n\t"                           \
+  "@act add.u32 %1, %1, eb;\n\t"                                  \
+  "@act add.u32 %6, zn, 1;\n\t"
+#define ANSB_SP_STEP_W(STS_)                                      \
+  "ld.shared.v2.u32 {ea, eb}, [%0];\n\t"                          \
+  "bfe.u32 av, ea, 8, 4;\n\t"                                     \
+  "add.u32 zn, %6, av;\n\t"                                       \
+  "setp.lt.u32 act, zn, %10;\n\t"                                 \
+  "mad.lo.u32 ad, zn, %13, %9;\n\t"                               \
+  "shr.u32 vv, ea, 16;\n\t"                                       \
+  "@act " STS_ " [ad], eb;\n\t"                                   \
+  "@act shf.l.wrap.b32 tt, x, vv, ea;\n\t"                        \
+  "@act shf.l.wrap.b32 x, 0, x, ea;\n\t"                          \
+  "@act mad.lo.u32 %0, tt, %8, %7;\n\t"                           \
+  "@act mad.lo.u32 %1, ea, %11, %1;\n\t"                          \
+  "@act add.u32 %6, zn, 1;\n\t"
+
+// The walk of one window, entirely in PTX (loop included).  Groups of K look-ups share one
+// 32-bit extract of the bit window and one refill check: K = 4 when no state of the table takes
+// more than 8 bits, else 2.  The loop ends when no lane took the last look-up of a group; every
+// look-up a lane takes moves its position on, so a window costs at most its symbols in trips.
+//   st: shared address of the state's entry      z: the lane's next position (symbols it has decoded)
+//   abase: window address of the lane's first symbol, minus the window's first row (a row holds one
+//          symbol of every lane)
+//   lim: first position the lane may not write (end of the window, or of the lane)
+template <int ES, int K, bool SHORT>
+__device__ __forceinline__ void strip_window_walk(uint32_t& st, uint32_t& bitpos, uint32_t& w0, uint32_t& w1,
+                                                  uint32_t& w2, uint32_t& sp, uint32_t& z, uint32_t tab_lane,
+                                                  uint32_t stride, uint32_t abase, uint32_t lim, uint32_t unit,
+                                                  uint32_t sp_limit) {
+#define ANSB_SP_ASM(LBL_, BODY_)                                                            \
+  asm volatile(                                                                             \
+      "{\n\t"                                                                               \
+      ".reg .pred act, pq, pany;\n\t"                                                       \
+      ".reg .u32 x, ea, eb, av, zn, tt, ad, vv, nw;\n"                                      \
+      LBL_ ":\n\t"                                                                          \
+      BODY_                                                                                 \
+      "vote.sync.any.pred pany, act, 0xffffffff;\n\t"                                       \
+      "@pany bra " LBL_ ";\n\t"                                                             \
+      "min.u32 %5, %5, %12;\n\t"                                                            \
+      "}"                                                                                   \
+      : "+r"(st), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp), "+r"(z)             \
+      : "r"(tab_lane), "r"(stride), "r"(abase), "r"(lim), "r"(unit), "r"(sp_limit),         \
+        "n"(32 * ES)                                                                        \
+      : "memory")
+#define ANSB_SP_G4(ST_, STS_) ANSB_SP_BEGIN ST_(STS_) ST_(STS_) ST_(STS_) ST_(STS_) ANSB_SP_END
+#define ANSB_SP_G2(ST_, STS_) ANSB_SP_BEGIN ST_(STS_) ST_(STS_) ANSB_SP_END
+  if (SHORT) {                                             // (tables of up to 256 states: no state takes more than 8 bits)
+    if (ES == 1) ANSB_SP_ASM("ANSB_SPS1", ANSB_SP_G4(ANSB_SP_STEP_S, "st.shared.u8"));
+    if (ES == 2) ANSB_SP_ASM("ANSB_SPS2", ANSB_SP_G4(ANSB_SP_STEP_S, "st.shared.u16"));
+  } else if (K == 4) {
+    if (ES == 1) ANSB_SP_ASM("ANSB_SP41", ANSB_SP_G4(ANSB_SP_STEP_N, "st.shared.u8"));
+    if (ES == 2) ANSB_SP_ASM("ANSB_SP42", ANSB_SP_G4(ANSB_SP_STEP_N, "st.shared.u16"));
+    if (ES == 4) ANSB_SP_ASM("ANSB_SP44", ANSB_SP_G4(ANSB_SP_STEP_W, "st.shared.u32"));
+  } else {
+    if (ES == 1) ANSB_SP_ASM("ANSB_SP21", ANSB_SP_G2(ANSB_SP_STEP_N, "st.shared.u8"));
+    if (ES == 2) ANSB_SP_ASM("ANSB_SP22", ANSB_SP_G2(ANSB_SP_STEP_N, "st.shared.u16"));
+    if (ES == 4) ANSB_SP_ASM("ANSB_SP24", ANSB_SP_G2(ANSB_SP_STEP_W, "st.shared.u32"));
+  }
+#undef ANSB_SP_G2
+#undef ANSB_SP_G4
+#undef ANSB_SP_ASM
+}
+
+__device__ __forceinline__ uint4 lds_v4(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_v4(uint32_t a, uint4 v) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" :: "r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+struct StripGeom {                 // one sub-stream's place in its layer
+  uint64_t first;                  // first symbol of the strip in the layer
+  uint32_t ns;                     // symbols in the strip
+};
+
+// Decode one sub-stream.  win_abs: the warp's window (kStripWindow bytes, holding `fill`);
+// words: the sub-stream in shared memory (STAGED, at stage_abs) or in global memory.
+template <int ES, bool STAGED, bool SHORT>
+__device__ __noinline__ uint32_t decode_strip(
+    uint32_t tab_lane, uint32_t stride_log, uint32_t succ_abs, uint32_t win_abs, uint32_t stage_abs,
+    const uint32_t* __restrict__ words, uint32_t ext_words, uint32_t R, uint32_t ns, uint8_t* __restrict__ out_strip,
+    uint32_t fill, bool wide_steps, uint32_t unit, uint32_t lane) {
+  constexpr uint32_t RB = 32u * ES;                        // bytes of a row (one symbol of every lane)
+  constexpr uint32_t P = kStripWindow / RB;                // rows of a window
+  const uint32_t word_limit = STAGED ? ext_words + 4u : ext_words;
+  auto load_word = [&](uint32_t i) -> uint32_t {     // (staged: the words after the sub-stream are zero, up to kStripPad)
+    if (STAGED) return lds_u32(stage_abs + min(i, word_limit + 8u) * 4u);
+    return i < word_limit ? __ldg(words + i) : 0u;
+  };
+  uint32_t bad = 0;
+
+  const uint32_t count = lane_symbols(ns, 32u, lane);     // symbols of this lane
+  const uint32_t rows = (ns + 31u) >> 5;
+
+  // the lanes' bit lengths head the sub-stream; their running sum places every lane's string
+  const uint32_t hw = load_word(lane >> 1);
+  const uint32_t len = (lane & 1u) ? hw >> 16 : hw & 0xFFFFu;
+  uint32_t incl = len;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t up = __shfl_up_sync(kFull, incl, d);
+    if (lane >= static_cast<uint32_t>(d)) incl += up;
+  }
+  const uint32_t total_bits = __shfl_sync(kFull, incl, 31);
+  // the sub-stream must be exactly its header, the words its bits need, and the padding
+  if (ext_words < kStripHeader / 4u || (((kStripHeader / 4u + ((total_bits + 31u) >> 5)) + 3u) & ~3u) != ext_words)
+    bad |= ANS_STATUS_BAD_LENGTH;
+  const uint32_t bit0 = kStripHeader * 8u + (incl - len);
+  uint32_t idx = bit0 >> 5, bitpos = bit0 & 31u;
+  uint32_t w0 = load_word(idx), w1 = load_word(idx + 1), w2 = load_word(idx + 2);
+  idx += 3;
+  uint32_t state = 0;
+  if (count) {                                             // the string begins with the state, R bits
+    state = __funnelshift_l(w1, w0, bitpos) >> (32u - R);
+    bitpos += R;
+    if (bitpos >= 32u) { w0 = w1; w1 = w2; w2 = load_word(idx); ++idx; bitpos -= 32u; }
+  }
+  const uint32_t stride = 1u << stride_log;
+  uint32_t st = tab_lane + (state << stride_log);
+  uint32_t z = 0;                                          // the lane's next position
+  const uint32_t sp_limit = stage_abs + word_limit * 4u;
+  uint32_t sp = min(stage_abs + min(idx, word_limit) * 4u, sp_limit);   // (lengths that lead outside are flagged below)
+  const bool vec_ok = (reinterpret_cast<uintptr_t>(out_strip) & 15u) == 0;
+  const uint4 fill4 = make_uint4(fill, fill, fill, fill);
+
+  for (uint32_t t0 = 0; t0 < rows; t0 += P) {
+    const uint32_t lim = min(t0 + P, count);
+    const uint32_t abase = win_abs + lane * ES - t0 * RB;
+    __syncwarp();
+    if (STAGED) {
+      if (SHORT || wide_steps)
+        strip_window_walk<ES, 4, SHORT>(st, bitpos, w0, w1, w2, sp, z, tab_lane, stride, abase, lim, unit, sp_limit);
+      else
+        strip_window_walk<ES, 2, false>(st, bitpos, w0, w1, w2, sp, z, tab_lane, stride, abase, lim, unit, sp_limit);
+    } else {                                               // the same walk in plain code, words from global memory
+      bool any = true;
+      while (any) {
+        const uint32_t ea = lds_u32(st), eb = SHORT ? 0u : lds_u32(st + 4u);
+        const uint32_t nb = SHORT ? (ea >> 16) & 15u : ea & 31u, zn = z + (SHORT ? (ea >> 20) & 15u : (ea >> 8) & 15u);
+        const bool act = zn < lim;
+        if (act) {
+          const uint32_t q = SHORT ? ea >> 24 : ES == 4 ? ea >> 16 : eb, val = SHORT ? ea : ES == 4 ? eb : ea >> 16;
+          sts_elem<ES>(abase + zn * RB, val);
+          const uint32_t x = __funnelshift_l(w1, w0, bitpos);
+          st = tab_lane + (__funnelshift_l(x, q, nb) << stride_log);
+          z = zn + 1u;
+          bitpos += nb;
+          if (bitpos >= 32u) { w0 = w1; w1 = w2; w2 = load_word(idx); ++idx; bitpos -= 32u; }
+        }
+        any = __any_sync(kFull, act);
+      }
+    }
+    __syncwarp();
+    // the window is complete: write it out (it is contiguous in the output) and fill it again
+    const uint32_t wbytes = min(kStripWindow, ns * ES - t0 * RB);
+    uint8_t* gdst = out_strip + size_t(t0) * RB;
+    const bool more = t0 + P < rows;
+    if (vec_ok && (wbytes & 15u) == 0) {
+      // one bulk copy from shared memory to the output; the window may be filled again once the
+      // copy has read it
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) {
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" :: "l"(gdst), "r"(win_abs), "r"(wbytes) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      }
+      __syncwarp();
+      if (more)
+        for (uint32_t i = lane * 16u; i < kStripWindow; i += 512u) sts_v4(win_abs + i, fill4);
+    } else if (vec_ok) {
+      for (uint32_t i = lane * 16u; i + 16u <= wbytes; i += 512u) {
+        const uint4 v = lds_v4(win_abs + i);
+        *reinterpret_cast<uint4*>(gdst + i) = v;
+        if (more) sts_v4(win_abs + i, fill4);
+      }
+      const uint32_t tail0 = wbytes & ~15u;                // a ragged end: only in a layer's last strip
+      if (tail0 + lane * ES < wbytes) {
+        const uint32_t a = win_abs + tail0 + lane * ES;
+        const uint32_t v = ES == 1 ? lds_u32(a & ~3u) >> (8u * (a & 3u)) : ES == 2 ? lds_u16(a) : lds_u32(a);
+        stg_elem<ES>(gdst + tail0 + lane * ES, v);
+      }
+    } else {
+      for (uint32_t i = lane * ES; i < wbytes; i += 32u * ES) {
+        const uint32_t a = win_abs + i;
+        const uint32_t v = ES == 1 ? lds_u32(a & ~3u) >> (8u * (a & 3u)) : ES == 2 ? lds_u16(a) : lds_u32(a);
+        stg_elem<ES>(gdst + i, v);
+      }
+      __syncwarp();
+      if (more)
+        for (uint32_t i = lane * 16u; i < kStripWindow; i += 512u) sts_v4(win_abs + i, fill4);
+    }
+  }
+  if (STAGED) {
+    if (sp >= sp_limit) bad |= ANS_STATUS_BAD_LENGTH;
+    idx = (sp - stage_abs) >> 2;
+  }
+  // What is left of the lane lies inside the run of the entry it stopped at: zero-bit states,
+  // the dominant symbol already in place.  Walk them one by one to reach the final state.
+  uint32_t s = (st - tab_lane) >> stride_log;
+  for (uint32_t left = count - z; left != 0 && left <= uint32_t(kMaxRun); --left) s = lds_u16(succ_abs + s * 2u);
+  if (count - z > uint32_t(kMaxRun)) bad |= ANS_STATUS_BAD_FINAL_STATE;
+  if (s != 0) bad |= ANS_STATUS_BAD_FINAL_STATE;
+  // the lane must have used exactly its bits
+  const uint32_t used = (idx - 3u) * 32u + bitpos - bit0;
+  if (used != len) bad |= ANS_STATUS_BAD_LENGTH;
+  return bad;
+}
+
+__global__ void __launch_bounds__(kStripWarps * 32) ans_decode_strips_kernel(const __grid_constant__ StripArgs args) {
+  extern __shared__ __align__(16) uint8_t sm[];
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  // dynamic shared memory: [table, in copies][successors][windows][stages], each 16-byte aligned
+  const uint32_t sm_abs = smem_u32(sm);
+  const uint32_t tab_abs = sm_abs;
+  const uint32_t succ_abs = tab_abs + args.table_bytes;
+  const uint32_t win_abs = succ_abs + args.succ_bytes + warp * kStripWindow;
+  const uint32_t stage_abs = succ_abs + args.succ_bytes + kStripWarps * kStripWindow + warp * args.stage_bytes;
+
+  // let the next launch of the stream get its CTAs in place while this one runs (it waits, as this
+  // one does below, before it touches memory)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // the layer of this CTA: its first CTA is the last one at or before blockIdx.x
+  int lo = 0;
+  if (args.ctas <= kStripCtaTable) {
+    lo = args.cta_layer[blockIdx.x];
+  } else {
+    int hi = args.n_layers;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (args.cta_begin[mid] <= blockIdx.x) lo = mid; else hi = mid;
+    }
+  }
+  const StripLayer& L = args.layer[lo];
+  const uint32_t zero_point = L.packed & 0xFFu, R = (L.packed >> 8) & 15u, bitwidth = (L.packed >> 12) & 15u;
+  const int dtype = static_cast<int>((L.packed >> 16) & 3u);
+  const uint32_t G = (L.packed >> 18) & 127u;
+  const uint32_t es = dtype == ANS_U8 ? 1u : dtype == ANS_F32 ? 4u : 2u;
+  const uint32_t sub = (blockIdx.x - args.cta_begin[lo]) * kStripWarps + warp;
+  const bool have = sub < L.n_sub;
+
+  // whatever an earlier launch of the stream wrote is visible from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // everything the CTA needs from memory is requested before any of it is used: the
+  // sub-stream's offsets, the table's header and its entries (the first batch)
+  uint64_t off0 = 0, off1 = 0;
+  if (have) {
+    off0 = __ldg(L.sub_offsets + sub);
+    off1 = __ldg(L.sub_offsets + sub + 1);
+  }
+  const TableHeader* hdr = reinterpret_cast<const TableHeader*>(L.blob);
+  const uint32_t* g_single = reinterpret_cast<const uint32_t*>(L.blob + single_offset());
+  const uint32_t* g_multi = reinterpret_cast<const uint32_t*>(L.blob + multi_offset(static_cast<int>(R)));
+  const uint32_t h_magic = __ldg(&hdr->magic), h_log = __ldg(&hdr->table_log), h_alphabet = __ldg(&hdr->alphabet),
+                 h_dominant = __ldg(&hdr->dominant);
+  const uint32_t n_states = 1u << R;
+  uint32_t gm[kStripBatch], gs[kStripBatch];
+  auto request_entries = [&](uint32_t b0) {
+#pragma unroll
+    for (uint32_t k = 0; k < kStripBatch; ++k) {
+      const uint32_t i = b0 + k * blockDim.x + threadIdx.x;
+      gm[k] = i < n_states ? __ldg(g_multi + i) : 0u;
+      gs[k] = i < n_states ? __ldg(g_single + i) : 0u;
+    }
+  };
+  request_entries(0);
+
+  // the sub-stream's bytes: asynchronous 16-byte copies into shared memory, started as soon as its
+  // offsets are here, so that they travel while the table is being staged.  Both ends on 16-byte
+  // boundaries, inside the stream.
+  uint32_t bad = 0;
+  uint64_t extent = 0;
+  if (have) {
+    extent = off1 - off0;
+    if (off1 < off0 || off1 > L.stream_bytes || ((off0 | off1) & 15u) || extent > 0xFFFFFFF0ull) {
+      extent = 0;
+      off0 = 0;
+      bad |= ANS_STATUS_BAD_LENGTH;
+    }
+  }
+  const bool staged = extent > 0 && extent + kStripPad <= args.stage_bytes;
+  if (staged) {
+    const uint8_t* src = L.stream + off0;
+    for (uint32_t o = lane * 16u; o < static_cast<uint32_t>(extent); o += 512u)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(stage_abs + o), "l"(src + o) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    for (uint32_t i = lane; i < kStripPad / 4u; i += 32u)
+      asm volatile("st.shared.u32 [%0], %1;" :: "r"(stage_abs + static_cast<uint32_t>(extent) + i * 4u), "r"(0u) : "memory");
+  }
+
+  // stage the table: copies interleaved entry by entry (entry i of copy c at slot i * copies + c;
+  // lane l reads copy l mod copies), the dequantised value folded into every entry
+  // (a table smaller than the launch's largest uses the room for more copies, up to one per lane)
+  const bool short_entries = R <= 8u && es != 4u;
+  const uint32_t entry_log = short_entries ? 2u : 3u;
+  const uint32_t rep_log = min(short_entries ? 5u : 4u, 31u - static_cast<uint32_t>(__clz(args.table_bytes >> (R + entry_log))));
+  const uint32_t reps = 1u << rep_log;
+  const uint32_t stride_log = entry_log + rep_log;
+  const uint32_t tab_lane = tab_abs + ((lane & (reps - 1u)) << entry_log);
+  uint32_t most_bits = 0;
+  for (uint32_t b0 = 0; b0 < n_states; b0 += blockDim.x * kStripBatch) {
+    if (b0 != 0) request_entries(b0);
+#pragma unroll
+    for (uint32_t k = 0; k < kStripBatch; ++k) {
+      const uint32_t i = b0 + k * blockDim.x + threadIdx.x;
+      if (i < n_states) {
+        const uint32_t val = dequant_bits(static_cast<int>(entry_sym(gm[k])), static_cast<int>(zero_point), L.scale, dtype);
+        const uint2 e = to_strip_entry(gm[k], val, es != 4u);
+        const uint32_t e1 = to_strip_entry_short(gm[k], val);
+        const uint32_t slot = tab_abs + (i << stride_log);
+        if (stride_log >= 4u) {
+          // the entry's copies lie side by side: written 16 bytes at a time, every lane starting
+          // at another 16 bytes so that the stores of a warp spread over the banks
+          const uint4 v = short_entries ? make_uint4(e1, e1, e1, e1) : make_uint4(e.x, e.y, e.x, e.y);
+          const uint32_t pieces = 1u << (stride_log - 4u), turn = lane & (pieces - 1u);
+#pragma unroll
+          for (uint32_t p = 0; p < 8u; ++p)
+            if (p < pieces) sts_v4(slot + ((p ^ turn) << 4), v);
+        } else {
+          for (uint32_t c = 0; c < reps; ++c) {
+            const uint32_t a = slot + (c << entry_log);
+            if (short_entries) asm volatile("st.shared.u32 [%0], %1;" :: "r"(a), "r"(e1) : "memory");
+            else asm volatile("st.shared.v2.u32 [%0], {%1, %2};" :: "r"(a), "r"(e.x), "r"(e.y) : "memory");
+          }
+        }
+        asm volatile("st.shared.u16 [%0], %1;" :: "r"(succ_abs + i * 2u), "r"(entry_newx(gs[k])) : "memory");
+        most_bits = max(most_bits, entry_nb(gm[k]));
+      }
+    }
+  }
+  if (threadIdx.x == 0 && (h_magic != kTableMagic || h_log != R || h_alphabet > (1u << bitwidth))) bad |= ANS_STATUS_BAD_SYMBOL;
+  // four look-ups share one 32-bit extract only if no state takes more than 8 bits
+  const bool wide_steps = __syncthreads_or(most_bits > 8u) == 0;
+
+  if (have) {
+    // the warp's window starts out holding the dominant symbol's value (the symbol of every
+    // zero-bit state; without one no look-up skips a position and the fill is never seen)
+    const uint32_t dom = dequant_bits(static_cast<int>(h_dominant < 256u ? h_dominant : 0u), static_cast<int>(zero_point), L.scale, dtype);
+    const uint32_t fill = es == 4u ? dom : es == 2u ? (dom & 0xFFFFu) * 0x10001u : (dom & 0xFFu) * 0x01010101u;
+    const uint4 fill4 = make_uint4(fill, fill, fill, fill);
+    for (uint32_t i = lane * 16u; i < kStripWindow; i += 512u) sts_v4(win_abs + i, fill4);
+
+    // the strip of this sub-stream
+    const uint64_t chunk = sub / G;
+    const uint32_t g = sub - static_cast<uint32_t>(chunk) * G;
+    const uint32_t S = L.chunk_symbols / (32u * G);
+    const uint64_t c0 = chunk * L.chunk_symbols;
+    const uint64_t nc = min(uint64_t(L.chunk_symbols), L.n_symbols - c0);
+    const uint64_t sfirst = uint64_t(g) * 32u * S;
+    const uint32_t ns = nc > sfirst ? static_cast<uint32_t>(min(nc - sfirst, uint64_t(32u) * S)) : 0u;
+    uint8_t* out_strip = L.out + (c0 + sfirst) * es;
+    const uint32_t ext_words = static_cast<uint32_t>(extent >> 2);
+    const uint32_t* words = reinterpret_cast<const uint32_t*>(L.stream + off0);
+
+    if (staged) {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      __syncwarp();
+    }
+    if (extent == 0) {
+      // unusable offsets (flagged above): nothing is read; an empty strip needs nothing either
+      if (ns != 0) bad |= ANS_STATUS_BAD_LENGTH;
+    } else {
+#define ANSB_SCALL(ES_, ST_, SH_)                                                                     \
+  bad |= decode_strip<ES_, ST_, SH_>(tab_lane, stride_log, succ_abs, win_abs, stage_abs, words, ext_words, R, ns, \
+                                     out_strip, fill, wide_steps, args.unit, lane)
+      if (short_entries) {
+        if (staged) { if (es == 1u) ANSB_SCALL(1, true, true); else ANSB_SCALL(2, true, true); }
+        else { if (es == 1u) ANSB_SCALL(1, false, true); else ANSB_SCALL(2, false, true); }
+      } else if (staged) {
+        if (es == 1u) ANSB_SCALL(1, true, false); else if (es == 2u) ANSB_SCALL(2, true, false); else ANSB_SCALL(4, true, false);
+      } else {
+        if (es == 1u) ANSB_SCALL(1, false, false); else if (es == 2u) ANSB_SCALL(2, false, false); else ANSB_SCALL(4, false, false);
+      }
+#undef ANSB_SCALL
+    }
+  }
+  bad = __reduce_or_sync(kFull, bad);
+  if (lane == 0 && bad && args.d_status) atomicOr(args.d_status, bad);
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+struct StripFacts { int sms = 0; int smem_sm = 0; int smem_block = 0; size_t smem_set = 0; };
+static StripFacts g_strip_facts[64];     // per device; racing writers store equal values
+
+int launch_strips(const ans_layer_desc* h_descs, int n_layers, uint8_t* d_symbols_override, uint32_t* d_status,
+                  cudaStream_t st) {
+  int dev = 0;
+  ANSB_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return ANS_ERR_UNSUPPORTED;
+  StripFacts& facts = g_strip_facts[dev];
+  if (!facts.sms) {
+    int sms = 0, per_sm = 0, per_block = 0;
+    ANSB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    ANSB_CUDA(cudaDeviceGetAttribute(&per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev));
+    ANSB_CUDA(cudaDeviceGetAttribute(&per_block, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    ANSB_CUDA(cudaFuncSetAttribute(ans_decode_strips_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                   cudaSharedmemCarveoutMaxShared));
+    facts.smem_sm = per_sm;
+    facts.smem_block = per_block;
+    facts.sms = sms;
+  }
+  for (int l0 = 0; l0 < n_layers; l0 += kStripParamLayers) {
+    const int cnt = (n_layers - l0) < kStripParamLayers ? (n_layers - l0) : kStripParamLayers;
+    StripArgs a{};
+    a.n_layers = 0;
+    a.d_status = d_status;
+    a.unit = 1u;
+    int max_log = 1;
+    uint64_t ctas = 0;
+    size_t max_avg_sub = 0, one_table = 0;
+    for (int i = 0; i < cnt; ++i) {
+      const ans_layer_desc& d = h_descs[l0 + i];
+      if (d.work_count == 0) continue;
+      const uint64_t n_sub = subs_of(d);
+      if (n_sub > 0xFFFFFFFFull) return ANS_ERR_UNSUPPORTED;
+      StripLayer& L = a.layer[a.n_layers];
+      L.blob = static_cast<const uint8_t*>(d.d_table);
+      L.stream = d.d_stream;
+      L.sub_offsets = d.d_sub_offsets;
+      L.out = d_symbols_override ? d_symbols_override : static_cast<uint8_t*>(d.d_out);
+      L.stream_bytes = d.stream_bytes;
+      L.n_symbols = d.n_symbols;
+      L.chunk_symbols = d.chunk_symbols;
+      L.n_sub = static_cast<uint32_t>(n_sub);
+      L.scale = d.scale;
+      const uint32_t dtype = d_symbols_override ? ANS_U8 : static_cast<uint32_t>(d.out_dtype);
+      L.packed = static_cast<uint32_t>(d.zero_point) | (static_cast<uint32_t>(d.table_log) << 8) |
+                 (static_cast<uint32_t>(d.bitwidth) << 12) | (dtype << 16) | ((d.lanes / 32u) << 18);
+      a.cta_begin[a.n_layers] = static_cast<uint32_t>(ctas);
+      ctas += d.work_count;
+      ++a.n_layers;
+      if (d.table_log > max_log) max_log = d.table_log;
+      const size_t tb = size_t((d.table_log <= 8 && dtype != ANS_F32) ? 4 : 8) << d.table_log;   // one copy, in its entry form
+      if (tb > one_table) one_table = tb;
+      const size_t avg = d.stream_bytes / n_sub;
+      if (avg > max_avg_sub) max_avg_sub = avg;
+    }
+    if (a.n_layers == 0) continue;
+    if (ctas > 0x7FFFFFFFull) return ANS_ERR_UNSUPPORTED;
+    a.cta_begin[a.n_layers] = static_cast<uint32_t>(ctas);
+    a.max_log = static_cast<uint32_t>(max_log);
+    a.ctas = static_cast<uint32_t>(ctas);
+    if (ctas <= kStripCtaTable)
+      for (int l = 0; l < a.n_layers; ++l)
+        for (uint32_t c = a.cta_begin[l]; c < a.cta_begin[l + 1]; ++c) a.cta_layer[c] = static_cast<uint8_t>(l);
+
+    // shared memory of a CTA: table copies, successors, barriers, four windows, four staging buffers.
+    // A staging buffer holds the largest layer-average sub-stream plus a margin (a longer one is read
+    // from global memory).  What room is left under the share of an SM that one wave of CTAs
+    // leaves to each goes to more copies of the table (fewer bank conflicts on the look-ups).
+    size_t want = max_avg_sub + max_avg_sub / 8 + 256 + kStripPad;
+    want = (want + 127) & ~size_t(127);
+    const size_t succ = ((size_t(2) << max_log) + 15) & ~size_t(15);
+    const size_t fixed = succ + size_t(kStripWarps) * kStripWindow;
+    const size_t block_max = static_cast<size_t>(facts.smem_block);
+    if (fixed + one_table + kStripWarps * 1024 > block_max) return ANS_ERR_UNSUPPORTED;
+    size_t stage = want;
+    if (fixed + one_table + kStripWarps * stage > block_max) stage = ((block_max - fixed - one_table) / kStripWarps) & ~size_t(127);
+    uint64_t per_sm = (ctas + facts.sms - 1) / facts.sms;
+    if (per_sm > 8) per_sm = 8;
+    if (per_sm < 1) per_sm = 1;
+    size_t cap = static_cast<size_t>(facts.smem_sm) / per_sm;
+    cap = cap > 2048 ? cap - 1024 : cap;                   // the system's share per CTA
+    if (cap > block_max) cap = block_max;
+    size_t smem = fixed + one_table + kStripWarps * stage;
+    uint32_t rep_log = 0;
+    while (rep_log < 5 && smem + (one_table << rep_log) <= cap) {
+      smem += one_table << rep_log;
+      ++rep_log;
+    }
+    a.succ_bytes = static_cast<uint32_t>(succ);
+    a.table_bytes = static_cast<uint32_t>(one_table << rep_log);
+    a.stage_bytes = static_cast<uint32_t>(stage);
+    if (smem > facts.smem_set) {
+      ANSB_CUDA(cudaFuncSetAttribute(ans_decode_strips_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(smem)));
+      facts.smem_set = smem;
+    }
+    // launched so that it may take its place on the device while the launch before it on the
+    // stream is still running; the kernel waits for that launch before it reads memory
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>(ctas));
+    cfg.blockDim = dim3(kStripWarps * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ANSB_CUDA(cudaLaunchKernelEx(&cfg, ans_decode_strips_kernel, a));
+  }
+  return ANS_OK;
+}
+
+}  // namespace ansb

@@ -125,6 +125,36 @@ inline size_t quad_lane_count(size_t nc, size_t W, size_t lambda) {
 }
 inline size_t quad_position(size_t W, size_t lambda, size_t t) { return ((t / 4) * W + lambda) * 4 + t % 4; }
 
+// One sub-stream of the strips container: `strip` holds its ns symbols (a contiguous part of the
+// chunk), dealt to the 32 lanes round-robin.  Appended to `bytes`: the lanes' bit lengths, then
+// their strings (state in R bits, then the fields) back to back from the top bit of 32-bit words.
+bool pack_strip(const EncTable& T, const uint8_t* strip, size_t ns, std::vector<uint8_t>& bytes,
+                std::vector<uint8_t>& nb, std::vector<uint16_t>& val) {
+  const size_t base = bytes.size();
+  bytes.resize(base + 64, 0);
+  const size_t max_lane = (ns + 31) / 32 + 1;
+  nb.resize(max_lane);
+  val.resize(max_lane);
+  TopBitWriter bw(bytes);
+  for (size_t k = 0; k < 32; ++k) {
+    const size_t cnt = lane_count(ns, 32, k);
+    uint64_t len = 0;
+    if (cnt) {
+      const int init = encode_lane(T, strip + k, cnt, 32, nb.data(), val.data());
+      if (init < 0) return false;
+      bw.put(static_cast<uint32_t>(init), T.R);
+      len = static_cast<uint64_t>(T.R);
+      for (size_t t = 0; t < cnt; ++t) { bw.put(val[t], nb[t]); len += nb[t]; }
+    }
+    if (len > 0xFFFF) return false;
+    bytes[base + 2 * k] = static_cast<uint8_t>(len & 0xFF);        // (the writer only appends, so the header stays put)
+    bytes[base + 2 * k + 1] = static_cast<uint8_t>(len >> 8);
+  }
+  bw.finish();
+  while ((bytes.size() - base) % 16) bytes.push_back(0);
+  return true;
+}
+
 // One sub-stream (32 lanes) into `bytes` (appended) and meta (32 entries).
 bool pack_sub(const EncTable& T, const uint8_t* chunk, size_t nc, size_t W, size_t g, int layout,
               std::vector<uint8_t>& bytes, void* meta32, std::vector<uint8_t>& nb, std::vector<uint16_t>& val,
@@ -248,11 +278,11 @@ ANS_EXPORT int ans_host_normalize_freqs(const uint64_t* h_counts, int alphabet, 
 ANS_EXPORT int ans_host_pack_bound(uint64_t n_symbols, uint32_t chunk_symbols, uint32_t lanes, int layout,
                                    uint64_t* h_bytes_out) {
   if (!h_bytes_out || chunk_symbols == 0 || lanes == 0 || lanes % 32) return ANS_ERR_INVALID_ARG;
-  if (layout != ANS_LAYOUT_INTERLEAVED && layout != ANS_LAYOUT_PRIVATE && layout != ANS_LAYOUT_QUADS)
-    return ANS_ERR_UNSUPPORTED;
+  if (layout < ANS_LAYOUT_INTERLEAVED || layout > ANS_LAYOUT_STRIPS) return ANS_ERR_UNSUPPORTED;
   const uint64_t chunks = n_symbols ? (n_symbols + chunk_symbols - 1) / chunk_symbols : 0;
   const uint64_t subs = chunks * (lanes / 32);
-  // <= 14 bits per symbol, plus per lane a last unit/word, plus per sub-stream 16 bytes of pad
+  // <= 14 bits per symbol, plus per lane a last unit/word (strips: a length and a state), plus
+  // per sub-stream 16 bytes of pad
   *h_bytes_out = n_symbols * 2 + subs * (32 * 4 + 16) + 16;
   return ANS_OK;
 }
@@ -266,9 +296,11 @@ ANS_EXPORT int ans_host_pack_layer(const uint8_t* h_symbols, uint64_t n_symbols,
   if (alphabet < 1 || alphabet > ANS_MAX_ALPHABET || chunk_symbols == 0) return ANS_ERR_INVALID_ARG;
   if (table_log < 1 || table_log > ANS_MAX_TABLE_LOG) return ANS_ERR_UNSUPPORTED;
   if (lanes < 32 || lanes > ANS_MAX_LANES || lanes % 32) return ANS_ERR_UNSUPPORTED;
-  if (layout != ANS_LAYOUT_INTERLEAVED && layout != ANS_LAYOUT_PRIVATE && layout != ANS_LAYOUT_QUADS)
+  if (layout < ANS_LAYOUT_INTERLEAVED || layout > ANS_LAYOUT_STRIPS) return ANS_ERR_UNSUPPORTED;
+  const bool strips = layout == ANS_LAYOUT_STRIPS;
+  if (strips && (chunk_symbols % lanes || chunk_symbols / lanes > ANS_MAX_STRIP_LANE_SYMBOLS))
     return ANS_ERR_UNSUPPORTED;
-  if (n_symbols && (!h_symbols || !h_stream_out || !h_lane_meta_out)) return ANS_ERR_INVALID_ARG;
+  if (n_symbols && (!h_symbols || !h_stream_out || (!h_lane_meta_out && !strips))) return ANS_ERR_INVALID_ARG;
   EncTable T;
   if (!make_enc_table(h_freqs, alphabet, table_log, T)) return ANS_ERR_BAD_FREQS;
 
@@ -292,6 +324,15 @@ ANS_EXPORT int ans_host_pack_layer(const uint8_t* h_symbols, uint64_t n_symbols,
       const size_t nc = std::min<uint64_t>(C, n_symbols - c * C);
       for (size_t g = 0; g < G; ++g) {
         part_offs[ti].push_back(part[ti].size());
+        if (strips) {
+          const size_t first = g * 32 * (C / W);
+          const size_t ns = nc > first ? std::min(nc - first, 32 * (C / W)) : 0;
+          if (!pack_strip(T, h_symbols + c * C + first, ns, part[ti], nb, val)) {
+            part_rc[ti] = ANS_ERR_BAD_FREQS;
+            return;
+          }
+          continue;
+        }
         void* meta = static_cast<uint8_t*>(h_lane_meta_out) + (c * G + g) * 32 * meta_es;
         if (!pack_sub(T, h_symbols + c * C, nc, W, g, layout, part[ti], meta, nb, val, lane_bytes)) {
           part_rc[ti] = ANS_ERR_BAD_FREQS;

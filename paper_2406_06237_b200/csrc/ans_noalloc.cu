@@ -50,7 +50,8 @@ ANS_EXPORT int ans_decode_dequant_host_noalloc(const ans_layer_desc* h_desc, con
   if (!h_desc || !h_norm_freqs) return ANS_ERR_INVALID_ARG;
   if (h_desc->chunk_symbols == 0 || h_desc->lanes == 0 || h_desc->lanes % 32) return ANS_ERR_INVALID_ARG;
   if (h_desc->n_symbols == 0) return validate_desc(*h_desc, false);   // nothing to decode, but still a sound layer?
-  if (!h_stream || !h_sub_offsets || !h_lane_meta || !h_out) return ANS_ERR_INVALID_ARG;
+  if (!h_stream || !h_sub_offsets || !h_out) return ANS_ERR_INVALID_ARG;
+  if (!h_lane_meta && lane_meta_size(h_desc->layout)) return ANS_ERR_INVALID_ARG;
 
   // lay the call out in the fixed area and refuse what does not fit.  Every term is bounded by
   // the area before it enters a sum, so that no size, however absurd, can wrap around and pass.
@@ -61,7 +62,7 @@ ANS_EXPORT int ans_decode_dequant_host_noalloc(const ans_layer_desc* h_desc, con
   const uint64_t n_sub = subs_of(*h_desc);               // <= n_symbols * 64 groups: no overflow
   if (n_sub > kNoAllocBytes / 128) return ANS_ERR_BUFFER_TOO_SMALL;
   const size_t offs_bytes = (n_sub + 1) * 8;
-  const size_t meta_bytes = n_sub * 32 * (h_desc->layout == ANS_LAYOUT_INTERLEAVED ? 2 : 4);
+  const size_t meta_bytes = n_sub * 32 * lane_meta_size(h_desc->layout);
   const size_t out_bytes = h_desc->n_symbols * elem_size(h_desc->out_dtype);
   const size_t need = 256 + up256(table_bytes) + up256(stream_bytes) + up256(offs_bytes) + up256(meta_bytes) +
                       up256(out_bytes);
@@ -88,7 +89,7 @@ ANS_EXPORT int ans_decode_dequant_host_noalloc(const ans_layer_desc* h_desc, con
   if (rc != ANS_OK) return rc;
   ANSB_CUDA(cudaMemcpyAsync(d_stream, h_stream, stream_bytes, cudaMemcpyHostToDevice, st));
   ANSB_CUDA(cudaMemcpyAsync(d_offs, h_sub_offsets, offs_bytes, cudaMemcpyHostToDevice, st));
-  ANSB_CUDA(cudaMemcpyAsync(d_meta, h_lane_meta, meta_bytes, cudaMemcpyHostToDevice, st));
+  if (meta_bytes) ANSB_CUDA(cudaMemcpyAsync(d_meta, h_lane_meta, meta_bytes, cudaMemcpyHostToDevice, st));
   ans_layer_desc d = *h_desc;
   d.d_table = d_table + table_off;
   d.d_stream = d_stream;

@@ -59,6 +59,23 @@ def test_host_packer_equals_oracle_encoder(layout, n, C, lanes, R, b):
         assert (o == P.sub_offsets).all() and (m == P.lane_meta).all()
 
 
+@pytest.mark.parametrize("n,C,lanes,R,b", [(36864, 4096, 32, 12, 4), (5000, 1024, 64, 8, 3), (100_003, 16384, 128, 11, 6),
+                                           (33, 128, 32, 6, 2), (70_000, 65536, 256, 14, 8), (4097, 4096, 32, 12, 1),
+                                           (130, 512, 32, 5, 3), (300_000, 16384, 64, 8, 4), (0, 4096, 32, 8, 4)])
+def test_host_packer_equals_oracle_encoder_strips(n, C, lanes, R, b):
+    spec = tiny_spec(max(n, 1), bitwidth=b, pzp=0.9, table_log=R, chunk=C)
+    sym = sg.draw_symbols(spec)
+    T, P, f256 = oracle_pack_spec(spec, sym, oracle.STRIPS, lanes)
+    sym = sym[:n]
+    P = oracle.pack(T, sym, C, lanes // 32, oracle.STRIPS)
+    for threads in (1, 3):
+        s, o, m = ans.ans_host_pack_layer(sym, f256, spec.alphabet, R, C, lanes, ans.ANS_LAYOUT_STRIPS, threads)
+        assert s.size == P.stream.size and (s == P.stream).all()
+        assert (o == P.sub_offsets).all() and m.size == 0
+    with pytest.raises(ans.AnsError):                      # chunk no multiple of 4 * lanes
+        ans.ans_host_pack_layer(sym, f256, spec.alphabet, R, 1000, 32, ans.ANS_LAYOUT_STRIPS, 1)
+
+
 def test_plan_batch_counts_groups_of_four_sub_streams():
     arr = (ans.ans_layer_desc * 3)()
     for d, (n, C, lanes) in zip(arr, [(36864, 4096, 32), (0, 4096, 64), (10, 4, 128)]):

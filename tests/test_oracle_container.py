@@ -226,7 +226,7 @@ def test_quads_word_of_the_hand_trace(name):
 # ---- strips container -----------------------------------------------------------------------
 STRIP_CASES = [(0, 512, 1), (1, 512, 1), (6, 512, 1), (130, 512, 1), (511, 512, 1), (512, 512, 1), (513, 512, 1),
                (5000, 1024, 2), (4096, 1024, 1), (777, 4096, 4), (65536 + 17, 16384, 2), (3000, 2048, 2),
-               (1000, 128, 1), (1000, 256, 2), (40001, 16384, 4)]
+               (1000, 32, 1), (1000, 192, 2), (40001, 16384, 4), (33, 96, 3)]
 
 
 @pytest.mark.parametrize("n,C,G", STRIP_CASES)
@@ -242,9 +242,9 @@ def test_strips_round_trip(n, C, G):
     assert rc == oracle.OK and (out == msg).all()
 
 
-def test_strips_chunk_must_be_a_multiple_of_four_times_the_lanes():
+def test_strips_chunk_must_be_a_multiple_of_the_lanes():
     T = oracle.Table([3, 1], 2)
-    for C, G in ((1000, 1), (64, 1), (384, 2)):
+    for C, G in ((1000, 1), (48, 1), (96, 2), (32 * 4097, 1)):
         with pytest.raises(oracle.OracleError):
             oracle.pack(T, np.zeros(10, dtype=np.uint8), C, G, oracle.STRIPS)
 
@@ -252,7 +252,7 @@ def test_strips_chunk_must_be_a_multiple_of_four_times_the_lanes():
 @pytest.mark.parametrize("n,C,G", [(3000, 2048, 2), (1000, 1024, 1), (517, 512, 4), (130, 4096, 1), (40000, 16384, 2)])
 def test_strips_equal_plain_single_lane_coding(n, C, G):
     """Independent build of every sub-stream in Python.  Sub-stream g owns the strip
-    [g*32*S, (g+1)*32*S) of its chunk; the strip is dealt to 32 lanes four symbols at a time;
+    [g*32*S, (g+1)*32*S) of its chunk; the strip is dealt to 32 lanes round-robin;
     a lane's string is the plain one-lane coder's initial state in R bits followed by that
     coder's fields, most significant bit first; the sub-stream is the 32 lengths as
     little-endian uint16, then the strings back to back in 32-bit little-endian words filled
@@ -268,11 +268,9 @@ def test_strips_equal_plain_single_lane_coding(n, C, G):
         for g in range(G):
             sub = c * G + g
             strip = chunk[g * 32 * S:(g + 1) * 32 * S]
-            owned = _quads_lanes(strip.size, 32)
-            assert sorted(q for l in owned for q in l) == list(range(strip.size))
             lens, bits = [], ""
             for k in range(32):
-                mine = strip[owned[k]]
+                mine = strip[k::32]
                 s = ""
                 if mine.size:
                     init, nb, val = oracle.encode_lane_fields(T, mine)
@@ -296,14 +294,14 @@ def _body_bits(stream, nbits):
 
 @pytest.mark.parametrize("name", ["trace_T1.txt", "trace_T2.txt"])
 def test_strips_bytes_of_the_hand_trace(name):
-    """Lane 0 of a one-strip layer carrying the hand trace's message (positions 0..3, 128..131,
-    ...; the other positions hold the first symbol): its length and bits are the ones worked
-    out by hand in the fixture; for T1 so are the other lanes' and the first word."""
+    """Lane 0 of a one-strip layer carrying the hand trace's message (positions 0, 32, 64, ...;
+    the other positions hold the first symbol): its length and bits are the ones worked out by
+    hand in the fixture; for T1 so are the other lanes' and the first word."""
     g = read_golden(name)
     R = int(g["table_log"])
     T = oracle.Table(_ints(g["freqs"]), R)
     msg = _ints(g["message"])
-    pos = [(t // 4) * 128 + t % 4 for t in range(len(msg))]
+    pos = [32 * t for t in range(len(msg))]
     sym = np.full(pos[-1] + 1, msg[0], dtype=np.uint8)
     sym[pos] = msg
     P = oracle.pack(T, sym, 512, 1, oracle.STRIPS)
@@ -324,37 +322,35 @@ def test_strips_same_symbols_for_every_chunking_and_threads():
     rng = np.random.default_rng(21)
     msg = _source(rng, 50000)
     T = _table(msg, 15, 11)
-    for C, G in [(1024, 1), (4096, 1), (4096, 4), (16384, 2), (65536, 8), (128, 1), (131072, 1)]:
+    for C, G in [(1024, 1), (4096, 1), (4096, 4), (16384, 2), (65536, 8), (32, 1), (131072, 1), (480, 3)]:
         P = oracle.pack(T, msg, C, G, oracle.STRIPS)
         for th in (1, 4):
             out, rc = oracle.unpack(T, P, threads=th)
             assert rc == oracle.OK and (out == msg).all()
 
 
-def test_strips_with_one_group_own_the_symbols_of_quads():
+def test_strips_with_one_group_own_the_symbols_of_the_private_lanes():
     """With 32 lanes per chunk the strip is the whole chunk, so lane k owns the very symbols it
-    owns in the quads container: same initial states, same fields."""
+    owns in the private container: same initial states, same number of bits."""
     rng = np.random.default_rng(23)
     msg = _source(rng, 9000)
     T = _table(msg, 15, 9)
-    Pq = oracle.pack(T, msg, 4096, 1, oracle.QUADS)
+    Pp = oracle.pack(T, msg, 4096, 1, oracle.PRIVATE)
     Ps = oracle.pack(T, msg, 4096, 1, oracle.STRIPS)
-    for sub in range(Pq.n_sub):
+    for sub in range(Pp.n_sub):
         b0 = int(Ps.sub_offsets[sub])
         lens = np.frombuffer(bytes(Ps.stream[b0:b0 + 64]), dtype="<u2").astype(int)
         body = _body_bits(Ps.stream[b0:], int(lens.sum()))
+        chunk = msg[sub * 4096:(sub + 1) * 4096]
         start = 0
         for k in range(32):
-            meta = int(Pq.lane_meta[sub, k])
             mine = body[start:start + lens[k]]
             start += lens[k]
             if not lens[k]:
+                assert chunk[k::32].size == 0
                 continue
-            assert int(mine[:9], 2) == (meta & 0xFFFF)
-            q0 = int(Pq.sub_offsets[sub]) + 4 * (meta >> 16)
-            nw = (lens[k] - 9 + 31) // 32
-            qbits = "".join(format(int(w), "032b") for w in np.frombuffer(bytes(Pq.stream[q0:q0 + 4 * nw]), dtype="<u4"))
-            assert qbits[:lens[k] - 9] == mine[9:]
+            assert int(mine[:9], 2) == (int(Pp.lane_meta[sub, k]) & 0xFFFF)
+            assert lens[k] - 9 == oracle.encode_plain(T, chunk[k::32])[2]
 
 
 def test_strips_corruption_is_reported():
@@ -392,8 +388,8 @@ def test_strips_overhead_per_lane_is_the_state_and_a_length():
     bits = 0
     for sub in range(P.n_sub):
         strip = msg[sub * 32 * S:(sub + 1) * 32 * S]
-        for mine in _quads_lanes(strip.size, 32):
-            bits += oracle.encode_plain(T, strip[mine])[2] + R + 16
+        for k in range(32):
+            bits += oracle.encode_plain(T, strip[k::32])[2] + R + 16
     pad = 0
     for sub in range(P.n_sub):
         b0, b1 = int(P.sub_offsets[sub]), int(P.sub_offsets[sub + 1])
