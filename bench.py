@@ -32,9 +32,11 @@ NOMINAL_PEAK_GBS = 8000.0
 FALLBACK_PEAK_GBS = 6650.0
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, scaled from the 2-matrix capture in
-# profiles/ans_decode_kernel_quads_large.md to the 8 matrices of a full launch
-NCU_TRAFFIC = {("large", "quads", 32, 8, 8192, 0, 0): 1021.9e6}      # 256-state table (the default)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the 8 matrices, from the 2-matrix capture in
+# profiles/ans_decode_kernel_quads_large.md: reads scale with the matrices (4 x 27.31 MB); writes are the
+# output (1073.74 MB) less what is still in L2 when the kernel ends, which the capture shows as
+# 268.44 - 228.17 = 40.27 MB whatever the size
+NCU_TRAFFIC = {("large", "quads", 32, 8, 8192, 0, 0): 4 * 27.31e6 + 1073.74e6 - 40.27e6}      # 256-state table (the default)
 
 
 def measured_peak():
@@ -70,8 +72,11 @@ WORKLOAD_TEXT = {
 }
 
 
-# the container each workload is timed on unless --layout says otherwise: the fastest measured
-DEFAULT_LAYOUT = {"large": "quads", "resnet18": "quads", "resnet50": "quads", "sweep": "quads", "conv3x3": "quads"}
+# the container and lanes per chunk each workload is timed on unless --layout / --lanes say otherwise: the
+# fastest measured (quads: one symbol per look-up, lanes in step; strips: a look-up may stand for a run of the
+# dominant symbol, which pays when one symbol owns most of the states, as in the ResNet-50 workload)
+DEFAULTS = {"large": ("quads", 32), "resnet18": ("strips", 64), "resnet50": ("strips", 64), "sweep": ("quads", 32),
+            "conv3x3": ("quads", 32)}
 
 
 class ClockSampler:
@@ -82,7 +87,7 @@ class ClockSampler:
 
     def __init__(self, index):
         self.index, self.rows, self.proc = index, [], None
-        self.first, self.last, self.in_timed = 0, None, None     # rows taken under the timed load
+        self.first, self.last = 0, None                       # rows taken while the timed rounds ran
 
     def start(self):
         try:
@@ -106,6 +111,10 @@ class ClockSampler:
                 self.proc.wait(timeout=5)
             except Exception:
                 pass
+
+    def summary(self):
+        """Median SM clock and the throttle reasons seen in rows [first, last): the samples taken
+        while the timed rounds ran."""
         rows = self.rows[self.first:self.last]
         sm = [float(r[1]) for r in rows if len(r) >= 9 and r[1].replace(".", "").isdigit()]
         mx = [float(r[2]) for r in rows if len(r) >= 9 and r[2].replace(".", "").isdigit()]
@@ -116,13 +125,8 @@ class ClockSampler:
             for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
-        out = {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-               "reasons": sorted(reasons), "samples": len(sm)}
-        if self.in_timed is not None and self.in_timed < len(sm):
-            out["samples_in_timed_region"] = self.in_timed
-            out["note"] = ("the timed region is shorter than a few sampling periods (20 ms): the same launches "
-                           "were kept running right after it until 5 samples were in")
-        return out
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples_in_timed_region": len(sm)}
 
 
 def cpu_baseline(specs, syms, layout_name, args_lanes=32):
@@ -205,7 +209,7 @@ def run_reference(args):
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": "weights/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": specs[0].out_dtype if len({sp.out_dtype for sp in specs}) == 1 else "mixed", "data": "synthetic",
         "config": {"workload": WORKLOAD_TEXT[args.workload], "layout": args.layout, "sample": sample_txt},
         "cpu_baseline": {"value": value, "unit": "weights/s", "cores": cores, "kind": "oracle", "sample": sample_txt},
         "e2e": {"value": value, "unit": "weights/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -223,77 +227,81 @@ def reduce_max(x: float, world: int) -> float:
     return float(t.item())
 
 
-def time_workload(db, steps, warmup, flush, n_sets, world, sampler=None):
-    """K timed steps, each bracketed by CUDA events on the launching stream; the L2 flush (if
-    any) sits outside the brackets.  Returns per-step milliseconds (max over ranks of the sum)."""
+MIN_REGION_S = 0.5          # device time the timed rounds of a workload add up to, at least
+
+
+def time_workload(db, steps, warmup, n_sets, world, min_region_s=MIN_REGION_S, max_rounds=2000):
+    """Rounds of K back-to-back launches, each round bracketed by CUDA events on the launching
+    stream.  The host must not be what is timed, so every round goes behind a device-side spin of
+    a few milliseconds (outside the brackets): by the time the device reaches the first launch all
+    K are queued.  The first round is the K steps the command line asked for; further rounds
+    repeat them until the rounds add up to min_region_s of device time, so that clock samples
+    fall inside the timed region.  A last round brackets every launch by itself.
+    Returns (per-round milliseconds per step, per-launch milliseconds of the last round)."""
     import torch
     import torch.distributed as dist
     st = torch.cuda.current_stream()
     for i in range(warmup):
-        if flush is not None:
-            flush.add_(1)
         db.decode(i % n_sets)
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-    if sampler is not None:
-        sampler.first = len(sampler.rows)
-    # The host must not be what is timed: a spin of a few milliseconds goes first (outside every
-    # bracket), so that the K launches and their events are all queued by the time the device
-    # reaches them and run back to back.
-    torch.cuda._sleep(int(2e7))
-    for i in range(steps):
-        if flush is not None:
-            flush.add_(1)
-        ev[i][0].record(st)
-        db.decode(i % n_sets)
-        ev[i][1].record(st)
-    torch.cuda.synchronize()
-    if sampler is not None and sampler.proc is not None:
-        # a clock reading needs a few sampling periods of load: keep the same launches going
-        # (outside every timing bracket) until they are in
-        sampler.in_timed = len(sampler.rows) - sampler.first
-        t_end = time.perf_counter() + 2.0
-        while len(sampler.rows) - sampler.first < 5 and time.perf_counter() < t_end:
+    spin = int(2e7)                                       # cycles: about 10 ms
+
+    def one_round(per_launch=False):
+        evs = []
+        torch.cuda._sleep(spin)
+        if per_launch:
+            for i in range(steps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(st)
+                db.decode(i % n_sets)
+                b.record(st)
+                evs.append((a, b))
+        else:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(st)
             for i in range(steps):
                 db.decode(i % n_sets)
-            torch.cuda.synchronize()
-        sampler.last = len(sampler.rows)
+            b.record(st)
+            evs.append((a, b))
+        return evs
+
+    rounds, total_ms = [], 0.0
+    while True:
+        ev = one_round()
+        torch.cuda.synchronize()
+        ms = ev[0][0].elapsed_time(ev[0][1])
+        rounds.append(ms / steps)
+        total_ms += ms
+        if total_ms >= min_region_s * 1e3 or len(rounds) >= max_rounds:
+            break
+    pairs = one_round(per_launch=True)
+    torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    ms = [a.elapsed_time(b) for a, b in ev]               # each launch by itself
-    span = ev[0][0].elapsed_time(ev[-1][1])               # the K steps as one region, gaps included
+    each = [a.elapsed_time(b) for a, b in pairs]
     assert db.read_status() == 0, "decoder flagged a stream"
-    return ms, span
+    return rounds, each
 
 
-def run_ours(args):
-    import torch
-    import paper_2406_06237_b200 as ans
-    from paper_2406_06237_b200.runtime import DeviceBatch, pack_layer
+LAYOUT_IDS = {"private": "ANS_LAYOUT_PRIVATE", "interleaved": "ANS_LAYOUT_INTERLEAVED", "quads": "ANS_LAYOUT_QUADS",
+              "strips": "ANS_LAYOUT_STRIPS"}
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
-    torch.cuda.set_device(local)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    ans.lib()                                           # fail loudly if the library is missing
 
-    layout = {"private": ans.ANS_LAYOUT_PRIVATE, "interleaved": ans.ANS_LAYOUT_INTERLEAVED,
-              "quads": ans.ANS_LAYOUT_QUADS, "strips": ans.ANS_LAYOUT_STRIPS}[args.layout]
-    specs = make_specs(args)
-    t_setup = time.perf_counter()
+def build_case(ans, args, workload, layout_name, lanes, table_log=0, chunk=0, local=0, by_channel=False):
+    """Draw the workload's symbols, pack them with the library's host packer, put everything on
+    the device.  Returns (specs, syms, layers, db, n_sets, working-set text)."""
+    import copy
     from concurrent.futures import ThreadPoolExecutor
+    from paper_2406_06237_b200.runtime import DeviceBatch, pack_layer
+    a2 = copy.copy(args)
+    a2.workload, a2.table_log, a2.chunk = workload, table_log, chunk
+    specs = make_specs(a2)
+    layout = getattr(ans, LAYOUT_IDS[layout_name])
     cores = os.cpu_count() or 1
-
-    by_channel = args.grouping == "channel"
     if by_channel:
         # the paper's own grouping (Section III-B): one chunk per layer, one lane per input channel,
         # weights stored channels-last so that lane c carries input channel c; layers whose input
@@ -301,15 +309,14 @@ def run_ours(args):
         import dataclasses
         specs = [dataclasses.replace(sp, chunk_symbols=sp.n) for sp in specs
                  if len(sp.shape) == 4 and sp.shape[1] % 32 == 0 and sp.shape[1] <= 2048]
-        args.no_cpu_baseline = args.no_e2e = True
 
     def prep(spec):
         sym = sg.draw_symbols(spec, threads=max(1, cores // 4))
-        lanes = args.lanes
+        ln = lanes
         if by_channel:
             sym = np.ascontiguousarray(sym.reshape(spec.shape).transpose(0, 2, 3, 1)).ravel()
-            lanes = spec.shape[1]
-        pl = pack_layer(sym, spec.alphabet, spec.table_log, spec.chunk_symbols, lanes, layout, spec.bitwidth,
+            ln = spec.shape[1]
+        pl = pack_layer(sym, spec.alphabet, spec.table_log, spec.chunk_symbols, ln, layout, spec.bitwidth,
                         spec.zero_point, spec.scale, ans.DTYPES[spec.out_dtype], n_threads=max(1, cores // 2))
         return sym, pl
 
@@ -325,90 +332,149 @@ def run_ours(args):
     small = ws < (512 << 20)
     n_sets = min(64, max(2, -(-(512 << 20) // max(ws, 1)))) if small else 1
     db = DeviceBatch(layers, f"cuda:{local}", n_out_sets=n_sets)
-    flush = None
-    setup_s = time.perf_counter() - t_setup
+    policy = (f"inputs larger than L2: launches rotate over {n_sets} full copies of the workload "
+              f"({n_sets * ws / 2**20:.0f} MB in all)" if small else "working set (compressed + output) is larger than L2")
+    return specs, syms, layers, db, n_sets, policy
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    ms, span = time_workload(db, args.steps, args.warmup, flush, n_sets, world, sampler if rank == 0 else None)
-    clocks = sampler.stop() if rank == 0 else None
-    total_ms = reduce_max(span, world)
-    ms_per_step = total_ms / args.steps
+
+def figures(ans, layers, db, rounds, each, peak):
+    """Throughput and roofline figures of one measured case."""
     n_w = db.n_symbols()
-    value = world * n_w / (ms_per_step * 1e-3)
-
+    out_bytes = sum(L.n_symbols * ans.ELEM_SIZE[L.out_dtype] for L in layers)
     # algorithmic bytes of one launch: everything compressed read once, each layer's table
     # once, every decoded element written once
     table_read = sum(4 << L.table_log for L in layers)
     comp_bytes = db.compressed_bytes()
     algo_bytes = comp_bytes + table_read + out_bytes
-    peak, peak_kind = measured_peak()
-    kernel_ms = statistics.mean(ms)
+    kernel_ms = statistics.mean(rounds)                   # average launch duration over all timed rounds
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-    kname = f"ans_decode_kernel<{args.layout}>"
+    return {"n_w": n_w, "out_bytes": out_bytes, "comp_bytes": comp_bytes, "algo_bytes": algo_bytes,
+            "kernel_ms": kernel_ms, "achieved": achieved, "frac": achieved / peak,
+            "frac_nominal": achieved / NOMINAL_PEAK_GBS,
+            "coded_bits": 8.0 * comp_bytes / max(1, n_w)}
+
+
+def entropy_bits(specs, syms):
+    ent = 0.0
+    for spec, sym in zip(specs, syms):
+        c = np.bincount(sym, minlength=256).astype(np.float64)
+        p = c[c > 0] / max(1, sym.size)
+        ent += float(-(p * np.log2(p)).sum()) * sym.size
+    return ent
+
+
+# (workload, container, lanes, table_log, chunk) measured beside the headline: the other table size
+# quoted for the large layers, the two ResNets, one cell of the granularity sweep
+VARIANTS = [("large", "quads", 32, 12, 0), ("resnet50", "strips", 64, 0, 0), ("resnet50", "quads", 32, 0, 0),
+            ("resnet18", "strips", 64, 0, 0), ("resnet18", "quads", 32, 0, 0), ("sweep", "quads", 32, 12, 16384)]
+
+
+def run_ours(args):
+    import torch
+    import paper_2406_06237_b200 as ans
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    ans.lib()                                           # fail loudly if the library is missing
+
+    t_setup = time.perf_counter()
+    by_channel = args.grouping == "channel"
+    if by_channel:
+        args.no_cpu_baseline = args.no_e2e = True
+    specs, syms, layers, db, n_sets, policy = build_case(ans, args, args.workload, args.layout, args.lanes,
+                                                         args.table_log, args.chunk, local, by_channel)
+    setup_s = time.perf_counter() - t_setup
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    peak, peak_kind = measured_peak()
+    sampler.first = len(sampler.rows)
+    rounds, each = time_workload(db, args.steps, args.warmup, n_sets, world)
+    sampler.last = len(sampler.rows)
+    clocks = sampler.summary() if rank == 0 else None
+    ms_per_step = reduce_max(rounds[0], world)          # the K steps asked for: the first round
+    fg = figures(ans, layers, db, rounds, each, peak)
+    n_w = fg["n_w"]
+    value = world * n_w / (ms_per_step * 1e-3)
+
+    kname = "ans_decode_strips_kernel" if args.layout == "strips" else f"ans_decode_kernel<{args.layout}>"
     # DRAM bytes per launch from an ncu capture of this kernel (see profiles/), only for the
     # configuration that capture covers; None otherwise
     traffic = NCU_TRAFFIC.get((args.workload, args.layout, args.lanes, args.mats, args.dim, args.chunk, args.table_log))
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+    roofline = {"bound": "hbm", "achieved": fg["achieved"], "peak": peak, "unit": "GB/s", "frac": fg["frac"],
                 "traffic": traffic, "kernel": kname, "peak_kind": f"of {peak_kind}",
-                "algorithmic_bytes_per_launch": algo_bytes, "kernel_ms_mean": kernel_ms,
-                "kernel_ms_median": statistics.median(ms), "kernel_ms_min": min(ms),
-                "frac_of_nominal_8TBs": achieved / NOMINAL_PEAK_GBS,
-                "note": "HBM is the metric's roofline; ncu shows the kernel held by instruction issue, the integer "
-                        "pipe and shared-memory wavefronts together (see profiles/)"}
+                "algorithmic_bytes_per_launch": fg["algo_bytes"], "kernel_ms_mean": fg["kernel_ms"],
+                "timed_rounds": len(rounds), "launches_per_round": args.steps,
+                "round_ms_per_launch_min": min(rounds), "round_ms_per_launch_max": max(rounds),
+                "launch_bracketed_alone_ms_median": statistics.median(each), "launch_bracketed_alone_ms_min": min(each),
+                "frac_of_nominal_8TBs": fg["frac_nominal"],
+                "note": "kernel_ms_mean: CUDA events around rounds of back-to-back launches, divided by the launches "
+                        "(gaps between launches included); HBM is the metric's roofline, the kernels themselves are "
+                        "held by instruction issue and shared-memory wavefronts (see profiles/)"}
 
     # end to end through the host-buffer entry point: pinned host buffers in, pinned out
     e2e = None
     if not args.no_e2e:
         e2e = run_e2e(ans, db, layers, args, world)
+    ent_bits = entropy_bits(specs, syms)
+    cpu = cpu_baseline(specs, syms, args.layout, args.lanes) if world == 1 and rank == 0 and not args.no_cpu_baseline else None
+    head_specs = specs
+    launches = (len(rounds) + 1) * args.steps * db.launches_per_decode()
 
-    # the same workload with the other table size the design notes quote (2^12 states)
+    # the other workloads and table sizes, each measured the same way (shorter regions)
     variants = []
-    if args.workload == "large" and not args.table_log and world == 1 and not args.no_variants:
-        db = None
+    if args.workload == "large" and not args.table_log and not args.chunk and world == 1 and not args.no_variants \
+            and args.mats == 8 and args.dim == 8192:
+        del db
         torch.cuda.empty_cache()
-        with ThreadPoolExecutor(4) as ex:
-            layers12 = list(ex.map(lambda sp_sy: pack_layer(sp_sy[1], sp_sy[0].alphabet, 12, sp_sy[0].chunk_symbols,
-                                                            args.lanes, layout, sp_sy[0].bitwidth, sp_sy[0].zero_point,
-                                                            sp_sy[0].scale, ans.DTYPES[sp_sy[0].out_dtype],
-                                                            n_threads=max(1, cores // 2)), zip(specs, syms)))
-        db12 = DeviceBatch(layers12, f"cuda:{local}", n_out_sets=1)
-        ms12, _ = time_workload(db12, min(args.steps, 50), 5, None, 1, 1)
-        bytes12 = db12.compressed_bytes() + sum(4 << 12 for _ in layers12) + out_bytes
-        k12 = statistics.mean(ms12)
-        variants.append({"table_log": 12, "layout": args.layout, "kernel_ms_mean": k12, "value": n_w / (k12 * 1e-3), "unit": "weights/s",
-                         "achieved_gbs": bytes12 / (k12 * 1e-3) / 1e9, "frac": bytes12 / (k12 * 1e-3) / 1e9 / peak,
-                         "coded_bits_per_weight": 8.0 * db12.compressed_bytes() / n_w})
-        del db12
-
+        for wl, lay, ln, tl, ck in VARIANTS:
+            vs, vy, vl, vdb, vsets, vpol = build_case(ans, args, wl, lay, ln, tl, ck, local)
+            sampler.first = len(sampler.rows)
+            vr, ve = time_workload(vdb, min(args.steps, 200) if wl in ("large", "sweep") else max(args.steps, 100), 5, vsets, 1,
+                                   min_region_s=0.3)
+            sampler.last = len(sampler.rows)
+            vf = figures(ans, vl, vdb, vr, ve, peak)
+            variants.append({"workload": wl, "layout": lay, "lanes": ln, "table_log": vl[0].table_log,
+                             "chunk_symbols": vl[0].chunk_symbols, "weights": vf["n_w"], "out_dtype": vs[0].out_dtype,
+                             "kernel_ms_mean": vf["kernel_ms"], "timed_rounds": len(vr),
+                             "launch_bracketed_alone_ms_median": statistics.median(ve),
+                             "value": vf["n_w"] / (vf["kernel_ms"] * 1e-3), "unit": "weights/s",
+                             "achieved_gbs": vf["achieved"], "frac": vf["frac"], "frac_of_nominal_8TBs": vf["frac_nominal"],
+                             "coded_bits_per_weight": vf["coded_bits"],
+                             "entropy_bits_per_weight": entropy_bits(vs, vy) / max(1, vf["n_w"]),
+                             "l2_policy": vpol, "clocks": sampler.summary()})
+            launches += (len(vr) + 1) * (min(args.steps, 200) if wl in ("large", "sweep") else max(args.steps, 100)) * vdb.launches_per_decode()
+            del vdb
+            torch.cuda.empty_cache()
+    if rank == 0:
+        sampler.stop()
     if rank != 0:
         return
-    hist = np.zeros(256, dtype=np.float64)
-    ent_bits = 0.0
-    for spec, sym in zip(specs, syms):
-        c = np.bincount(sym, minlength=256).astype(np.float64)
-        p = c[c > 0] / max(1, sym.size)
-        ent_bits += float(-(p * np.log2(p)).sum()) * sym.size
-    coded_bits = 8.0 * comp_bytes
-    cpu = cpu_baseline(specs, syms, args.layout, args.lanes) if world == 1 and not args.no_cpu_baseline else None
+    dts = sorted({sp.out_dtype for sp in head_specs})
     out = {
         "metric": METRIC, "value": value, "unit": "weights/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "vs_baseline": None, "dtype": dts[0] if len(dts) == 1 else "mixed", "data": "synthetic",
         "config": {"workload": WORKLOAD_TEXT[args.workload], "name": args.workload, "layout": args.layout,
-                   "lanes": "one per input channel" if args.grouping == "channel" else args.lanes,
+                   "lanes": "one per input channel" if by_channel else args.lanes,
                    "grouping": args.grouping, "table_log": layers[0].table_log, "chunk_symbols": layers[0].chunk_symbols,
-                   "layers": len(layers), "weights": n_w, "out_dtype": specs[0].out_dtype,
-                   "l2_policy": (f"inputs larger than L2: launches rotate over {n_sets} full copies of the workload "
-                                 f"({n_sets * ws / 2**20:.0f} MB in all)"
-                                 if small else "working set (compressed + output) is larger than L2"),
+                   "layers": len(layers), "weights": n_w, "out_dtype": head_specs[0].out_dtype,
+                   "arithmetic": "integer decode, one fp32 multiply per weight, round-to-nearest-even to the output type",
+                   "l2_policy": policy,
                    "per_gpu": "every rank decodes its own replica of the workload; no collective on the data path"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "roofline": roofline, "cpu_baseline": cpu,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
         "variants": variants,
-        "compression": {"coded_bits_per_weight": coded_bits / max(1, n_w), "entropy_bits_per_weight": ent_bits / max(1, n_w),
-                        "gap_bits_per_weight": (coded_bits - ent_bits) / max(1, n_w),
-                        "compressed_bytes": comp_bytes, "output_bytes": out_bytes},
+        "compression": {"coded_bits_per_weight": fg["coded_bits"], "entropy_bits_per_weight": ent_bits / max(1, n_w),
+                        "gap_bits_per_weight": fg["coded_bits"] - ent_bits / max(1, n_w),
+                        "compressed_bytes": fg["comp_bytes"], "output_bytes": fg["out_bytes"]},
         "setup_s": setup_s,
     }
     print(json.dumps(out))
@@ -467,7 +533,7 @@ def main():
     ap.add_argument("--workload", default="large", choices=list(WORKLOAD_TEXT))
     ap.add_argument("--layout", default=None, choices=["private", "interleaved", "quads", "strips"],
                     help="container; default: the fastest measured for the workload")
-    ap.add_argument("--lanes", type=int, default=32)
+    ap.add_argument("--lanes", type=int, default=0, help="lanes per chunk (a multiple of 32); default: per workload")
     ap.add_argument("--grouping", default="chunks", choices=["chunks", "channel"],
                     help="channel (ResNet workloads): one stream per input channel of every conv, as in the paper")
     ap.add_argument("--chunk", type=int, default=0)
@@ -480,12 +546,38 @@ def main():
     ap.add_argument("--no-variants", action="store_true")
     args = ap.parse_args()
     if args.layout is None:
-        args.layout = DEFAULT_LAYOUT[args.workload]
+        args.layout = DEFAULTS[args.workload][0]
+    if not args.lanes:
+        args.lanes = DEFAULTS[args.workload][1] if args.layout == DEFAULTS[args.workload][0] else 32
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_ranks(args.gpus, run_impl, args)              # not under torchrun: start the N ranks here
+    else:
+        run_impl(args)
+
+
+def run_impl(args):
     if args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
+
+
+def _rank_entry(rank, n, port, target, targs):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    target(*targs)
+
+
+def spawn_ranks(n, target, *targs):
+    """Start n local ranks, one process per GPU, with the environment torchrun would give them
+    (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR = 127.0.0.1, a free MASTER_PORT), and wait for them."""
+    import socket
+    import torch.multiprocessing as mp
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    mp.spawn(_rank_entry, args=(n, port, target, targs), nprocs=n, join=True)
 
 
 if __name__ == "__main__":

@@ -136,6 +136,15 @@ class DeviceBatch:
     def n_symbols(self) -> int:
         return sum(L.n_symbols for L in self.layers)
 
+    def launches_per_decode(self) -> int:
+        """Kernel launches one decode() makes: one, except that the strips kernel takes the
+        layers 64 at a time (a group in which every layer is empty is not launched)."""
+        if not any(L.n_symbols for L in self.layers):
+            return 0
+        if self.layers[0].layout == B.ANS_LAYOUT_STRIPS:
+            return sum(1 for g in range(0, len(self.layers), 64) if any(L.n_symbols for L in self.layers[g:g + 64]))
+        return 1
+
     # -- calls ---------------------------------------------------------------------------
     def decode(self, out_set: int = 0, stream: int | None = None) -> None:
         """ONE launch for all layers (asynchronous)."""
