@@ -80,8 +80,11 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
     const int R = L.table_log;
     // copies of this layer's table: a table smaller than the launch's largest uses the room for
     // more of them (the pre-walked walk keeps an extra entry after the table, so it does not)
-    // quads with 1-byte outputs: one-word entries, so twice the copies (up to 32) in the same room
-    const bool short_entries = kQuads && (args.d_symbols_override || L.out_dtype == ANS_U8);
+    // quads with 1-byte outputs: one-word entries, so twice the copies (up to 32) in the same room;
+    // quads with 2-byte outputs and 2^10 to 2^12 states likewise (smaller tables already have a
+    // conflict-free copy per lane pair in the two-word form, larger ones do not fit one word)
+    const bool short_entries = kQuads && (args.d_symbols_override || L.out_dtype == ANS_U8 ||
+                                          (L.out_dtype == ANS_BF16 && R >= 10 && R <= 12));
     const uint32_t rep_two = min(4u, args.rep_log + (args.max_log - static_cast<uint32_t>(R)));
     const uint32_t rep_log = (kPrivate && !lock) ? args.rep_log : short_entries ? rep_two + 1u : rep_two;
     const uint32_t reps = 1u << rep_log;
@@ -184,8 +187,9 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
                                  : to_smem_entry(g[k], vals[entry_sym(g[k])], 32u * static_cast<uint32_t>(es));
           // every lane starts at another copy: the stores of a warp spread over the banks
           if (short_entries) {
-            const uint32_t e1 = entry_nb(g[k]) | ((entry_newx(g[k]) >> entry_nb(g[k])) << 8) |
-                                (vals[entry_sym(g[k])] << 24);
+            const uint32_t qq = entry_newx(g[k]) >> entry_nb(g[k]);
+            const uint32_t e1 = es == 2 ? entry_nb(g[k]) | (qq << 4) | (vals[entry_sym(g[k])] << 16)
+                                        : entry_nb(g[k]) | (qq << 8) | (vals[entry_sym(g[k])] << 24);
             for (uint32_t c = 0; c < reps; ++c)
               reinterpret_cast<uint32_t*>(tab)[(i << rep_log) + ((c + lane) & (reps - 1u))] = e1;
           } else {
@@ -282,10 +286,12 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
                                       s_maxnb <= 8u, args.unit)
         if constexpr (kQuads) {                           // (1-byte outputs: one-word entries, see above)
           if (staged) {
-            if (es == 1) ANSB_QCALL(1, true, true); else if (es == 2) ANSB_QCALL(2, true, false);
+            if (es == 1) ANSB_QCALL(1, true, true);
+            else if (es == 2) { if (short_entries) ANSB_QCALL(2, true, true); else ANSB_QCALL(2, true, false); }
             else ANSB_QCALL(4, true, false);
           } else {
-            if (es == 1) ANSB_QCALL(1, false, true); else if (es == 2) ANSB_QCALL(2, false, false);
+            if (es == 1) ANSB_QCALL(1, false, true);
+            else if (es == 2) { if (short_entries) ANSB_QCALL(2, false, true); else ANSB_QCALL(2, false, false); }
             else ANSB_QCALL(4, false, false);
           }
         } else if constexpr (lock) {

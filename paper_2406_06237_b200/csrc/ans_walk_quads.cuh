@@ -19,6 +19,8 @@ namespace ansb {
 // or, for 1-byte outputs, ONE word: nb [4:0] | q [21:8] | value [31:24].  Half the bytes per
 // table, so twice the copies fit: it pays where copies are short (tables of 2^11 states and up,
 // whose random look-ups collide), at the price of one more instruction per look-up.
+// 2-byte outputs have a one-word form too, for tables of 2^10 to 2^12 states:
+// nb [3:0] | q [15:4] | value [31:16] (two more instructions per look-up, half the wavefronts).
 // =============================================================================================
 __device__ __forceinline__ uint2 to_quads_entry(uint32_t g, uint32_t val, bool narrow) {
   const uint32_t nb = entry_nb(g), q = entry_newx(g) >> nb;
@@ -38,6 +40,14 @@ __device__ __forceinline__ uint2 to_quads_entry(uint32_t g, uint32_t val, bool n
   "shf.l.wrap.b32 x, 0, x, ea" I_ ";\n\t"                         \
   "mad.lo.u32 %0, t, %7, %6;\n\t"                                 \
   "mad.lo.u32 %1, ea" I_ ", %9, %1;\n\t"
+#define ANSB_QD_STEP_S2(I_)                                       \
+  "ld.shared.u32 ea" I_ ", [%0];\n\t"                             \
+  "and.b32 nbb, ea" I_ ", 15;\n\t"                                \
+  "bfe.u32 nx, ea" I_ ", 4, 12;\n\t"                              \
+  "shf.l.wrap.b32 t, x, nx, nbb;\n\t"                            \
+  "shf.l.wrap.b32 x, 0, x, nbb;\n\t"                             \
+  "mad.lo.u32 %0, t, %7, %6;\n\t"                                 \
+  "add.u32 %1, %1, nbb;\n\t"
 #define ANSB_QD_STEP_W(I_)                                        \
   "ld.shared.v2.u32 {ea" I_ ", eb" I_ "}, [%0];\n\t"              \
   "shr.u32 nx, ea" I_ ", 8;\n\t"                                  \
@@ -82,7 +92,7 @@ __device__ __forceinline__ void quads_loop(uint32_t& st, uint32_t& bitpos, uint3
   asm volatile(                                                                             \
       "{\n\t"                                                                               \
       ".reg .pred q;\n\t"                                                                   \
-      ".reg .u32 x, t, nx, nw, v0, v1, cnt, ea0, ea1, ea2, ea3, eb0, eb1, eb2, eb3;\n\t"     \
+      ".reg .u32 x, t, nx, nbb, nw, v0, v1, cnt, ea0, ea1, ea2, ea3, eb0, eb1, eb2, eb3;\n\t" \
       ".reg .u64 gpp;\n\t"                                                                  \
       "mov.u64 gpp, %8;\n\t"                                                                \
       "mov.u32 cnt, %10;\n"                                                                 \
@@ -103,7 +113,7 @@ __device__ __forceinline__ void quads_loop(uint32_t& st, uint32_t& bitpos, uint3
   asm volatile(                                                                             \
       "{\n\t"                                                                               \
       ".reg .pred q;\n\t"                                                                   \
-      ".reg .u32 x, t, nx, nw, v0, v1, cnt, ea0, ea1, ea2, ea3, eb0, eb1, eb2, eb3;\n\t"     \
+      ".reg .u32 x, t, nx, nbb, nw, v0, v1, cnt, ea0, ea1, ea2, ea3, eb0, eb1, eb2, eb3;\n\t" \
       ".reg .u64 gpp;\n\t"                                                                  \
       "mov.u64 gpp, %8;\n\t"                                                                \
       "mov.u32 cnt, %10;\n"                                                                 \
@@ -123,7 +133,10 @@ __device__ __forceinline__ void quads_loop(uint32_t& st, uint32_t& bitpos, uint3
       : "memory")
 #define ANSB_QD_BOTH(L1_, LG_, TURN_, ST_, OUT_)                                            \
   if (groups == 1) ANSB_QD_ASM1(L1_, TURN_, ST_, OUT_); else ANSB_QD_ASMG(LG_, TURN_, ST_, OUT_)
-  if (SHORT) {     // one-word entries (1-byte outputs)
+  if (SHORT && ES == 2) {     // one-word entries, 2-byte outputs
+    if (K == 4) { ANSB_QD_BOTH("ANSB_QT41", "ANSB_QT4G", ANSB_QD_TURN4, ANSB_QD_STEP_S2, ANSB_QD_OUT2); }
+    else { ANSB_QD_BOTH("ANSB_QT21", "ANSB_QT2G", ANSB_QD_TURN2, ANSB_QD_STEP_S2, ANSB_QD_OUT2); }
+  } else if (SHORT) {     // one-word entries, 1-byte outputs
     if (K == 4) { ANSB_QD_BOTH("ANSB_QS41", "ANSB_QS4G", ANSB_QD_TURN4, ANSB_QD_STEP_S, ANSB_QD_OUT1S); }
     else { ANSB_QD_BOTH("ANSB_QS21", "ANSB_QS2G", ANSB_QD_TURN2, ANSB_QD_STEP_S, ANSB_QD_OUT1S); }
   } else if (K == 4) {
@@ -184,9 +197,10 @@ __device__ __noinline__ uint32_t decode_quads(
   // the rest in plain code, one symbol and one element store at a time
   for (; k < my_count; ++k) {
     const uint32_t ea = lds_u32(st), eb = SHORT ? 0u : lds_u32(st + 4u);
-    const uint32_t nb = ea & 31u;
-    const uint32_t q = SHORT ? (ea >> 8) & 0x3FFFu : NARROW ? eb : ea >> 8;
-    const uint32_t val = SHORT ? ea >> 24 : NARROW ? ea >> 16 : eb;
+    constexpr bool SHORT2 = SHORT && ES == 2;
+    const uint32_t nb = SHORT2 ? ea & 15u : ea & 31u;
+    const uint32_t q = SHORT2 ? (ea >> 4) & 0xFFFu : SHORT ? (ea >> 8) & 0x3FFFu : NARROW ? eb : ea >> 8;
+    const uint32_t val = SHORT2 ? ea >> 16 : SHORT ? ea >> 24 : NARROW ? ea >> 16 : eb;
     const uint32_t x = __funnelshift_l(w1, w0, bitpos);
     st = tab_abs + (__funnelshift_l(x, q, nb) << stride_log);
     stg_elem<ES>(out_lane + size_t(k >> 2) * turn_stride + (k & 3u) * ES, val);
