@@ -277,6 +277,52 @@ int ans_host_pack_layer(const uint8_t* h_symbols, uint64_t n_symbols,
                         uint8_t* h_stream_out, uint64_t stream_cap, uint64_t* h_stream_bytes_out,
                         uint64_t* h_sub_offsets_out, void* h_lane_meta_out, int n_threads);
 
+/* ------------------------------------------------------------------------------------
+ * The compress side on the device.  Off the inference path (the paper compresses offline,
+ * Section III-A); it serves training-time use, where the entropy of the quantised weights is
+ * wanted at every step (Section II-C, Eq. 3 regularises the entropy H_W of the weights) and
+ * the weights are already on the device.  All asynchronous on `stream`; every d_* buffer is
+ * the caller's.
+ * ------------------------------------------------------------------------------------ */
+
+/* Histogram of n_symbols bytes: d_counts[256] (zeroed by the call, then counted). */
+int ans_histogram_device(const uint8_t* d_symbols, uint64_t n_symbols, uint64_t* d_counts, void* stream);
+
+/*
+ * Entropy of a histogram over its first `alphabet` entries, in double precision:
+ * d_entropy_out[0] = -sum_s p_s log2 p_s (bits per symbol, p_s = count_s / total; 0 for an empty
+ * histogram), d_entropy_out[1] = that times the total (bits for the layer): the H_W of Eq. 3.
+ */
+int ans_entropy_device(const uint64_t* d_counts, int alphabet, double* d_entropy_out, void* stream);
+
+/*
+ * Histogram -> frequencies summing to 1 << table_log, the rule of ans_host_normalize_freqs
+ * (floor share, at least one state per symbol that occurs, largest remainders up, largest
+ * shares down, ties to the lower symbol), in integer arithmetic: d_freqs_out[256].
+ * Bit 1 of *d_status (optional, OR-ed) is set if the histogram is empty, has more symbols than
+ * states or more than 2^50 counts.
+ */
+int ans_normalize_freqs_device(const uint64_t* d_counts, int alphabet, int table_log, uint32_t* d_freqs_out,
+                               uint32_t* d_status, void* stream);
+
+/*
+ * Encode one layer on the device into the strips container (Section II-A: encoding follows a
+ * transition of the automaton and appends the bits that label it), byte for byte what
+ * ans_host_pack_layer writes for ANS_LAYOUT_STRIPS (the only layout this call takes).
+ *   d_symbols[n_symbols]; d_table: the layer's table from ans_build_decode_tables (it carries
+ *   the frequencies the encoder needs); d_stream_out: stream_cap bytes, 16-byte aligned, zeroed
+ *   and filled by the call (ans_host_pack_bound gives a sufficient stream_cap);
+ *   d_sub_offsets_out[n_sub + 1]: byte offsets, the last one the stream's size;
+ *   d_scratch: ans_encode_scratch_bytes(...) bytes, 256-byte aligned.
+ * *d_status (OR-ed): bit 2 = the stream did not fit stream_cap (what did not fit is not
+ * written), bit 4 = a symbol without a state in the table, or a lane longer than 65535 bits.
+ */
+int ans_encode_scratch_bytes(uint64_t n_symbols, uint32_t chunk_symbols, uint32_t lanes, size_t* h_bytes_out);
+int ans_encode_layer_device(const uint8_t* d_symbols, uint64_t n_symbols, const void* d_table, int table_log,
+                            uint32_t chunk_symbols, uint32_t lanes, int layout, uint8_t* d_stream_out,
+                            uint64_t stream_cap, uint64_t* d_sub_offsets_out, void* d_scratch,
+                            size_t d_scratch_bytes, uint32_t* d_status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,6 +27,8 @@ EXPORTS = [
     "ans_read_status", "ans_host_scratch_bytes", "ans_decode_dequant_host",
     "ans_host_normalize_freqs", "ans_host_pack_bound", "ans_host_pack_layer",
     "ans_noalloc_max_bytes", "ans_decode_dequant_host_noalloc",
+    "ans_histogram_device", "ans_entropy_device", "ans_normalize_freqs_device",
+    "ans_encode_scratch_bytes", "ans_encode_layer_device",
 ]
 
 
@@ -83,6 +85,11 @@ def lib():
         L.ans_host_normalize_freqs.argtypes = [vp, i32, i32, vp]
         L.ans_host_pack_bound.argtypes = [u64, u32, u32, i32, P(u64)]
         L.ans_host_pack_layer.argtypes = [vp, u64, vp, i32, i32, u32, u32, i32, vp, u64, P(u64), vp, vp, i32]
+        L.ans_histogram_device.argtypes = [vp, u64, vp, vp]
+        L.ans_entropy_device.argtypes = [vp, i32, vp, vp]
+        L.ans_normalize_freqs_device.argtypes = [vp, i32, i32, vp, vp, vp]
+        L.ans_encode_scratch_bytes.argtypes = [u64, u32, u32, P(sz)]
+        L.ans_encode_layer_device.argtypes = [vp, u64, vp, i32, u32, u32, i32, vp, u64, vp, vp, sz, vp, vp]
         _LIB = L
     return _LIB
 
@@ -222,3 +229,37 @@ def ans_host_pack_layer(symbols: np.ndarray, freqs: np.ndarray, alphabet: int, t
                                      ctypes.byref(used), offs.ctypes.data, meta.ctypes.data, n_threads),
            "ans_host_pack_layer")
     return stream[:used.value].copy(), offs, meta
+
+
+def ans_histogram_device(d_symbols: int, n_symbols: int, d_counts: int, stream: int = 0) -> None:
+    _check(lib().ans_histogram_device(d_symbols, n_symbols, d_counts, stream), "ans_histogram_device")
+
+
+def ans_entropy_device(d_counts: int, alphabet: int, d_entropy_out: int, stream: int = 0) -> None:
+    _check(lib().ans_entropy_device(d_counts, alphabet, d_entropy_out, stream), "ans_entropy_device")
+
+
+def ans_normalize_freqs_device(d_counts: int, alphabet: int, table_log: int, d_freqs_out: int, d_status: int = 0,
+                               stream: int = 0) -> None:
+    _check(lib().ans_normalize_freqs_device(d_counts, alphabet, table_log, d_freqs_out, d_status, stream),
+           "ans_normalize_freqs_device")
+
+
+def ans_encode_scratch_bytes(n_symbols: int, chunk_symbols: int, lanes: int) -> int:
+    out = ctypes.c_size_t()
+    _check(lib().ans_encode_scratch_bytes(n_symbols, chunk_symbols, lanes, ctypes.byref(out)), "ans_encode_scratch_bytes")
+    return out.value
+
+
+def ans_host_pack_bound(n_symbols: int, chunk_symbols: int, lanes: int, layout: int) -> int:
+    cap = ctypes.c_uint64()
+    _check(lib().ans_host_pack_bound(n_symbols, chunk_symbols, lanes, layout, ctypes.byref(cap)), "ans_host_pack_bound")
+    return cap.value
+
+
+def ans_encode_layer_device(d_symbols: int, n_symbols: int, d_table: int, table_log: int, chunk_symbols: int,
+                            lanes: int, layout: int, d_stream_out: int, stream_cap: int, d_sub_offsets_out: int,
+                            d_scratch: int, d_scratch_bytes: int, d_status: int, stream: int = 0) -> None:
+    _check(lib().ans_encode_layer_device(d_symbols, n_symbols, d_table, table_log, chunk_symbols, lanes, layout,
+                                         d_stream_out, stream_cap, d_sub_offsets_out, d_scratch, d_scratch_bytes,
+                                         d_status, stream), "ans_encode_layer_device")
