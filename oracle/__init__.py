@@ -61,6 +61,9 @@ def _lib():
         L.anso_pack_strips.argtypes = [vp, vp, i64, i64, i32, vp, u64, vp]
         L.anso_pack_strips.restype = i64
         L.anso_unpack_strips.argtypes = [vp, vp, vp, i64, i64, i32, i64, i64, vp]
+        L.anso_pack_channels.argtypes = [vp, vp, i64, i64, i32, i32, vp, u64, vp]
+        L.anso_pack_channels.restype = i64
+        L.anso_unpack_channels.argtypes = [vp, vp, vp, i64, i64, i32, i32, i64, i64, vp]
         L.anso_dequant_f32.argtypes = [vp, i64, i32, ctypes.c_float, vp]
         L.anso_dequant_f32.restype = None
         L.anso_dequant_bf16.argtypes = [vp, i64, i32, ctypes.c_float, vp]
@@ -76,7 +79,7 @@ def _p(a: np.ndarray):
     return a.ctypes.data
 
 
-INTERLEAVED, PRIVATE, QUADS, STRIPS = 0, 1, 2, 3
+INTERLEAVED, PRIVATE, QUADS, STRIPS, CHANNELS = 0, 1, 2, 3, 4
 
 
 class Table:
@@ -159,9 +162,9 @@ def decode_plain(T: Table, data, init: int, n: int, want_trace: bool = False):
 class Packed:
     """One layer in a container: stream bytes, per-sub-stream offsets, per-lane metadata."""
 
-    def __init__(self, layout, stream, sub_offsets, lane_meta, n, chunk, groups):
+    def __init__(self, layout, stream, sub_offsets, lane_meta, n, chunk, groups, piece=1):
         self.layout, self.stream, self.sub_offsets, self.lane_meta = layout, stream, sub_offsets, lane_meta
-        self.n, self.chunk, self.groups = n, chunk, groups
+        self.n, self.chunk, self.groups, self.piece = n, chunk, groups, piece
 
     @property
     def n_chunks(self):
@@ -176,7 +179,7 @@ class Packed:
         return int(self.stream.nbytes + self.sub_offsets.nbytes + self.lane_meta.nbytes)
 
 
-def pack(T: Table, symbols, chunk: int, groups: int = 1, layout: int = INTERLEAVED) -> Packed:
+def pack(T: Table, symbols, chunk: int, groups: int = 1, layout: int = INTERLEAVED, piece: int = 1) -> Packed:
     symbols = np.ascontiguousarray(symbols, dtype=np.uint8)
     n = symbols.size
     n_chunks = (n + chunk - 1) // chunk
@@ -189,7 +192,12 @@ def pack(T: Table, symbols, chunk: int, groups: int = 1, layout: int = INTERLEAV
     stream = np.zeros(cap, dtype=np.uint8)
     offs = np.zeros(n_sub + 1, dtype=np.uint64)
     lib = _lib()
-    if layout == STRIPS:
+    if layout == CHANNELS:
+        cap = n_sub * (64 + 4 * (chunk // (32 * groups) + 1) * T.R + 36) + 64
+        stream = np.zeros(cap, dtype=np.uint8)
+        meta = np.zeros((n_sub, 0), dtype=np.uint32)
+        total = lib.anso_pack_channels(T.ptr, _p(symbols), n, chunk, groups, piece, _p(stream), cap, _p(offs))
+    elif layout == STRIPS:
         meta = np.zeros((n_sub, 0), dtype=np.uint32)       # this container has no per-lane array
         total = lib.anso_pack_strips(T.ptr, _p(symbols), n, chunk, groups, _p(stream), cap, _p(offs))
     elif layout == INTERLEAVED:
@@ -201,7 +209,7 @@ def pack(T: Table, symbols, chunk: int, groups: int = 1, layout: int = INTERLEAV
         total = fn(T.ptr, _p(symbols), n, chunk, groups, _p(stream), cap, _p(offs), _p(meta))
     if total < 0:
         raise OracleError(total, "pack")
-    return Packed(layout, stream[:total].copy(), offs, meta, n, chunk, groups)
+    return Packed(layout, stream[:total].copy(), offs, meta, n, chunk, groups, piece)
 
 
 def unpack(T: Table, P: Packed, threads: int = 1, chunk_range=None):
@@ -209,7 +217,11 @@ def unpack(T: Table, P: Packed, threads: int = 1, chunk_range=None):
     out = np.zeros(max(P.n, 1), dtype=np.uint8)
     lib = _lib()
     lo, hi = chunk_range if chunk_range is not None else (0, P.n_chunks)
-    if P.layout == STRIPS:
+    if P.layout == CHANNELS:
+        def work(rng):
+            return lib.anso_unpack_channels(T.ptr, _p(P.stream), _p(P.sub_offsets), P.n, P.chunk, P.groups, P.piece,
+                                            rng[0], rng[1], _p(out))
+    elif P.layout == STRIPS:
         def work(rng):
             return lib.anso_unpack_strips(T.ptr, _p(P.stream), _p(P.sub_offsets), P.n, P.chunk, P.groups,
                                             rng[0], rng[1], _p(out))

@@ -34,6 +34,9 @@
  *                      round-robin to its lanes; a lane's bits begin with its
  *                      initial state; a sub-stream carries its lanes' bit
  *                      lengths and their strings back to back.
+ *       "channels":    the paper's grouping: pieces of H*W symbols dealt to the
+ *                      lanes, so that a lane is an input channel of a layer
+ *                      stored O x I x H x W; bytes laid out as in "strips".
  *   - frequency normalisation (largest-remainder, every present symbol >= 1).
  *
  * Pins (see tests): hand-enumerated state traces, table tiling invariants,
@@ -687,6 +690,118 @@ int anso_unpack_strips(const anso_table* T, const uint8_t* stream, const uint64_
         start += len;
       }
       /* the sub-stream holds exactly the header, the words its bits need, and the pad */
+      uint64_t want = ANSO_STRIP_HEADER + ((start + 31) / 32) * 4;
+      want = (want + 15) / 16 * 16;
+      if (want != extent) rc = ANSO_ERR_CORRUPT;
+    }
+  }
+  return rc;
+}
+
+/*
+ * Channels container: the paper's own grouping (Section III-B: the weights of a
+ * layer are split into streams by INPUT CHANNEL, so that the streams feed the
+ * input-channel-parallel multipliers side by side).  For a convolution tensor
+ * stored output-channel major, O x I x H x W, the weights of input channel c are
+ * O pieces of E = H*W consecutive symbols, one piece every I*E symbols.  Hence:
+ *   - a chunk's symbols come in pieces of E consecutive symbols; piece j of the
+ *     chunk belongs to lane j mod W (W = 32*G lanes) as that lane's
+ *     (j div W)-th piece.  With one chunk per layer and W = I, lane c is input
+ *     channel c.  C and n must be multiples of W*E, so every lane of a chunk
+ *     owns the same number of whole pieces.
+ *   - sub-stream g holds lanes 32g .. 32g+31; its bytes are laid out exactly as
+ *     in the strips container (32 lengths, then the strings, each headed by its
+ *     initial state, most significant bit first).
+ */
+static int64_t channels_position(int W, int E, int lambda, int64_t t) {
+  return ((t / E) * W + lambda) * E + t % E;    /* chunk-relative place of lane lambda's t-th symbol */
+}
+
+int64_t anso_pack_channels(const anso_table* T, const uint8_t* symbols, int64_t n,
+                           int64_t C, int G, int E, uint8_t* stream, uint64_t cap_bytes,
+                           uint64_t* sub_offsets) {
+  if (!T || C < 1 || G < 1 || E < 1 || n < 0) return ANSO_ERR_ARG;
+  const int W = 32 * G;
+  if (C % ((int64_t)W * E) || n % ((int64_t)W * E)) return ANSO_ERR_ARG;
+  const int64_t n_chunks = (n + C - 1) / C;
+  const int64_t max_lane = C / W;
+  uint8_t* mine = (uint8_t*)malloc((size_t)max_lane);
+  uint8_t* fnb = (uint8_t*)malloc((size_t)max_lane);
+  uint16_t* fval = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)max_lane);
+  uint64_t off = 0;
+  int64_t rc = ANSO_OK;
+  for (int64_t c = 0; c < n_chunks && rc >= 0; ++c) {
+    const uint8_t* cs = symbols + c * C;
+    const int64_t nc = (n - c * C) < C ? (n - c * C) : C;
+    const int64_t cnt = nc / W;                        /* symbols of every lane of this chunk */
+    for (int g = 0; g < G && rc >= 0; ++g) {
+      const int64_t sub = c * G + g;
+      sub_offsets[sub] = off;
+      const uint64_t worst = ANSO_STRIP_HEADER + (uint64_t)(32 * (cnt + 1) * T->R + 7) / 8 + 20;
+      if (off + worst > cap_bytes) { rc = ANSO_ERR_SPACE; break; }
+      memset(stream + off, 0, (size_t)worst);
+      uint8_t* body = stream + off + ANSO_STRIP_HEADER;
+      uint64_t pos = 0;
+      for (int k = 0; k < 32; ++k) {
+        const uint64_t pos0 = pos;
+        if (cnt > 0) {
+          for (int64_t t = 0; t < cnt; ++t) mine[t] = cs[channels_position(W, E, 32 * g + k, t)];
+          int init = anso_encode_lane(T, mine, cnt, 1, fnb, fval);
+          if (init < 0) { rc = init; break; }
+          put_bits_msb(body, &pos, (uint32_t)init, T->R);
+          for (int64_t t = 0; t < cnt; ++t) put_bits_msb(body, &pos, fval[t], fnb[t]);
+        }
+        const uint64_t len = pos - pos0;
+        if (len > 0xFFFF) { rc = ANSO_ERR_ARG; break; }   /* a lane's length must fit its 16-bit field */
+        stream[off + 2 * k] = (uint8_t)(len & 0xFF);
+        stream[off + 2 * k + 1] = (uint8_t)(len >> 8);
+      }
+      if (rc < 0) break;
+      off += ANSO_STRIP_HEADER + ((pos + 31) / 32) * 4;
+      while (off % 16) ++off;
+    }
+  }
+  if (rc >= 0) sub_offsets[n_chunks * G] = off;
+  free(mine); free(fnb); free(fval);
+  return rc < 0 ? rc : (int64_t)off;
+}
+
+int anso_unpack_channels(const anso_table* T, const uint8_t* stream, const uint64_t* sub_offsets,
+                         int64_t n, int64_t C, int G, int E,
+                         int64_t chunk_begin, int64_t chunk_end, uint8_t* out) {
+  const int W = 32 * G;
+  if (E < 1 || C % ((int64_t)W * E) || n % ((int64_t)W * E)) return ANSO_ERR_ARG;
+  int rc = ANSO_OK;
+  for (int64_t c = chunk_begin; c < chunk_end; ++c) {
+    uint8_t* co = out + c * C;
+    const int64_t nc = (n - c * C) < C ? (n - c * C) : C;
+    const int64_t cnt = nc / W;
+    for (int g = 0; g < G; ++g) {
+      const int64_t sub = c * G + g;
+      const uint8_t* p = stream + sub_offsets[sub];
+      const uint64_t extent = sub_offsets[sub + 1] - sub_offsets[sub];
+      if (extent < ANSO_STRIP_HEADER) { rc = ANSO_ERR_CORRUPT; continue; }
+      const uint8_t* body = p + ANSO_STRIP_HEADER;
+      const uint64_t body_bytes = extent - ANSO_STRIP_HEADER;
+      uint64_t start = 0;
+      for (int k = 0; k < 32; ++k) {
+        const uint64_t len = (uint64_t)p[2 * k] | ((uint64_t)p[2 * k + 1] << 8);
+        uint64_t pos = start;
+        if (cnt > 0) {
+          uint32_t i = get_bits_msb(body, body_bytes, pos, T->R);
+          pos += (uint64_t)T->R;
+          for (int64_t t = 0; t < cnt; ++t) {
+            co[channels_position(W, E, 32 * g + k, t)] = T->sym[i];
+            const int nb = T->nb[i];
+            const uint32_t v = get_bits_msb(body, body_bytes, pos, nb);
+            pos += (uint64_t)nb;
+            i = T->newx[i] + v;
+          }
+          if (i != 0) rc = ANSO_ERR_CORRUPT;
+        }
+        if (pos - start != len) rc = ANSO_ERR_CORRUPT;
+        start += len;
+      }
       uint64_t want = ANSO_STRIP_HEADER + ((start + 31) / 32) * 4;
       want = (want + 15) / 16 * 16;
       if (want != extent) rc = ANSO_ERR_CORRUPT;

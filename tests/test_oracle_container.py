@@ -398,3 +398,66 @@ def test_strips_overhead_per_lane_is_the_state_and_a_length():
         pad += (b1 - b0 - 64) * 8 - body
     assert P.stream.size * 8 == bits + pad
     assert P.total_bytes() < oracle.pack(T, msg, C, G, oracle.QUADS).total_bytes()
+
+
+# ---- channels container (the paper's grouping by input channel, Section III-B) ------------------
+@pytest.mark.parametrize("O,I,H,W", [(8, 64, 3, 3), (5, 32, 1, 1), (16, 96, 7, 7), (3, 128, 3, 3), (64, 64, 1, 1)])
+def test_channels_lane_is_an_input_channel(O, I, H, W):
+    """A conv tensor stored O x I x H x W as one chunk with I lanes and pieces of H*W symbols:
+    lane c's string is the plain one-lane coder's state and fields for tensor[:, c, :, :] read in
+    memory order; the sub-stream bytes are built here independently (lengths, strings from the
+    top bit of 32-bit little-endian words, zero padding to 16 bytes)."""
+    rng = np.random.default_rng(O * I + H)
+    R = 9
+    w = _source(rng, O * I * H * W).reshape(O, I, H, W)
+    T = _table(w.ravel(), 15, R)
+    P = oracle.pack(T, w.ravel(), w.size, I // 32, oracle.CHANNELS, piece=H * W)
+    assert P.n_sub == I // 32 and P.lane_meta.size == 0
+    for g in range(I // 32):
+        lens, bits = [], ""
+        for k in range(32):
+            mine = np.ascontiguousarray(w[:, 32 * g + k]).ravel()
+            init, nb, val = oracle.encode_lane_fields(T, mine)
+            s = format(init, "b").zfill(R) + "".join(format(int(v), "b").zfill(int(b)) if b else "" for b, v in zip(nb, val))
+            lens.append(len(s))
+            bits += s
+        words = (len(bits) + 31) // 32
+        bits = bits.ljust(32 * words, "0")
+        want = b"".join(int(x).to_bytes(2, "little") for x in lens)
+        want += b"".join(int(bits[32 * i:32 * i + 32], 2).to_bytes(4, "little") for i in range(words))
+        want += bytes(-len(want) % 16)
+        assert bytes(P.stream[int(P.sub_offsets[g]):int(P.sub_offsets[g + 1])]) == want
+    out, rc = oracle.unpack(T, P)
+    assert rc == oracle.OK and (out == w.ravel()).all()
+
+
+def test_channels_with_pieces_of_one_symbol_and_32_lanes_is_the_strips_container():
+    rng = np.random.default_rng(31)
+    msg = _source(rng, 32 * 300)
+    T = _table(msg, 15, 10)
+    a = oracle.pack(T, msg, 3200, 1, oracle.CHANNELS, piece=1)
+    b = oracle.pack(T, msg, 3200, 1, oracle.STRIPS)
+    assert bytes(a.stream) == bytes(b.stream) and (a.sub_offsets == b.sub_offsets).all()
+
+
+def test_channels_chunks_threads_sizes_and_corruption():
+    rng = np.random.default_rng(33)
+    O, I, E = 24, 64, 9
+    w = _source(rng, O * I * E)
+    T = _table(w, 15, 11)
+    for C in (w.size, 8 * I * E, I * E):                   # one chunk per layer, or chunks of whole rows
+        P = oracle.pack(T, w, C, I // 32, oracle.CHANNELS, piece=E)
+        for th in (1, 3):
+            out, rc = oracle.unpack(T, P, threads=th)
+            assert rc == oracle.OK and (out == w).all()
+    for C, n, E2 in ((w.size + 1, w.size, 9), (w.size, w.size - 64, 9), (w.size, w.size, 7)):
+        with pytest.raises(oracle.OracleError):            # sizes that are no multiple of lanes * piece
+            oracle.pack(T, w[:n], C, I // 32, oracle.CHANNELS, piece=E2)
+    P = oracle.pack(T, w, w.size, I // 32, oracle.CHANNELS, piece=E)
+    flagged = 0
+    positions = list(range(3, P.stream.size, 131))
+    for pos in positions:
+        Q = oracle.Packed(P.layout, P.stream.copy(), P.sub_offsets, P.lane_meta, P.n, P.chunk, P.groups, P.piece)
+        Q.stream[pos] ^= 0x5A
+        flagged += (oracle.unpack(T, Q)[1] == oracle.ERR_CORRUPT)
+    assert flagged > len(positions) // 2
