@@ -303,21 +303,22 @@ def build_case(ans, args, workload, layout_name, lanes, table_log=0, chunk=0, lo
     layout = getattr(ans, LAYOUT_IDS[layout_name])
     cores = os.cpu_count() or 1
     if by_channel:
-        # the paper's own grouping (Section III-B): one chunk per layer, one lane per input channel,
-        # weights stored channels-last so that lane c carries input channel c; layers whose input
-        # channels are no multiple of 32 (the first conv, which the paper leaves uncompressed) are left out
+        # the paper's own grouping (Section III-B): one chunk per layer, one lane per input channel of the
+        # tensor as stored (O x I x H x W), pieces of H * W symbols; layers whose input channels are no
+        # multiple of 32 (the first conv, which the paper leaves uncompressed) are left out
         import dataclasses
         specs = [dataclasses.replace(sp, chunk_symbols=sp.n) for sp in specs
                  if len(sp.shape) == 4 and sp.shape[1] % 32 == 0 and sp.shape[1] <= 2048]
+        layout = ans.ANS_LAYOUT_CHANNELS
 
     def prep(spec):
         sym = sg.draw_symbols(spec, threads=max(1, cores // 4))
-        ln = lanes
+        ln, piece = lanes, 1
         if by_channel:
-            sym = np.ascontiguousarray(sym.reshape(spec.shape).transpose(0, 2, 3, 1)).ravel()
-            ln = spec.shape[1]
+            ln, piece = spec.shape[1], spec.shape[2] * spec.shape[3]
         pl = pack_layer(sym, spec.alphabet, spec.table_log, spec.chunk_symbols, ln, layout, spec.bitwidth,
-                        spec.zero_point, spec.scale, ans.DTYPES[spec.out_dtype], n_threads=max(1, cores // 2))
+                        spec.zero_point, spec.scale, ans.DTYPES[spec.out_dtype], n_threads=max(1, cores // 2),
+                        piece_symbols=piece)
         return sym, pl
 
     with ThreadPoolExecutor(4) as ex:
@@ -464,7 +465,7 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": dts[0] if len(dts) == 1 else "mixed", "data": "synthetic",
         "config": {"workload": WORKLOAD_TEXT[args.workload], "name": args.workload, "layout": args.layout,
-                   "lanes": "one per input channel" if by_channel else args.lanes,
+                   "lanes": "one per input channel (channels container)" if by_channel else args.lanes,
                    "grouping": args.grouping, "table_log": layers[0].table_log, "chunk_symbols": layers[0].chunk_symbols,
                    "layers": len(layers), "weights": n_w, "out_dtype": head_specs[0].out_dtype,
                    "arithmetic": "integer decode, one fp32 multiply per weight, round-to-nearest-even to the output type",

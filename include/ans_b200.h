@@ -65,6 +65,16 @@
  *       without gaps, filling 32-bit little-endian words from the most significant bit down,
  *       zero-padded to a multiple of 16 bytes.  There is no per-lane array: d_lane_meta is
  *       ignored and may be NULL.
+ *     ANS_LAYOUT_CHANNELS: the paper's own grouping (Section III-B: a layer's weights are split
+ *       into streams by input channel).  A chunk's symbols come in pieces of `piece_symbols`
+ *       consecutive symbols; piece j of the chunk is the (j / lanes)-th piece of lane j % lanes.
+ *       For a convolution tensor stored O x I x H x W, with piece_symbols = H * W, lanes = I
+ *       and one chunk per layer (chunk_symbols = n_symbols), lane c carries input channel c and
+ *       the decoded tensor comes out in its own O x I x H x W order.  chunk_symbols and
+ *       n_symbols must be multiples of lanes * piece_symbols; a lane owns at most 32768
+ *       symbols per chunk and its string at most 65535 bits; piece_symbols * element size of
+ *       the output at most 128 bytes (an 8 x 8 kernel in bf16).  Sub-stream g holds lanes
+ *       32 g .. 32 g + 31; its bytes are laid out as for ANS_LAYOUT_STRIPS; no d_lane_meta.
  */
 #ifndef ANS_B200_H
 #define ANS_B200_H
@@ -92,11 +102,14 @@ extern "C" {
 #define ANS_LAYOUT_PRIVATE     1
 #define ANS_LAYOUT_QUADS       2
 #define ANS_LAYOUT_STRIPS      3
+#define ANS_LAYOUT_CHANNELS    4
 
 #define ANS_MAX_TABLE_LOG 14
 #define ANS_MAX_LANES     2048   /* lanes per chunk: any multiple of 32 up to this */
 #define ANS_MAX_ALPHABET  256
 #define ANS_MAX_STRIP_LANE_SYMBOLS 4096   /* ANS_LAYOUT_STRIPS: chunk_symbols / lanes at most */
+#define ANS_MAX_CHANNEL_LANE_SYMBOLS 32768 /* ANS_LAYOUT_CHANNELS: chunk_symbols / lanes at most */
+#define ANS_MAX_PIECE_SYMBOLS 127         /* ANS_LAYOUT_CHANNELS: piece_symbols at most */
 
 /* bits of the device status word (0 = every stream sound) */
 #define ANS_STATUS_BAD_FINAL_STATE 1u   /* a lane did not end in state index 0          */
@@ -130,6 +143,9 @@ typedef struct ans_layer_desc {
   uint32_t        work_begin;     /* written by ans_plan_batch: first work item of the layer */
   uint32_t        work_count;     /* written by ans_plan_batch: the layer's work items (a work
                                      item is a group of up to 4 consecutive sub-streams)     */
+  uint32_t        piece_symbols;  /* ANS_LAYOUT_CHANNELS: symbols of a piece (H * W of the conv
+                                     kernel), 1 .. 127; ignored by the other layouts           */
+  uint32_t        reserved;       /* 0 */
 } ans_layer_desc;
 
 /* Library version (major*100 + minor). */
@@ -257,7 +273,7 @@ int ans_decode_dequant_host_noalloc(const ans_layer_desc* h_desc, const uint32_t
 int ans_host_normalize_freqs(const uint64_t* h_counts, int alphabet, int table_log,
                              uint32_t* h_freqs_out);
 
-/* Upper bound of the stream bytes ans_host_pack_layer can produce. */
+/* Upper bound of the stream bytes ans_host_pack_layer / ans_host_pack_channels can produce. */
 int ans_host_pack_bound(uint64_t n_symbols, uint32_t chunk_symbols, uint32_t lanes,
                         int layout, uint64_t* h_bytes_out);
 
@@ -276,6 +292,17 @@ int ans_host_pack_layer(const uint8_t* h_symbols, uint64_t n_symbols,
                         uint32_t chunk_symbols, uint32_t lanes, int layout,
                         uint8_t* h_stream_out, uint64_t stream_cap, uint64_t* h_stream_bytes_out,
                         uint64_t* h_sub_offsets_out, void* h_lane_meta_out, int n_threads);
+
+/*
+ * The same for ANS_LAYOUT_CHANNELS (Section III-B: one stream per input channel), which needs
+ * the piece size: h_symbols is the tensor as stored (O x I x H x W), piece_symbols = H * W,
+ * lanes = I, chunk_symbols = n_symbols for one chunk per layer.  No lane metadata is written.
+ */
+int ans_host_pack_channels(const uint8_t* h_symbols, uint64_t n_symbols,
+                           const uint32_t* h_freqs, int alphabet, int table_log,
+                           uint32_t chunk_symbols, uint32_t lanes, uint32_t piece_symbols,
+                           uint8_t* h_stream_out, uint64_t stream_cap, uint64_t* h_stream_bytes_out,
+                           uint64_t* h_sub_offsets_out, int n_threads);
 
 /* ------------------------------------------------------------------------------------
  * The compress side on the device.  Off the inference path (the paper compresses offline,

@@ -17,7 +17,7 @@ ANS_OK = 0
 ANS_ERR_INVALID_ARG, ANS_ERR_BAD_FREQS, ANS_ERR_UNSUPPORTED = -1, -2, -3
 ANS_ERR_BUFFER_TOO_SMALL, ANS_ERR_CUDA, ANS_ERR_CORRUPT = -4, -5, -6
 ANS_U8, ANS_F32, ANS_BF16 = 0, 1, 2
-ANS_LAYOUT_INTERLEAVED, ANS_LAYOUT_PRIVATE, ANS_LAYOUT_QUADS, ANS_LAYOUT_STRIPS = 0, 1, 2, 3
+ANS_LAYOUT_INTERLEAVED, ANS_LAYOUT_PRIVATE, ANS_LAYOUT_QUADS, ANS_LAYOUT_STRIPS, ANS_LAYOUT_CHANNELS = 0, 1, 2, 3, 4
 DTYPES = {"u8": ANS_U8, "f32": ANS_F32, "bf16": ANS_BF16}
 ELEM_SIZE = {ANS_U8: 1, ANS_F32: 4, ANS_BF16: 2}
 
@@ -25,7 +25,7 @@ EXPORTS = [
     "ans_version", "ans_strerror", "ans_last_cuda_error", "ans_table_bytes", "ans_build_decode_tables",
     "ans_plan_batch", "ans_decode_layer", "ans_decode_dequant", "ans_decode_dequant_batch",
     "ans_read_status", "ans_host_scratch_bytes", "ans_decode_dequant_host",
-    "ans_host_normalize_freqs", "ans_host_pack_bound", "ans_host_pack_layer",
+    "ans_host_normalize_freqs", "ans_host_pack_bound", "ans_host_pack_layer", "ans_host_pack_channels",
     "ans_noalloc_max_bytes", "ans_decode_dequant_host_noalloc",
     "ans_histogram_device", "ans_entropy_device", "ans_normalize_freqs_device",
     "ans_encode_scratch_bytes", "ans_encode_layer_device",
@@ -40,6 +40,7 @@ class ans_layer_desc(ctypes.Structure):
         ("table_log", ctypes.c_int32), ("bitwidth", ctypes.c_int32), ("zero_point", ctypes.c_int32),
         ("scale", ctypes.c_float), ("out_dtype", ctypes.c_int32), ("layout", ctypes.c_int32),
         ("work_begin", ctypes.c_uint32), ("work_count", ctypes.c_uint32),
+        ("piece_symbols", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
     ]
 
 
@@ -85,6 +86,7 @@ def lib():
         L.ans_host_normalize_freqs.argtypes = [vp, i32, i32, vp]
         L.ans_host_pack_bound.argtypes = [u64, u32, u32, i32, P(u64)]
         L.ans_host_pack_layer.argtypes = [vp, u64, vp, i32, i32, u32, u32, i32, vp, u64, P(u64), vp, vp, i32]
+        L.ans_host_pack_channels.argtypes = [vp, u64, vp, i32, i32, u32, u32, u32, vp, u64, P(u64), vp, i32]
         L.ans_histogram_device.argtypes = [vp, u64, vp, vp]
         L.ans_entropy_device.argtypes = [vp, i32, vp, vp]
         L.ans_normalize_freqs_device.argtypes = [vp, i32, i32, vp, vp, vp]
@@ -263,3 +265,20 @@ def ans_encode_layer_device(d_symbols: int, n_symbols: int, d_table: int, table_
     _check(lib().ans_encode_layer_device(d_symbols, n_symbols, d_table, table_log, chunk_symbols, lanes, layout,
                                          d_stream_out, stream_cap, d_sub_offsets_out, d_scratch, d_scratch_bytes,
                                          d_status, stream), "ans_encode_layer_device")
+
+
+def ans_host_pack_channels(symbols: np.ndarray, freqs: np.ndarray, alphabet: int, table_log: int,
+                           chunk_symbols: int, lanes: int, piece_symbols: int, n_threads: int = 0):
+    """ANS_LAYOUT_CHANNELS: returns (stream uint8[], sub_offsets uint64[n_sub+1], empty lane_meta)."""
+    sym = np.ascontiguousarray(symbols, dtype=np.uint8)
+    f = np.ascontiguousarray(freqs, dtype=np.uint32)
+    assert f.size == 256
+    cap = ans_host_pack_bound(sym.size, chunk_symbols, lanes, ANS_LAYOUT_CHANNELS)
+    n_sub = -(-sym.size // chunk_symbols) * (lanes // 32)
+    stream = np.empty(cap, dtype=np.uint8)
+    offs = np.zeros(n_sub + 1, dtype=np.uint64)
+    used = ctypes.c_uint64()
+    _check(lib().ans_host_pack_channels(sym.ctypes.data, sym.size, f.ctypes.data, alphabet, table_log, chunk_symbols,
+                                        lanes, piece_symbols, stream.ctypes.data, cap, ctypes.byref(used),
+                                        offs.ctypes.data, n_threads), "ans_host_pack_channels")
+    return stream[:used.value].copy(), offs, np.zeros((n_sub, 0), dtype=np.uint32)

@@ -19,6 +19,13 @@ int validate_desc(const ans_layer_desc& d, bool need_out) {
   if (d.layout == ANS_LAYOUT_STRIPS &&
       (d.chunk_symbols % d.lanes || d.chunk_symbols / d.lanes > ANS_MAX_STRIP_LANE_SYMBOLS))
     return ANS_ERR_UNSUPPORTED;
+  if (d.layout == ANS_LAYOUT_CHANNELS) {
+    if (d.piece_symbols < 1 || d.piece_symbols > ANS_MAX_PIECE_SYMBOLS) return ANS_ERR_UNSUPPORTED;
+    const uint64_t unit = uint64_t(d.lanes) * d.piece_symbols;
+    if (d.chunk_symbols % unit || d.n_symbols % unit || d.chunk_symbols / d.lanes > ANS_MAX_CHANNEL_LANE_SYMBOLS)
+      return ANS_ERR_UNSUPPORTED;
+    if (d.piece_symbols * elem_size(d.out_dtype) > 128) return ANS_ERR_UNSUPPORTED;
+  }
   if (d.bitwidth < 1 || d.bitwidth > 8) return ANS_ERR_INVALID_ARG;
   if (d.zero_point < 0 || d.zero_point >= (1 << d.bitwidth)) return ANS_ERR_INVALID_ARG;
   if (!std::isfinite(d.scale)) return ANS_ERR_INVALID_ARG;

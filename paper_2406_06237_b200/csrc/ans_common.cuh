@@ -66,8 +66,8 @@ inline uint64_t granules_of(const ans_layer_desc& d) { return (subs_of(d) + kGra
 inline size_t elem_size(int dtype) { return dtype == ANS_U8 ? 1 : dtype == ANS_F32 ? 4 : 2; }
 // bytes of d_lane_meta per lane (the strips layout has no such array)
 inline size_t lane_meta_size(int layout) {
-  return layout == ANS_LAYOUT_INTERLEAVED ? 2 : layout == ANS_LAYOUT_STRIPS ? 0 : 4;
+  return layout == ANS_LAYOUT_INTERLEAVED ? 2 : (layout == ANS_LAYOUT_STRIPS || layout == ANS_LAYOUT_CHANNELS) ? 0 : 4;
 }
-inline bool known_layout(int layout) { return layout >= ANS_LAYOUT_INTERLEAVED && layout <= ANS_LAYOUT_STRIPS; }
+inline bool known_layout(int layout) { return layout >= ANS_LAYOUT_INTERLEAVED && layout <= ANS_LAYOUT_CHANNELS; }
 
 }  // namespace ansb

@@ -366,7 +366,8 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   }
   if (total == 0) return ANS_OK;
   if (total > 0xFFFFFFFFull) return ANS_ERR_UNSUPPORTED;
-  if (layout == ANS_LAYOUT_STRIPS) return launch_strips(h_descs, n_layers, d_symbols_override, d_status, st);
+  if (layout == ANS_LAYOUT_STRIPS || layout == ANS_LAYOUT_CHANNELS)
+    return launch_strips(h_descs, n_layers, d_symbols_override, d_status, st);
 
   LaunchArgs a{};
   a.d_descs = d_descs;
@@ -550,6 +551,6 @@ ANS_EXPORT int ans_decode_dequant_batch(const ans_layer_desc* d_descs, const ans
                                         int n_layers, uint32_t* d_status, void* stream) {
   if (n_layers < 0 || !d_status) return ANS_ERR_INVALID_ARG;
   if (n_layers == 0) return ANS_OK;
-  if (!h_descs || (!d_descs && h_descs[0].layout != ANS_LAYOUT_STRIPS)) return ANS_ERR_INVALID_ARG;
+  if (!h_descs || (!d_descs && lane_meta_size(h_descs[0].layout))) return ANS_ERR_INVALID_ARG;
   return launch(d_descs, h_descs, n_layers, nullptr, d_status, static_cast<cudaStream_t>(stream));
 }

@@ -13,6 +13,11 @@
 // memory, pre-filled with the dominant symbol's value; a lane only writes the symbol that ends a
 // run; a full window is contiguous in the output and leaves in 16-byte stores.
 //
+// The channels container (Section III-B: one stream per input channel of a tensor stored
+// O x I x H x W) is walked by the same kernel: a row of the window is then one piece (H * W
+// symbols) of every lane, rows lie a whole tensor row apart in the output, and a window leaves in
+// one bulk store per row.
+//
 // One CTA = one work item of the batch plan (up to four consecutive sub-streams of ONE layer,
 // a warp each).  Up to kStripParamLayers layer records travel in the kernel parameters, so a
 // CTA reaches its layer without a trip to memory; the trips that remain are the sub-stream's
@@ -42,6 +47,7 @@ struct StripLayer {                // what the kernel needs of one layer, 64 byt
   uint32_t n_sub;
   float scale;
   uint32_t packed;                 // zero_point [7:0] | table_log [11:8] | bitwidth [15:12] | dtype [17:16] | lanes / 32 [24:18]
+                                   // | piece_symbols [31:25] (channels container; 0: strips)
 };
 
 struct StripArgs {
@@ -89,12 +95,12 @@ __device__ __forceinline__ uint32_t to_strip_entry_short(uint32_t g, uint32_t va
 // One look-up.  %6: the lane's next position; zn: the position of the symbol that ends the run;
 // the lane takes the step only if that position is inside the window (and the lane), else it
 // keeps its state and waits.
-#define ANSB_SP_STEP_N(STS_)                                      \
+#define ANSB_SP_STEP_N(STS_, ADDR_)                                      \
   "ld.shared.v2.u32 {ea, eb}, [%0];\n\t"                          \
   "bfe.u32 av, ea, 8, 4;\n\t"                                     \
   "add.u32 zn, %6, av;\n\t"                                       \
   "setp.lt.u32 act, zn, %10;\n\t"                                 \
-  "mad.lo.u32 ad, zn, %13, %9;\n\t"                               \
+  ADDR_                                                           \
   "shr.u32 vv, ea, 16;\n\t"                                       \
   "@act " STS_ " [ad], vv;\n\t"                                   \
   "@act shf.l.wrap.b32 tt, x, eb, ea;\n\t"                        \
@@ -102,12 +108,12 @@ __device__ __forceinline__ uint32_t to_strip_entry_short(uint32_t g, uint32_t va
   "@act mad.lo.u32 %0, tt, %8, %7;\n\t"                           \
   "@act mad.lo.u32 %1, ea, %11, %1;\n\t"                          \
   "@act add.u32 %6, zn, 1;\n\t"
-#define ANSB_SP_STEP_S(STS_)                                      \
+#define ANSB_SP_STEP_S(STS_, ADDR_)                                      \
   "ld.shared.u32 ea, [%0];\n\t"                                   \
   "bfe.u32 av, ea, 20, 4;\n\t"                                    \
   "add.u32 zn, %6, av;\n\t"                                       \
   "setp.lt.u32 act, zn, %10;\n\t"                                 \
-  "mad.lo.u32 ad, zn, %13, %9;\n\t"                               \
+  ADDR_                                                           \
   "@act " STS_ " [ad], ea;\n\t"                                   \
   "bfe.u32 eb, ea, 16, 4;\n\t"                                    \
   "shr.u32 av, ea, 24;\n\t"                                       \
@@ -116,12 +122,12 @@ __device__ __forceinline__ uint32_t to_strip_entry_short(uint32_t g, uint32_t va
   "@act mad.lo.u32 %0, tt, %8, %7;\n\t"                           \
   "@act add.u32 %1, %1, eb;\n\t"                                  \
   "@act add.u32 %6, zn, 1;\n\t"
-#define ANSB_SP_STEP_W(STS_)                                      \
+#define ANSB_SP_STEP_W(STS_, ADDR_)                                      \
   "ld.shared.v2.u32 {ea, eb}, [%0];\n\t"                          \
   "bfe.u32 av, ea, 8, 4;\n\t"                                     \
   "add.u32 zn, %6, av;\n\t"                                       \
   "setp.lt.u32 act, zn, %10;\n\t"                                 \
-  "mad.lo.u32 ad, zn, %13, %9;\n\t"                               \
+  ADDR_                                                           \
   "shr.u32 vv, ea, 16;\n\t"                                       \
   "@act " STS_ " [ad], eb;\n\t"                                   \
   "@act shf.l.wrap.b32 tt, x, vv, ea;\n\t"                        \
@@ -129,6 +135,15 @@ __device__ __forceinline__ uint32_t to_strip_entry_short(uint32_t g, uint32_t va
   "@act mad.lo.u32 %0, tt, %8, %7;\n\t"                           \
   "@act mad.lo.u32 %1, ea, %11, %1;\n\t"                          \
   "@act add.u32 %6, zn, 1;\n\t"
+
+// where the symbol at position zn goes in the window.  Strips: a row is one symbol of every lane.
+// Channels: a row is one piece of E symbols of every lane; zn / E by a multiplication (%15 =
+// 2^32 / E rounded up, exact for positions below 2^32 / E), %16 = 31 * E * ES.
+#define ANSB_SP_ADDR_STRIPS "mad.lo.u32 ad, zn, %13, %9;\n\t"
+#define ANSB_SP_ADDR_PIECES                                       \
+  "mul.hi.u32 tt, zn, %15;\n\t"                                   \
+  "mad.lo.u32 ad, tt, %16, %9;\n\t"                               \
+  "mad.lo.u32 ad, zn, %14, ad;\n\t"
 
 // The walk of one window, entirely in PTX (loop included).  Groups of K look-ups share one
 // 32-bit extract of the bit window and one refill check: K = 4 when no state of the table takes
@@ -138,12 +153,12 @@ __device__ __forceinline__ uint32_t to_strip_entry_short(uint32_t g, uint32_t va
 //   abase: window address of the lane's first symbol, minus the window's first row (a row holds one
 //          symbol of every lane)
 //   lim: first position the lane may not write (end of the window, or of the lane)
-template <int ES, int K, bool SHORT>
+template <int ES, int K, bool SHORT, bool PIECES>
 __device__ __forceinline__ void strip_window_walk(uint32_t& st, uint32_t& bitpos, uint32_t& w0, uint32_t& w1,
                                                   uint32_t& w2, uint32_t& sp, uint32_t& z, uint32_t tab_lane,
                                                   uint32_t stride, uint32_t abase, uint32_t lim, uint32_t unit,
-                                                  uint32_t sp_limit) {
-#define ANSB_SP_ASM(LBL_, BODY_)                                                            \
+                                                  uint32_t sp_limit, uint32_t magic, uint32_t row_skip) {
+#define ANSB_SP_ASM(LBL_, BODY_, MORE_)                                                     \
   asm volatile(                                                                             \
       "{\n\t"                                                                               \
       ".reg .pred act, pq, pany;\n\t"                                                       \
@@ -156,22 +171,29 @@ __device__ __forceinline__ void strip_window_walk(uint32_t& st, uint32_t& bitpos
       "}"                                                                                   \
       : "+r"(st), "+r"(bitpos), "+r"(w0), "+r"(w1), "+r"(w2), "+r"(sp), "+r"(z)             \
       : "r"(tab_lane), "r"(stride), "r"(abase), "r"(lim), "r"(unit), "r"(sp_limit),         \
-        "n"(32 * ES)                                                                        \
+        "n"(32 * ES), "n"(ES) MORE_()                                                       \
       : "memory")
-#define ANSB_SP_G4(ST_, STS_) ANSB_SP_BEGIN ST_(STS_) ST_(STS_) ST_(STS_) ST_(STS_) ANSB_SP_END
-#define ANSB_SP_G2(ST_, STS_) ANSB_SP_BEGIN ST_(STS_) ST_(STS_) ANSB_SP_END
-  if (SHORT) {                                             // (tables of up to 256 states: no state takes more than 8 bits)
-    if (ES == 1) ANSB_SP_ASM("ANSB_SPS1", ANSB_SP_G4(ANSB_SP_STEP_S, "st.shared.u8"));
-    if (ES == 2) ANSB_SP_ASM("ANSB_SPS2", ANSB_SP_G4(ANSB_SP_STEP_S, "st.shared.u16"));
-  } else if (K == 4) {
-    if (ES == 1) ANSB_SP_ASM("ANSB_SP41", ANSB_SP_G4(ANSB_SP_STEP_N, "st.shared.u8"));
-    if (ES == 2) ANSB_SP_ASM("ANSB_SP42", ANSB_SP_G4(ANSB_SP_STEP_N, "st.shared.u16"));
-    if (ES == 4) ANSB_SP_ASM("ANSB_SP44", ANSB_SP_G4(ANSB_SP_STEP_W, "st.shared.u32"));
-  } else {
-    if (ES == 1) ANSB_SP_ASM("ANSB_SP21", ANSB_SP_G2(ANSB_SP_STEP_N, "st.shared.u8"));
-    if (ES == 2) ANSB_SP_ASM("ANSB_SP22", ANSB_SP_G2(ANSB_SP_STEP_N, "st.shared.u16"));
-    if (ES == 4) ANSB_SP_ASM("ANSB_SP24", ANSB_SP_G2(ANSB_SP_STEP_W, "st.shared.u32"));
+#define ANSB_SP_G4(ST_, STS_, AD_) ANSB_SP_BEGIN ST_(STS_, AD_) ST_(STS_, AD_) ST_(STS_, AD_) ST_(STS_, AD_) ANSB_SP_END
+#define ANSB_SP_G2(ST_, STS_, AD_) ANSB_SP_BEGIN ST_(STS_, AD_) ST_(STS_, AD_) ANSB_SP_END
+#define ANSB_SP_NONE()
+#define ANSB_SP_PIECE_OPS() , "r"(magic), "r"(row_skip)
+#define ANSB_SP_ALL(AD_, P_, MORE_)                                                              \
+  if (SHORT) {                                             /* (tables of up to 256 states: no state takes more than 8 bits) */ \
+    if (ES == 1) ANSB_SP_ASM("ANSB_SPS1" P_, ANSB_SP_G4(ANSB_SP_STEP_S, "st.shared.u8", AD_), MORE_);     \
+    if (ES == 2) ANSB_SP_ASM("ANSB_SPS2" P_, ANSB_SP_G4(ANSB_SP_STEP_S, "st.shared.u16", AD_), MORE_);    \
+  } else if (K == 4) {                                                                           \
+    if (ES == 1) ANSB_SP_ASM("ANSB_SP41" P_, ANSB_SP_G4(ANSB_SP_STEP_N, "st.shared.u8", AD_), MORE_);     \
+    if (ES == 2) ANSB_SP_ASM("ANSB_SP42" P_, ANSB_SP_G4(ANSB_SP_STEP_N, "st.shared.u16", AD_), MORE_);    \
+    if (ES == 4) ANSB_SP_ASM("ANSB_SP44" P_, ANSB_SP_G4(ANSB_SP_STEP_W, "st.shared.u32", AD_), MORE_);    \
+  } else {                                                                                       \
+    if (ES == 1) ANSB_SP_ASM("ANSB_SP21" P_, ANSB_SP_G2(ANSB_SP_STEP_N, "st.shared.u8", AD_), MORE_);     \
+    if (ES == 2) ANSB_SP_ASM("ANSB_SP22" P_, ANSB_SP_G2(ANSB_SP_STEP_N, "st.shared.u16", AD_), MORE_);    \
+    if (ES == 4) ANSB_SP_ASM("ANSB_SP24" P_, ANSB_SP_G2(ANSB_SP_STEP_W, "st.shared.u32", AD_), MORE_);    \
   }
+  if (PIECES) { ANSB_SP_ALL(ANSB_SP_ADDR_PIECES, "P", ANSB_SP_PIECE_OPS) } else { ANSB_SP_ALL(ANSB_SP_ADDR_STRIPS, "", ANSB_SP_NONE) }
+#undef ANSB_SP_ALL
+#undef ANSB_SP_PIECE_OPS
+#undef ANSB_SP_NONE
 #undef ANSB_SP_G2
 #undef ANSB_SP_G4
 #undef ANSB_SP_ASM
@@ -186,20 +208,26 @@ __device__ __forceinline__ void sts_v4(uint32_t a, uint4 v) {
   asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" :: "r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-struct StripGeom {                 // one sub-stream's place in its layer
-  uint64_t first;                  // first symbol of the strip in the layer
-  uint32_t ns;                     // symbols in the strip
+struct StripGeom {                 // one sub-stream's place in the output
+  uint32_t count;                  // symbols of this lane
+  uint32_t rows;                   // rows of the sub-stream (a row: E symbols of every lane, contiguous in the output)
+  uint32_t E;                      // symbols of a lane per row: 1 for strips, the piece for channels
+  uint32_t last_row_bytes;         // bytes of the last row (strips: it may be short)
+  uint32_t row_stride;             // bytes from one row to the next in the output
 };
 
 // Decode one sub-stream.  win_abs: the warp's window (kStripWindow bytes, holding `fill`);
 // words: the sub-stream in shared memory (STAGED, at stage_abs) or in global memory.
-template <int ES, bool STAGED, bool SHORT>
+template <int ES, bool STAGED, bool SHORT, bool PIECES>
 __device__ __noinline__ uint32_t decode_strip(
     uint32_t tab_lane, uint32_t stride_log, uint32_t succ_abs, uint32_t win_abs, uint32_t stage_abs,
-    const uint32_t* __restrict__ words, uint32_t ext_words, uint32_t R, uint32_t ns, uint8_t* __restrict__ out_strip,
+    const uint32_t* __restrict__ words, uint32_t ext_words, uint32_t R, uint32_t count, uint32_t rows, uint32_t piece,
+    uint32_t last_row_bytes, uint32_t row_stride, uint8_t* __restrict__ out_strip,
     uint32_t fill, bool wide_steps, uint32_t unit, uint32_t lane) {
-  constexpr uint32_t RB = 32u * ES;                        // bytes of a row (one symbol of every lane)
-  constexpr uint32_t P = kStripWindow / RB;                // rows of a window
+  const uint32_t E = PIECES ? piece : 1u;
+  const uint32_t magic = PIECES ? 0xFFFFFFFFu / piece + 1u : 0u;   // 2^32 / E rounded up (E >= 2)
+  const uint32_t RB = 32u * ES * E;                        // bytes of a row
+  const uint32_t P = kStripWindow / RB;                    // rows of a window
   const uint32_t word_limit = STAGED ? ext_words + 4u : ext_words;
   auto load_word = [&](uint32_t i) -> uint32_t {     // (staged: the words after the sub-stream are zero, up to kStripPad)
     if (STAGED) return lds_u32(stage_abs + min(i, word_limit + 8u) * 4u);
@@ -207,8 +235,6 @@ __device__ __noinline__ uint32_t decode_strip(
   };
   uint32_t bad = 0;
 
-  const uint32_t count = lane_symbols(ns, 32u, lane);     // symbols of this lane
-  const uint32_t rows = (ns + 31u) >> 5;
 
   // the lanes' bit lengths head the sub-stream; their running sum places every lane's string
   const uint32_t hw = load_word(lane >> 1);
@@ -242,14 +268,16 @@ __device__ __noinline__ uint32_t decode_strip(
   const uint4 fill4 = make_uint4(fill, fill, fill, fill);
 
   for (uint32_t t0 = 0; t0 < rows; t0 += P) {
-    const uint32_t lim = min(t0 + P, count);
-    const uint32_t abase = win_abs + lane * ES - t0 * RB;
+    const uint32_t lim = min((t0 + P) * E, count);
+    const uint32_t abase = win_abs + lane * ES * E - t0 * RB;
     __syncwarp();
     if (STAGED) {
       if (SHORT || wide_steps)
-        strip_window_walk<ES, 4, SHORT>(st, bitpos, w0, w1, w2, sp, z, tab_lane, stride, abase, lim, unit, sp_limit);
+        strip_window_walk<ES, 4, SHORT, PIECES>(st, bitpos, w0, w1, w2, sp, z, tab_lane, stride, abase, lim, unit, sp_limit,
+                                                magic, 31u * E * ES);
       else
-        strip_window_walk<ES, 2, false>(st, bitpos, w0, w1, w2, sp, z, tab_lane, stride, abase, lim, unit, sp_limit);
+        strip_window_walk<ES, 2, false, PIECES>(st, bitpos, w0, w1, w2, sp, z, tab_lane, stride, abase, lim, unit, sp_limit,
+                                                magic, 31u * E * ES);
     } else {                                               // the same walk in plain code, words from global memory
       bool any = true;
       while (any) {
@@ -258,7 +286,7 @@ __device__ __noinline__ uint32_t decode_strip(
         const bool act = zn < lim;
         if (act) {
           const uint32_t q = SHORT ? ea >> 24 : ES == 4 ? ea >> 16 : eb, val = SHORT ? ea : ES == 4 ? eb : ea >> 16;
-          sts_elem<ES>(abase + zn * RB, val);
+          sts_elem<ES>(PIECES ? abase + zn * ES + (zn / E) * (31u * E * ES) : abase + zn * RB, val);
           const uint32_t x = __funnelshift_l(w1, w0, bitpos);
           st = tab_lane + (__funnelshift_l(x, q, nb) << stride_log);
           z = zn + 1u;
@@ -269,40 +297,46 @@ __device__ __noinline__ uint32_t decode_strip(
       }
     }
     __syncwarp();
-    // the window is complete: write it out (it is contiguous in the output) and fill it again
-    const uint32_t wbytes = min(kStripWindow, ns * ES - t0 * RB);
-    uint8_t* gdst = out_strip + size_t(t0) * RB;
+    // the window is complete: write it out and fill it again.  Its rows are contiguous in the
+    // output for strips (one bulk store); for channels every row is a store of its own.
+    const uint32_t wrows = min(P, rows - t0);
+    const uint32_t wbytes = (wrows - 1u) * RB + (t0 + wrows == rows ? last_row_bytes : RB);
+    uint8_t* gdst = out_strip + size_t(t0) * row_stride;
     const bool more = t0 + P < rows;
     if (vec_ok && (wbytes & 15u) == 0) {
-      // one bulk copy from shared memory to the output; the window may be filled again once the
-      // copy has read it
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0) {
-        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" :: "l"(gdst), "r"(win_abs), "r"(wbytes) : "memory");
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      if (row_stride == RB) {                          // rows side by side in the output: one store
+        if (lane == 0) {
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" :: "l"(gdst), "r"(win_abs), "r"(wbytes) : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        }
+      } else {
+        bool mine = false;
+        for (uint32_t r = lane; r < wrows; r += 32u) {
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                       :: "l"(gdst + size_t(r) * row_stride), "r"(win_abs + r * RB), "r"(RB) : "memory");
+          mine = true;
+        }
+        if (mine) {
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        }
       }
       __syncwarp();
       if (more)
         for (uint32_t i = lane * 16u; i < kStripWindow; i += 512u) sts_v4(win_abs + i, fill4);
-    } else if (vec_ok) {
-      for (uint32_t i = lane * 16u; i + 16u <= wbytes; i += 512u) {
-        const uint4 v = lds_v4(win_abs + i);
-        *reinterpret_cast<uint4*>(gdst + i) = v;
-        if (more) sts_v4(win_abs + i, fill4);
-      }
-      const uint32_t tail0 = wbytes & ~15u;                // a ragged end: only in a layer's last strip
-      if (tail0 + lane * ES < wbytes) {
-        const uint32_t a = win_abs + tail0 + lane * ES;
-        const uint32_t v = ES == 1 ? lds_u32(a & ~3u) >> (8u * (a & 3u)) : ES == 2 ? lds_u16(a) : lds_u32(a);
-        stg_elem<ES>(gdst + tail0 + lane * ES, v);
-      }
     } else {
-      for (uint32_t i = lane * ES; i < wbytes; i += 32u * ES) {
-        const uint32_t a = win_abs + i;
-        const uint32_t v = ES == 1 ? lds_u32(a & ~3u) >> (8u * (a & 3u)) : ES == 2 ? lds_u16(a) : lds_u32(a);
-        stg_elem<ES>(gdst + i, v);
+      // ragged ends (a layer's last strip) and outputs off a 16-byte boundary leave through registers
+      for (uint32_t r = 0; r < wrows; ++r) {
+        const uint32_t rb = (t0 + r + 1u == rows) ? last_row_bytes : RB;
+        uint8_t* grow = gdst + size_t(r) * row_stride;
+        for (uint32_t i = lane * ES; i < rb; i += 32u * ES) {
+          const uint32_t a = win_abs + r * RB + i;
+          const uint32_t v = ES == 1 ? lds_u32(a & ~3u) >> (8u * (a & 3u)) : ES == 2 ? lds_u16(a) : lds_u32(a);
+          stg_elem<ES>(grow + i, v);
+        }
       }
       __syncwarp();
       if (more)
@@ -352,7 +386,7 @@ __global__ void __launch_bounds__(kStripWarps * 32) ans_decode_strips_kernel(con
   const StripLayer& L = args.layer[lo];
   const uint32_t zero_point = L.packed & 0xFFu, R = (L.packed >> 8) & 15u, bitwidth = (L.packed >> 12) & 15u;
   const int dtype = static_cast<int>((L.packed >> 16) & 3u);
-  const uint32_t G = (L.packed >> 18) & 127u;
+  const uint32_t G = (L.packed >> 18) & 127u, piece = L.packed >> 25;
   const uint32_t es = dtype == ANS_U8 ? 1u : dtype == ANS_F32 ? 4u : 2u;
   const uint32_t sub = (blockIdx.x - args.cta_begin[lo]) * kStripWarps + warp;
   const bool have = sub < L.n_sub;
@@ -458,15 +492,36 @@ __global__ void __launch_bounds__(kStripWarps * 32) ans_decode_strips_kernel(con
     const uint4 fill4 = make_uint4(fill, fill, fill, fill);
     for (uint32_t i = lane * 16u; i < kStripWindow; i += 512u) sts_v4(win_abs + i, fill4);
 
-    // the strip of this sub-stream
+    // the place of this sub-stream in the output
     const uint64_t chunk = sub / G;
     const uint32_t g = sub - static_cast<uint32_t>(chunk) * G;
-    const uint32_t S = L.chunk_symbols / (32u * G);
     const uint64_t c0 = chunk * L.chunk_symbols;
-    const uint64_t nc = min(uint64_t(L.chunk_symbols), L.n_symbols - c0);
-    const uint64_t sfirst = uint64_t(g) * 32u * S;
-    const uint32_t ns = nc > sfirst ? static_cast<uint32_t>(min(nc - sfirst, uint64_t(32u) * S)) : 0u;
-    uint8_t* out_strip = L.out + (c0 + sfirst) * es;
+    const uint32_t nc = static_cast<uint32_t>(min(uint64_t(L.chunk_symbols), L.n_symbols - c0));
+    StripGeom geo;
+    uint8_t* out_strip;
+    uint32_t ns;                                           // symbols of the sub-stream
+    if (piece) {
+      // channels: lanes 32 g .. 32 g + 31 of a chunk dealt in pieces; every lane owns nc / W symbols
+      const uint32_t W = 32u * G;
+      geo.count = nc / W;
+      geo.E = piece;
+      geo.rows = geo.count / piece;
+      geo.last_row_bytes = 32u * piece * es;
+      geo.row_stride = W * piece * es;
+      ns = 32u * geo.count;
+      out_strip = L.out + (c0 + uint64_t(32u * g) * piece) * es;
+    } else {
+      // strips: a contiguous part of the chunk dealt round-robin
+      const uint32_t S = L.chunk_symbols / (32u * G);
+      const uint32_t sfirst = g * 32u * S;                 // (inside the chunk: below 2^32)
+      ns = nc > sfirst ? min(nc - sfirst, 32u * S) : 0u;
+      geo.count = lane_symbols(ns, 32u, lane);
+      geo.E = 1u;
+      geo.rows = (ns + 31u) >> 5;
+      geo.last_row_bytes = (ns - (geo.rows ? (geo.rows - 1u) * 32u : 0u)) * es;
+      geo.row_stride = 32u * es;
+      out_strip = L.out + (c0 + sfirst) * es;
+    }
     const uint32_t ext_words = static_cast<uint32_t>(extent >> 2);
     const uint32_t* words = reinterpret_cast<const uint32_t*>(L.stream + off0);
 
@@ -479,8 +534,12 @@ __global__ void __launch_bounds__(kStripWarps * 32) ans_decode_strips_kernel(con
       if (ns != 0) bad |= ANS_STATUS_BAD_LENGTH;
     } else {
 #define ANSB_SCALL(ES_, ST_, SH_)                                                                     \
-  bad |= decode_strip<ES_, ST_, SH_>(tab_lane, stride_log, succ_abs, win_abs, stage_abs, words, ext_words, R, ns, \
-                                     out_strip, fill, wide_steps, args.unit, lane)
+  bad |= piece > 1u ? decode_strip<ES_, ST_, SH_, true>(tab_lane, stride_log, succ_abs, win_abs, stage_abs, words, ext_words, \
+                                                        R, geo.count, geo.rows, geo.E, geo.last_row_bytes, geo.row_stride, \
+                                                        out_strip, fill, wide_steps, args.unit, lane)                \
+                    : decode_strip<ES_, ST_, SH_, false>(tab_lane, stride_log, succ_abs, win_abs, stage_abs, words, ext_words, \
+                                                         R, geo.count, geo.rows, geo.E, geo.last_row_bytes, geo.row_stride, \
+                                                         out_strip, fill, wide_steps, args.unit, lane)
       if (short_entries) {
         if (staged) { if (es == 1u) ANSB_SCALL(1, true, true); else ANSB_SCALL(2, true, true); }
         else { if (es == 1u) ANSB_SCALL(1, false, true); else ANSB_SCALL(2, false, true); }
@@ -545,7 +604,10 @@ int launch_strips(const ans_layer_desc* h_descs, int n_layers, uint8_t* d_symbol
       L.scale = d.scale;
       const uint32_t dtype = d_symbols_override ? ANS_U8 : static_cast<uint32_t>(d.out_dtype);
       L.packed = static_cast<uint32_t>(d.zero_point) | (static_cast<uint32_t>(d.table_log) << 8) |
-                 (static_cast<uint32_t>(d.bitwidth) << 12) | (dtype << 16) | ((d.lanes / 32u) << 18);
+                 (static_cast<uint32_t>(d.bitwidth) << 12) | (dtype << 16) | ((d.lanes / 32u) << 18) |
+                 ((d.layout == ANS_LAYOUT_CHANNELS ? d.piece_symbols : 0u) << 25);
+      if (d.layout == ANS_LAYOUT_CHANNELS && d.piece_symbols * (dtype == ANS_U8 ? 1u : dtype == ANS_F32 ? 4u : 2u) > 128u)
+        return ANS_ERR_UNSUPPORTED;
       a.cta_begin[a.n_layers] = static_cast<uint32_t>(ctas);
       ctas += d.work_count;
       ++a.n_layers;

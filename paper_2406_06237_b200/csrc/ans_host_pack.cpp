@@ -155,6 +155,37 @@ bool pack_strip(const EncTable& T, const uint8_t* strip, size_t ns, std::vector<
   return true;
 }
 
+// One sub-stream of the channels container: lanes 32 g .. 32 g + 31 of a chunk whose symbols come
+// in pieces of E, piece j belonging to lane j mod W; every lane owns cnt symbols.  Bytes as for strips.
+bool pack_channels_sub(const EncTable& T, const uint8_t* chunk, size_t cnt, size_t W, size_t E, size_t g,
+                       std::vector<uint8_t>& bytes, std::vector<uint8_t>& nb, std::vector<uint16_t>& val,
+                       std::vector<uint8_t>& mine) {
+  const size_t base = bytes.size();
+  bytes.resize(base + 64, 0);
+  nb.resize(cnt + 1);
+  val.resize(cnt + 1);
+  mine.resize(cnt + 1);
+  TopBitWriter bw(bytes);
+  for (size_t k = 0; k < 32; ++k) {
+    uint64_t len = 0;
+    if (cnt) {
+      const size_t lambda = 32 * g + k;
+      for (size_t t = 0; t < cnt; ++t) mine[t] = chunk[((t / E) * W + lambda) * E + t % E];
+      const int init = encode_lane(T, mine.data(), cnt, 1, nb.data(), val.data());
+      if (init < 0) return false;
+      bw.put(static_cast<uint32_t>(init), T.R);
+      len = static_cast<uint64_t>(T.R);
+      for (size_t t = 0; t < cnt; ++t) { bw.put(val[t], nb[t]); len += nb[t]; }
+    }
+    if (len > 0xFFFF) return false;
+    bytes[base + 2 * k] = static_cast<uint8_t>(len & 0xFF);
+    bytes[base + 2 * k + 1] = static_cast<uint8_t>(len >> 8);
+  }
+  bw.finish();
+  while ((bytes.size() - base) % 16) bytes.push_back(0);
+  return true;
+}
+
 // One sub-stream (32 lanes) into `bytes` (appended) and meta (32 entries).
 bool pack_sub(const EncTable& T, const uint8_t* chunk, size_t nc, size_t W, size_t g, int layout,
               std::vector<uint8_t>& bytes, void* meta32, std::vector<uint8_t>& nb, std::vector<uint16_t>& val,
@@ -278,7 +309,7 @@ ANS_EXPORT int ans_host_normalize_freqs(const uint64_t* h_counts, int alphabet, 
 ANS_EXPORT int ans_host_pack_bound(uint64_t n_symbols, uint32_t chunk_symbols, uint32_t lanes, int layout,
                                    uint64_t* h_bytes_out) {
   if (!h_bytes_out || chunk_symbols == 0 || lanes == 0 || lanes % 32) return ANS_ERR_INVALID_ARG;
-  if (layout < ANS_LAYOUT_INTERLEAVED || layout > ANS_LAYOUT_STRIPS) return ANS_ERR_UNSUPPORTED;
+  if (layout < ANS_LAYOUT_INTERLEAVED || layout > ANS_LAYOUT_CHANNELS) return ANS_ERR_UNSUPPORTED;
   const uint64_t chunks = n_symbols ? (n_symbols + chunk_symbols - 1) / chunk_symbols : 0;
   const uint64_t subs = chunks * (lanes / 32);
   // <= 14 bits per symbol, plus per lane a last unit/word (strips: a length and a state), plus
@@ -287,20 +318,51 @@ ANS_EXPORT int ans_host_pack_bound(uint64_t n_symbols, uint32_t chunk_symbols, u
   return ANS_OK;
 }
 
+static int pack_any(const uint8_t* h_symbols, uint64_t n_symbols, const uint32_t* h_freqs,
+                    int alphabet, int table_log, uint32_t chunk_symbols, uint32_t lanes,
+                    int layout, uint32_t piece, uint8_t* h_stream_out, uint64_t stream_cap,
+                    uint64_t* h_stream_bytes_out, uint64_t* h_sub_offsets_out,
+                    void* h_lane_meta_out, int n_threads);
+
 ANS_EXPORT int ans_host_pack_layer(const uint8_t* h_symbols, uint64_t n_symbols, const uint32_t* h_freqs,
                                    int alphabet, int table_log, uint32_t chunk_symbols, uint32_t lanes,
                                    int layout, uint8_t* h_stream_out, uint64_t stream_cap,
                                    uint64_t* h_stream_bytes_out, uint64_t* h_sub_offsets_out,
                                    void* h_lane_meta_out, int n_threads) {
+  if (layout == ANS_LAYOUT_CHANNELS) return ANS_ERR_UNSUPPORTED;     // needs the piece size: ans_host_pack_channels
+  return pack_any(h_symbols, n_symbols, h_freqs, alphabet, table_log, chunk_symbols, lanes, layout, 1, h_stream_out,
+                  stream_cap, h_stream_bytes_out, h_sub_offsets_out, h_lane_meta_out, n_threads);
+}
+
+ANS_EXPORT int ans_host_pack_channels(const uint8_t* h_symbols, uint64_t n_symbols, const uint32_t* h_freqs,
+                                      int alphabet, int table_log, uint32_t chunk_symbols, uint32_t lanes,
+                                      uint32_t piece_symbols, uint8_t* h_stream_out, uint64_t stream_cap,
+                                      uint64_t* h_stream_bytes_out, uint64_t* h_sub_offsets_out, int n_threads) {
+  return pack_any(h_symbols, n_symbols, h_freqs, alphabet, table_log, chunk_symbols, lanes, ANS_LAYOUT_CHANNELS,
+                  piece_symbols, h_stream_out, stream_cap, h_stream_bytes_out, h_sub_offsets_out, nullptr, n_threads);
+}
+
+static int pack_any(const uint8_t* h_symbols, uint64_t n_symbols, const uint32_t* h_freqs,
+                    int alphabet, int table_log, uint32_t chunk_symbols, uint32_t lanes,
+                    int layout, uint32_t piece, uint8_t* h_stream_out, uint64_t stream_cap,
+                    uint64_t* h_stream_bytes_out, uint64_t* h_sub_offsets_out,
+                    void* h_lane_meta_out, int n_threads) {
   if (!h_freqs || !h_stream_bytes_out || !h_sub_offsets_out) return ANS_ERR_INVALID_ARG;
   if (alphabet < 1 || alphabet > ANS_MAX_ALPHABET || chunk_symbols == 0) return ANS_ERR_INVALID_ARG;
   if (table_log < 1 || table_log > ANS_MAX_TABLE_LOG) return ANS_ERR_UNSUPPORTED;
   if (lanes < 32 || lanes > ANS_MAX_LANES || lanes % 32) return ANS_ERR_UNSUPPORTED;
-  if (layout < ANS_LAYOUT_INTERLEAVED || layout > ANS_LAYOUT_STRIPS) return ANS_ERR_UNSUPPORTED;
+  if (layout < ANS_LAYOUT_INTERLEAVED || layout > ANS_LAYOUT_CHANNELS) return ANS_ERR_UNSUPPORTED;
+  const bool channels = layout == ANS_LAYOUT_CHANNELS;
+  if (channels) {
+    if (piece < 1 || piece > ANS_MAX_PIECE_SYMBOLS) return ANS_ERR_UNSUPPORTED;
+    const uint64_t unit = uint64_t(lanes) * piece;
+    if (chunk_symbols % unit || n_symbols % unit || chunk_symbols / lanes > ANS_MAX_CHANNEL_LANE_SYMBOLS)
+      return ANS_ERR_UNSUPPORTED;
+  }
   const bool strips = layout == ANS_LAYOUT_STRIPS;
   if (strips && (chunk_symbols % lanes || chunk_symbols / lanes > ANS_MAX_STRIP_LANE_SYMBOLS))
     return ANS_ERR_UNSUPPORTED;
-  if (n_symbols && (!h_symbols || !h_stream_out || (!h_lane_meta_out && !strips))) return ANS_ERR_INVALID_ARG;
+  if (n_symbols && (!h_symbols || !h_stream_out || (!h_lane_meta_out && !strips && !channels))) return ANS_ERR_INVALID_ARG;
   EncTable T;
   if (!make_enc_table(h_freqs, alphabet, table_log, T)) return ANS_ERR_BAD_FREQS;
 
@@ -324,6 +386,13 @@ ANS_EXPORT int ans_host_pack_layer(const uint8_t* h_symbols, uint64_t n_symbols,
       const size_t nc = std::min<uint64_t>(C, n_symbols - c * C);
       for (size_t g = 0; g < G; ++g) {
         part_offs[ti].push_back(part[ti].size());
+        if (channels) {
+          if (!pack_channels_sub(T, h_symbols + c * C, nc / W, W, piece, g, part[ti], nb, val, lane_bytes)) {
+            part_rc[ti] = ANS_ERR_BAD_FREQS;
+            return;
+          }
+          continue;
+        }
         if (strips) {
           const size_t first = g * 32 * (C / W);
           const size_t ns = nc > first ? std::min(nc - first, 32 * (C / W)) : 0;

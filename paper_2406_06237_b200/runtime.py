@@ -29,6 +29,7 @@ class PackedLayer:
     scale: float
     out_dtype: int
     layout: int
+    piece_symbols: int = 1      # ANS_LAYOUT_CHANNELS: symbols of a piece (H * W)
 
     def compressed_bytes(self) -> int:
         return int(self.stream.nbytes + self.sub_offsets.nbytes + self.lane_meta.nbytes)
@@ -36,14 +37,18 @@ class PackedLayer:
 
 def pack_layer(symbols: np.ndarray, alphabet: int, table_log: int, chunk_symbols: int, lanes: int,
                layout: int, bitwidth: int, zero_point: int, scale: float, out_dtype: int,
-               n_threads: int = 0) -> PackedLayer:
+               n_threads: int = 0, piece_symbols: int = 1) -> PackedLayer:
     """Histogram, normalise and encode one layer with the library's host packer."""
     counts = np.bincount(symbols, minlength=256).astype(np.uint64)
     freqs = B.ans_host_normalize_freqs(counts[:alphabet], alphabet, table_log)
-    stream, offs, meta = B.ans_host_pack_layer(symbols, freqs, alphabet, table_log, chunk_symbols, lanes,
-                                               layout, n_threads)
+    if layout == B.ANS_LAYOUT_CHANNELS:
+        stream, offs, meta = B.ans_host_pack_channels(symbols, freqs, alphabet, table_log, chunk_symbols, lanes,
+                                                      piece_symbols, n_threads)
+    else:
+        stream, offs, meta = B.ans_host_pack_layer(symbols, freqs, alphabet, table_log, chunk_symbols, lanes,
+                                                   layout, n_threads)
     return PackedLayer(stream, offs, meta, freqs, alphabet, int(symbols.size), chunk_symbols, lanes,
-                       table_log, bitwidth, zero_point, float(scale), out_dtype, layout)
+                       table_log, bitwidth, zero_point, float(scale), out_dtype, layout, piece_symbols)
 
 
 _TORCH_DTYPE = {B.ANS_U8: torch.uint8, B.ANS_F32: torch.float32, B.ANS_BF16: torch.bfloat16}
@@ -116,7 +121,7 @@ class DeviceBatch:
                 d.stream_bytes = L.stream.nbytes
                 d.n_symbols, d.chunk_symbols, d.lanes = L.n_symbols, L.chunk_symbols, L.lanes
                 d.table_log, d.bitwidth, d.zero_point, d.scale = L.table_log, L.bitwidth, L.zero_point, L.scale
-                d.out_dtype, d.layout = L.out_dtype, L.layout
+                d.out_dtype, d.layout, d.piece_symbols = L.out_dtype, L.layout, L.piece_symbols
             self.total_work = B.ans_plan_batch(arr) if n else 0
             raw = torch.frombuffer(bytearray(bytes(arr)), dtype=torch.uint8)
             self.h_descs.append(arr)
@@ -141,7 +146,7 @@ class DeviceBatch:
         layers 64 at a time (a group in which every layer is empty is not launched)."""
         if not any(L.n_symbols for L in self.layers):
             return 0
-        if self.layers[0].layout == B.ANS_LAYOUT_STRIPS:
+        if self.layers[0].layout in (B.ANS_LAYOUT_STRIPS, B.ANS_LAYOUT_CHANNELS):
             return sum(1 for g in range(0, len(self.layers), 64) if any(L.n_symbols for L in self.layers[g:g + 64]))
         return 1
 

@@ -31,7 +31,7 @@ def to_packed_layer(spec, P, f256, table_log=None, out_dtype=None):
     from paper_2406_06237_b200.runtime import PackedLayer
     return PackedLayer(P.stream, P.sub_offsets, P.lane_meta, f256, spec.alphabet, P.n, P.chunk,
                        32 * P.groups, table_log or spec.table_log, spec.bitwidth, spec.zero_point,
-                       spec.scale, ans.DTYPES[out_dtype or spec.out_dtype], P.layout)
+                       spec.scale, ans.DTYPES[out_dtype or spec.out_dtype], P.layout, getattr(P, "piece", 1))
 
 
 def oracle_expected(spec, T, P, threads=1, out_dtype=None):

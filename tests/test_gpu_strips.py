@@ -258,3 +258,81 @@ def test_full_size_resnet50_in_the_benchmark_configuration():
     """Config 3 as bench.py times it (64 lanes per 16 K-symbol chunk, 256-state tables, one launch),
     every output element against the oracle."""
     run_and_compare(sg.workload_resnet50(), STRIPS, 64, threads=16)
+
+
+# ---- channels container: one stream per input channel of an O x I x H x W tensor (Section III-B) ----
+CHANNELS = ans.ANS_LAYOUT_CHANNELS
+
+
+def _channels_case(shape, b, pzp, R, dt, index=0, chunk_rows=0):
+    O, I, H, W = shape
+    n = O * I * H * W
+    spec = sg.LayerSpec(f"conv{index}", shape, b, *sg.alphabet_for_bits(b), sg.theta_for_pzp(*sg.alphabet_for_bits(b), pzp),
+                        0.02, R, (chunk_rows * I * H * W) if chunk_rows else n, dt, sg.stream_key(21, index))
+    sym = sg.draw_symbols(spec)
+    f = oracle.normalize_freqs(oracle.histogram(sym), spec.alphabet, R)
+    T = oracle.Table(f, R)
+    P = oracle.pack(T, sym, spec.chunk_symbols, I // 32, oracle.CHANNELS, piece=H * W)
+    f256 = np.zeros(256, dtype=np.uint32)
+    f256[:spec.alphabet] = f
+    want_sym, rc = oracle.unpack(T, P)
+    assert rc == oracle.OK and (want_sym == sym).all()
+    return spec, T, P, f256, sym, oracle.dequant(sym, spec.zero_point, spec.scale, dt)
+
+
+def _decode_and_compare(cases, per_layer=False):
+    db = DeviceBatch([to_packed_layer(c[0], c[2], c[3]) for c in cases])
+    for o in db.out_sets[0]:
+        o.view(torch.uint8).fill_(0xA5)
+    (db.decode_per_layer if per_layer else db.decode)()
+    assert db.read_status() == 0
+    for i, c in enumerate(cases):
+        assert np.array_equal(bits_view(db.output(i)), expected_bits(c[5])), f"layer {i} {c[0].shape}"
+    return db
+
+
+@pytest.mark.parametrize("dt", ["bf16", "u8", "f32"])
+def test_channels_conv_shapes(dt):
+    """3x3, 1x1 and 7x7 kernels, 32 to 512 input channels, one chunk per layer or chunks of whole
+    output-channel rows; the decoded tensor is in the tensor's own O x I x H x W order."""
+    shapes = [((64, 64, 3, 3), 0), ((128, 32, 1, 1), 0), ((16, 96, 7, 7) if dt != "f32" else (16, 96, 5, 5), 0),
+              ((256, 512, 1, 1), 0), ((40, 128, 3, 3), 8), ((7, 64, 1, 1), 1), ((512, 256, 3, 3), 64)]
+    cases = [_channels_case(sh, 1 + i % 6, 0.6 + 0.06 * i, 6 + i % 6, dt, i, rows) for i, (sh, rows) in enumerate(shapes)]
+    db = _decode_and_compare(cases)
+    assert (db.decode_symbols(0).cpu().numpy() == cases[0][4]).all() and db.read_status() == 0
+    _decode_and_compare(cases[:3], per_layer=True)
+
+
+def test_channels_resnet50_by_input_channel():
+    """Every ResNet-50 conv but the first (3 input channels; the paper leaves the first layer
+    uncompressed, Section III-A) as one chunk with a lane per input channel."""
+    cases = []
+    for i, spec in enumerate(sg.workload_resnet50()):
+        if spec.shape[1] % 32:
+            continue
+        cases.append(_channels_case(spec.shape, spec.bitwidth, 0.9, 8, "bf16", i))
+    assert len(cases) == 52
+    _decode_and_compare(cases)
+
+
+def test_channels_corruption_and_bad_sizes():
+    c = _channels_case((64, 64, 3, 3), 4, 0.8, 10, "bf16")
+    spec, T, P, f256 = c[0], c[1], c[2], c[3]
+    rng = np.random.default_rng(5)
+    flagged = 0
+    for trial in range(6):
+        s = P.stream.copy()
+        pos = rng.integers(0, s.size, size=4)
+        s[pos] ^= rng.integers(1, 256, size=4).astype(np.uint8)
+        P2 = oracle.Packed(P.layout, s, P.sub_offsets, P.lane_meta, P.n, P.chunk, P.groups, P.piece)
+        db = DeviceBatch([to_packed_layer(spec, P2, f256)])
+        db.decode()
+        st = db.read_status()
+        assert (st != 0) == (oracle.unpack(T, P2)[1] != oracle.OK)
+        flagged += st != 0
+    assert flagged > 0
+    pl = to_packed_layer(spec, P, f256)
+    pl.piece_symbols = 7                                   # 64 * 64 * 9 is no multiple of 64 * 7
+    with pytest.raises(ans.AnsError) as e:
+        DeviceBatch([pl]).decode()
+    assert e.value.code == ans.ANS_ERR_UNSUPPORTED

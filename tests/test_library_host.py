@@ -29,8 +29,9 @@ def test_every_declared_symbol_is_exported():
 
 def test_descriptor_layout_matches_header():
     # 5 pointers, 2 u64, then 4-byte fields: the ctypes mirror must have the C struct's size
-    assert ctypes.sizeof(ans.ans_layer_desc) == 5 * 8 + 2 * 8 + 10 * 4
+    assert ctypes.sizeof(ans.ans_layer_desc) == 5 * 8 + 2 * 8 + 12 * 4
     assert ans.ans_layer_desc.n_symbols.offset == 48 and ans.ans_layer_desc.work_count.offset == 92
+    assert ans.ans_layer_desc.piece_symbols.offset == 96
 
 
 def test_table_bytes():
@@ -74,6 +75,23 @@ def test_host_packer_equals_oracle_encoder_strips(n, C, lanes, R, b):
         assert (o == P.sub_offsets).all() and m.size == 0
     with pytest.raises(ans.AnsError):                      # chunk no multiple of 4 * lanes
         ans.ans_host_pack_layer(sym, f256, spec.alphabet, R, 1000, 32, ans.ANS_LAYOUT_STRIPS, 1)
+
+
+@pytest.mark.parametrize("O,I,E,R,chunk_rows", [(8, 64, 9, 8, 0), (5, 32, 1, 6, 0), (16, 96, 49, 11, 4), (64, 128, 9, 8, 16)])
+def test_host_packer_equals_oracle_encoder_channels(O, I, E, R, chunk_rows):
+    """ANS_LAYOUT_CHANNELS: a stream per input channel of a tensor stored O x I x (H*W)."""
+    spec = tiny_spec(O * I * E, bitwidth=4, pzp=0.85, table_log=R, chunk=O * I * E)
+    sym = sg.draw_symbols(spec)
+    C = chunk_rows * I * E if chunk_rows else sym.size
+    T, _, f256 = oracle_pack_spec(spec, sym, oracle.STRIPS, 32, chunk=32)
+    P = oracle.pack(T, sym, C, I // 32, oracle.CHANNELS, piece=E)
+    for threads in (1, 3):
+        s, o, m = ans.ans_host_pack_channels(sym, f256, spec.alphabet, R, C, I, E, threads)
+        assert s.size == P.stream.size and (s == P.stream).all() and (o == P.sub_offsets).all() and m.size == 0
+    with pytest.raises(ans.AnsError):                      # the layer is no multiple of lanes * piece
+        ans.ans_host_pack_channels(sym[:-1], f256, spec.alphabet, R, C, I, E, 1)
+    with pytest.raises(ans.AnsError):                      # the plain call cannot know the piece size
+        ans.ans_host_pack_layer(sym, f256, spec.alphabet, R, C, I, ans.ANS_LAYOUT_CHANNELS, 1)
 
 
 def test_plan_batch_counts_groups_of_four_sub_streams():
