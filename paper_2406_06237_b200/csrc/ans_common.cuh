@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 #include <stdint.h>
 
 #include "ans_b200.h"
@@ -54,6 +55,14 @@ inline int cuda_fail(cudaError_t e) {
     cudaError_t e__ = (call);                             \
     if (e__ != cudaSuccess) return ::ansb::cuda_fail(e__); \
   } while (0)
+
+// NVTX range around an API call (visible in a profiler's timeline; costs nothing without one)
+struct ApiRange {
+  explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+  ~ApiRange() { nvtxRangePop(); }
+  ApiRange(const ApiRange&) = delete;
+  ApiRange& operator=(const ApiRange&) = delete;
+};
 
 int validate_desc(const ans_layer_desc& d, bool need_out);
 inline uint32_t groups_of(const ans_layer_desc& d) { return d.lanes / 32u; }

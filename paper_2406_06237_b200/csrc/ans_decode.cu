@@ -530,6 +530,7 @@ ANS_EXPORT int ans_plan_batch(ans_layer_desc* h_descs, int n_layers, uint64_t* h
 
 ANS_EXPORT int ans_decode_layer(const ans_layer_desc* h_desc, uint8_t* d_symbols_out, uint32_t* d_status,
                                 void* stream) {
+  ApiRange range("ans_decode_layer");
   if (!h_desc || !d_status) return ANS_ERR_INVALID_ARG;
   if (!d_symbols_out && h_desc->n_symbols) return ANS_ERR_INVALID_ARG;
   ans_layer_desc d = *h_desc;
@@ -540,6 +541,7 @@ ANS_EXPORT int ans_decode_layer(const ans_layer_desc* h_desc, uint8_t* d_symbols
 }
 
 ANS_EXPORT int ans_decode_dequant(const ans_layer_desc* h_desc, uint32_t* d_status, void* stream) {
+  ApiRange range("ans_decode_dequant");
   if (!h_desc || !d_status) return ANS_ERR_INVALID_ARG;
   ans_layer_desc d = *h_desc;
   const int rc = ans_plan_batch(&d, 1, nullptr);
@@ -549,6 +551,7 @@ ANS_EXPORT int ans_decode_dequant(const ans_layer_desc* h_desc, uint32_t* d_stat
 
 ANS_EXPORT int ans_decode_dequant_batch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs,
                                         int n_layers, uint32_t* d_status, void* stream) {
+  ApiRange range("ans_decode_dequant_batch");
   if (n_layers < 0 || !d_status) return ANS_ERR_INVALID_ARG;
   if (n_layers == 0) return ANS_OK;
   if (!h_descs || (!d_descs && lane_meta_size(h_descs[0].layout))) return ANS_ERR_INVALID_ARG;

@@ -98,6 +98,7 @@ ANS_EXPORT int ans_build_decode_tables(const uint32_t* h_norm_freqs, const int32
                                        const int32_t* h_table_log, int n_layers, void* d_tables,
                                        size_t d_tables_bytes, uint64_t* h_table_offsets_out,
                                        void* stream) {
+  ApiRange range("ans_build_decode_tables");
   if (!h_norm_freqs || !h_alphabet || !h_table_log || !h_table_offsets_out || n_layers < 0)
     return ANS_ERR_INVALID_ARG;
   if (n_layers == 0) return ANS_OK;
