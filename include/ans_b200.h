@@ -350,6 +350,23 @@ int ans_encode_layer_device(const uint8_t* d_symbols, uint64_t n_symbols, const 
                             uint64_t stream_cap, uint64_t* d_sub_offsets_out, void* d_scratch,
                             size_t d_scratch_bytes, uint32_t* d_status, void* stream);
 
+/* ------------------------------------------------------------------------------------
+ * Decode fused into its consumer (Section I, Section III-C: the weights are decompressed just
+ * before the computation that uses them and the decoded weights never travel through DRAM):
+ *   Y[M x N] = X[M x K] * W^T,  W[N x K] read in compressed form,
+ * X bfloat16 row-major, Y float row-major, the product on the tensor cores with fp32
+ * accumulation (the order of the K-direction sums is the hardware's).  W is dequantised to
+ * bfloat16 exactly as ans_decode_dequant would (Section II-B).
+ *   h_desc: W's layer: ANS_LAYOUT_STRIPS, chunk_symbols = 4096, lanes = 32, table_log <= 12,
+ *           n_symbols = N * K, the symbols being W in blocks of 64 x 64: block (n / 64, k / 64)
+ *           holds 4096 consecutive symbols, row-major inside the block, blocks ordered
+ *           [N / 64][K / 64].  d_out / out_dtype are ignored.
+ *   1 <= M <= 128; N and K multiples of 64; d_x and d_y 16-byte aligned.
+ * d_status as for the decode calls.  Asynchronous on `stream`.
+ * ------------------------------------------------------------------------------------ */
+int ans_decode_gemm_bf16(const ans_layer_desc* h_desc, const void* d_x, int M, int N, int K, float* d_y,
+                         uint32_t* d_status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

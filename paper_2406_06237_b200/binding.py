@@ -28,7 +28,7 @@ EXPORTS = [
     "ans_host_normalize_freqs", "ans_host_pack_bound", "ans_host_pack_layer", "ans_host_pack_channels",
     "ans_noalloc_max_bytes", "ans_decode_dequant_host_noalloc",
     "ans_histogram_device", "ans_entropy_device", "ans_normalize_freqs_device",
-    "ans_encode_scratch_bytes", "ans_encode_layer_device",
+    "ans_encode_scratch_bytes", "ans_encode_layer_device", "ans_decode_gemm_bf16",
 ]
 
 
@@ -86,6 +86,7 @@ def lib():
         L.ans_host_normalize_freqs.argtypes = [vp, i32, i32, vp]
         L.ans_host_pack_bound.argtypes = [u64, u32, u32, i32, P(u64)]
         L.ans_host_pack_layer.argtypes = [vp, u64, vp, i32, i32, u32, u32, i32, vp, u64, P(u64), vp, vp, i32]
+        L.ans_decode_gemm_bf16.argtypes = [P(ans_layer_desc), vp, i32, i32, i32, vp, vp, vp]
         L.ans_host_pack_channels.argtypes = [vp, u64, vp, i32, i32, u32, u32, u32, vp, u64, P(u64), vp, i32]
         L.ans_histogram_device.argtypes = [vp, u64, vp, vp]
         L.ans_entropy_device.argtypes = [vp, i32, vp, vp]
@@ -282,3 +283,8 @@ def ans_host_pack_channels(symbols: np.ndarray, freqs: np.ndarray, alphabet: int
                                         lanes, piece_symbols, stream.ctypes.data, cap, ctypes.byref(used),
                                         offs.ctypes.data, n_threads), "ans_host_pack_channels")
     return stream[:used.value].copy(), offs, np.zeros((n_sub, 0), dtype=np.uint32)
+
+
+def ans_decode_gemm_bf16(h_desc: ans_layer_desc, d_x: int, M: int, N: int, K: int, d_y: int, d_status: int,
+                         stream: int = 0) -> None:
+    _check(lib().ans_decode_gemm_bf16(ctypes.byref(h_desc), d_x, M, N, K, d_y, d_status, stream), "ans_decode_gemm_bf16")

@@ -1,0 +1,289 @@
+// Decode fused into its consumer: Y = X * W^T with W read in compressed form, for sm_100a.
+//
+// Paper Section I and Section III-C: the weights stay compressed in memory and are decompressed
+// just before the computation that uses them, so that the decoded weights never travel to or from
+// DRAM.  Here the consumer is a bf16 matrix product on the 5th-generation tensor cores: a CTA
+// decodes 64 x 64 blocks of W (tANS states of a sub-stream's 32 lanes walked in step, Section
+// II-A; dequantised to bf16, Section II-B) straight into shared memory in the layout
+// tcgen05.mma reads its B operand from, and multiplies them with the matching 128 x 64 slices
+// of X into a 128 x 64 fp32 accumulator in tensor memory.
+//
+// W (N x K, row n = output feature) must be stored for this call in blocks of 64 x 64:
+// block (n / 64, k / 64) is 4096 consecutive symbols, row-major inside the block, blocks
+// ordered [N / 64][K / 64]; coded in the strips container with chunk_symbols = 4096 and 32
+// lanes, so that one sub-stream is one block.  X is M x K bf16 row-major, M <= 128; Y is
+// M x N fp32 row-major.
+//
+// One CTA per block row of W (64 output features).  Warps 0-3 produce: warp w takes the blocks
+// k / 64 = w, w + 4, ... of its block row, copies the slice of X and decodes the block of W into
+// stage w, and hands the stage over through an mbarrier; warp 4 owns the tensor memory and issues
+// the tcgen05.mma instructions in block order (four of K = 16 per stage), committing each stage
+// back to its producer; at the end warps 0-3 read the accumulator with tcgen05.ld and store it.
+// Every wait is bounded; a wait that runs out sets a status bit and the kernel carries on to its
+// end (tensor memory is freed on every path).
+#include "ans_decode_common.cuh"
+
+namespace ansb {
+
+constexpr uint32_t kFgBlock = 64;                 // W is cut into kFgBlock x kFgBlock blocks
+constexpr uint32_t kFgStages = 4;                 // = producer warps
+constexpr uint32_t kFgATile = 128 * 128;          // bytes: 128 rows of X, 64 bf16 each
+constexpr uint32_t kFgBTile = 64 * 128;           // bytes: 64 rows of W, 64 bf16 each
+constexpr uint32_t kFgHeader = 64;                // bytes: 32 lanes x 16-bit length (strips container)
+constexpr uint32_t kFgCols = 64;                  // tensor-memory columns: 64 fp32 accumulators per row
+
+struct FgArgs {
+  const uint8_t* blob;          // W's decode table
+  const uint8_t* stream;
+  const uint64_t* sub_offsets;
+  uint64_t stream_bytes;
+  const uint16_t* x;            // bf16 [M][K]
+  float* y;                     // [M][N]
+  uint32_t M, N, K;
+  uint32_t R, zero_point, bitwidth;
+  float scale;
+  uint32_t* d_status;
+};
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
+
+// A wait on an mbarrier phase with a limit in clock cycles (about 0.1 s); once any wait of the
+// thread has run out (a bit in `bad`), later ones only look once, so that a broken run ends fast.
+__device__ __forceinline__ bool fg_wait(uint32_t bar, uint32_t parity, uint32_t bad) {
+  const long long t0 = clock64();
+  for (;;) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+    if ((bad & kStatusTimeout) || clock64() - t0 > 200000000ll) return false;
+  }
+}
+
+// where element (row, k) of a tile of 64 bf16 per row lies: rows of 128 bytes, eight rows to a
+// 1 KB group, the 16-byte pieces of a row exchanged by the row's number in its group (the
+// 128-byte swizzle of the tensor-core operand layouts, K-major)
+__device__ __forceinline__ uint32_t tile_offset(uint32_t row, uint32_t k) {
+  return (row >> 3) * 1024u + (row & 7u) * 128u + ((((k >> 3) ^ row) & 7u) << 4) + (k & 7u) * 2u;
+}
+
+// shared-memory operand descriptor: start address, 16-byte units; leading offset 1 (unused for a
+// swizzled K-major tile); stride between 8-row groups 1024 bytes; descriptor version 1;
+// 128-byte swizzle
+__device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
+  return uint64_t((smem_addr & 0x3FFFFu) >> 4) | (uint64_t(1) << 16) | (uint64_t(1024 >> 4) << 32) |
+         (uint64_t(1) << 46) | (uint64_t(2) << 61);
+}
+
+// instruction descriptor of kind::f16: D fp32, A and B bf16, both K-major, N = 64, M = 128
+constexpr uint32_t kFgIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((kFgBlock >> 3) << 17) | ((128u >> 4) << 24);
+
+// Decode one 64 x 64 block (one sub-stream of the strips container, 128 symbols per lane, lanes in
+// step) into the B tile at b_abs.  tab: one word per state (symbol, nb_bits, newX); vals: the
+// dequantised bf16 of every symbol.  Returns status bits.
+__device__ __noinline__ uint32_t decode_block(const FgArgs& a, uint64_t sub, uint32_t tab_abs, uint32_t vals_abs,
+                                              uint32_t b_abs, uint32_t lane) {
+  uint32_t bad = 0;
+  uint64_t off0 = __ldg(a.sub_offsets + sub), off1 = __ldg(a.sub_offsets + sub + 1);
+  if (off1 < off0 || off1 > a.stream_bytes || ((off0 | off1) & 15u) || off1 - off0 < kFgHeader || off1 - off0 > 0x3FFFFFFFull) {
+    // unusable offsets: the block is left as zeros
+    for (uint32_t i = lane * 16u; i < kFgBTile; i += 512u)
+      asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" :: "r"(b_abs + i), "r"(0u) : "memory");
+    return ANS_STATUS_BAD_LENGTH;
+  }
+  const uint32_t* words = reinterpret_cast<const uint32_t*>(a.stream + off0);
+  const uint32_t ext_words = static_cast<uint32_t>((off1 - off0) >> 2);
+  auto load_word = [&](uint32_t i) -> uint32_t { return i < ext_words ? __ldg(words + i) : 0u; };
+  const uint32_t hw = load_word(lane >> 1);
+  const uint32_t len = (lane & 1u) ? hw >> 16 : hw & 0xFFFFu;
+  uint32_t incl = len;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t up = __shfl_up_sync(kFull, incl, d);
+    if (lane >= static_cast<uint32_t>(d)) incl += up;
+  }
+  const uint32_t total_bits = __shfl_sync(kFull, incl, 31);
+  if ((((kFgHeader / 4u + ((total_bits + 31u) >> 5)) + 3u) & ~3u) != ext_words) bad |= ANS_STATUS_BAD_LENGTH;
+  const uint32_t bit0 = kFgHeader * 8u + (incl - len);
+  uint32_t idx = bit0 >> 5, bitpos = bit0 & 31u;
+  uint32_t w0 = load_word(idx), w1 = load_word(idx + 1);
+  idx += 2;
+  auto take = [&](uint32_t nb) -> uint32_t {           // the next nb bits, most significant first
+    const uint32_t x = __funnelshift_l(w1, w0, bitpos);
+    const uint32_t v = nb ? x >> (32u - nb) : 0u;
+    bitpos += nb;
+    if (bitpos >= 32u) { w0 = w1; w1 = load_word(idx); ++idx; bitpos -= 32u; }
+    return v;
+  };
+  uint32_t state = take(a.R);
+  constexpr uint32_t kPerLane = kFgBlock * kFgBlock / 32u;
+  for (uint32_t t = 0; t < kPerLane; ++t) {
+    const uint32_t e = lds_u32(tab_abs + state * 4u);
+    const uint32_t q = t * 32u + lane;                   // the symbol's place in the block, row-major
+    const uint32_t val = lds_u32(vals_abs + (e & 0xFFu) * 4u);
+    sts_elem<2>(b_abs + tile_offset(q >> 6, q & 63u), val);
+    state = (e >> 16) + take((e >> 8) & 15u);
+  }
+  if (state != 0) bad |= ANS_STATUS_BAD_FINAL_STATE;
+  if ((idx - 2u) * 32u + bitpos - bit0 != len) bad |= ANS_STATUS_BAD_LENGTH;
+  return bad;
+}
+
+__global__ void __launch_bounds__(160, 1) ans_decode_gemm_kernel(const FgArgs a) {
+  extern __shared__ uint8_t sm_raw[];
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  // [A tiles][B tiles], 1 KB aligned; [table 4 << R][values 1 KB][barriers]
+  const uint32_t base = (smem_u32(sm_raw) + 1023u) & ~1023u;
+  const uint32_t a_abs = base, b_abs = base + kFgStages * kFgATile;
+  const uint32_t tab_abs = b_abs + kFgStages * kFgBTile;
+  const uint32_t vals_abs = tab_abs + (4u << a.R);
+  const uint32_t bars_abs = vals_abs + 1024u;
+  const uint32_t full_bar = bars_abs, empty_bar = bars_abs + 8u * kFgStages, done_bar = bars_abs + 16u * kFgStages;
+  const uint32_t slot_abs = done_bar + 8u;
+  uint32_t bad = 0;
+
+  if (threadIdx.x == 0) {
+    for (uint32_t s = 0; s < kFgStages; ++s) { mbar_init(full_bar + 8u * s, 1); mbar_init(empty_bar + 8u * s, 1); }
+    mbar_init(done_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 4) {                                         // this warp owns the tensor memory
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(slot_abs), "r"(kFgCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // the table, one word per state, and the dequantised value of every symbol
+  {
+    const uint32_t* g_single = reinterpret_cast<const uint32_t*>(a.blob + single_offset());
+    for (uint32_t i = threadIdx.x; i < (1u << a.R); i += blockDim.x)
+      asm volatile("st.shared.u32 [%0], %1;" :: "r"(tab_abs + i * 4u), "r"(__ldg(g_single + i)) : "memory");
+    for (uint32_t s = threadIdx.x; s < 256u; s += blockDim.x)
+      asm volatile("st.shared.u32 [%0], %1;" :: "r"(vals_abs + s * 4u),
+                   "r"(dequant_bits(static_cast<int>(s), static_cast<int>(a.zero_point), a.scale, ANS_BF16)) : "memory");
+    const TableHeader* hdr = reinterpret_cast<const TableHeader*>(a.blob);
+    if (threadIdx.x == 0 && (__ldg(&hdr->magic) != kTableMagic || __ldg(&hdr->table_log) != a.R ||
+                             __ldg(&hdr->alphabet) > (1u << a.bitwidth)))
+      bad |= ANS_STATUS_BAD_SYMBOL;
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = lds_u32(slot_abs);
+
+  const uint32_t nb_row = blockIdx.x;                      // block row of W: output features 64 nb_row ...
+  const uint32_t KB = a.K / kFgBlock;
+  if (warp < kFgStages) {
+    // ---- producers --------------------------------------------------------------------------
+    const uint32_t my_a = a_abs + warp * kFgATile, my_b = b_abs + warp * kFgBTile;
+    for (uint32_t kb = warp, it = 0; kb < KB; kb += kFgStages, ++it) {
+      if (it > 0 && !__all_sync(kFull, fg_wait(empty_bar + 8u * warp, (it - 1u) & 1u, bad))) bad |= kStatusTimeout;
+      // the slice of X: rows beyond M are zeros
+      for (uint32_t i = lane; i < 128u * 8u; i += 32u) {
+        const uint32_t r = i >> 3, c = i & 7u;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (r < a.M) v = __ldg(reinterpret_cast<const uint4*>(a.x + size_t(r) * a.K + size_t(kb) * kFgBlock + c * 8u));
+        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};"
+                     :: "r"(my_a + tile_offset(r, c * 8u)), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+      }
+      bad |= decode_block(a, uint64_t(nb_row) * KB + kb, tab_abs, vals_abs, my_b, lane);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads shared memory through the async proxy
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full_bar + 8u * warp);
+    }
+  } else if (lane == 0) {
+    // ---- the thread that issues the matrix instructions ----------------------------------------
+    for (uint32_t kb = 0; kb < KB; ++kb) {
+      const uint32_t s = kb & (kFgStages - 1u), it = kb / kFgStages;
+      if (!fg_wait(full_bar + 8u * s, it & 1u, bad)) bad |= kStatusTimeout;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint64_t da = operand_desc(a_abs + s * kFgATile), db = operand_desc(b_abs + s * kFgBTile);
+#pragma unroll
+      for (uint32_t j = 0; j < kFgBlock / 16u; ++j) {      // K = 16 per instruction: 32 bytes further along the rows
+        const uint32_t accumulate = (kb | j) ? 1u : 0u;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+            :: "r"(tmem), "l"(da + 2u * j), "l"(db + 2u * j), "r"(kFgIdesc), "r"(accumulate), "r"(0u) : "memory");
+      }
+      // the stage is free again once these have read it
+      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(empty_bar + 8u * s) : "memory");
+    }
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(done_bar) : "memory");
+  }
+
+  // ---- the accumulator: row m of Y in lane m of the tensor memory, 64 columns -------------------
+  if (warp < 4) {
+    __syncwarp();
+    if (!__all_sync(kFull, fg_wait(done_bar, 0, bad))) bad |= kStatusTimeout;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t row = warp * 32u + lane;
+    float* yrow = a.y + size_t(row) * a.N + size_t(nb_row) * kFgBlock;
+#pragma unroll
+    for (uint32_t c0 = 0; c0 < kFgCols; c0 += 8u) {
+      uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
+      asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                   : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3), "=r"(r4), "=r"(r5), "=r"(r6), "=r"(r7)
+                   : "r"(tmem + ((warp * 32u) << 16) + c0) : "memory");
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      if (row < a.M) {
+        *reinterpret_cast<uint4*>(yrow + c0) = make_uint4(r0, r1, r2, r3);
+        *reinterpret_cast<uint4*>(yrow + c0 + 4) = make_uint4(r4, r5, r6, r7);
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 4) {
+    __syncwarp();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kFgCols) : "memory");
+  }
+  bad = __reduce_or_sync(kFull, bad);
+  if (lane == 0 && bad && a.d_status) atomicOr(a.d_status, bad);
+}
+
+}  // namespace ansb
+
+using namespace ansb;
+
+ANS_EXPORT int ans_decode_gemm_bf16(const ans_layer_desc* h_desc, const void* d_x, int M, int N, int K, float* d_y,
+                                    uint32_t* d_status, void* stream) {
+  ApiRange range("ans_decode_gemm_bf16");
+  if (!h_desc || !d_x || !d_y || !d_status) return ANS_ERR_INVALID_ARG;
+  const ans_layer_desc& d = *h_desc;
+  int rc = validate_desc(d, false);
+  if (rc != ANS_OK) return rc;
+  if (d.layout != ANS_LAYOUT_STRIPS || d.chunk_symbols != kFgBlock * kFgBlock || d.lanes != 32 || d.table_log > 12)
+    return ANS_ERR_UNSUPPORTED;
+  if (M < 1 || M > 128 || N < 64 || K < 64 || N % 64 || K % 64 || N > (1 << 20) || K > (1 << 20)) return ANS_ERR_UNSUPPORTED;
+  if (d.n_symbols != uint64_t(N) * uint64_t(K)) return ANS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_x) & 15) || (reinterpret_cast<uintptr_t>(d_y) & 15)) return ANS_ERR_INVALID_ARG;
+  FgArgs a{};
+  a.blob = static_cast<const uint8_t*>(d.d_table);
+  a.stream = d.d_stream;
+  a.sub_offsets = d.d_sub_offsets;
+  a.stream_bytes = d.stream_bytes;
+  a.x = static_cast<const uint16_t*>(d_x);
+  a.y = d_y;
+  a.M = static_cast<uint32_t>(M);
+  a.N = static_cast<uint32_t>(N);
+  a.K = static_cast<uint32_t>(K);
+  a.R = static_cast<uint32_t>(d.table_log);
+  a.zero_point = static_cast<uint32_t>(d.zero_point);
+  a.bitwidth = static_cast<uint32_t>(d.bitwidth);
+  a.scale = d.scale;
+  a.d_status = d_status;
+  const size_t smem = 1024 + kFgStages * (kFgATile + kFgBTile) + (size_t(4) << d.table_log) + 1024 + 128;
+  ANSB_CUDA(cudaFuncSetAttribute(ans_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  ans_decode_gemm_kernel<<<static_cast<unsigned>(N / 64), 160, smem, static_cast<cudaStream_t>(stream)>>>(a);
+  ANSB_CUDA(cudaGetLastError());
+  return ANS_OK;
+}

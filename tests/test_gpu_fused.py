@@ -1,0 +1,78 @@
+"""Decode fused into a bf16 matrix product (Section I, Section III-C: weights are decompressed
+just before the computation that uses them) against the oracle: W is decoded and dequantised by
+the ORACLE, the product is taken in float64 on the host, and the GPU's fp32-accumulated result
+must agree within the bound of fp32 accumulation over K terms."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synthgen as sg
+import paper_2406_06237_b200 as ans
+from paper_2406_06237_b200.runtime import DeviceBatch
+from helpers import oracle_pack_spec, to_packed_layer
+
+pytestmark = pytest.mark.gpu
+
+
+def _bf16_bits_to_f64(bits):
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def _blocked(w):
+    """N x K -> the order the fused call wants: blocks of 64 x 64, [N/64][K/64][64][64]."""
+    n, k = w.shape
+    return np.ascontiguousarray(w.reshape(n // 64, 64, k // 64, 64).transpose(0, 2, 1, 3)).ravel()
+
+
+def _case(M, N, K, b, pzp, R, seed, scale=0.03125):
+    A, zp = sg.alphabet_for_bits(b)
+    spec = sg.LayerSpec(f"w{N}x{K}", (N, K), b, A, zp, sg.theta_for_pzp(A, zp, pzp), scale, R, 4096, "bf16",
+                        sg.stream_key(31, seed))
+    w_sym = sg.draw_symbols(spec).reshape(N, K)
+    T, P, f256 = oracle_pack_spec(spec, _blocked(w_sym), oracle.STRIPS, 32)
+    dec, rc = oracle.unpack(T, P)
+    assert rc == oracle.OK
+    w_bits = oracle.dequant(dec, zp, scale, "bf16")           # blocked order
+    w = _bf16_bits_to_f64(w_bits).reshape(N // 64, K // 64, 64, 64).transpose(0, 2, 1, 3).reshape(N, K)
+    rng = np.random.default_rng(seed)
+    x = torch.from_numpy(rng.standard_normal((M, K)).astype(np.float32)).to(torch.bfloat16)
+    x64 = x.to(torch.float32).numpy().astype(np.float64)
+    return spec, P, f256, x, x64, w
+
+
+@pytest.mark.parametrize("M,N,K,b,pzp,R", [(128, 64, 64, 3, 0.7, 8), (128, 128, 256, 4, 0.6, 8), (1, 64, 128, 2, 0.9, 6),
+                                           (77, 192, 320, 5, 0.85, 10), (128, 512, 1024, 3, 0.7, 12),
+                                           (16, 64, 2048, 8, 0.9, 8)])
+def test_fused_product_equals_the_oracles_weights_times_x(M, N, K, b, pzp, R):
+    spec, P, f256, x, x64, w = _case(M, N, K, b, pzp, R, seed=M + N + K)
+    db = DeviceBatch([to_packed_layer(spec, P, f256)])         # the table and the compressed bytes on the device
+    xd = x.cuda()
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    guard = torch.full((4096,), 7.0, dtype=torch.float32, device="cuda")
+    ans.ans_decode_gemm_bf16(db.h_descs[0][0], xd.data_ptr(), M, N, K, y.data_ptr(), db.status.data_ptr(),
+                             torch.cuda.current_stream().cuda_stream)
+    assert db.read_status() == 0
+    got = y.cpu().numpy().astype(np.float64)
+    want = x64 @ w.T
+    # products of two bf16 values are exact in fp32; the sums over K terms are rounded to fp32
+    bound = (np.abs(x64) @ np.abs(w).T) * (K * 2.0 ** -24) + 1e-30
+    assert np.isfinite(got).all() and (np.abs(got - want) <= bound).all(), float(np.abs(got - want).max())
+    assert (guard == 7.0).all()
+
+
+def test_fused_call_flags_a_corrupt_block_and_refuses_what_it_does_not_support():
+    spec, P, f256, x, x64, w = _case(32, 128, 128, 3, 0.7, 8, seed=5)
+    s = P.stream.copy()
+    s[int(P.sub_offsets[2]) + 100] ^= 0x55
+    P2 = oracle.Packed(P.layout, s, P.sub_offsets, P.lane_meta, P.n, P.chunk, P.groups)
+    T = oracle.Table(f256[:spec.alphabet], 8)
+    assert oracle.unpack(T, P2)[1] == oracle.ERR_CORRUPT
+    db = DeviceBatch([to_packed_layer(spec, P2, f256)])
+    y = torch.zeros((32, 128), dtype=torch.float32, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    ans.ans_decode_gemm_bf16(db.h_descs[0][0], x.cuda().data_ptr(), 32, 128, 128, y.data_ptr(), db.status.data_ptr(), st)
+    assert db.read_status() != 0
+    for M, N, K in ((129, 128, 128), (32, 100, 128), (32, 128, 64)):   # too many rows; N no multiple of 64; N * K != n_symbols
+        with pytest.raises(ans.AnsError):
+            ans.ans_decode_gemm_bf16(db.h_descs[0][0], x.cuda().data_ptr(), M, N, K, y.data_ptr(), db.status.data_ptr(), st)
