@@ -22,6 +22,7 @@
 // Every wait is bounded; a wait that runs out sets a status bit and the kernel carries on to its
 // end (tensor memory is freed on every path).
 #include "ans_decode_common.cuh"
+#include "ans_walk_strips.cuh"
 
 namespace ansb {
 
@@ -250,6 +251,291 @@ __global__ void __launch_bounds__(160, 1) ans_decode_gemm_kernel(const FgArgs a)
   if (lane == 0 && bad && a.d_status) atomicOr(a.d_status, bad);
 }
 
+// ---------------------------------------------------------------------------------------------
+// The wide form, for tables of up to 256 states (the paper's sizes) and N a multiple of 256.
+//
+// A CTA owns 256 output features (four block rows of W) and a range of K (the K dimension is
+// split over CTAs so that the grid fills the device; partial sums meet in Y by fp32 atomic
+// adds when there is more than one range).  Sixteen producer warps: stage s = warp / 4 holds a
+// 128 x 64 slice of X and the four 64 x 64 blocks of W under it, warp 4 s + i decodes block i
+// with the strips kernel's walk (pre-walked table: a look-up stands for a run of the dominant
+// symbol plus one symbol, Section II-A) into a plain row-major tile pre-filled with the
+// dominant value, then puts the tile's 16-byte pieces in the swizzled order in place.  The
+// sub-stream's bytes come into shared memory by asynchronous copies issued one block ahead.
+// Warp 16 issues one tcgen05.mma of N = 256 per 16 columns of K.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kF2Stages = 4;
+constexpr uint32_t kF2Rows = 4;                   // block rows of W per CTA
+constexpr uint32_t kF2Producers = kF2Stages * kF2Rows;
+constexpr uint32_t kF2Threads = (kF2Producers + 1) * 32;
+constexpr uint32_t kF2BTile = kF2Rows * kFgBTile; // bytes: 256 rows of W, 64 bf16 each
+constexpr uint32_t kF2Cols = kF2Rows * kFgBlock;  // tensor-memory columns
+constexpr uint32_t kF2Pad = 256;                  // zero bytes after a staged sub-stream: more than a lane can
+                                                  // advance in the 128 look-ups of a block (8 bits each at most)
+constexpr uint32_t kF2Idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((kF2Cols >> 3) << 17) | ((128u >> 4) << 24);
+
+struct F2Args {
+  FgArgs g;
+  uint32_t kb_per_split;        // blocks of K per CTA range
+  uint32_t stage_bytes;         // per producer: room for a sub-stream's bytes and the padding
+  uint32_t rep_log;             // copies of the table, log2
+  uint32_t unit;                // the value 1
+};
+
+// Decode one block (one sub-stream: 128 symbols per lane) into the row-major tile at tile_abs,
+// which holds the dominant value everywhere.  The sub-stream's words are in shared memory at
+// stage_abs (staged, zero words after them) or in global memory.  Returns status bits.
+__device__ __noinline__ uint32_t decode_block_wide(uint32_t tab_lane, uint32_t stride_log, uint32_t succ_abs,
+                                                   uint32_t tile_abs, uint32_t stage_abs,
+                                                   const uint32_t* __restrict__ words, uint32_t ext_words, bool staged,
+                                                   uint32_t R, uint32_t unit, uint32_t lane) {
+  constexpr uint32_t count = kFgBlock * kFgBlock / 32u;
+  const uint32_t word_limit = staged ? ext_words + 4u : ext_words;
+  auto load_word = [&](uint32_t i) -> uint32_t {
+    if (staged) return lds_u32(stage_abs + min(i, word_limit + 8u) * 4u);
+    return i < word_limit ? __ldg(words + i) : 0u;
+  };
+  uint32_t bad = 0;
+  const uint32_t hw = load_word(lane >> 1);
+  const uint32_t len = (lane & 1u) ? hw >> 16 : hw & 0xFFFFu;
+  uint32_t incl = len;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t up = __shfl_up_sync(kFull, incl, d);
+    if (lane >= static_cast<uint32_t>(d)) incl += up;
+  }
+  const uint32_t total_bits = __shfl_sync(kFull, incl, 31);
+  if (ext_words < kFgHeader / 4u || (((kFgHeader / 4u + ((total_bits + 31u) >> 5)) + 3u) & ~3u) != ext_words)
+    bad |= ANS_STATUS_BAD_LENGTH;
+  const uint32_t bit0 = kFgHeader * 8u + (incl - len);
+  uint32_t idx = bit0 >> 5, bitpos = bit0 & 31u;
+  uint32_t w0 = load_word(idx), w1 = load_word(idx + 1), w2 = load_word(idx + 2);
+  idx += 3;
+  uint32_t state = __funnelshift_l(w1, w0, bitpos) >> (32u - R);   // the string begins with the state, R bits
+  bitpos += R;
+  if (bitpos >= 32u) { w0 = w1; w1 = w2; w2 = load_word(idx); ++idx; bitpos -= 32u; }
+  const uint32_t stride = 1u << stride_log;
+  uint32_t st = tab_lane + (state << stride_log);
+  uint32_t z = 0;
+  const uint32_t abase = tile_abs + lane * 2u;             // position z of this lane: row z / 2 of the tile
+  if (staged) {
+    const uint32_t sp_limit = stage_abs + word_limit * 4u;
+    uint32_t sp = min(stage_abs + min(idx, word_limit) * 4u, sp_limit);
+    strip_window_walk<2, 4, true, false>(st, bitpos, w0, w1, w2, sp, z, tab_lane, stride, abase, count, unit, sp_limit, 0u, 0u);
+    if (sp >= sp_limit) bad |= ANS_STATUS_BAD_LENGTH;
+    idx = (sp - stage_abs) >> 2;
+  } else {
+    bool any = true;
+    while (any) {
+      const uint32_t ea = lds_u32(st);
+      const uint32_t nb = (ea >> 16) & 15u, zn = z + ((ea >> 20) & 15u);
+      const bool act = zn < count;
+      if (act) {
+        sts_elem<2>(abase + zn * 64u, ea);
+        const uint32_t x = __funnelshift_l(w1, w0, bitpos);
+        st = tab_lane + (__funnelshift_l(x, ea >> 24, nb) << stride_log);
+        z = zn + 1u;
+        bitpos += nb;
+        if (bitpos >= 32u) { w0 = w1; w1 = w2; w2 = load_word(idx); ++idx; bitpos -= 32u; }
+      }
+      any = __any_sync(kFull, act);
+    }
+  }
+  // what is left of the lane lies inside the run of the entry it stopped at
+  uint32_t s = (st - tab_lane) >> stride_log;
+  for (uint32_t left = count - z; left != 0 && left <= uint32_t(kMaxRun); --left) s = lds_u16(succ_abs + s * 2u);
+  if (count - z > uint32_t(kMaxRun) || s != 0) bad |= ANS_STATUS_BAD_FINAL_STATE;
+  if ((idx - 3u) * 32u + bitpos - bit0 != len) bad |= ANS_STATUS_BAD_LENGTH;
+  return bad;
+}
+
+__global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(const F2Args args) {
+  extern __shared__ uint8_t sm_raw[];
+  const FgArgs& a = args.g;
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  // [A tiles][B tiles], 1 KB aligned; [table copies][successors][byte stages][barriers]
+  const uint32_t base = (smem_u32(sm_raw) + 1023u) & ~1023u;
+  const uint32_t a_abs = base, b_abs = base + kF2Stages * kFgATile;
+  const uint32_t tab_abs = b_abs + kF2Stages * kF2BTile;
+  const uint32_t stride_log = 2u + args.rep_log;
+  const uint32_t succ_abs = tab_abs + (1u << (a.R + stride_log));
+  const uint32_t succ_bytes = max(2u << a.R, 16u);
+  const uint32_t stages_abs = succ_abs + succ_bytes;
+  const uint32_t bars_abs = stages_abs + kF2Producers * args.stage_bytes;
+  const uint32_t full_bar = bars_abs, empty_bar = bars_abs + 8u * kF2Stages, done_bar = bars_abs + 16u * kF2Stages;
+  const uint32_t slot_abs = done_bar + 8u;
+  uint32_t bad = 0;
+
+  if (threadIdx.x == 0) {
+    for (uint32_t s = 0; s < kF2Stages; ++s) { mbar_init(full_bar + 8u * s, kF2Rows); mbar_init(empty_bar + 8u * s, 1); }
+    mbar_init(done_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kF2Producers) {                              // this warp owns the tensor memory
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(slot_abs), "r"(kF2Cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // the pre-walked table in one-word entries, the bf16 value folded in, copies side by side
+  const TableHeader* hdr = reinterpret_cast<const TableHeader*>(a.blob);
+  const uint32_t h_dominant = __ldg(&hdr->dominant);
+  {
+    const uint32_t* g_single = reinterpret_cast<const uint32_t*>(a.blob + single_offset());
+    const uint32_t* g_multi = reinterpret_cast<const uint32_t*>(a.blob + multi_offset(static_cast<int>(a.R)));
+    for (uint32_t i = threadIdx.x; i < (1u << a.R); i += blockDim.x) {
+      const uint32_t gm = __ldg(g_multi + i), gs = __ldg(g_single + i);
+      const uint32_t val = dequant_bits(static_cast<int>(entry_sym(gm)), static_cast<int>(a.zero_point), a.scale, ANS_BF16);
+      const uint32_t e = to_strip_entry_short(gm, val);
+      for (uint32_t c = 0; c < (1u << args.rep_log); ++c)
+        asm volatile("st.shared.u32 [%0], %1;" :: "r"(tab_abs + (i << stride_log) + c * 4u), "r"(e) : "memory");
+      asm volatile("st.shared.u16 [%0], %1;" :: "r"(succ_abs + i * 2u), "r"(entry_newx(gs)) : "memory");
+    }
+    if (threadIdx.x == 0 && (__ldg(&hdr->magic) != kTableMagic || __ldg(&hdr->table_log) != a.R ||
+                             __ldg(&hdr->alphabet) > (1u << a.bitwidth)))
+      bad |= ANS_STATUS_BAD_SYMBOL;
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = lds_u32(slot_abs);
+
+  const uint32_t KB = a.K / kFgBlock;
+  const uint32_t kb0 = blockIdx.y * args.kb_per_split;
+  const uint32_t nk = min(KB, kb0 + args.kb_per_split) - kb0;   // (the host leaves no range empty)
+  if (warp < kF2Producers) {
+    // ---- producers --------------------------------------------------------------------------
+    const uint32_t s = warp / kF2Rows, i = warp % kF2Rows;
+    const uint32_t my_a = a_abs + s * kFgATile, my_b = b_abs + s * kF2BTile + i * kFgBTile;
+    const uint32_t my_stage = stages_abs + warp * args.stage_bytes;
+    const uint32_t tab_lane = tab_abs + ((lane & ((1u << args.rep_log) - 1u)) << 2);
+    const uint32_t dom = dequant_bits(static_cast<int>(h_dominant < 256u ? h_dominant : 0u), static_cast<int>(a.zero_point),
+                                      a.scale, ANS_BF16);
+    const uint32_t fill = (dom & 0xFFFFu) * 0x10001u;
+    const uint4 fill4 = make_uint4(fill, fill, fill, fill);
+    const uint64_t sub0 = uint64_t(blockIdx.x * kF2Rows + i) * KB + kb0;   // the block row's first sub-stream of the range
+
+    // the extent of a sub-stream, checked; its bytes requested into the warp's stage when they fit
+    uint64_t off0 = 0;
+    uint32_t extent = 0;
+    bool staged = false;
+    auto locate = [&](uint64_t o0, uint64_t o1) {
+      off0 = o0;
+      extent = static_cast<uint32_t>(o1 - o0);
+      if (o1 < o0 || o1 > a.stream_bytes || ((o0 | o1) & 15u) || o1 - o0 < kFgHeader || o1 - o0 > 0x3FFFFFFFull) {
+        extent = 0;
+        off0 = 0;
+        bad |= ANS_STATUS_BAD_LENGTH;
+      }
+      staged = extent > 0 && extent + kF2Pad <= args.stage_bytes;
+      if (staged) {
+        const uint8_t* src = a.stream + off0;
+        for (uint32_t o = lane * 16u; o < extent; o += 512u)
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(my_stage + o), "l"(src + o) : "memory");
+        for (uint32_t q = lane; q < kF2Pad / 4u; q += 32u)
+          asm volatile("st.shared.u32 [%0], %1;" :: "r"(my_stage + extent + q * 4u), "r"(0u) : "memory");
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    uint64_t n0 = 0, n1 = 0;                               // offsets of the block after this one
+    if (s < nk) locate(__ldg(a.sub_offsets + sub0 + s), __ldg(a.sub_offsets + sub0 + s + 1));
+    for (uint32_t j = s, it = 0; j < nk; j += kF2Stages, ++it) {
+      const bool more = j + kF2Stages < nk;
+      if (more) {
+        n0 = __ldg(a.sub_offsets + sub0 + j + kF2Stages);
+        n1 = __ldg(a.sub_offsets + sub0 + j + kF2Stages + 1);
+      }
+      if (it > 0 && !__all_sync(kFull, fg_wait(empty_bar + 8u * s, (it - 1u) & 1u, bad))) bad |= kStatusTimeout;
+      // this warp's quarter of the slice of X: rows beyond M are zeros
+#pragma unroll
+      for (uint32_t q = 0; q < 8u; ++q) {
+        const uint32_t c = lane & 7u, r = i * 32u + q * 4u + (lane >> 3);
+        const uint32_t bytes = r < a.M ? 16u : 0u;
+        const uint16_t* src = a.x + size_t(r < a.M ? r : 0u) * a.K + size_t(kb0 + j) * kFgBlock + c * 8u;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(my_a + tile_offset(r, c * 8u)), "l"(src), "r"(bytes) : "memory");
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      for (uint32_t o = lane * 16u; o < kFgBTile; o += 512u) sts_v4(my_b + o, fill4);
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      __syncwarp();
+      if (extent)
+        bad |= decode_block_wide(tab_lane, stride_log, succ_abs, my_b, my_stage,
+                                 reinterpret_cast<const uint32_t*>(a.stream + off0), extent >> 2, staged, a.R, args.unit, lane);
+      __syncwarp();
+      // the stage's bytes are used up: the next block's may come while the tile is put in order
+      if (more) locate(n0, n1);
+      // rows of 128 bytes, their 16-byte pieces exchanged by the row's number in its group of
+      // eight (the 128-byte swizzle): four rows a round, every lane one piece
+#pragma unroll 4
+      for (uint32_t q = 0; q < kFgBlock / 4u; ++q) {
+        const uint32_t r = q * 4u + (lane >> 3), c = lane & 7u;
+        const uint4 v = lds_v4(my_b + r * 128u + c * 16u);
+        __syncwarp();
+        sts_v4(my_b + r * 128u + ((c ^ (r & 7u)) << 4), v);
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads shared memory through the async proxy
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full_bar + 8u * s);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+  } else if (lane == 0) {
+    // ---- the thread that issues the matrix instructions ----------------------------------------
+    for (uint32_t j = 0; j < nk; ++j) {
+      const uint32_t s = j & (kF2Stages - 1u), it = j / kF2Stages;
+      if (!fg_wait(full_bar + 8u * s, it & 1u, bad)) bad |= kStatusTimeout;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint64_t da = operand_desc(a_abs + s * kFgATile), db = operand_desc(b_abs + s * kF2BTile);
+#pragma unroll
+      for (uint32_t k = 0; k < kFgBlock / 16u; ++k) {      // K = 16 per instruction: 32 bytes further along the rows
+        const uint32_t accumulate = (j | k) ? 1u : 0u;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+            :: "r"(tmem), "l"(da + 2u * k), "l"(db + 2u * k), "r"(kF2Idesc), "r"(accumulate), "r"(0u) : "memory");
+      }
+      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(empty_bar + 8u * s) : "memory");
+    }
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(done_bar) : "memory");
+  }
+
+  // ---- the accumulator: row m of Y in lane m of the tensor memory, 256 columns -------------------
+  if (warp < 4) {
+    __syncwarp();
+    if (!__all_sync(kFull, fg_wait(done_bar, 0, bad))) bad |= kStatusTimeout;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t row = warp * 32u + lane;
+    float* yrow = a.y + size_t(row) * a.N + size_t(blockIdx.x) * kF2Cols;
+    const bool add = gridDim.y > 1;
+#pragma unroll 4
+    for (uint32_t c0 = 0; c0 < kF2Cols; c0 += 8u) {
+      uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
+      asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                   : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3), "=r"(r4), "=r"(r5), "=r"(r6), "=r"(r7)
+                   : "r"(tmem + ((warp * 32u) << 16) + c0) : "memory");
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      if (row < a.M) {
+        if (add) {
+          atomicAdd(reinterpret_cast<float4*>(yrow + c0),
+                    make_float4(__uint_as_float(r0), __uint_as_float(r1), __uint_as_float(r2), __uint_as_float(r3)));
+          atomicAdd(reinterpret_cast<float4*>(yrow + c0 + 4),
+                    make_float4(__uint_as_float(r4), __uint_as_float(r5), __uint_as_float(r6), __uint_as_float(r7)));
+        } else {
+          *reinterpret_cast<uint4*>(yrow + c0) = make_uint4(r0, r1, r2, r3);
+          *reinterpret_cast<uint4*>(yrow + c0 + 4) = make_uint4(r4, r5, r6, r7);
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == kF2Producers) {
+    __syncwarp();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kF2Cols) : "memory");
+  }
+  bad = __reduce_or_sync(kFull, bad);
+  if (lane == 0 && bad && a.d_status) atomicOr(a.d_status, bad);
+}
+
 }  // namespace ansb
 
 using namespace ansb;
@@ -281,9 +567,50 @@ ANS_EXPORT int ans_decode_gemm_bf16(const ans_layer_desc* h_desc, const void* d_
   a.bitwidth = static_cast<uint32_t>(d.bitwidth);
   a.scale = d.scale;
   a.d_status = d_status;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int dev = 0, sms = 0, smem_max = 0;
+  ANSB_CUDA(cudaGetDevice(&dev));
+  ANSB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  ANSB_CUDA(cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+  if (d.table_log <= 8 && N % static_cast<int>(kF2Cols) == 0) {
+    // the wide form: room for a sub-stream of up to 1.25 times the average plus the padding per
+    // producer, less if shared memory is short (a sub-stream that does not fit is read from global
+    // memory); what shared memory is left goes to copies of the table
+    const uint64_t n_sub = uint64_t(N / 64) * uint64_t(K / 64);
+    size_t stage = static_cast<size_t>(d.stream_bytes / n_sub);
+    stage = (stage + stage / 4 + 128 + kF2Pad + 127) & ~size_t(127);
+    const size_t succ = (size_t(2) << d.table_log) < 16 ? 16 : (size_t(2) << d.table_log);
+    const size_t one_table = size_t(4) << d.table_log;
+    const size_t rest = 1024 + kF2Stages * (kFgATile + kF2BTile) + succ + 128;
+    const size_t room = static_cast<size_t>(smem_max) > rest + one_table ? static_cast<size_t>(smem_max) - rest - one_table : 0;
+    if (kF2Producers * stage > room) stage = (room / kF2Producers) & ~size_t(127);
+    const size_t fixed = rest + kF2Producers * stage;
+    if (stage >= 512) {
+      uint32_t rep_log = 0;
+      while (rep_log < 5 && fixed + (one_table << (rep_log + 1)) <= static_cast<size_t>(smem_max)) ++rep_log;
+      const uint32_t KB = static_cast<uint32_t>(K / 64), tiles = static_cast<uint32_t>(N) / kF2Cols;
+      uint32_t splits = static_cast<uint32_t>(sms) / tiles;
+      if (splits < 1) splits = 1;
+      if (splits > KB) splits = KB;
+      const uint32_t per = (KB + splits - 1) / splits;
+      splits = (KB + per - 1) / per;                       // no range is empty
+      F2Args w{};
+      w.g = a;
+      w.kb_per_split = per;
+      w.stage_bytes = static_cast<uint32_t>(stage);
+      w.rep_log = rep_log;
+      w.unit = 1u;
+      const size_t smem = fixed + (one_table << rep_log);
+      if (splits > 1) ANSB_CUDA(cudaMemsetAsync(d_y, 0, size_t(M) * size_t(N) * sizeof(float), st));
+      ANSB_CUDA(cudaFuncSetAttribute(ans_decode_gemm_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+      ans_decode_gemm_wide_kernel<<<dim3(tiles, splits), kF2Threads, smem, st>>>(w);
+      ANSB_CUDA(cudaGetLastError());
+      return ANS_OK;
+    }
+  }
   const size_t smem = 1024 + kFgStages * (kFgATile + kFgBTile) + (size_t(4) << d.table_log) + 1024 + 128;
   ANSB_CUDA(cudaFuncSetAttribute(ans_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-  ans_decode_gemm_kernel<<<static_cast<unsigned>(N / 64), 160, smem, static_cast<cudaStream_t>(stream)>>>(a);
+  ans_decode_gemm_kernel<<<static_cast<unsigned>(N / 64), 160, smem, st>>>(a);
   ANSB_CUDA(cudaGetLastError());
   return ANS_OK;
 }

@@ -25,11 +25,14 @@ def _blocked(w):
     return np.ascontiguousarray(w.reshape(n // 64, 64, k // 64, 64).transpose(0, 2, 1, 3)).ravel()
 
 
-def _case(M, N, K, b, pzp, R, seed, scale=0.03125):
+def _case(M, N, K, b, pzp, R, seed, scale=0.03125, quiet_rows=0):
     A, zp = sg.alphabet_for_bits(b)
     spec = sg.LayerSpec(f"w{N}x{K}", (N, K), b, A, zp, sg.theta_for_pzp(A, zp, pzp), scale, R, 4096, "bf16",
                         sg.stream_key(31, seed))
     w_sym = sg.draw_symbols(spec).reshape(N, K)
+    if quiet_rows:                          # only every quiet_rows-th block row keeps its weights: sub-streams of very unequal length
+        keep = (np.arange(N) // 64) % quiet_rows == 0
+        w_sym[~keep] = zp
     T, P, f256 = oracle_pack_spec(spec, _blocked(w_sym), oracle.STRIPS, 32)
     dec, rc = oracle.unpack(T, P)
     assert rc == oracle.OK
@@ -59,6 +62,48 @@ def test_fused_product_equals_the_oracles_weights_times_x(M, N, K, b, pzp, R):
     bound = (np.abs(x64) @ np.abs(w).T) * (K * 2.0 ** -24) + 1e-30
     assert np.isfinite(got).all() and (np.abs(got - want) <= bound).all(), float(np.abs(got - want).max())
     assert (guard == 7.0).all()
+
+
+# The wide form of the kernel (tables of up to 256 states, N a multiple of 256): K split over CTAs
+# with the partial sums added in Y, stages reused many times, one range only (plain stores), a
+# ragged last range, M below a full tile.
+@pytest.mark.parametrize("M,N,K,b,pzp,R,quiet", [(128, 256, 256, 3, 0.7, 8, 0), (50, 512, 1024, 4, 0.6, 8, 0),
+                                                 (128, 2048, 4800, 3, 0.8, 8, 0), (8, 19200, 640, 2, 0.9, 6, 0),
+                                                 (33, 256, 64, 3, 0.7, 7, 0), (128, 1024, 2048, 6, 0.5, 8, 3),
+                                                 (64, 256, 19008, 3, 0.7, 8, 0)])
+def test_wide_form_equals_the_oracles_weights_times_x(M, N, K, b, pzp, R, quiet):
+    spec, P, f256, x, x64, w = _case(M, N, K, b, pzp, R, seed=M + N + K, quiet_rows=quiet)
+    if quiet:                               # the kept block rows' sub-streams are far above the average: they do not fit the staging room
+        ext = np.diff(P.sub_offsets.astype(np.int64))
+        assert ext.max() > 1.25 * ext.mean() + 512
+    db = DeviceBatch([to_packed_layer(spec, P, f256)])
+    xd = x.cuda()
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    guard = torch.full((4096,), 7.0, dtype=torch.float32, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    for _ in range(2):                      # twice: the second call must not add to the first call's sums
+        ans.ans_decode_gemm_bf16(db.h_descs[0][0], xd.data_ptr(), M, N, K, y.data_ptr(), db.status.data_ptr(), st)
+    assert db.read_status() == 0
+    got = y.cpu().numpy().astype(np.float64)
+    want = x64 @ w.T
+    bound = (np.abs(x64) @ np.abs(w).T) * ((K + 64) * 2.0 ** -24) + 1e-30
+    assert np.isfinite(got).all() and (np.abs(got - want) <= bound).all(), float(np.abs(got - want).max())
+    assert (guard == 7.0).all()
+
+
+def test_wide_form_flags_a_corrupt_block():
+    spec, P, f256, x, x64, w = _case(32, 256, 256, 3, 0.7, 8, seed=6)
+    for where in (100, 3):                  # inside a lane's bits; inside the lengths that head the sub-stream
+        s = P.stream.copy()
+        s[int(P.sub_offsets[5]) + where] ^= 0x55
+        P2 = oracle.Packed(P.layout, s, P.sub_offsets, P.lane_meta, P.n, P.chunk, P.groups)
+        assert oracle.unpack(oracle.Table(f256[:spec.alphabet], 8), P2)[1] == oracle.ERR_CORRUPT
+        db = DeviceBatch([to_packed_layer(spec, P2, f256)])
+        y = torch.zeros((32, 256), dtype=torch.float32, device="cuda")
+        ans.ans_decode_gemm_bf16(db.h_descs[0][0], x.cuda().data_ptr(), 32, 256, 256, y.data_ptr(), db.status.data_ptr(),
+                                 torch.cuda.current_stream().cuda_stream)
+        assert db.read_status() != 0
+        assert torch.isfinite(y).all()
 
 
 def test_fused_call_flags_a_corrupt_block_and_refuses_what_it_does_not_support():
