@@ -359,8 +359,11 @@ int ans_encode_layer_device(const uint8_t* d_symbols, uint64_t n_symbols, const 
  * bfloat16 exactly as ans_decode_dequant would (Section II-B).
  *   h_desc: W's layer: ANS_LAYOUT_STRIPS, chunk_symbols = 4096, lanes = 32, table_log <= 12,
  *           n_symbols = N * K, the symbols being W in blocks of 64 x 64: block (n / 64, k / 64)
- *           holds 4096 consecutive symbols, row-major inside the block, blocks ordered
- *           [N / 64][K / 64].  d_out / out_dtype are ignored.
+ *           holds 4096 consecutive symbols, blocks ordered [N / 64][K / 64].  Inside a block
+ *           element (r, c) (r: output feature, c: input feature, both modulo 64) is symbol
+ *             (r / 8) * 512 + (r % 8) * 64 + ((c / 8) ^ (r % 8)) * 8 + c % 8
+ *           (the order in which the tensor core reads a 128-byte-swizzled K-major tile, so
+ *           that a decoded block is an operand as it lies).  d_out / out_dtype are ignored.
  *   1 <= M <= 128; N and K multiples of 64; d_x and d_y 16-byte aligned.
  * d_status as for the decode calls.  Asynchronous on `stream`.
  * ------------------------------------------------------------------------------------ */

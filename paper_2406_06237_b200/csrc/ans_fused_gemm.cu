@@ -9,9 +9,11 @@
 // of X into a 128 x 64 fp32 accumulator in tensor memory.
 //
 // W (N x K, row n = output feature) must be stored for this call in blocks of 64 x 64:
-// block (n / 64, k / 64) is 4096 consecutive symbols, row-major inside the block, blocks
-// ordered [N / 64][K / 64]; coded in the strips container with chunk_symbols = 4096 and 32
-// lanes, so that one sub-stream is one block.  X is M x K bf16 row-major, M <= 128; Y is
+// block (n / 64, k / 64) is 4096 consecutive symbols, blocks ordered [N / 64][K / 64]; coded in
+// the strips container with chunk_symbols = 4096 and 32 lanes, so that one sub-stream is one
+// block.  Inside a block the symbols lie in the order the tensor core reads the tile from shared
+// memory (rows of 64, the eight 8-element pieces of row r exchanged by r mod 8: tile_offset
+// below), so that symbol q of the block is simply the q-th bf16 of the tile.  X is M x K bf16 row-major, M <= 128; Y is
 // M x N fp32 row-major.
 //
 // One CTA per block row of W (64 output features).  Warps 0-3 produce: warp w takes the blocks
@@ -55,13 +57,15 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 
 // A wait on an mbarrier phase with a limit in clock cycles (about 0.1 s); once any wait of the
 // thread has run out (a bit in `bad`), later ones only look once, so that a broken run ends fast.
+// try_wait lets the hardware park the thread for a while instead of having it poll: a waiting
+// warp then leaves the issue slots to the warps that decode.
 __device__ __forceinline__ bool fg_wait(uint32_t bar, uint32_t parity, uint32_t bad) {
   const long long t0 = clock64();
   for (;;) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     if (done) return true;
@@ -128,9 +132,9 @@ __device__ __noinline__ uint32_t decode_block(const FgArgs& a, uint64_t sub, uin
   constexpr uint32_t kPerLane = kFgBlock * kFgBlock / 32u;
   for (uint32_t t = 0; t < kPerLane; ++t) {
     const uint32_t e = lds_u32(tab_abs + state * 4u);
-    const uint32_t q = t * 32u + lane;                   // the symbol's place in the block, row-major
+    const uint32_t q = t * 32u + lane;                   // the symbol's place in the block = in the tile
     const uint32_t val = lds_u32(vals_abs + (e & 0xFFu) * 4u);
-    sts_elem<2>(b_abs + tile_offset(q >> 6, q & 63u), val);
+    sts_elem<2>(b_abs + q * 2u, val);
     state = (e >> 16) + take((e >> 8) & 15u);
   }
   if (state != 0) bad |= ANS_STATUS_BAD_FINAL_STATE;
@@ -256,17 +260,18 @@ __global__ void __launch_bounds__(160, 1) ans_decode_gemm_kernel(const FgArgs a)
 //
 // A CTA owns 256 output features (four block rows of W) and a range of K (the K dimension is
 // split over CTAs so that the grid fills the device; partial sums meet in Y by fp32 atomic
-// adds when there is more than one range).  Sixteen producer warps: stage s = warp / 4 holds a
-// 128 x 64 slice of X and the four 64 x 64 blocks of W under it, warp 4 s + i decodes block i
+// adds when there is more than one range).  A stage holds a 128 x 64 slice of X and the four
+// 64 x 64 blocks of W under it; three stages.  Sixteen producer warps take the blocks of the
+// CTA's range in turn (block b = 4 j + i: row i of step j of K, stage j mod 3) and decode them
 // with the strips kernel's walk (pre-walked table: a look-up stands for a run of the dominant
-// symbol plus one symbol, Section II-A) into a plain row-major tile pre-filled with the
-// dominant value, then puts the tile's 16-byte pieces in the swizzled order in place.  The
-// sub-stream's bytes come into shared memory by asynchronous copies issued one block ahead.
+// symbol plus one symbol, Section II-A) into the tile, pre-filled with the dominant value.  The
+// sub-stream's bytes come into shared memory by asynchronous copies issued one block ahead, and
+// the table lies there in up to 32 copies (a lane reads its own: no bank conflicts).
 // Warp 16 issues one tcgen05.mma of N = 256 per 16 columns of K.
 // ---------------------------------------------------------------------------------------------
-constexpr uint32_t kF2Stages = 4;
+constexpr uint32_t kF2Stages = 4;   // (three stages leave room for 32 copies of the table, but twelve tiles in flight instead of sixteen: slower)
 constexpr uint32_t kF2Rows = 4;                   // block rows of W per CTA
-constexpr uint32_t kF2Producers = kF2Stages * kF2Rows;
+constexpr uint32_t kF2Producers = 16;
 constexpr uint32_t kF2Threads = (kF2Producers + 1) * 32;
 constexpr uint32_t kF2BTile = kF2Rows * kFgBTile; // bytes: 256 rows of W, 64 bf16 each
 constexpr uint32_t kF2Cols = kF2Rows * kFgBlock;  // tensor-memory columns
@@ -282,8 +287,8 @@ struct F2Args {
   uint32_t unit;                // the value 1
 };
 
-// Decode one block (one sub-stream: 128 symbols per lane) into the row-major tile at tile_abs,
-// which holds the dominant value everywhere.  The sub-stream's words are in shared memory at
+// Decode one block (one sub-stream: 128 symbols per lane) into the tile at tile_abs, which holds
+// the dominant value everywhere.  The sub-stream's words are in shared memory at
 // stage_abs (staged, zero words after them) or in global memory.  Returns status bits.
 __device__ __noinline__ uint32_t decode_block_wide(uint32_t tab_lane, uint32_t stride_log, uint32_t succ_abs,
                                                    uint32_t tile_abs, uint32_t stage_abs,
@@ -317,7 +322,7 @@ __device__ __noinline__ uint32_t decode_block_wide(uint32_t tab_lane, uint32_t s
   const uint32_t stride = 1u << stride_log;
   uint32_t st = tab_lane + (state << stride_log);
   uint32_t z = 0;
-  const uint32_t abase = tile_abs + lane * 2u;             // position z of this lane: row z / 2 of the tile
+  const uint32_t abase = tile_abs + lane * 2u;             // position z of this lane: symbol 32 z + lane of the block
   if (staged) {
     const uint32_t sp_limit = stage_abs + word_limit * 4u;
     uint32_t sp = min(stage_abs + min(idx, word_limit) * 4u, sp_limit);
@@ -362,12 +367,21 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
   const uint32_t succ_bytes = max(2u << a.R, 16u);
   const uint32_t stages_abs = succ_abs + succ_bytes;
   const uint32_t bars_abs = stages_abs + kF2Producers * args.stage_bytes;
-  const uint32_t full_bar = bars_abs, empty_bar = bars_abs + 8u * kF2Stages, done_bar = bars_abs + 16u * kF2Stages;
+  // A wait on an mbarrier tells the current phase from the one before it and no more.  The thread
+  // that issues the products takes the steps in order, but a producer may be several steps ahead
+  // of the others; so a stage has two "empty" barriers used in turn (fill u of stage s frees
+  // barrier 2 s + u mod 2): the phase before the one a producer waits for then lies nine steps
+  // back, and the producer has seen step j - 7 consumed when it took its last block.
+  const uint32_t full_bar = bars_abs, empty_bar = bars_abs + 8u * kF2Stages, done_bar = bars_abs + 24u * kF2Stages;
   const uint32_t slot_abs = done_bar + 8u;
   uint32_t bad = 0;
 
   if (threadIdx.x == 0) {
-    for (uint32_t s = 0; s < kF2Stages; ++s) { mbar_init(full_bar + 8u * s, kF2Rows); mbar_init(empty_bar + 8u * s, 1); }
+    for (uint32_t s = 0; s < kF2Stages; ++s) {
+      mbar_init(full_bar + 8u * s, kF2Rows);
+      mbar_init(empty_bar + 16u * s, 1);
+      mbar_init(empty_bar + 16u * s + 8u, 1);
+    }
     mbar_init(done_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -385,8 +399,15 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
       const uint32_t gm = __ldg(g_multi + i), gs = __ldg(g_single + i);
       const uint32_t val = dequant_bits(static_cast<int>(entry_sym(gm)), static_cast<int>(a.zero_point), a.scale, ANS_BF16);
       const uint32_t e = to_strip_entry_short(gm, val);
-      for (uint32_t c = 0; c < (1u << args.rep_log); ++c)
-        asm volatile("st.shared.u32 [%0], %1;" :: "r"(tab_abs + (i << stride_log) + c * 4u), "r"(e) : "memory");
+      if (stride_log >= 4u) {                              // 16 bytes at a time, every lane starting at another piece
+        const uint32_t pieces = 1u << (stride_log - 4u), turn = lane & (pieces - 1u);
+#pragma unroll
+        for (uint32_t q = 0; q < 8u; ++q)
+          if (q < pieces) sts_v4(tab_abs + (i << stride_log) + ((q ^ turn) << 4), make_uint4(e, e, e, e));
+      } else {
+        for (uint32_t c = 0; c < (1u << args.rep_log); ++c)
+          asm volatile("st.shared.u32 [%0], %1;" :: "r"(tab_abs + (i << stride_log) + c * 4u), "r"(e) : "memory");
+      }
       asm volatile("st.shared.u16 [%0], %1;" :: "r"(succ_abs + i * 2u), "r"(entry_newx(gs)) : "memory");
     }
     if (threadIdx.x == 0 && (__ldg(&hdr->magic) != kTableMagic || __ldg(&hdr->table_log) != a.R ||
@@ -403,8 +424,9 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
   const uint32_t nk = min(KB, kb0 + args.kb_per_split) - kb0;   // (the host leaves no range empty)
   if (warp < kF2Producers) {
     // ---- producers --------------------------------------------------------------------------
-    const uint32_t s = warp / kF2Rows, i = warp % kF2Rows;
-    const uint32_t my_a = a_abs + s * kFgATile, my_b = b_abs + s * kF2BTile + i * kFgBTile;
+    const uint32_t i = warp % kF2Rows, j0 = warp / kF2Rows;
+    constexpr uint32_t kStep = kF2Producers / kF2Rows;     // steps of K between two blocks of a warp
+    static_assert(kStep <= 2 * kF2Stages, "a producer must have seen the phase before the one it waits for");
     const uint32_t my_stage = stages_abs + warp * args.stage_bytes;
     const uint32_t tab_lane = tab_abs + ((lane & ((1u << args.rep_log) - 1u)) << 2);
     const uint32_t dom = dequant_bits(static_cast<int>(h_dominant < 256u ? h_dominant : 0u), static_cast<int>(a.zero_point),
@@ -436,14 +458,17 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
     uint64_t n0 = 0, n1 = 0;                               // offsets of the block after this one
-    if (s < nk) locate(__ldg(a.sub_offsets + sub0 + s), __ldg(a.sub_offsets + sub0 + s + 1));
-    for (uint32_t j = s, it = 0; j < nk; j += kF2Stages, ++it) {
-      const bool more = j + kF2Stages < nk;
+    if (j0 < nk) locate(__ldg(a.sub_offsets + sub0 + j0), __ldg(a.sub_offsets + sub0 + j0 + 1));
+    for (uint32_t j = j0; j < nk; j += kStep) {
+      const bool more = j + kStep < nk;
       if (more) {
-        n0 = __ldg(a.sub_offsets + sub0 + j + kF2Stages);
-        n1 = __ldg(a.sub_offsets + sub0 + j + kF2Stages + 1);
+        n0 = __ldg(a.sub_offsets + sub0 + j + kStep);
+        n1 = __ldg(a.sub_offsets + sub0 + j + kStep + 1);
       }
-      if (it > 0 && !__all_sync(kFull, fg_wait(empty_bar + 8u * s, (it - 1u) & 1u, bad))) bad |= kStatusTimeout;
+      const uint32_t s = j % kF2Stages, use = j / kF2Stages;   // the stage and how often it has been filled before
+      const uint32_t my_a = a_abs + s * kFgATile, my_b = b_abs + s * kF2BTile + i * kFgBTile;
+      if (use > 0 && !__all_sync(kFull, fg_wait(empty_bar + 16u * s + 8u * ((use - 1u) & 1u), ((use - 1u) >> 1) & 1u, bad)))
+        bad |= kStatusTimeout;
       // this warp's quarter of the slice of X: rows beyond M are zeros
 #pragma unroll
       for (uint32_t q = 0; q < 8u; ++q) {
@@ -460,17 +485,8 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
         bad |= decode_block_wide(tab_lane, stride_log, succ_abs, my_b, my_stage,
                                  reinterpret_cast<const uint32_t*>(a.stream + off0), extent >> 2, staged, a.R, args.unit, lane);
       __syncwarp();
-      // the stage's bytes are used up: the next block's may come while the tile is put in order
+      // the warp's bytes are used up: the next block's may come
       if (more) locate(n0, n1);
-      // rows of 128 bytes, their 16-byte pieces exchanged by the row's number in its group of
-      // eight (the 128-byte swizzle): four rows a round, every lane one piece
-#pragma unroll 4
-      for (uint32_t q = 0; q < kFgBlock / 4u; ++q) {
-        const uint32_t r = q * 4u + (lane >> 3), c = lane & 7u;
-        const uint4 v = lds_v4(my_b + r * 128u + c * 16u);
-        __syncwarp();
-        sts_v4(my_b + r * 128u + ((c ^ (r & 7u)) << 4), v);
-      }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads shared memory through the async proxy
       __syncwarp();
       if (lane == 0) mbar_arrive(full_bar + 8u * s);
@@ -479,8 +495,8 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
   } else if (lane == 0) {
     // ---- the thread that issues the matrix instructions ----------------------------------------
     for (uint32_t j = 0; j < nk; ++j) {
-      const uint32_t s = j & (kF2Stages - 1u), it = j / kF2Stages;
-      if (!fg_wait(full_bar + 8u * s, it & 1u, bad)) bad |= kStatusTimeout;
+      const uint32_t s = j % kF2Stages, use = j / kF2Stages;
+      if (!fg_wait(full_bar + 8u * s, use & 1u, bad)) bad |= kStatusTimeout;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint64_t da = operand_desc(a_abs + s * kFgATile), db = operand_desc(b_abs + s * kF2BTile);
 #pragma unroll
@@ -492,7 +508,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
             "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
             :: "r"(tmem), "l"(da + 2u * k), "l"(db + 2u * k), "r"(kF2Idesc), "r"(accumulate), "r"(0u) : "memory");
       }
-      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(empty_bar + 8u * s) : "memory");
+      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(empty_bar + 16u * s + 8u * (use & 1u)) : "memory");
     }
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(done_bar) : "memory");
   }

@@ -19,10 +19,26 @@ def _bf16_bits_to_f64(bits):
     return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 
 
+def _block_order():
+    """Where element (r, c) of a 64 x 64 block lies among the block's 4096 symbols."""
+    r, c = np.meshgrid(np.arange(64), np.arange(64), indexing="ij")
+    return (r // 8) * 512 + (r % 8) * 64 + ((c // 8) ^ (r % 8)) * 8 + c % 8
+
+
 def _blocked(w):
-    """N x K -> the order the fused call wants: blocks of 64 x 64, [N/64][K/64][64][64]."""
+    """N x K -> the order the fused call wants: blocks of 64 x 64, [N/64][K/64][4096], each block
+    in the tensor core's operand order."""
     n, k = w.shape
-    return np.ascontiguousarray(w.reshape(n // 64, 64, k // 64, 64).transpose(0, 2, 1, 3)).ravel()
+    blocks = w.reshape(n // 64, 64, k // 64, 64).transpose(0, 2, 1, 3).reshape(n // 64, k // 64, 4096)
+    out = np.empty_like(blocks)
+    out[:, :, _block_order().ravel()] = blocks
+    return out.ravel()
+
+
+def _unblocked(flat, n, k):
+    """The inverse of _blocked."""
+    blocks = flat.reshape(n // 64, k // 64, 4096)[:, :, _block_order().ravel()]
+    return blocks.reshape(n // 64, k // 64, 64, 64).transpose(0, 2, 1, 3).reshape(n, k)
 
 
 def _case(M, N, K, b, pzp, R, seed, scale=0.03125, quiet_rows=0):
@@ -37,7 +53,8 @@ def _case(M, N, K, b, pzp, R, seed, scale=0.03125, quiet_rows=0):
     dec, rc = oracle.unpack(T, P)
     assert rc == oracle.OK
     w_bits = oracle.dequant(dec, zp, scale, "bf16")           # blocked order
-    w = _bf16_bits_to_f64(w_bits).reshape(N // 64, K // 64, 64, 64).transpose(0, 2, 1, 3).reshape(N, K)
+    w = _unblocked(_bf16_bits_to_f64(w_bits), N, K)
+    assert (_unblocked(_blocked(w_sym), N, K) == w_sym).all()
     rng = np.random.default_rng(seed)
     x = torch.from_numpy(rng.standard_normal((M, K)).astype(np.float32)).to(torch.bfloat16)
     x64 = x.to(torch.float32).numpy().astype(np.float64)
@@ -70,7 +87,7 @@ def test_fused_product_equals_the_oracles_weights_times_x(M, N, K, b, pzp, R):
 @pytest.mark.parametrize("M,N,K,b,pzp,R,quiet", [(128, 256, 256, 3, 0.7, 8, 0), (50, 512, 1024, 4, 0.6, 8, 0),
                                                  (128, 2048, 4800, 3, 0.8, 8, 0), (8, 19200, 640, 2, 0.9, 6, 0),
                                                  (33, 256, 64, 3, 0.7, 7, 0), (128, 1024, 2048, 6, 0.5, 8, 3),
-                                                 (64, 256, 19008, 3, 0.7, 8, 0)])
+                                                 (64, 256, 19008, 3, 0.7, 8, 0), (4, 19200, 1408, 3, 0.7, 8, 0)])
 def test_wide_form_equals_the_oracles_weights_times_x(M, N, K, b, pzp, R, quiet):
     spec, P, f256, x, x64, w = _case(M, N, K, b, pzp, R, seed=M + N + K, quiet_rows=quiet)
     if quiet:                               # the kept block rows' sub-streams are far above the average: they do not fit the staging room
