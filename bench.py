@@ -370,6 +370,92 @@ VARIANTS = [("large", "quads", 32, 12, 0), ("resnet50", "strips", 64, 0, 0), ("r
             ("resnet18", "strips", 64, 0, 0), ("resnet18", "quads", 32, 0, 0), ("sweep", "quads", 32, 12, 16384)]
 
 
+FUSED_COPIES = 12           # device copies of the compressed matrix the fused launches rotate over (> L2 in all)
+
+
+def run_fused(ans, args, local, sampler=None, M=128, min_region_s=0.3):
+    """Decode fused into its consumer (paper Section I, Section III-C): Y = X W^T for one matrix of
+    the `large` workload (dim x dim, 256-state table, strips container in blocks of 64 x 64), M rows
+    of X, against the same product taken in two steps (ans_decode_dequant to bf16, then
+    torch.matmul).  Rounds of back-to-back calls behind a device-side spin, as for the decode
+    workloads; the calls rotate over FUSED_COPIES copies of the compressed matrix so that it comes
+    from DRAM."""
+    import torch
+    from paper_2406_06237_b200.runtime import DeviceBatch, pack_layer
+    spec = sg.workload_large(n_mats=1, dim=args.dim, chunk=4096, table_log=8)[0]
+    N = K = args.dim
+    cores = os.cpu_count() or 1
+    sym = sg.draw_symbols(spec, threads=max(1, cores // 4))
+    pl = pack_layer(sym, spec.alphabet, 8, 4096, 32, ans.ANS_LAYOUT_STRIPS, spec.bitwidth, spec.zero_point, spec.scale,
+                    ans.ANS_BF16, n_threads=max(1, cores // 2))
+    db = DeviceBatch([pl] * FUSED_COPIES, f"cuda:{local}")
+    x = torch.randn(M, K, device=f"cuda:{local}").to(torch.bfloat16)
+    y = torch.empty(M, N, dtype=torch.float32, device=f"cuda:{local}")
+    st = torch.cuda.current_stream()
+    descs = db.h_descs[0]
+    outs = [db.output(i).view(N, K) for i in range(FUSED_COPIES)]
+
+    def fused(i):
+        ans.ans_decode_gemm_bf16(descs[i], x.data_ptr(), M, N, K, y.data_ptr(), db.status.data_ptr(), st.cuda_stream)
+
+    def two_steps(i):
+        ans.ans_decode_dequant(descs[i], db.status.data_ptr(), st.cuda_stream)
+        return torch.matmul(x, outs[i].t())
+
+    def timed(fn, steps):
+        for i in range(5):
+            fn(i % FUSED_COPIES)
+        torch.cuda.synchronize()
+        rounds, total = [], 0.0
+        while total < min_region_s * 1e3 and len(rounds) < 500:
+            torch.cuda._sleep(int(2e7))
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(st)
+            for i in range(steps):
+                fn(i % FUSED_COPIES)
+            b.record(st)
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b)
+            rounds.append(ms / steps)
+            total += ms
+        return rounds
+
+    if sampler:
+        sampler.first = len(sampler.rows)
+    steps = 4 * FUSED_COPIES
+    rf = timed(fused, steps)
+    rt = timed(two_steps, steps)
+    if sampler:
+        sampler.last = len(sampler.rows)
+    assert db.read_status() == 0, "decoder flagged a stream"
+    # agreement of the two routes on the last copy (W's blocks put back in row-major order)
+    r, c = torch.meshgrid(torch.arange(64), torch.arange(64), indexing="ij")
+    order = ((r // 8) * 512 + (r % 8) * 64 + ((c // 8) ^ (r % 8)) * 8 + c % 8).reshape(-1).to(x.device)
+    last = FUSED_COPIES - 1
+    fused(last)
+    w = db.output(last).view(N // 64, K // 64, 4096)[:, :, order].view(N // 64, K // 64, 64, 64).permute(0, 2, 1, 3)
+    ref = x.float() @ w.reshape(N, K).float().t()
+    err = float((y - ref).abs().max() / ref.abs().max())
+    f_ms, t_ms = sum(rf) / len(rf), sum(rt) / len(rt)
+    comp = pl.compressed_bytes()
+    res = {"workload": f"Y = X W^T, X {M} x {K} bf16, W {N} x {K} compressed ({comp * 8 / (N * K):.3f} bit/weight, 256-state table)",
+           "kernel": "ans_decode_gemm_wide_kernel (tcgen05.mma, fp32 accumulator in tensor memory)",
+           "fused_ms_mean": f_ms, "decode_then_matmul_ms_mean": t_ms, "speedup_over_two_steps": t_ms / f_ms,
+           "weights_per_s": N * K / (f_ms * 1e-3), "tensor_tflops": 2.0 * M * N * K / (f_ms * 1e-3) / 1e12,
+           "dram_bytes_fused_algorithmic": comp + M * K * 2 + M * N * 4,
+           "dram_bytes_two_steps_algorithmic": comp + 2 * (N * K * 2) + M * K * 2 + M * N * 2,
+           "timed_rounds": [len(rf), len(rt)], "launches_per_round": steps,
+           "max_rel_difference_between_the_routes": err,
+           "l2_policy": f"calls rotate over {FUSED_COPIES} device copies of the compressed matrix "
+                        f"({FUSED_COPIES * comp / 2**20:.0f} MB in all)",
+           "bound": "the decode's instruction issue, as for the decode kernels (see profiles/); not the tensor cores",
+           "clocks": sampler.summary() if sampler else None}
+    launches = (len(rf) + len(rt)) * steps + 11
+    del db
+    torch.cuda.empty_cache()
+    return res, launches
+
+
 def run_ours(args):
     import torch
     import paper_2406_06237_b200 as ans
@@ -455,6 +541,15 @@ def run_ours(args):
             launches += (len(vr) + 1) * (min(args.steps, 200) if wl in ("large", "sweep") else max(args.steps, 100)) * vdb.launches_per_decode()
             del vdb
             torch.cuda.empty_cache()
+    fused = None
+    if world == 1 and not args.no_fused and args.workload == "large" and args.dim % 256 == 0:
+        try:
+            del db
+        except NameError:
+            pass
+        torch.cuda.empty_cache()
+        fused, fl = run_fused(ans, args, local, sampler)
+        launches += fl
     if rank == 0:
         sampler.stop()
     if rank != 0:
@@ -472,7 +567,7 @@ def run_ours(args):
                    "l2_policy": policy,
                    "per_gpu": "every rank decodes its own replica of the workload; no collective on the data path"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
-        "variants": variants,
+        "variants": variants, "fused": fused,
         "compression": {"coded_bits_per_weight": fg["coded_bits"], "entropy_bits_per_weight": ent_bits / max(1, n_w),
                         "gap_bits_per_weight": fg["coded_bits"] - ent_bits / max(1, n_w),
                         "compressed_bytes": fg["comp_bytes"], "output_bytes": fg["out_bytes"]},
@@ -545,6 +640,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-variants", action="store_true")
+    ap.add_argument("--no-fused", action="store_true", help="skip the fused decode + matrix product measurement")
+    ap.add_argument("--fused-only", action="store_true",
+                    help="only the fused decode + matrix product measurement (one short region), as one JSON line")
     args = ap.parse_args()
     if args.layout is None:
         args.layout = DEFAULTS[args.workload][0]
@@ -560,6 +658,14 @@ def main():
 def run_impl(args):
     if args.impl == "reference":
         run_reference(args)
+    elif args.fused_only:
+        import torch
+        import paper_2406_06237_b200 as ans
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+        ans.lib()
+        res, launches = run_fused(ans, args, 0, None, min_region_s=0.02)
+        print(json.dumps({"fused": res, "gpu_launches": launches}))
     else:
         run_ours(args)
 
