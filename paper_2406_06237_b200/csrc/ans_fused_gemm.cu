@@ -258,30 +258,33 @@ __global__ void __launch_bounds__(160, 1) ans_decode_gemm_kernel(const FgArgs a)
 // ---------------------------------------------------------------------------------------------
 // The wide form, for tables of up to 256 states (the paper's sizes) and N a multiple of 256.
 //
-// A CTA owns 256 output features (four block rows of W) and a range of K (the K dimension is
-// split over CTAs so that the grid fills the device; partial sums meet in Y by fp32 atomic
-// adds when there is more than one range).  A stage holds a 128 x 64 slice of X and the four
-// 64 x 64 blocks of W under it; three stages.  Sixteen producer warps take the blocks of the
-// CTA's range in turn (block b = 4 j + i: row i of step j of K, stage j mod 3) and decode them
-// with the strips kernel's walk (pre-walked table: a look-up stands for a run of the dominant
-// symbol plus one symbol, Section II-A) into the tile, pre-filled with the dominant value.  The
-// sub-stream's bytes come into shared memory by asynchronous copies issued one block ahead, and
-// the table lies there in up to 32 copies (a lane reads its own: no bank conflicts).
-// Warp 16 issues one tcgen05.mma of N = 256 per 16 columns of K.
+// The work is cut into units: 256 output features (four block rows of W) by one step of 64 along
+// K; the units, ordered by features and then by K, are dealt to the CTAs (one per SM) in equal
+// contiguous ranges.  A range is a sequence of segments, each a run of K steps under the same 256
+// features: a segment is accumulated in tensor memory and then leaves for Y, by plain stores if
+// it covers all of K and by fp32 atomic adds (into a Y zeroed beforehand) if not.  Two
+// accumulators take turns, so that a segment is stored while the next is being multiplied.
+// A stage holds a 128 x 64 slice of X and the four 64 x 64 blocks of W under it.  Sixteen producer
+// warps take the blocks of the range in turn (row i = warp mod 4 of unit warp / 4, + 4, ...) and
+// decode them with the strips kernel's walk (pre-walked table: a look-up stands for a run of the
+// dominant symbol plus one symbol, Section II-A) into the tile, pre-filled with the dominant
+// value.  The sub-stream's bytes come into shared memory by asynchronous copies issued one block
+// ahead.  Warp 16 issues one tcgen05.mma of N = 256 per 16 columns of K; warps 17-20 read the
+// finished accumulators with tcgen05.ld.
 // ---------------------------------------------------------------------------------------------
 constexpr uint32_t kF2Stages = 4;   // (three stages leave room for 32 copies of the table, but twelve tiles in flight instead of sixteen: slower)
 constexpr uint32_t kF2Rows = 4;                   // block rows of W per CTA
 constexpr uint32_t kF2Producers = 16;
-constexpr uint32_t kF2Threads = (kF2Producers + 1) * 32;
+constexpr uint32_t kF2Threads = (kF2Producers + 1 + 4) * 32;   // producers, the issuing warp, four warps that store
 constexpr uint32_t kF2BTile = kF2Rows * kFgBTile; // bytes: 256 rows of W, 64 bf16 each
-constexpr uint32_t kF2Cols = kF2Rows * kFgBlock;  // tensor-memory columns
+constexpr uint32_t kF2Cols = kF2Rows * kFgBlock;  // tensor-memory columns of one accumulator (there are two)
 constexpr uint32_t kF2Pad = 256;                  // zero bytes after a staged sub-stream: more than a lane can
                                                   // advance in the 128 look-ups of a block (8 bits each at most)
 constexpr uint32_t kF2Idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((kF2Cols >> 3) << 17) | ((128u >> 4) << 24);
 
 struct F2Args {
   FgArgs g;
-  uint32_t kb_per_split;        // blocks of K per CTA range
+  uint32_t units;               // work units in all: (N / 256) * (K / 64), one per 256 x 64 piece of W
   uint32_t stage_bytes;         // per producer: room for a sub-stream's bytes and the padding
   uint32_t rep_log;             // copies of the table, log2
   uint32_t unit;                // the value 1
@@ -372,8 +375,9 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
   // of the others; so a stage has two "empty" barriers used in turn (fill u of stage s frees
   // barrier 2 s + u mod 2): the phase before the one a producer waits for then lies nine steps
   // back, and the producer has seen step j - 7 consumed when it took its last block.
-  const uint32_t full_bar = bars_abs, empty_bar = bars_abs + 8u * kF2Stages, done_bar = bars_abs + 24u * kF2Stages;
-  const uint32_t slot_abs = done_bar + 8u;
+  const uint32_t full_bar = bars_abs, empty_bar = bars_abs + 8u * kF2Stages;
+  const uint32_t acc_full = bars_abs + 24u * kF2Stages, acc_empty = acc_full + 16u;   // two accumulators
+  const uint32_t slot_abs = acc_empty + 16u;
   uint32_t bad = 0;
 
   if (threadIdx.x == 0) {
@@ -382,11 +386,11 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
       mbar_init(empty_bar + 16u * s, 1);
       mbar_init(empty_bar + 16u * s + 8u, 1);
     }
-    mbar_init(done_bar, 1);
+    for (uint32_t b = 0; b < 2u; ++b) { mbar_init(acc_full + 8u * b, 1); mbar_init(acc_empty + 8u * b, 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kF2Producers) {                              // this warp owns the tensor memory
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(slot_abs), "r"(kF2Cols) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(slot_abs), "r"(2u * kF2Cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // the pre-walked table in one-word entries, the bf16 value folded in, copies side by side
@@ -420,12 +424,13 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
   const uint32_t tmem = lds_u32(slot_abs);
 
   const uint32_t KB = a.K / kFgBlock;
-  const uint32_t kb0 = blockIdx.y * args.kb_per_split;
-  const uint32_t nk = min(KB, kb0 + args.kb_per_split) - kb0;   // (the host leaves no range empty)
+  // this CTA's units [u0, u0 + nu)
+  const uint32_t u0 = static_cast<uint32_t>(uint64_t(args.units) * blockIdx.x / gridDim.x);
+  const uint32_t nu = static_cast<uint32_t>(uint64_t(args.units) * (blockIdx.x + 1u) / gridDim.x) - u0;
   if (warp < kF2Producers) {
     // ---- producers --------------------------------------------------------------------------
     const uint32_t i = warp % kF2Rows, j0 = warp / kF2Rows;
-    constexpr uint32_t kStep = kF2Producers / kF2Rows;     // steps of K between two blocks of a warp
+    constexpr uint32_t kStep = kF2Producers / kF2Rows;     // units between two blocks of a warp
     static_assert(kStep <= 2 * kF2Stages, "a producer must have seen the phase before the one it waits for");
     const uint32_t my_stage = stages_abs + warp * args.stage_bytes;
     const uint32_t tab_lane = tab_abs + ((lane & ((1u << args.rep_log) - 1u)) << 2);
@@ -433,7 +438,11 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
                                       a.scale, ANS_BF16);
     const uint32_t fill = (dom & 0xFFFFu) * 0x10001u;
     const uint4 fill4 = make_uint4(fill, fill, fill, fill);
-    const uint64_t sub0 = uint64_t(blockIdx.x * kF2Rows + i) * KB + kb0;   // the block row's first sub-stream of the range
+    // the sub-stream of this warp's row of unit u: block (4 tile + i, step) of W
+    auto sub_of = [&](uint32_t u) -> uint64_t {
+      const uint32_t tile = u / KB;
+      return uint64_t(tile * kF2Rows + i) * KB + (u - tile * KB);
+    };
 
     // the extent of a sub-stream, checked; its bytes requested into the warp's stage when they fit
     uint64_t off0 = 0;
@@ -458,15 +467,20 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
     uint64_t n0 = 0, n1 = 0;                               // offsets of the block after this one
-    if (j0 < nk) locate(__ldg(a.sub_offsets + sub0 + j0), __ldg(a.sub_offsets + sub0 + j0 + 1));
-    for (uint32_t j = j0; j < nk; j += kStep) {
-      const bool more = j + kStep < nk;
+    if (j0 < nu) {
+      const uint64_t sub = sub_of(u0 + j0);
+      locate(__ldg(a.sub_offsets + sub), __ldg(a.sub_offsets + sub + 1));
+    }
+    for (uint32_t j = j0; j < nu; j += kStep) {
+      const bool more = j + kStep < nu;
       if (more) {
-        n0 = __ldg(a.sub_offsets + sub0 + j + kStep);
-        n1 = __ldg(a.sub_offsets + sub0 + j + kStep + 1);
+        const uint64_t sub = sub_of(u0 + j + kStep);
+        n0 = __ldg(a.sub_offsets + sub);
+        n1 = __ldg(a.sub_offsets + sub + 1);
       }
       const uint32_t s = j % kF2Stages, use = j / kF2Stages;   // the stage and how often it has been filled before
       const uint32_t my_a = a_abs + s * kFgATile, my_b = b_abs + s * kF2BTile + i * kFgBTile;
+      const uint32_t kb = (u0 + j) % KB;
       if (use > 0 && !__all_sync(kFull, fg_wait(empty_bar + 16u * s + 8u * ((use - 1u) & 1u), ((use - 1u) >> 1) & 1u, bad)))
         bad |= kStatusTimeout;
       // this warp's quarter of the slice of X: rows beyond M are zeros
@@ -474,7 +488,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
       for (uint32_t q = 0; q < 8u; ++q) {
         const uint32_t c = lane & 7u, r = i * 32u + q * 4u + (lane >> 3);
         const uint32_t bytes = r < a.M ? 16u : 0u;
-        const uint16_t* src = a.x + size_t(r < a.M ? r : 0u) * a.K + size_t(kb0 + j) * kFgBlock + c * 8u;
+        const uint16_t* src = a.x + size_t(r < a.M ? r : 0u) * a.K + size_t(kb) * kFgBlock + c * 8u;
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(my_a + tile_offset(r, c * 8u)), "l"(src), "r"(bytes) : "memory");
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
@@ -492,53 +506,74 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
       if (lane == 0) mbar_arrive(full_bar + 8u * s);
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-  } else if (lane == 0) {
+  } else if (warp == kF2Producers) {
     // ---- the thread that issues the matrix instructions ----------------------------------------
-    for (uint32_t j = 0; j < nk; ++j) {
-      const uint32_t s = j % kF2Stages, use = j / kF2Stages;
-      if (!fg_wait(full_bar + 8u * s, use & 1u, bad)) bad |= kStatusTimeout;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint64_t da = operand_desc(a_abs + s * kFgATile), db = operand_desc(b_abs + s * kF2BTile);
+    if (lane == 0) {
+      uint32_t seg = 0;
+      for (uint32_t j = 0; j < nu; ++j) {
+        const uint32_t s = j % kF2Stages, use = j / kF2Stages;
+        const uint32_t kb = (u0 + j) % KB;
+        const bool first = j == 0 || kb == 0, last = j + 1u == nu || kb + 1u == KB;
+        const uint32_t buf = seg & 1u;
+        if (first && seg >= 2u) {                          // the accumulator must have been read out
+          if (!fg_wait(acc_empty + 8u * buf, ((seg >> 1) - 1u) & 1u, bad)) bad |= kStatusTimeout;
+        }
+        if (!fg_wait(full_bar + 8u * s, use & 1u, bad)) bad |= kStatusTimeout;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint64_t da = operand_desc(a_abs + s * kFgATile), db = operand_desc(b_abs + s * kF2BTile);
 #pragma unroll
-      for (uint32_t k = 0; k < kFgBlock / 16u; ++k) {      // K = 16 per instruction: 32 bytes further along the rows
-        const uint32_t accumulate = (j | k) ? 1u : 0u;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-            :: "r"(tmem), "l"(da + 2u * k), "l"(db + 2u * k), "r"(kF2Idesc), "r"(accumulate), "r"(0u) : "memory");
-      }
-      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(empty_bar + 16u * s + 8u * (use & 1u)) : "memory");
-    }
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(done_bar) : "memory");
-  }
-
-  // ---- the accumulator: row m of Y in lane m of the tensor memory, 256 columns -------------------
-  if (warp < 4) {
-    __syncwarp();
-    if (!__all_sync(kFull, fg_wait(done_bar, 0, bad))) bad |= kStatusTimeout;
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t row = warp * 32u + lane;
-    float* yrow = a.y + size_t(row) * a.N + size_t(blockIdx.x) * kF2Cols;
-    const bool add = gridDim.y > 1;
-#pragma unroll 4
-    for (uint32_t c0 = 0; c0 < kF2Cols; c0 += 8u) {
-      uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
-      asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                   : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3), "=r"(r4), "=r"(r5), "=r"(r6), "=r"(r7)
-                   : "r"(tmem + ((warp * 32u) << 16) + c0) : "memory");
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      if (row < a.M) {
-        if (add) {
-          atomicAdd(reinterpret_cast<float4*>(yrow + c0),
-                    make_float4(__uint_as_float(r0), __uint_as_float(r1), __uint_as_float(r2), __uint_as_float(r3)));
-          atomicAdd(reinterpret_cast<float4*>(yrow + c0 + 4),
-                    make_float4(__uint_as_float(r4), __uint_as_float(r5), __uint_as_float(r6), __uint_as_float(r7)));
-        } else {
-          *reinterpret_cast<uint4*>(yrow + c0) = make_uint4(r0, r1, r2, r3);
-          *reinterpret_cast<uint4*>(yrow + c0 + 4) = make_uint4(r4, r5, r6, r7);
+        for (uint32_t k = 0; k < kFgBlock / 16u; ++k) {    // K = 16 per instruction: 32 bytes further along the rows
+          const uint32_t accumulate = (!first || k) ? 1u : 0u;
+          asm volatile(
+              "{\n\t.reg .pred p;\n\t"
+              "setp.ne.b32 p, %4, 0;\n\t"
+              "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+              :: "r"(tmem + buf * kF2Cols), "l"(da + 2u * k), "l"(db + 2u * k), "r"(kF2Idesc), "r"(accumulate), "r"(0u) : "memory");
+        }
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                     :: "r"(empty_bar + 16u * s + 8u * (use & 1u)) : "memory");
+        if (last) {
+          asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(acc_full + 8u * buf) : "memory");
+          ++seg;
         }
       }
+    }
+  } else {
+    // ---- the accumulators: row m of Y in lane m of the tensor memory, 256 columns ------------------
+    const uint32_t quarter = warp & 3u;                    // the lanes of tensor memory this warp may read
+    const uint32_t row = quarter * 32u + lane;
+    uint32_t seg = 0;
+    for (uint32_t j = 0; j < nu; ++seg) {
+      const uint32_t tile = (u0 + j) / KB, kb = (u0 + j) - tile * KB;
+      const uint32_t len = min(KB - kb, nu - j);
+      const bool add = len != KB;                          // part of K only: the parts meet in Y
+      const uint32_t buf = seg & 1u;
+      if (!__all_sync(kFull, fg_wait(acc_full + 8u * buf, (seg >> 1) & 1u, bad))) bad |= kStatusTimeout;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      float* yrow = a.y + size_t(row) * a.N + size_t(tile) * kF2Cols;
+#pragma unroll 4
+      for (uint32_t c0 = 0; c0 < (quarter * 32u < a.M ? kF2Cols : 0u); c0 += 8u) {   // (a warp whose rows are all beyond M has nothing to store)
+        uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3), "=r"(r4), "=r"(r5), "=r"(r6), "=r"(r7)
+                     : "r"(tmem + ((quarter * 32u) << 16) + buf * kF2Cols + c0) : "memory");
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (row < a.M) {
+          if (add) {
+            atomicAdd(reinterpret_cast<float4*>(yrow + c0),
+                      make_float4(__uint_as_float(r0), __uint_as_float(r1), __uint_as_float(r2), __uint_as_float(r3)));
+            atomicAdd(reinterpret_cast<float4*>(yrow + c0 + 4),
+                      make_float4(__uint_as_float(r4), __uint_as_float(r5), __uint_as_float(r6), __uint_as_float(r7)));
+          } else {
+            *reinterpret_cast<uint4*>(yrow + c0) = make_uint4(r0, r1, r2, r3);
+            *reinterpret_cast<uint4*>(yrow + c0 + 4) = make_uint4(r4, r5, r6, r7);
+          }
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty + 8u * buf);
+      j += len;
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -546,7 +581,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
   if (warp == kF2Producers) {
     __syncwarp();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kF2Cols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(2u * kF2Cols) : "memory");
   }
   bad = __reduce_or_sync(kFull, bad);
   if (lane == 0 && bad && a.d_status) atomicOr(a.d_status, bad);
@@ -605,21 +640,37 @@ ANS_EXPORT int ans_decode_gemm_bf16(const ans_layer_desc* h_desc, const void* d_
       uint32_t rep_log = 0;
       while (rep_log < 5 && fixed + (one_table << (rep_log + 1)) <= static_cast<size_t>(smem_max)) ++rep_log;
       const uint32_t KB = static_cast<uint32_t>(K / 64), tiles = static_cast<uint32_t>(N) / kF2Cols;
-      uint32_t splits = static_cast<uint32_t>(sms) / tiles;
-      if (splits < 1) splits = 1;
-      if (splits > KB) splits = KB;
-      const uint32_t per = (KB + splits - 1) / splits;
-      splits = (KB + per - 1) / per;                       // no range is empty
+      const uint64_t units = uint64_t(tiles) * KB;
+      if (units > 0x7FFFFFFFull) return ANS_ERR_UNSUPPORTED;
+      // CTAs: one per SM with the units dealt evenly, or, if that saves no round of the producers
+      // (four units are decoded at a time), a whole number of CTAs per 256 features, so that no
+      // range crosses from one accumulator's features to the next
+      uint32_t ctas = units < static_cast<uint64_t>(sms) ? static_cast<uint32_t>(units) : static_cast<uint32_t>(sms);
+      {
+        uint32_t per_tile = static_cast<uint32_t>(sms) / tiles;
+        if (per_tile > KB) per_tile = KB;
+        const uint32_t aligned = tiles * per_tile;
+        constexpr uint32_t kAtATime = kF2Producers / kF2Rows;
+        auto rounds = [&](uint32_t n) { return ((units + n - 1) / n + kAtATime - 1) / kAtATime; };
+        if (aligned >= 1 && rounds(aligned) <= rounds(ctas)) {
+          // and no more CTAs than that number of rounds needs: fewer partial sums to add
+          while (per_tile > 1 && rounds(tiles * (per_tile - 1)) == rounds(aligned)) --per_tile;
+          ctas = tiles * per_tile;
+        }
+      }
+      // Y is zeroed first if any range ends inside the K steps of its 256 features (those parts are added)
+      bool whole = true;
+      for (uint32_t c = 1; c < ctas && whole; ++c) whole = (units * c / ctas) % KB == 0;
       F2Args w{};
       w.g = a;
-      w.kb_per_split = per;
+      w.units = static_cast<uint32_t>(units);
       w.stage_bytes = static_cast<uint32_t>(stage);
       w.rep_log = rep_log;
       w.unit = 1u;
       const size_t smem = fixed + (one_table << rep_log);
-      if (splits > 1) ANSB_CUDA(cudaMemsetAsync(d_y, 0, size_t(M) * size_t(N) * sizeof(float), st));
+      if (!whole) ANSB_CUDA(cudaMemsetAsync(d_y, 0, size_t(M) * size_t(N) * sizeof(float), st));
       ANSB_CUDA(cudaFuncSetAttribute(ans_decode_gemm_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-      ans_decode_gemm_wide_kernel<<<dim3(tiles, splits), kF2Threads, smem, st>>>(w);
+      ans_decode_gemm_wide_kernel<<<ctas, kF2Threads, smem, st>>>(w);
       ANSB_CUDA(cudaGetLastError());
       return ANS_OK;
     }
