@@ -381,13 +381,13 @@ def run_fused(ans, args, local, sampler=None, M=128, min_region_s=0.3):
     workloads; the calls rotate over FUSED_COPIES copies of the compressed matrix so that it comes
     from DRAM."""
     import torch
-    from paper_2406_06237_b200.runtime import DeviceBatch, pack_layer
+    from paper_2406_06237_b200.runtime import DeviceBatch, gemm_block_order, pack_gemm_layer
     spec = sg.workload_large(n_mats=1, dim=args.dim, chunk=4096, table_log=8)[0]
     N = K = args.dim
     cores = os.cpu_count() or 1
     sym = sg.draw_symbols(spec, threads=max(1, cores // 4))
-    pl = pack_layer(sym, spec.alphabet, 8, 4096, 32, ans.ANS_LAYOUT_STRIPS, spec.bitwidth, spec.zero_point, spec.scale,
-                    ans.ANS_BF16, n_threads=max(1, cores // 2))
+    pl = pack_gemm_layer(sym.reshape(N, K), spec.alphabet, 8, spec.bitwidth, spec.zero_point, spec.scale,
+                         n_threads=max(1, cores // 2))
     db = DeviceBatch([pl] * FUSED_COPIES, f"cuda:{local}")
     x = torch.randn(M, K, device=f"cuda:{local}").to(torch.bfloat16)
     y = torch.empty(M, N, dtype=torch.float32, device=f"cuda:{local}")
@@ -429,8 +429,7 @@ def run_fused(ans, args, local, sampler=None, M=128, min_region_s=0.3):
         sampler.last = len(sampler.rows)
     assert db.read_status() == 0, "decoder flagged a stream"
     # agreement of the two routes on the last copy (W's blocks put back in row-major order)
-    r, c = torch.meshgrid(torch.arange(64), torch.arange(64), indexing="ij")
-    order = ((r // 8) * 512 + (r % 8) * 64 + ((c // 8) ^ (r % 8)) * 8 + c % 8).reshape(-1).to(x.device)
+    order = torch.from_numpy(gemm_block_order().ravel()).to(x.device)
     last = FUSED_COPIES - 1
     fused(last)
     w = db.output(last).view(N // 64, K // 64, 4096)[:, :, order].view(N // 64, K // 64, 64, 64).permute(0, 2, 1, 3)

@@ -51,6 +51,29 @@ def pack_layer(symbols: np.ndarray, alphabet: int, table_log: int, chunk_symbols
                        table_log, bitwidth, zero_point, float(scale), out_dtype, layout, piece_symbols)
 
 
+def gemm_block_order() -> np.ndarray:
+    """Where element (r, c) of a 64 x 64 block of W lies among the block's 4096 symbols for
+    ans_decode_gemm_bf16 (the order in which the tensor core reads a 128-byte-swizzled K-major
+    tile): index [r, c] -> symbol number."""
+    r, c = np.meshgrid(np.arange(64), np.arange(64), indexing="ij")
+    return (r // 8) * 512 + (r % 8) * 64 + ((c // 8) ^ (r % 8)) * 8 + c % 8
+
+
+def pack_gemm_layer(w_symbols: np.ndarray, alphabet: int, table_log: int, bitwidth: int, zero_point: int,
+                    scale: float, n_threads: int = 0) -> PackedLayer:
+    """Encode W (N x K symbols, row n = output feature; N and K multiples of 64) the way
+    ans_decode_gemm_bf16 reads it: blocks of 64 x 64 ordered [N / 64][K / 64], each block in
+    gemm_block_order(), one sub-stream of the strips container per block."""
+    n, k = w_symbols.shape
+    if n % 64 or k % 64:
+        raise ValueError("N and K must be multiples of 64")
+    blocks = w_symbols.reshape(n // 64, 64, k // 64, 64).transpose(0, 2, 1, 3).reshape(n // 64, k // 64, 4096)
+    ordered = np.empty_like(blocks)
+    ordered[:, :, gemm_block_order().ravel()] = blocks
+    return pack_layer(np.ascontiguousarray(ordered).ravel(), alphabet, table_log, 4096, 32, B.ANS_LAYOUT_STRIPS,
+                      bitwidth, zero_point, scale, B.ANS_BF16, n_threads)
+
+
 _TORCH_DTYPE = {B.ANS_U8: torch.uint8, B.ANS_F32: torch.float32, B.ANS_BF16: torch.bfloat16}
 
 

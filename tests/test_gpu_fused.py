@@ -9,7 +9,7 @@ import torch
 import oracle
 import synthgen as sg
 import paper_2406_06237_b200 as ans
-from paper_2406_06237_b200.runtime import DeviceBatch
+from paper_2406_06237_b200.runtime import DeviceBatch, pack_gemm_layer
 from helpers import oracle_pack_spec, to_packed_layer
 
 pytestmark = pytest.mark.gpu
@@ -108,6 +108,27 @@ def test_wide_form_equals_the_oracles_weights_times_x(M, N, K, b, pzp, R, quiet)
     bound = (np.abs(x64) @ np.abs(w).T) * ((K + 64) * 2.0 ** -24) + 1e-30
     assert np.isfinite(got).all() and (np.abs(got - want) <= bound).all(), float(np.abs(got - want).max())
     assert (guard == 7.0).all()
+
+
+def test_the_librarys_own_packer_feeds_the_fused_call():
+    """pack_gemm_layer (blocks in the operand's order, library encoder) -> fused call, against the
+    weights dequantised by the oracle from the symbols as drawn."""
+    M, N, K, b, R = 40, 512, 384, 3, 8
+    A, zp = sg.alphabet_for_bits(b)
+    spec = sg.LayerSpec("w", (N, K), b, A, zp, sg.theta_for_pzp(A, zp, 0.7), 0.0625, R, 4096, "bf16", sg.stream_key(31, 77))
+    w_sym = sg.draw_symbols(spec).reshape(N, K)
+    pl = pack_gemm_layer(w_sym, A, R, b, zp, 0.0625)
+    w = _bf16_bits_to_f64(oracle.dequant(w_sym.ravel(), zp, 0.0625, "bf16")).reshape(N, K)
+    x = torch.from_numpy(np.random.default_rng(3).standard_normal((M, K)).astype(np.float32)).to(torch.bfloat16)
+    x64 = x.to(torch.float32).numpy().astype(np.float64)
+    db = DeviceBatch([pl])
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    ans.ans_decode_gemm_bf16(db.h_descs[0][0], x.cuda().data_ptr(), M, N, K, y.data_ptr(), db.status.data_ptr(),
+                             torch.cuda.current_stream().cuda_stream)
+    assert db.read_status() == 0
+    got = y.cpu().numpy().astype(np.float64)
+    bound = (np.abs(x64) @ np.abs(w).T) * ((K + 64) * 2.0 ** -24) + 1e-30
+    assert (np.abs(got - x64 @ w.T) <= bound).all()
 
 
 def test_wide_form_flags_a_corrupt_block():

@@ -136,3 +136,15 @@ def test_no_cpu_fallback_in_product_path():
     for fn in os.listdir(os.path.join(ROOT, "oracle")):
         if fn.endswith((".py", ".c")):
             assert "paper_2406_06237_b200" not in open(os.path.join(ROOT, "oracle", fn)).read()
+
+
+def test_gemm_block_order_is_the_128_byte_swizzle_of_a_k_major_tile():
+    """Rows of 64 bf16 = 128 bytes lie one after the other; inside row r the eight 16-byte pieces
+    (8 elements each) are exchanged by r mod 8; elements keep their place inside a piece."""
+    from paper_2406_06237_b200.runtime import gemm_block_order
+    o = gemm_block_order()
+    assert sorted(o.ravel().tolist()) == list(range(4096))
+    r, c = np.meshgrid(np.arange(64), np.arange(64), indexing="ij")
+    assert (o // 64 == r).all()
+    assert ((o % 64) // 8 == ((c // 8) ^ (r % 8))).all()
+    assert (o % 8 == c % 8).all()
