@@ -291,7 +291,7 @@ LAYOUT_IDS = {"private": "ANS_LAYOUT_PRIVATE", "interleaved": "ANS_LAYOUT_INTERL
               "strips": "ANS_LAYOUT_STRIPS"}
 
 
-def build_case(ans, args, workload, layout_name, lanes, table_log=0, chunk=0, local=0, by_channel=False):
+def build_case(ans, args, workload, layout_name, lanes, table_log=0, chunk=0, local=0, by_channel=False, settled=True):
     """Draw the workload's symbols, pack them with the library's host packer, put everything on
     the device.  Returns (specs, syms, layers, db, n_sets, working-set text)."""
     import copy
@@ -332,7 +332,13 @@ def build_case(ans, args, workload, layout_name, lanes, table_log=0, chunk=0, lo
     ws = out_bytes + sum(L.compressed_bytes() for L in layers)
     small = ws < (512 << 20)
     n_sets = min(64, max(2, -(-(512 << 20) // max(ws, 1)))) if small else 1
-    db = DeviceBatch(layers, f"cuda:{local}", n_out_sets=n_sets)
+    # the tables and the compressed bytes are on the device before the first timed launch and never
+    # change: the descriptors say so (ANS_DESC_INPUTS_SETTLED), which lets a strips launch fetch them
+    # and begin while the launch before it drains; where the launches rotate over several output
+    # sets, a launch writes a set that the launch before it does not touch (ANS_DESC_OUTPUT_IDLE)
+    settled = settled and not args.no_settled
+    db = DeviceBatch(layers, f"cuda:{local}", n_out_sets=n_sets, inputs_settled=settled,
+                     output_idle=n_sets >= 2 and settled)
     policy = (f"inputs larger than L2: launches rotate over {n_sets} full copies of the workload "
               f"({n_sets * ws / 2**20:.0f} MB in all)" if small else "working set (compressed + output) is larger than L2")
     return specs, syms, layers, db, n_sets, policy
@@ -366,9 +372,12 @@ def entropy_bits(specs, syms):
 
 # (workload, container, lanes, table_log, chunk) measured beside the headline: the other table size
 # quoted for the large layers, the two ResNets, one cell of the granularity sweep
-VARIANTS = [("large", "quads", 32, 12, 0), ("resnet50", "strips", 64, 0, 0), ("resnet50", "quads", 32, 0, 0),
-            ("resnet50", "strips", 64, 12, 0), ("resnet18", "strips", 64, 0, 0), ("resnet18", "quads", 32, 0, 0),
-            ("sweep", "quads", 32, 12, 16384)]
+# last field: whether the descriptors carry ANS_DESC_INPUTS_SETTLED / ANS_DESC_OUTPUT_IDLE (only the strips
+# kernel reads them); resnet50 is measured both ways
+VARIANTS = [("large", "quads", 32, 12, 0, True), ("resnet50", "strips", 64, 0, 0, True),
+            ("resnet50", "strips", 64, 0, 0, False), ("resnet50", "quads", 32, 0, 0, True),
+            ("resnet50", "strips", 64, 12, 0, True), ("resnet18", "strips", 64, 0, 0, True),
+            ("resnet18", "quads", 32, 0, 0, True), ("sweep", "quads", 32, 12, 16384, True)]
 
 
 FUSED_COPIES = 12           # device copies of the compressed matrix the fused launches rotate over (> L2 in all)
@@ -486,6 +495,7 @@ def run_ours(args):
     sampler.first = len(sampler.rows)
     rounds, each = time_workload(db, args.steps, args.warmup, n_sets, world)
     sampler.last = len(sampler.rows)
+    db_flags = db.h_descs[0][0].flags if layers else 0
     clocks = sampler.summary() if rank == 0 else None
     ms_per_step = reduce_max(rounds[0], world)          # the K steps asked for: the first round
     fg = figures(ans, layers, db, rounds, each, peak)
@@ -522,8 +532,8 @@ def run_ours(args):
             and args.mats == 8 and args.dim == 8192:
         del db
         torch.cuda.empty_cache()
-        for wl, lay, ln, tl, ck in VARIANTS:
-            vs, vy, vl, vdb, vsets, vpol = build_case(ans, args, wl, lay, ln, tl, ck, local)
+        for wl, lay, ln, tl, ck, vflag in VARIANTS:
+            vs, vy, vl, vdb, vsets, vpol = build_case(ans, args, wl, lay, ln, tl, ck, local, settled=vflag)
             sampler.first = len(sampler.rows)
             vr, ve = time_workload(vdb, min(args.steps, 200) if wl in ("large", "sweep") else max(args.steps, 100), 5, vsets, 1,
                                    min_region_s=0.3)
@@ -537,6 +547,7 @@ def run_ours(args):
                              "achieved_gbs": vf["achieved"], "frac": vf["frac"], "frac_of_nominal_8TBs": vf["frac_nominal"],
                              "coded_bits_per_weight": vf["coded_bits"],
                              "entropy_bits_per_weight": entropy_bits(vs, vy) / max(1, vf["n_w"]),
+                             "desc_flags": int(vdb.h_descs[0][0].flags),
                              "l2_policy": vpol, "clocks": sampler.summary()})
             launches += (len(vr) + 1) * (min(args.steps, 200) if wl in ("large", "sweep") else max(args.steps, 100)) * vdb.launches_per_decode()
             del vdb
@@ -574,7 +585,7 @@ def run_ours(args):
                    "grouping": args.grouping, "table_log": layers[0].table_log, "chunk_symbols": layers[0].chunk_symbols,
                    "layers": len(layers), "weights": n_w, "out_dtype": head_specs[0].out_dtype,
                    "arithmetic": "integer decode, one fp32 multiply per weight, round-to-nearest-even to the output type",
-                   "l2_policy": policy,
+                   "l2_policy": policy, "desc_flags": int(db_flags),
                    "per_gpu": "every rank decodes its own replica of the workload; no collective on the data path"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
         "targets": targets, "variants": variants, "fused": fused,
@@ -651,6 +662,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-variants", action="store_true")
     ap.add_argument("--no-fused", action="store_true", help="skip the fused decode + matrix product measurement")
+    ap.add_argument("--no-settled", action="store_true",
+                    help="set neither ANS_DESC_INPUTS_SETTLED nor ANS_DESC_OUTPUT_IDLE: every launch waits for the one "
+                         "before it before it reads anything")
     ap.add_argument("--fused-only", action="store_true",
                     help="only the fused decode + matrix product measurement (one short region), as one JSON line")
     args = ap.parse_args()

@@ -18,6 +18,7 @@ ANS_ERR_INVALID_ARG, ANS_ERR_BAD_FREQS, ANS_ERR_UNSUPPORTED = -1, -2, -3
 ANS_ERR_BUFFER_TOO_SMALL, ANS_ERR_CUDA, ANS_ERR_CORRUPT = -4, -5, -6
 ANS_U8, ANS_F32, ANS_BF16 = 0, 1, 2
 ANS_LAYOUT_INTERLEAVED, ANS_LAYOUT_PRIVATE, ANS_LAYOUT_QUADS, ANS_LAYOUT_STRIPS, ANS_LAYOUT_CHANNELS = 0, 1, 2, 3, 4
+ANS_DESC_INPUTS_SETTLED, ANS_DESC_OUTPUT_IDLE = 1, 2
 DTYPES = {"u8": ANS_U8, "f32": ANS_F32, "bf16": ANS_BF16}
 ELEM_SIZE = {ANS_U8: 1, ANS_F32: 4, ANS_BF16: 2}
 
@@ -40,7 +41,7 @@ class ans_layer_desc(ctypes.Structure):
         ("table_log", ctypes.c_int32), ("bitwidth", ctypes.c_int32), ("zero_point", ctypes.c_int32),
         ("scale", ctypes.c_float), ("out_dtype", ctypes.c_int32), ("layout", ctypes.c_int32),
         ("work_begin", ctypes.c_uint32), ("work_count", ctypes.c_uint32),
-        ("piece_symbols", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+        ("piece_symbols", ctypes.c_uint32), ("flags", ctypes.c_uint32),
     ]
 
 

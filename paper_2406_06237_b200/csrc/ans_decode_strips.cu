@@ -62,6 +62,8 @@ struct StripArgs {
   uint32_t stage_bytes;            // per-warp staging buffer for the sub-stream's bytes
   uint32_t unit;                   // the value 1 (keeps a multiply-add a multiply-add)
   uint32_t ctas;                   // CTAs of the launch
+  uint32_t early;                  // 1: every layer's inputs were settled before the preceding work began;
+                                   // 2: and the preceding work does not touch the outputs
   uint8_t cta_layer[kStripCtaTable];   // layer of every CTA when ctas <= kStripCtaTable: one look-up instead of a search
 };
 
@@ -80,7 +82,10 @@ __device__ __noinline__ uint32_t decode_strip(
     uint32_t tab_lane, uint32_t stride_log, uint32_t succ_abs, uint32_t win_abs, uint32_t stage_abs,
     const uint32_t* __restrict__ words, uint32_t ext_words, uint32_t R, uint32_t count, uint32_t rows, uint32_t piece,
     uint32_t last_row_bytes, uint32_t row_stride, uint8_t* __restrict__ out_strip,
-    uint32_t fill, bool wide_steps, uint32_t unit, uint32_t lane) {
+    uint32_t fill, bool wide_steps, uint32_t unit, uint32_t lane_early) {
+  // lane_early: the lane, and in bit 8 whether the wait for the preceding work on the stream is
+  // still to come (it then comes before the first byte is written; bit 9: no wait is needed)
+  const uint32_t lane = lane_early & 31u;
   const uint32_t E = PIECES ? piece : 1u;
   const uint32_t magic = PIECES ? 0xFFFFFFFFu / piece + 1u : 0u;   // 2^32 / E rounded up (E >= 2)
   const uint32_t RB = 32u * ES * E;                        // bytes of a row
@@ -156,6 +161,7 @@ __device__ __noinline__ uint32_t decode_strip(
     __syncwarp();
     // the window is complete: write it out and fill it again.  Its rows are contiguous in the
     // output for strips (one bulk store); for channels every row is a store of its own.
+    if (t0 == 0 && ((lane_early >> 8) & 1u)) asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t wrows = min(P, rows - t0);
     const uint32_t wbytes = (wrows - 1u) * RB + (t0 + wrows == rows ? last_row_bytes : RB);
     uint8_t* gdst = out_strip + size_t(t0) * row_stride;
@@ -248,8 +254,10 @@ __global__ void __launch_bounds__(kStripWarps * 32) ans_decode_strips_kernel(con
   const uint32_t sub = (blockIdx.x - args.cta_begin[lo]) * kStripWarps + warp;
   const bool have = sub < L.n_sub;
 
-  // whatever an earlier launch of the stream wrote is visible from here on
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // whatever an earlier launch of the stream wrote is visible from here on (unless the caller has
+  // stated that the inputs were settled before that launch: then the wait comes after the table
+  // and the bytes have been fetched, before anything is written)
+  if (!args.early) asm volatile("griddepcontrol.wait;" ::: "memory");
   // everything the CTA needs from memory is requested before any of it is used: the
   // sub-stream's offsets, the table's header and its entries (the first batch)
   uint64_t off0 = 0, off1 = 0;
@@ -393,10 +401,10 @@ __global__ void __launch_bounds__(kStripWarps * 32) ans_decode_strips_kernel(con
 #define ANSB_SCALL(ES_, ST_, SH_)                                                                     \
   bad |= piece > 1u ? decode_strip<ES_, ST_, SH_, true>(tab_lane, stride_log, succ_abs, win_abs, stage_abs, words, ext_words, \
                                                         R, geo.count, geo.rows, geo.E, geo.last_row_bytes, geo.row_stride, \
-                                                        out_strip, fill, wide_steps, args.unit, lane)                \
+                                                        out_strip, fill, wide_steps, args.unit, lane | (args.early << 8)) \
                     : decode_strip<ES_, ST_, SH_, false>(tab_lane, stride_log, succ_abs, win_abs, stage_abs, words, ext_words, \
                                                          R, geo.count, geo.rows, geo.E, geo.last_row_bytes, geo.row_stride, \
-                                                         out_strip, fill, wide_steps, args.unit, lane)
+                                                         out_strip, fill, wide_steps, args.unit, lane | (args.early << 8))
       if (short_entries) {
         if (staged) { if (es == 1u) ANSB_SCALL(1, true, true); else ANSB_SCALL(2, true, true); }
         else { if (es == 1u) ANSB_SCALL(1, false, true); else ANSB_SCALL(2, false, true); }
@@ -409,6 +417,7 @@ __global__ void __launch_bounds__(kStripWarps * 32) ans_decode_strips_kernel(con
     }
   }
   bad = __reduce_or_sync(kFull, bad);
+  if (args.early && bad) asm volatile("griddepcontrol.wait;" ::: "memory");   // (a warp that wrote nothing has not waited yet)
   if (lane == 0 && bad && args.d_status) atomicOr(args.d_status, bad);
 }
 
@@ -441,6 +450,8 @@ int launch_strips(const ans_layer_desc* h_descs, int n_layers, uint8_t* d_symbol
     a.n_layers = 0;
     a.d_status = d_status;
     a.unit = 1u;
+    a.early = 1u;
+    bool idle = true;
     int max_log = 1;
     uint64_t ctas = 0;
     size_t max_avg_sub = 0, one_table = 0;
@@ -449,6 +460,8 @@ int launch_strips(const ans_layer_desc* h_descs, int n_layers, uint8_t* d_symbol
       if (d.work_count == 0) continue;
       const uint64_t n_sub = subs_of(d);
       if (n_sub > 0xFFFFFFFFull) return ANS_ERR_UNSUPPORTED;
+      if (!(d.flags & ANS_DESC_INPUTS_SETTLED)) a.early = 0u;
+      if (!(d.flags & ANS_DESC_OUTPUT_IDLE)) idle = false;
       StripLayer& L = a.layer[a.n_layers];
       L.blob = static_cast<const uint8_t*>(d.d_table);
       L.stream = d.d_stream;
@@ -475,6 +488,7 @@ int launch_strips(const ans_layer_desc* h_descs, int n_layers, uint8_t* d_symbol
       if (avg > max_avg_sub) max_avg_sub = avg;
     }
     if (a.n_layers == 0) continue;
+    if (a.early && idle) a.early = 2u;
     if (ctas > 0x7FFFFFFFull) return ANS_ERR_UNSUPPORTED;
     a.cta_begin[a.n_layers] = static_cast<uint32_t>(ctas);
     a.max_log = static_cast<uint32_t>(max_log);

@@ -87,7 +87,13 @@ class DeviceBatch:
     outputs) exists that many times, so that a timing loop which rotates over the sets reads
     and writes memory that the launches in between have pushed out of L2."""
 
-    def __init__(self, layers: list[PackedLayer], device="cuda:0", n_out_sets: int = 1):
+    def __init__(self, layers: list[PackedLayer], device="cuda:0", n_out_sets: int = 1,
+                 inputs_settled: bool = False, output_idle: bool = False):
+        """inputs_settled: set ANS_DESC_INPUTS_SETTLED on every layer.  The tables and the compressed
+        bytes are put on the device (and the device synchronised) in this constructor, so the
+        statement holds for every decode call made through this object afterwards.
+        output_idle: also set ANS_DESC_OUTPUT_IDLE; the caller must then see to it that the work
+        queued before a decode call does not touch that call's output set."""
         self.layers = layers
         self.device = torch.device(device)
         if self.device.type != "cuda":
@@ -145,6 +151,7 @@ class DeviceBatch:
                 d.n_symbols, d.chunk_symbols, d.lanes = L.n_symbols, L.chunk_symbols, L.lanes
                 d.table_log, d.bitwidth, d.zero_point, d.scale = L.table_log, L.bitwidth, L.zero_point, L.scale
                 d.out_dtype, d.layout, d.piece_symbols = L.out_dtype, L.layout, L.piece_symbols
+                d.flags = (B.ANS_DESC_INPUTS_SETTLED | (B.ANS_DESC_OUTPUT_IDLE if output_idle else 0)) if inputs_settled else 0
             self.total_work = B.ans_plan_batch(arr) if n else 0
             raw = torch.frombuffer(bytearray(bytes(arr)), dtype=torch.uint8)
             self.h_descs.append(arr)

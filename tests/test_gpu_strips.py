@@ -108,6 +108,46 @@ def test_config5_reduced():
     run_and_compare(sg.workload_large(n_mats=2, dim=2048), STRIPS, 64)
 
 
+@pytest.mark.parametrize("idle", [False, True])
+def test_launches_queued_back_to_back_with_the_settled_inputs_flags(idle):
+    """ANS_DESC_INPUTS_SETTLED (and ANS_DESC_OUTPUT_IDLE): a launch may read its inputs, and begin,
+    while the launch before it on the stream still runs.  Thirty launches queued behind a device-side
+    spin, rotating over three output sets (so that a launch never writes the set the one before it
+    writes), every set poisoned first; every set must hold the oracle's bits afterwards.  A corrupt
+    stream is still flagged."""
+    specs = [tiny_spec(300_000, 3, 0.9, 8, 16384, "bf16", index=0), tiny_spec(70_001, 4, 0.7, 8, 4096, "f32", index=1),
+             tiny_spec(0, 2, 0.8, 6, 4096, "u8", index=2), tiny_spec(150_000, 2, 0.95, 7, 8192, "u8", index=3)]
+    prepared = []
+    for spec in specs:
+        sym = sg.draw_symbols(spec)
+        T, P, f256 = oracle_pack_spec(spec, sym, STRIPS, 64)
+        prepared.append((to_packed_layer(spec, P, f256), oracle_expected(spec, T, P)[1]))
+    db = DeviceBatch([p[0] for p in prepared], n_out_sets=3, inputs_settled=True, output_idle=idle)
+    want_flags = ans.ANS_DESC_INPUTS_SETTLED | (ans.ANS_DESC_OUTPUT_IDLE if idle else 0)
+    assert all(int(d.flags) == want_flags for k in range(3) for d in db.h_descs[k][:len(specs)])
+    for outs in db.out_sets:
+        for o in outs:
+            o.view(torch.uint8).fill_(0xA5)
+    torch.cuda.synchronize()
+    torch.cuda._sleep(20_000_000)
+    for i in range(30):
+        db.decode(i % 3)
+    assert db.read_status() == 0
+    for k in range(3):
+        for i, (pl, want) in enumerate(prepared):
+            got = bits_view(db.output(i, k))
+            assert (got == expected_bits(want)).all(), (k, i)
+    # a corrupt stream under the same flags
+    pl = prepared[0][0]
+    bad = pl.stream.copy()
+    bad[int(pl.sub_offsets[1]) + 70] ^= 0x5A
+    import dataclasses
+    db2 = DeviceBatch([dataclasses.replace(pl, stream=bad)], n_out_sets=2, inputs_settled=True, output_idle=idle)
+    for i in range(4):
+        db2.decode(i % 2)
+    assert db2.read_status() != 0
+
+
 def test_long_substreams_read_from_global_memory():
     """Sub-streams too long for the shared-memory staging buffer (here beside short ones of another
     layer, which size the buffer) are read word by word from global memory."""
