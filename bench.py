@@ -331,7 +331,8 @@ def build_case(ans, args, workload, layout_name, lanes, table_log=0, chunk=0, lo
     # rotate over them, so that between two uses of a copy at least 3 x L2 bytes have gone by
     ws = out_bytes + sum(L.compressed_bytes() for L in layers)
     small = ws < (512 << 20)
-    n_sets = min(64, max(2, -(-(512 << 20) // max(ws, 1)))) if small else 1
+    # (a big one in two, so that a launch never writes the buffers the launch before it writes)
+    n_sets = min(64, max(2, -(-(512 << 20) // max(ws, 1)))) if small else 2
     # the tables and the compressed bytes are on the device before the first timed launch and never
     # change: the descriptors say so (ANS_DESC_INPUTS_SETTLED), which lets a strips launch fetch them
     # and begin while the launch before it drains; where the launches rotate over several output
@@ -340,7 +341,8 @@ def build_case(ans, args, workload, layout_name, lanes, table_log=0, chunk=0, lo
     db = DeviceBatch(layers, f"cuda:{local}", n_out_sets=n_sets, inputs_settled=settled,
                      output_idle=n_sets >= 2 and settled)
     policy = (f"inputs larger than L2: launches rotate over {n_sets} full copies of the workload "
-              f"({n_sets * ws / 2**20:.0f} MB in all)" if small else "working set (compressed + output) is larger than L2")
+              f"({n_sets * ws / 2**20:.0f} MB in all)" if small
+              else f"working set (compressed + output) is larger than L2; launches alternate between {n_sets} full copies")
     return specs, syms, layers, db, n_sets, policy
 
 

@@ -150,10 +150,11 @@ typedef struct ans_layer_desc {
 
 /* ans_layer_desc.flags.
  * ANS_DESC_INPUTS_SETTLED: the caller states that this layer's table, stream, offsets and lane
- * metadata were complete in device memory before the work that precedes this call on the stream
- * began (weights loaded and tables built once, decoded many times: the usual case at inference
- * time).  The strips / channels kernel is launched so that it may take its place on the device
- * while the launch before it is still running (programmatic dependent launch); with this bit set
+ * metadata (and, for the *_batch call, the descriptor array in device memory) were complete
+ * before the work that precedes this call on the stream began (weights loaded and tables built
+ * once, decoded many times: the usual case at inference time).  The decode kernels are launched
+ * so that they may take their place on the device while the work before them is still running
+ * (programmatic dependent launch); with this bit set
  * on every layer of a launch it also reads its inputs, stages its table and begins to decode
  * (into shared memory) during that time, and waits for the preceding work only before its first
  * write to device memory.  Without the bit it waits before
@@ -162,8 +163,8 @@ typedef struct ans_layer_desc {
 /* ANS_DESC_OUTPUT_IDLE (only with ANS_DESC_INPUTS_SETTLED): the caller also states that the
  * work that precedes this call on the stream neither reads nor writes this layer's d_out (a
  * decode into one buffer while the layer before it is still being consumed from another).  The
- * strips / channels kernel then does not wait for the preceding work at all, except before it
- * sets a bit in *d_status; work that follows the call on the stream is ordered after it as
+ * kernel then does not wait for the preceding work at all, except before it sets a bit in
+ * *d_status; work that follows the call on the stream is ordered after it as
  * always. */
 #define ANS_DESC_OUTPUT_IDLE 2u
 

@@ -122,6 +122,7 @@ ANS_EXPORT int ans_decode_dequant_host(const ans_layer_desc* h_desc, const uint8
   ANSB_CUDA(cudaMemcpyAsync(d_offs, h_sub_offsets, (n_sub + 1) * 8, cudaMemcpyHostToDevice, st));
   if (meta_bytes) ANSB_CUDA(cudaMemcpyAsync(d_meta, h_lane_meta, meta_bytes, cudaMemcpyHostToDevice, st));
   ans_layer_desc d = *h_desc;
+  d.flags = 0;                                           // the inputs were copied in just now, on this stream
   d.stream_bytes = stream_bytes;
   d.d_stream = d_stream; d.d_sub_offsets = d_offs; d.d_lane_meta = d_meta; d.d_out = d_out;
   rc = ans_decode_dequant(&d, d_status, st);

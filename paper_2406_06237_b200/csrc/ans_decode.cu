@@ -56,6 +56,12 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
   const uint32_t bar = bars_abs + warp * 8u;
   __shared__ uint32_t s_dom, s_maxadv, s_maxnb;
   uint32_t parity = 0;
+  // let the next launch of the stream take its place as this one's CTAs leave; this launch waits
+  // for the work before it either here, before it reads anything, or (inputs settled before that
+  // work began, as the descriptors' flags say) only before its first write to device memory
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (!args.early) asm volatile("griddepcontrol.wait;" ::: "memory");
+  bool waited = args.early != 1u;
 
   uint64_t cursor = uint64_t(blockIdx.x) * args.items_per_cta;
   const uint64_t cta_end = min(cursor + uint64_t(args.items_per_cta), uint64_t(args.total_work));
@@ -271,6 +277,10 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
         parity ^= 1u;
         __syncwarp();
       }
+      if (!waited) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        waited = true;
+      }
       if (kPrivate) {
         const uint32_t* words = reinterpret_cast<const uint32_t*>(g_bytes);
 #define ANSB_CALL(ES_, ST_)                                                                              \
@@ -328,6 +338,7 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
     cursor = stop;
   }
   bad = __reduce_or_sync(kFull, bad);
+  if (args.early && bad) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (lane == 0 && bad && args.d_status) atomicOr(args.d_status, bad);
 }
 
@@ -345,6 +356,7 @@ int launch_strips(const ans_layer_desc* h_descs, int n_layers, uint8_t* d_symbol
 static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, int n_layers,
                   uint8_t* d_symbols_override, uint32_t* d_status, cudaStream_t st) {
   int max_log = 1, busy_layers = 0;
+  uint32_t flags_all = ~0u;                               // flags every layer with work carries
   uint64_t total = 0;
   size_t max_avg_sub = 0, max_es = 1;
   const int layout = h_descs[0].layout;
@@ -356,6 +368,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
       return ANS_ERR_INVALID_ARG;                         // ans_plan_batch was not run on this array
     total += h_descs[l].work_count;
     if (h_descs[l].work_count != 0) {
+      flags_all &= h_descs[l].flags;
       ++busy_layers;
       const size_t avg = h_descs[l].stream_bytes / subs_of(h_descs[l]);
       if (avg > max_avg_sub) max_avg_sub = avg;
@@ -377,6 +390,7 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   a.d_status = d_status;
   a.d_symbols_override = d_symbols_override;
   a.unit = 1u;
+  a.early = !(flags_all & ANS_DESC_INPUTS_SETTLED) ? 0u : (flags_all & ANS_DESC_OUTPUT_IDLE) ? 2u : 1u;
   a.max_log = static_cast<uint32_t>(max_log);
   a.table_words = 2u * ((1u << max_log) + 2u);           // two words per state, and a parking entry (one copy)
 
@@ -494,16 +508,30 @@ static int launch(const ans_layer_desc* d_descs, const ans_layer_desc* h_descs, 
   ipc = (ipc + step - 1) / step * step;
   a.items_per_cta = static_cast<uint32_t>(ipc);
   const unsigned blocks = static_cast<unsigned>((total + ipc - 1) / ipc);
-  const dim3 grid_dim(blocks), block_dim(static_cast<unsigned>(warps) * 32u);
-  switch (launch_which) {
-    case 0: ans_decode_kernel<ANS_LAYOUT_QUADS, true, false><<<grid_dim, block_dim, smem, st>>>(a); break;
-    case 1: ans_decode_kernel<ANS_LAYOUT_QUADS, true, true><<<grid_dim, block_dim, smem, st>>>(a); break;
-    case 2: ans_decode_kernel<ANS_LAYOUT_PRIVATE, true, false><<<grid_dim, block_dim, smem, st>>>(a); break;
-    case 3: ans_decode_kernel<ANS_LAYOUT_PRIVATE, true, true><<<grid_dim, block_dim, smem, st>>>(a); break;
-    case 4: case 5: ans_decode_kernel<ANS_LAYOUT_PRIVATE, false, false><<<grid_dim, block_dim, smem, st>>>(a); break;
-    case 6: ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, true, false><<<grid_dim, block_dim, smem, st>>>(a); break;
-    default: ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, true, true><<<grid_dim, block_dim, smem, st>>>(a); break;
-  }
+  // launched so that it may take its place on the device while the work before it on the stream
+  // is still running; the kernel waits for that work before it reads (or, with the descriptors'
+  // flags, before it writes) anything
+  const void* fns[8] = {
+      reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_QUADS, true, false>),
+      reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_QUADS, true, true>),
+      reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, true, false>),
+      reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, true, true>),
+      reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, false, false>),
+      reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_PRIVATE, false, false>),
+      reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, true, false>),
+      reinterpret_cast<const void*>(&ans_decode_kernel<ANS_LAYOUT_INTERLEAVED, true, true>)};
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(blocks);
+  cfg.blockDim = dim3(static_cast<unsigned>(warps) * 32u);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  void* kargs[1] = {&a};
+  ANSB_CUDA(cudaLaunchKernelExC(&cfg, fns[launch_which & 7], kargs));
   ANSB_CUDA(cudaGetLastError());
   return ANS_OK;
 }

@@ -30,6 +30,8 @@ struct LaunchArgs {
   uint32_t ring_bytes;             // private layout: per-warp output ring (kRingRows rows of the widest dtype)
   uint32_t unit;                   // the value 1 (a run-time operand keeps a multiply-add a multiply-add)
   uint32_t n_begin;                // entries of layer_begin in use (0: search the descriptors instead)
+  uint32_t early;                  // 1: every layer's inputs (and the descriptor array) were settled before the
+                                   // preceding work on the stream began; 2: and that work does not touch the outputs
   // Where each layer's work items start in the numbering the CTAs walk.  When the launch's layers
   // all fit here, every layer's count is rounded up to the items a CTA takes at a time, so that
   // a CTA's rounds line up with the start of every layer it meets (the padding items are empty);

@@ -91,6 +91,7 @@ ANS_EXPORT int ans_decode_dequant_host_noalloc(const ans_layer_desc* h_desc, con
   ANSB_CUDA(cudaMemcpyAsync(d_offs, h_sub_offsets, offs_bytes, cudaMemcpyHostToDevice, st));
   if (meta_bytes) ANSB_CUDA(cudaMemcpyAsync(d_meta, h_lane_meta, meta_bytes, cudaMemcpyHostToDevice, st));
   ans_layer_desc d = *h_desc;
+  d.flags = 0;                                           // the inputs were copied in just now, on this stream
   d.d_table = d_table + table_off;
   d.d_stream = d_stream;
   d.stream_bytes = stream_bytes;
