@@ -149,23 +149,28 @@ typedef struct ans_layer_desc {
 } ans_layer_desc;
 
 /* ans_layer_desc.flags.
+ *
+ * The decode kernels are launched so that they may take their place on the device while the
+ * work before them on the stream is still running (programmatic dependent launch).  By default
+ * a kernel waits for that work before it reads anything.
+ *
  * ANS_DESC_INPUTS_SETTLED: the caller states that this layer's table, stream, offsets and lane
  * metadata (and, for the *_batch call, the descriptor array in device memory) were complete
- * before the work that precedes this call on the stream began (weights loaded and tables built
- * once, decoded many times: the usual case at inference time).  The decode kernels are launched
- * so that they may take their place on the device while the work before them is still running
- * (programmatic dependent launch); with this bit set
- * on every layer of a launch it also reads its inputs, stages its table and begins to decode
- * (into shared memory) during that time, and waits for the preceding work only before its first
- * write to device memory.  Without the bit it waits before
- * it reads anything.  Outputs and the status word are never touched before the wait. */
-#define ANS_DESC_INPUTS_SETTLED 1u
-/* ANS_DESC_OUTPUT_IDLE (only with ANS_DESC_INPUTS_SETTLED): the caller also states that the
- * work that precedes this call on the stream neither reads nor writes this layer's d_out (a
+ * before the work that precedes this call on the stream began: weights loaded and tables built
+ * once, decoded many times, the usual case at inference time.  With the bit set on every layer
+ * of a launch the kernel reads its inputs, stages its table and begins to decode into shared
+ * memory while the preceding work drains, and waits for it only before its first write to
+ * device memory (outputs, status word).
+ *
+ * ANS_DESC_OUTPUT_IDLE (only together with ANS_DESC_INPUTS_SETTLED): the caller also states that
+ * the work that precedes this call on the stream neither reads nor writes this layer's d_out (a
  * decode into one buffer while the layer before it is still being consumed from another).  The
  * kernel then does not wait for the preceding work at all, except before it sets a bit in
- * *d_status; work that follows the call on the stream is ordered after it as
- * always. */
+ * *d_status.  Work that follows the call on the stream is ordered after it as always.
+ *
+ * The host-buffer calls (ans_decode_dequant_host, ans_decode_dequant_host_noalloc) copy their
+ * inputs in on the same stream and ignore the flags; so do the encoder and ans_decode_gemm_bf16. */
+#define ANS_DESC_INPUTS_SETTLED 1u
 #define ANS_DESC_OUTPUT_IDLE 2u
 
 /* Library version (major*100 + minor). */
