@@ -75,7 +75,7 @@ WORKLOAD_TEXT = {
 # the container and lanes per chunk each workload is timed on unless --layout / --lanes say otherwise: the
 # fastest measured (quads: one symbol per look-up, lanes in step; strips: a look-up may stand for a run of the
 # dominant symbol, which pays when one symbol owns most of the states, as in the ResNet-50 workload)
-DEFAULTS = {"large": ("quads", 32), "resnet18": ("strips", 64), "resnet50": ("strips", 64), "sweep": ("quads", 32),
+DEFAULTS = {"large": ("quads", 32), "resnet18": ("strips", 64), "resnet50": ("strips", 32), "sweep": ("quads", 32),
             "conv3x3": ("quads", 32)}
 
 
@@ -376,8 +376,9 @@ def entropy_bits(specs, syms):
 # quoted for the large layers, the two ResNets, one cell of the granularity sweep
 # last field: whether the descriptors carry ANS_DESC_INPUTS_SETTLED / ANS_DESC_OUTPUT_IDLE (only the strips
 # kernel reads them); resnet50 is measured both ways
-VARIANTS = [("large", "quads", 32, 12, 0, True), ("resnet50", "strips", 64, 0, 0, True),
-            ("resnet50", "strips", 64, 0, 0, False), ("resnet50", "quads", 32, 0, 0, True),
+VARIANTS = [("large", "quads", 32, 12, 0, True), ("resnet50", "strips", 32, 0, 0, True),
+            ("resnet50", "strips", 64, 0, 0, True), ("resnet50", "strips", 64, 0, 0, False),
+            ("resnet50", "strips", 32, 0, 0, False), ("resnet50", "quads", 32, 0, 0, True),
             ("resnet50", "strips", 64, 12, 0, True), ("resnet18", "strips", 64, 0, 0, True),
             ("resnet18", "quads", 32, 0, 0, True), ("sweep", "quads", 32, 12, 16384, True)]
 

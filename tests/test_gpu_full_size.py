@@ -15,7 +15,7 @@ from helpers import bits_view, expected_bits, parallel_map
 pytestmark = pytest.mark.gpu
 
 
-def full_size(specs, layout, lanes, sample_chunks=64):
+def full_size(specs, layout, lanes, sample_chunks=64, flagged=False):
     def prep(spec):
         sym = sg.draw_symbols(spec, threads=2)
         pl = pack_layer(sym, spec.alphabet, spec.table_log, spec.chunk_symbols, lanes, layout,
@@ -23,10 +23,22 @@ def full_size(specs, layout, lanes, sample_chunks=64):
         return sym, pl
 
     prepared = parallel_map(prep, specs, 8)
-    db = DeviceBatch([p[1] for p in prepared])
-    for o in db.out_sets[0]:
-        o.view(torch.uint8).fill_(0xA5)
-    db.decode()
+    if flagged:
+        # as bench.py launches it: descriptor flags set, launches queued back to back alternating
+        # between two output sets; the set checked below is written by the launch before the last
+        db = DeviceBatch([p[1] for p in prepared], n_out_sets=2, inputs_settled=True, output_idle=True)
+        for outs in db.out_sets:
+            for o in outs:
+                o.view(torch.uint8).fill_(0xA5)
+        torch.cuda.synchronize()
+        torch.cuda._sleep(20_000_000)
+        for k in (1, 0, 1):
+            db.decode(k)
+    else:
+        db = DeviceBatch([p[1] for p in prepared])
+        for o in db.out_sets[0]:
+            o.view(torch.uint8).fill_(0xA5)
+        db.decode()
     assert db.read_status() == 0
     rng = np.random.default_rng(1)
     for i, (spec, (sym, pl)) in enumerate(zip(specs, prepared)):
@@ -48,6 +60,10 @@ def full_size(specs, layout, lanes, sample_chunks=64):
 @pytest.mark.parametrize("table_log", [8, 12])
 def test_config5_large_layers_full(layout, table_log):
     full_size(sg.workload_large(table_log=table_log), layout, 32)
+
+
+def test_config5_large_layers_full_as_the_benchmark_launches_it():
+    full_size(sg.workload_large(), ans.ANS_LAYOUT_QUADS, 32, flagged=True)
 
 
 @pytest.mark.parametrize("layout", [ans.ANS_LAYOUT_INTERLEAVED, ans.ANS_LAYOUT_PRIVATE])
