@@ -23,7 +23,7 @@
  * or prints.
  *
  * Containers (how one layer's symbols are cut into independently decodable pieces;
- * the paper leaves this open beyond "one state per stream"):
+ * the paper fixes only that every stream has a state of its own):
  *   A layer of n symbols (the tensor flattened in memory order) is cut into chunks of
  *   `chunk_symbols` consecutive symbols.  Inside a chunk, `lanes` = 32*G lanes take the
  *   symbols round-robin (chunk-relative symbol q is the (q / lanes)-th symbol of lane

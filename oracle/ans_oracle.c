@@ -221,7 +221,7 @@ int anso_decode_plain(const anso_table* T, const uint8_t* bytes, uint64_t nbytes
  * symbols.  Inside a chunk, W = 32*G lanes take the symbols round-robin:
  * chunk-relative symbol q is the (q div W)-th symbol of lane q mod W.  Lane
  * lambda is lane k = lambda mod 32 of sub-stream g = lambda div 32.  Every lane
- * has its own state: the paper's "vector of states" (Section III-B).
+ * has its own state: the states of all streams kept side by side, as in Section III-B.
  * Sub-streams are numbered chunk-major: sub = chunk*G + g.
  * ------------------------------------------------------------------------- */
 
