@@ -272,15 +272,30 @@ __global__ void __launch_bounds__(160, 1) ans_decode_gemm_kernel(const FgArgs a)
 // ahead.  Warp 16 issues one tcgen05.mma of N = 256 per 16 columns of K; warps 17-20 read the
 // finished accumulators with tcgen05.ld.
 // ---------------------------------------------------------------------------------------------
-constexpr uint32_t kF2Stages = 4;   // (three stages leave room for 32 copies of the table, but twelve tiles in flight instead of sixteen: slower)
+// The kernel has two forms.  NM = 0: X is the 128-row operand (any M up to 128) and the 256 rows of W
+// are the N = 256 operand, as described above.  NM = 16 or 32, for M up to NM: the operands are
+// exchanged, Y^T = W X^T: the 256 rows of W are two 128-row operands and the NM rows of X (a tile
+// of NM * 128 bytes instead of 16 KB) the N = NM operand of both; the shared memory that X no
+// longer takes holds a fifth stage, so twenty producers decode instead of sixteen, and a row of
+// the accumulator is a feature, so that a warp stores 32 consecutive floats of a row of Y.
 constexpr uint32_t kF2Rows = 4;                   // block rows of W per CTA
-constexpr uint32_t kF2Producers = 16;
-constexpr uint32_t kF2Threads = (kF2Producers + 1 + 4) * 32;   // producers, the issuing warp, four warps that store
 constexpr uint32_t kF2BTile = kF2Rows * kFgBTile; // bytes: 256 rows of W, 64 bf16 each
-constexpr uint32_t kF2Cols = kF2Rows * kFgBlock;  // tensor-memory columns of one accumulator (there are two)
+constexpr uint32_t kF2Cols = kF2Rows * kFgBlock;  // features per unit
+template <uint32_t NM>
+struct F2Shape {
+  // (NM = 0: three stages would leave room for 32 copies of the table, but twelve tiles in flight
+  // instead of sixteen: measured slower)
+  static constexpr uint32_t kStages = NM ? 5 : 4;
+  static constexpr uint32_t kProducers = kStages * kF2Rows;
+  static constexpr uint32_t kThreads = (kProducers + 1 + 4) * 32;   // producers, the issuing warp, four warps that store
+  static constexpr uint32_t kXRows = NM ? NM : 128;                 // rows of X in a stage
+  static constexpr uint32_t kXTile = kXRows * 128;                  // bytes
+  static constexpr uint32_t kAccCols = NM ? 2 * NM : kF2Cols;       // tensor-memory columns of one accumulator (there are two)
+  // instruction descriptor of kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = NM or 256
+  static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (((NM ? NM : kF2Cols) >> 3) << 17) | ((128u >> 4) << 24);
+};
 constexpr uint32_t kF2Pad = 256;                  // zero bytes after a staged sub-stream: more than a lane can
                                                   // advance in the 128 look-ups of a block (8 bits each at most)
-constexpr uint32_t kF2Idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((kF2Cols >> 3) << 17) | ((128u >> 4) << 24);
 
 struct F2Args {
   FgArgs g;
@@ -357,13 +372,16 @@ __device__ __noinline__ uint32_t decode_block_wide(uint32_t tab_lane, uint32_t s
   return bad;
 }
 
-__global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(const F2Args args) {
+template <uint32_t NM>
+__global__ void __launch_bounds__(F2Shape<NM>::kThreads, 1) ans_decode_gemm_wide_kernel(const F2Args args) {
+  using Shape = F2Shape<NM>;
+  constexpr uint32_t kF2Stages = Shape::kStages, kF2Producers = Shape::kProducers;
   extern __shared__ uint8_t sm_raw[];
   const FgArgs& a = args.g;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   // [A tiles][B tiles], 1 KB aligned; [table copies][successors][byte stages][barriers]
   const uint32_t base = (smem_u32(sm_raw) + 1023u) & ~1023u;
-  const uint32_t a_abs = base, b_abs = base + kF2Stages * kFgATile;
+  const uint32_t a_abs = base, b_abs = base + kF2Stages * Shape::kXTile;   // (a: the slices of X; b: the tiles of W)
   const uint32_t tab_abs = b_abs + kF2Stages * kF2BTile;
   const uint32_t stride_log = 2u + args.rep_log;
   const uint32_t succ_abs = tab_abs + (1u << (a.R + stride_log));
@@ -390,7 +408,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kF2Producers) {                              // this warp owns the tensor memory
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(slot_abs), "r"(2u * kF2Cols) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(slot_abs), "r"(2u * Shape::kAccCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // the pre-walked table in one-word entries, the bf16 value folded in, copies side by side
@@ -432,6 +450,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
     const uint32_t i = warp % kF2Rows, j0 = warp / kF2Rows;
     constexpr uint32_t kStep = kF2Producers / kF2Rows;     // units between two blocks of a warp
     static_assert(kStep <= 2 * kF2Stages, "a producer must have seen the phase before the one it waits for");
+    static_assert(kStep == kF2Stages, "a producer keeps to one stage");
     const uint32_t my_stage = stages_abs + warp * args.stage_bytes;
     const uint32_t tab_lane = tab_abs + ((lane & ((1u << args.rep_log) - 1u)) << 2);
     const uint32_t dom = dequant_bits(static_cast<int>(h_dominant < 256u ? h_dominant : 0u), static_cast<int>(a.zero_point),
@@ -479,17 +498,20 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
         n1 = __ldg(a.sub_offsets + sub + 1);
       }
       const uint32_t s = j % kF2Stages, use = j / kF2Stages;   // the stage and how often it has been filled before
-      const uint32_t my_a = a_abs + s * kFgATile, my_b = b_abs + s * kF2BTile + i * kFgBTile;
+      const uint32_t my_a = a_abs + s * Shape::kXTile, my_b = b_abs + s * kF2BTile + i * kFgBTile;
       const uint32_t kb = (u0 + j) % KB;
       if (use > 0 && !__all_sync(kFull, fg_wait(empty_bar + 16u * s + 8u * ((use - 1u) & 1u), ((use - 1u) >> 1) & 1u, bad)))
         bad |= kStatusTimeout;
       // this warp's quarter of the slice of X: rows beyond M are zeros
+      constexpr uint32_t kQuarter = Shape::kXRows / kF2Rows;   // rows
 #pragma unroll
-      for (uint32_t q = 0; q < 8u; ++q) {
-        const uint32_t c = lane & 7u, r = i * 32u + q * 4u + (lane >> 3);
-        const uint32_t bytes = r < a.M ? 16u : 0u;
-        const uint16_t* src = a.x + size_t(r < a.M ? r : 0u) * a.K + size_t(kb) * kFgBlock + c * 8u;
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(my_a + tile_offset(r, c * 8u)), "l"(src), "r"(bytes) : "memory");
+      for (uint32_t q = 0; q < (kQuarter * 8u + 31u) / 32u; ++q) {
+        const uint32_t idx = q * 32u + lane, c = idx & 7u, r = i * kQuarter + (idx >> 3);
+        if (idx < kQuarter * 8u) {
+          const uint32_t bytes = r < a.M ? 16u : 0u;
+          const uint16_t* src = a.x + size_t(r < a.M ? r : 0u) * a.K + size_t(kb) * kFgBlock + c * 8u;
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(my_a + tile_offset(r, c * 8u)), "l"(src), "r"(bytes) : "memory");
+        }
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
       for (uint32_t o = lane * 16u; o < kFgBTile; o += 512u) sts_v4(my_b + o, fill4);
@@ -520,15 +542,22 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
         }
         if (!fg_wait(full_bar + 8u * s, use & 1u, bad)) bad |= kStatusTimeout;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t da = operand_desc(a_abs + s * kFgATile), db = operand_desc(b_abs + s * kF2BTile);
+        const uint64_t dx = operand_desc(a_abs + s * Shape::kXTile), dw = operand_desc(b_abs + s * kF2BTile);
 #pragma unroll
         for (uint32_t k = 0; k < kFgBlock / 16u; ++k) {    // K = 16 per instruction: 32 bytes further along the rows
           const uint32_t accumulate = (!first || k) ? 1u : 0u;
-          asm volatile(
-              "{\n\t.reg .pred p;\n\t"
-              "setp.ne.b32 p, %4, 0;\n\t"
-              "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-              :: "r"(tmem + buf * kF2Cols), "l"(da + 2u * k), "l"(db + 2u * k), "r"(kF2Idesc), "r"(accumulate), "r"(0u) : "memory");
+#pragma unroll
+          for (uint32_t h = 0; h < (NM ? 2u : 1u); ++h) {
+            // NM = 0: D[m][n] = X (128 rows) times the 256 rows of W.  Else D[n][m], one product for
+            // each half of the rows of W (128 rows = 16 KB further on), side by side in the accumulator
+            const uint64_t da = NM ? dw + uint64_t(h * (128u * 128u >> 4)) : dx, db = NM ? dx : dw;
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t"
+                "setp.ne.b32 p, %4, 0;\n\t"
+                "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+                :: "r"(tmem + buf * Shape::kAccCols + h * NM), "l"(da + 2u * k), "l"(db + 2u * k), "r"(Shape::kIdesc),
+                   "r"(accumulate), "r"(0u) : "memory");
+          }
         }
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
                      :: "r"(empty_bar + 16u * s + 8u * (use & 1u)) : "memory");
@@ -550,23 +579,48 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
       const uint32_t buf = seg & 1u;
       if (!__all_sync(kFull, fg_wait(acc_full + 8u * buf, (seg >> 1) & 1u, bad))) bad |= kStatusTimeout;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      float* yrow = a.y + size_t(row) * a.N + size_t(tile) * kF2Cols;
+      if constexpr (NM == 0) {
+        float* yrow = a.y + size_t(row) * a.N + size_t(tile) * kF2Cols;
 #pragma unroll 4
-      for (uint32_t c0 = 0; c0 < (quarter * 32u < a.M ? kF2Cols : 0u); c0 += 8u) {   // (a warp whose rows are all beyond M has nothing to store)
-        uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
-        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                     : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3), "=r"(r4), "=r"(r5), "=r"(r6), "=r"(r7)
-                     : "r"(tmem + ((quarter * 32u) << 16) + buf * kF2Cols + c0) : "memory");
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (row < a.M) {
-          if (add) {
-            atomicAdd(reinterpret_cast<float4*>(yrow + c0),
-                      make_float4(__uint_as_float(r0), __uint_as_float(r1), __uint_as_float(r2), __uint_as_float(r3)));
-            atomicAdd(reinterpret_cast<float4*>(yrow + c0 + 4),
-                      make_float4(__uint_as_float(r4), __uint_as_float(r5), __uint_as_float(r6), __uint_as_float(r7)));
-          } else {
-            *reinterpret_cast<uint4*>(yrow + c0) = make_uint4(r0, r1, r2, r3);
-            *reinterpret_cast<uint4*>(yrow + c0 + 4) = make_uint4(r4, r5, r6, r7);
+        for (uint32_t c0 = 0; c0 < (quarter * 32u < a.M ? kF2Cols : 0u); c0 += 8u) {   // (a warp whose rows are all beyond M has nothing to store)
+          uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
+          asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                       : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3), "=r"(r4), "=r"(r5), "=r"(r6), "=r"(r7)
+                       : "r"(tmem + ((quarter * 32u) << 16) + buf * kF2Cols + c0) : "memory");
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          if (row < a.M) {
+            if (add) {
+              atomicAdd(reinterpret_cast<float4*>(yrow + c0),
+                        make_float4(__uint_as_float(r0), __uint_as_float(r1), __uint_as_float(r2), __uint_as_float(r3)));
+              atomicAdd(reinterpret_cast<float4*>(yrow + c0 + 4),
+                        make_float4(__uint_as_float(r4), __uint_as_float(r5), __uint_as_float(r6), __uint_as_float(r7)));
+            } else {
+              *reinterpret_cast<uint4*>(yrow + c0) = make_uint4(r0, r1, r2, r3);
+              *reinterpret_cast<uint4*>(yrow + c0 + 4) = make_uint4(r4, r5, r6, r7);
+            }
+          }
+        }
+      } else {
+        // lane n of the tensor memory holds feature n of a half, its columns the rows of X: the
+        // warp's 32 lanes store 32 consecutive floats of one row of Y at a time
+#pragma unroll
+        for (uint32_t h = 0; h < 2u; ++h) {
+          float* ycol = a.y + size_t(tile) * kF2Cols + h * 128u + row;
+#pragma unroll
+          for (uint32_t c0 = 0; c0 < NM; c0 += 16u) {
+            uint32_t r[16];
+            asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                         : "r"(tmem + ((quarter * 32u) << 16) + buf * Shape::kAccCols + h * NM + c0) : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (uint32_t m = 0; m < 16u; ++m) {
+              if (c0 + m < a.M) {
+                if (add) atomicAdd(ycol + size_t(c0 + m) * a.N, __uint_as_float(r[m]));
+                else ycol[size_t(c0 + m) * a.N] = __uint_as_float(r[m]);
+              }
+            }
           }
         }
       }
@@ -581,10 +635,71 @@ __global__ void __launch_bounds__(kF2Threads, 1) ans_decode_gemm_wide_kernel(con
   if (warp == kF2Producers) {
     __syncwarp();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(2u * kF2Cols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(2u * Shape::kAccCols) : "memory");
   }
   bad = __reduce_or_sync(kFull, bad);
   if (lane == 0 && bad && a.d_status) atomicOr(a.d_status, bad);
+}
+
+}  // namespace ansb
+
+namespace ansb {
+
+// Launch the wide form NM (see F2Shape).  Returns ANS_OK, an error, or 1 if the form does not
+// fit this device's shared memory.
+template <uint32_t NM>
+static int launch_wide(const FgArgs& a, const ans_layer_desc& d, int sms, int smem_max, cudaStream_t st) {
+  using Shape = F2Shape<NM>;
+  const uint32_t M = a.M, N = a.N, K = a.K;
+  // room for a sub-stream of up to 1.25 times the average plus the padding per producer, less if
+  // shared memory is short (a sub-stream that does not fit is read from global memory); what
+  // shared memory is left goes to copies of the table
+  const uint64_t n_sub = uint64_t(N / 64) * uint64_t(K / 64);
+  size_t stage = static_cast<size_t>(d.stream_bytes / n_sub);
+  stage = (stage + stage / 4 + 128 + kF2Pad + 127) & ~size_t(127);
+  const size_t succ = (size_t(2) << d.table_log) < 16 ? 16 : (size_t(2) << d.table_log);
+  const size_t one_table = size_t(4) << d.table_log;
+  const size_t rest = 1024 + Shape::kStages * (Shape::kXTile + kF2BTile) + succ + 256;
+  const size_t room = static_cast<size_t>(smem_max) > rest + one_table ? static_cast<size_t>(smem_max) - rest - one_table : 0;
+  if (Shape::kProducers * stage > room) stage = (room / Shape::kProducers) & ~size_t(127);
+  const size_t fixed = rest + Shape::kProducers * stage;
+  if (stage < 512) return 1;
+  uint32_t rep_log = 0;
+  while (rep_log < 5 && fixed + (one_table << (rep_log + 1)) <= static_cast<size_t>(smem_max)) ++rep_log;
+  const uint32_t KB = K / 64, tiles = N / kF2Cols;
+  const uint64_t units = uint64_t(tiles) * KB;
+  if (units > 0x7FFFFFFFull) return ANS_ERR_UNSUPPORTED;
+  // CTAs: one per SM with the units dealt evenly, or, if that saves no round of the producers
+  // (a stage's worth of units is decoded at a time), a whole number of CTAs per 256 features, so
+  // that no range crosses from one accumulator's features to the next
+  uint32_t ctas = units < static_cast<uint64_t>(sms) ? static_cast<uint32_t>(units) : static_cast<uint32_t>(sms);
+  {
+    uint32_t per_tile = static_cast<uint32_t>(sms) / tiles;
+    if (per_tile > KB) per_tile = KB;
+    const uint32_t aligned = tiles * per_tile;
+    constexpr uint32_t kAtATime = Shape::kStages;
+    auto rounds = [&](uint32_t n) { return ((units + n - 1) / n + kAtATime - 1) / kAtATime; };
+    if (aligned >= 1 && rounds(aligned) <= rounds(ctas)) {
+      // and no more CTAs than that number of rounds needs: fewer partial sums to add
+      while (per_tile > 1 && rounds(tiles * (per_tile - 1)) == rounds(aligned)) --per_tile;
+      ctas = tiles * per_tile;
+    }
+  }
+  // Y is zeroed first if any range ends inside the K steps of its 256 features (those parts are added)
+  bool whole = true;
+  for (uint32_t c = 1; c < ctas && whole; ++c) whole = (units * c / ctas) % KB == 0;
+  F2Args w{};
+  w.g = a;
+  w.units = static_cast<uint32_t>(units);
+  w.stage_bytes = static_cast<uint32_t>(stage);
+  w.rep_log = rep_log;
+  w.unit = 1u;
+  const size_t smem = fixed + (one_table << rep_log);
+  if (!whole) ANSB_CUDA(cudaMemsetAsync(a.y, 0, size_t(M) * size_t(N) * sizeof(float), st));
+  ANSB_CUDA(cudaFuncSetAttribute(ans_decode_gemm_wide_kernel<NM>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  ans_decode_gemm_wide_kernel<NM><<<ctas, Shape::kThreads, smem, st>>>(w);
+  ANSB_CUDA(cudaGetLastError());
+  return ANS_OK;
 }
 
 }  // namespace ansb
@@ -624,56 +739,10 @@ ANS_EXPORT int ans_decode_gemm_bf16(const ans_layer_desc* h_desc, const void* d_
   ANSB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   ANSB_CUDA(cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
   if (d.table_log <= 8 && N % static_cast<int>(kF2Cols) == 0) {
-    // the wide form: room for a sub-stream of up to 1.25 times the average plus the padding per
-    // producer, less if shared memory is short (a sub-stream that does not fit is read from global
-    // memory); what shared memory is left goes to copies of the table
-    const uint64_t n_sub = uint64_t(N / 64) * uint64_t(K / 64);
-    size_t stage = static_cast<size_t>(d.stream_bytes / n_sub);
-    stage = (stage + stage / 4 + 128 + kF2Pad + 127) & ~size_t(127);
-    const size_t succ = (size_t(2) << d.table_log) < 16 ? 16 : (size_t(2) << d.table_log);
-    const size_t one_table = size_t(4) << d.table_log;
-    const size_t rest = 1024 + kF2Stages * (kFgATile + kF2BTile) + succ + 128;
-    const size_t room = static_cast<size_t>(smem_max) > rest + one_table ? static_cast<size_t>(smem_max) - rest - one_table : 0;
-    if (kF2Producers * stage > room) stage = (room / kF2Producers) & ~size_t(127);
-    const size_t fixed = rest + kF2Producers * stage;
-    if (stage >= 512) {
-      uint32_t rep_log = 0;
-      while (rep_log < 5 && fixed + (one_table << (rep_log + 1)) <= static_cast<size_t>(smem_max)) ++rep_log;
-      const uint32_t KB = static_cast<uint32_t>(K / 64), tiles = static_cast<uint32_t>(N) / kF2Cols;
-      const uint64_t units = uint64_t(tiles) * KB;
-      if (units > 0x7FFFFFFFull) return ANS_ERR_UNSUPPORTED;
-      // CTAs: one per SM with the units dealt evenly, or, if that saves no round of the producers
-      // (four units are decoded at a time), a whole number of CTAs per 256 features, so that no
-      // range crosses from one accumulator's features to the next
-      uint32_t ctas = units < static_cast<uint64_t>(sms) ? static_cast<uint32_t>(units) : static_cast<uint32_t>(sms);
-      {
-        uint32_t per_tile = static_cast<uint32_t>(sms) / tiles;
-        if (per_tile > KB) per_tile = KB;
-        const uint32_t aligned = tiles * per_tile;
-        constexpr uint32_t kAtATime = kF2Producers / kF2Rows;
-        auto rounds = [&](uint32_t n) { return ((units + n - 1) / n + kAtATime - 1) / kAtATime; };
-        if (aligned >= 1 && rounds(aligned) <= rounds(ctas)) {
-          // and no more CTAs than that number of rounds needs: fewer partial sums to add
-          while (per_tile > 1 && rounds(tiles * (per_tile - 1)) == rounds(aligned)) --per_tile;
-          ctas = tiles * per_tile;
-        }
-      }
-      // Y is zeroed first if any range ends inside the K steps of its 256 features (those parts are added)
-      bool whole = true;
-      for (uint32_t c = 1; c < ctas && whole; ++c) whole = (units * c / ctas) % KB == 0;
-      F2Args w{};
-      w.g = a;
-      w.units = static_cast<uint32_t>(units);
-      w.stage_bytes = static_cast<uint32_t>(stage);
-      w.rep_log = rep_log;
-      w.unit = 1u;
-      const size_t smem = fixed + (one_table << rep_log);
-      if (!whole) ANSB_CUDA(cudaMemsetAsync(d_y, 0, size_t(M) * size_t(N) * sizeof(float), st));
-      ANSB_CUDA(cudaFuncSetAttribute(ans_decode_gemm_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-      ans_decode_gemm_wide_kernel<<<ctas, kF2Threads, smem, st>>>(w);
-      ANSB_CUDA(cudaGetLastError());
-      return ANS_OK;
-    }
+    // the wide forms: the one with the operands exchanged when X has few rows
+    const int rc2 = M <= 16 ? launch_wide<16>(a, d, sms, smem_max, st)
+                  : M <= 32 ? launch_wide<32>(a, d, sms, smem_max, st) : launch_wide<0>(a, d, sms, smem_max, st);
+    if (rc2 != 1) return rc2;                              // (1: shared memory too short for it)
   }
   const size_t smem = 1024 + kFgStages * (kFgATile + kFgBTile) + (size_t(4) << d.table_log) + 1024 + 128;
   ANSB_CUDA(cudaFuncSetAttribute(ans_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));

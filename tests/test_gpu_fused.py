@@ -84,12 +84,16 @@ def test_fused_product_equals_the_oracles_weights_times_x(M, N, K, b, pzp, R):
 # The wide form of the kernel (tables of up to 256 states, N a multiple of 256): ranges that end
 # inside the K steps of their 256 features (partial sums added in Y) and ranges that do not (plain
 # stores: one unit per CTA with K = 64, or 37888 = 148 * 256 features with two steps each on a
-# 148-SM part), several segments per CTA, stages reused many times, M below a full tile.
+# 148-SM part), several segments per CTA, stages reused many times, M below a full tile; and the
+# forms with the operands exchanged that M <= 16 and M <= 32 take (Y^T = W X^T).
 @pytest.mark.parametrize("M,N,K,b,pzp,R,quiet", [(128, 256, 256, 3, 0.7, 8, 0), (50, 512, 1024, 4, 0.6, 8, 0),
                                                  (128, 2048, 4800, 3, 0.8, 8, 0), (8, 19200, 640, 2, 0.9, 6, 0),
                                                  (33, 256, 64, 3, 0.7, 7, 0), (128, 1024, 2048, 6, 0.5, 8, 3),
                                                  (64, 256, 19008, 3, 0.7, 8, 0), (4, 19200, 1408, 3, 0.7, 8, 0),
-                                                 (16, 37888, 128, 3, 0.7, 8, 0), (128, 1024, 64, 4, 0.6, 8, 0)])
+                                                 (16, 37888, 128, 3, 0.7, 8, 0), (128, 1024, 64, 4, 0.6, 8, 0),
+                                                 (32, 512, 1024, 3, 0.7, 8, 0), (17, 256, 2112, 4, 0.8, 8, 0),
+                                                 (31, 2048, 4800, 3, 0.8, 7, 0), (1, 256, 256, 3, 0.7, 8, 0),
+                                                 (12, 1024, 2048, 6, 0.5, 8, 3), (24, 19200, 640, 2, 0.9, 6, 0)])
 def test_wide_form_equals_the_oracles_weights_times_x(M, N, K, b, pzp, R, quiet):
     spec, P, f256, x, x64, w = _case(M, N, K, b, pzp, R, seed=M + N + K, quiet_rows=quiet)
     if quiet:                               # the kept block rows' sub-streams are far above the average: they do not fit the staging room
