@@ -402,14 +402,15 @@ def run_fused(ans, args, local, sampler=None, M=128, min_region_s=0.3):
     pl = pack_gemm_layer(sym.reshape(N, K), spec.alphabet, 8, spec.bitwidth, spec.zero_point, spec.scale,
                          n_threads=max(1, cores // 2))
     db = DeviceBatch([pl] * FUSED_COPIES, f"cuda:{local}")
-    x = torch.randn(M, K, device=f"cuda:{local}").to(torch.bfloat16)
+    x_full = torch.randn(M, K, device=f"cuda:{local}").to(torch.bfloat16)
+    x = x_full
     y = torch.empty(M, N, dtype=torch.float32, device=f"cuda:{local}")
     st = torch.cuda.current_stream()
     descs = db.h_descs[0]
     outs = [db.output(i).view(N, K) for i in range(FUSED_COPIES)]
 
     def fused(i):
-        ans.ans_decode_gemm_bf16(descs[i], x.data_ptr(), M, N, K, y.data_ptr(), db.status.data_ptr(), st.cuda_stream)
+        ans.ans_decode_gemm_bf16(descs[i], x.data_ptr(), x.shape[0], N, K, y.data_ptr(), db.status.data_ptr(), st.cuda_stream)
 
     def two_steps(i):
         ans.ans_decode_dequant(descs[i], db.status.data_ptr(), st.cuda_stream)
@@ -463,6 +464,14 @@ def run_fused(ans, args, local, sampler=None, M=128, min_region_s=0.3):
            "bound": "the decode's instruction issue, as for the decode kernels (see profiles/); not the tensor cores",
            "clocks": sampler.summary() if sampler else None}
     launches = (len(rf) + len(rt)) * steps + 11
+    # the same with 16 rows of X (the kernel then takes its form with the operands exchanged)
+    x = x_full[:16].contiguous()
+    r16f = timed(fused, steps)
+    r16t = timed(two_steps, steps)
+    assert db.read_status() == 0, "decoder flagged a stream"
+    res["rows_16"] = {"fused_ms_mean": sum(r16f) / len(r16f), "decode_then_matmul_ms_mean": sum(r16t) / len(r16t),
+                      "speedup_over_two_steps": (sum(r16t) / len(r16t)) / (sum(r16f) / len(r16f))}
+    launches += (len(r16f) + len(r16t)) * steps + 10
     del db
     torch.cuda.empty_cache()
     return res, launches
