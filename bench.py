@@ -509,6 +509,13 @@ def run_ours(args):
     sampler.last = len(sampler.rows)
     db_flags = db.h_descs[0][0].flags if layers else 0
     clocks = sampler.summary() if rank == 0 else None
+    # the same launches with the descriptor flags cleared: every launch waits for the one before it
+    waiting_ms = None
+    if db_flags and world == 1:
+        db.set_flags(0)
+        wr, _ = time_workload(db, args.steps, 3, n_sets, world, min_region_s=0.15)
+        waiting_ms = sum(wr) / len(wr)
+        db.set_flags(int(db_flags))
     ms_per_step = reduce_max(rounds[0], world)          # the K steps asked for: the first round
     fg = figures(ans, layers, db, rounds, each, peak)
     n_w = fg["n_w"]
@@ -525,8 +532,11 @@ def run_ours(args):
                 "round_ms_per_launch_min": min(rounds), "round_ms_per_launch_max": max(rounds),
                 "launch_bracketed_alone_ms_median": statistics.median(each), "launch_bracketed_alone_ms_min": min(each),
                 "frac_of_nominal_8TBs": fg["frac_nominal"],
+                "kernel_ms_mean_launches_waiting": waiting_ms,
+                "frac_launches_waiting": (fg["frac"] * fg["kernel_ms"] / waiting_ms) if waiting_ms else None,
                 "note": "kernel_ms_mean: CUDA events around rounds of back-to-back launches, divided by the launches "
-                        "(gaps between launches included); HBM is the metric's roofline, the kernels themselves are "
+                        "(gaps between launches included; the descriptors carry the flags in config.desc_flags, so a launch may "
+                        "begin while the one before it drains; *_launches_waiting: the same with the flags cleared); HBM is the metric's roofline, the kernels themselves are "
                         "held by instruction issue and shared-memory wavefronts (see profiles/)"}
 
     # end to end through the host-buffer entry point: pinned host buffers in, pinned out
@@ -537,6 +547,8 @@ def run_ours(args):
     cpu = cpu_baseline(specs, syms, args.layout, args.lanes) if world == 1 and rank == 0 and not args.no_cpu_baseline else None
     head_specs = specs
     launches = (len(rounds) + 1) * args.steps * db.launches_per_decode()
+    if waiting_ms is not None:
+        launches += (len(wr) + 1) * args.steps * db.launches_per_decode() + 3
 
     # the other workloads and table sizes, each measured the same way (shorter regions)
     variants = []

@@ -158,6 +158,15 @@ class DeviceBatch:
             self.d_descs.append(raw.to(self.device))
         torch.cuda.synchronize(self.device)
 
+    def set_flags(self, flags: int) -> None:
+        """Write `flags` (ANS_DESC_* bits) into every layer descriptor, host and device copies."""
+        torch.cuda.synchronize(self.device)
+        for k, arr in enumerate(self.h_descs):
+            for i in range(len(self.layers)):
+                arr[i].flags = flags
+            self.d_descs[k].copy_(torch.frombuffer(bytearray(bytes(arr)), dtype=torch.uint8))
+        torch.cuda.synchronize(self.device)
+
     # -- sizes for reporting -------------------------------------------------------------
     def compressed_bytes(self) -> int:
         return sum(L.compressed_bytes() for L in self.layers)
