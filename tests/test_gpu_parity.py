@@ -332,6 +332,37 @@ def test_substream_ends_off_a_16_byte_boundary_are_flagged(layout):
     assert db.read_status() == 0
 
 
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("idle", [False, True])
+@pytest.mark.parametrize("big", [False, True])
+def test_launches_queued_back_to_back_with_the_descriptor_flags(layout, idle, big):
+    """ANS_DESC_INPUTS_SETTLED / ANS_DESC_OUTPUT_IDLE on the general kernel: launches queued behind a
+    device-side spin, rotating over three output sets, every set poisoned first and compared with the
+    oracle afterwards; small layers (CTAs of four warps) and one big enough for the many-warp shape."""
+    if big:
+        specs = [tiny_spec(6_000_000, 3, 0.7, 8, 16384, "bf16", index=0)]
+    else:
+        specs = [tiny_spec(200_000, 3, 0.8, 9, 8192, "bf16", index=0), tiny_spec(50_001, 5, 0.6, 11, 4096, "f32", index=1),
+                 tiny_spec(0, 2, 0.8, 6, 4096, "u8", index=2), tiny_spec(99_999, 2, 0.9, 7, 16384, "u8", index=3)]
+    prepared = []
+    for spec in specs:
+        sym = sg.draw_symbols(spec)
+        T, P, f256 = oracle_pack_spec(spec, sym, layout, 32)
+        prepared.append((to_packed_layer(spec, P, f256), oracle_expected(spec, T, P)[1]))
+    db = DeviceBatch([p[0] for p in prepared], n_out_sets=3, inputs_settled=True, output_idle=idle)
+    for outs in db.out_sets:
+        for o in outs:
+            o.view(torch.uint8).fill_(0xA5)
+    torch.cuda.synchronize()
+    torch.cuda._sleep(20_000_000)
+    for i in range(12):
+        db.decode(i % 3)
+    assert db.read_status() == 0
+    for k in range(3):
+        for i, (pl, want) in enumerate(prepared):
+            assert (bits_view(db.output(i, k)) == expected_bits(want)).all(), (k, i)
+
+
 def test_bitwidth_check():
     spec = tiny_spec(5000, 4, 0.6, 12, 4096, "u8")
     sym = sg.draw_symbols(spec)

@@ -336,14 +336,24 @@ def _channels_case(shape, b, pzp, R, dt, index=0, chunk_rows=0):
     return spec, T, P, f256, sym, oracle.dequant(sym, spec.zero_point, spec.scale, dt)
 
 
-def _decode_and_compare(cases, per_layer=False):
-    db = DeviceBatch([to_packed_layer(c[0], c[2], c[3]) for c in cases])
-    for o in db.out_sets[0]:
-        o.view(torch.uint8).fill_(0xA5)
-    (db.decode_per_layer if per_layer else db.decode)()
+def _decode_and_compare(cases, per_layer=False, flagged=False):
+    """flagged: descriptor flags set, six launches queued back to back over two output sets."""
+    db = DeviceBatch([to_packed_layer(c[0], c[2], c[3]) for c in cases], n_out_sets=2 if flagged else 1,
+                     inputs_settled=flagged, output_idle=flagged)
+    for outs in db.out_sets:
+        for o in outs:
+            o.view(torch.uint8).fill_(0xA5)
+    if flagged:
+        torch.cuda.synchronize()
+        torch.cuda._sleep(10_000_000)
+        for k in range(6):
+            db.decode(k % 2)
+    else:
+        (db.decode_per_layer if per_layer else db.decode)()
     assert db.read_status() == 0
-    for i, c in enumerate(cases):
-        assert np.array_equal(bits_view(db.output(i)), expected_bits(c[5])), f"layer {i} {c[0].shape}"
+    for k in range(len(db.out_sets)):
+        for i, c in enumerate(cases):
+            assert np.array_equal(bits_view(db.output(i, k)), expected_bits(c[5])), f"set {k} layer {i} {c[0].shape}"
     return db
 
 
@@ -357,6 +367,7 @@ def test_channels_conv_shapes(dt):
     db = _decode_and_compare(cases)
     assert (db.decode_symbols(0).cpu().numpy() == cases[0][4]).all() and db.read_status() == 0
     _decode_and_compare(cases[:3], per_layer=True)
+    _decode_and_compare(cases, flagged=True)
 
 
 def test_channels_resnet50_by_input_channel():
