@@ -291,7 +291,7 @@ LAYOUT_IDS = {"private": "ANS_LAYOUT_PRIVATE", "interleaved": "ANS_LAYOUT_INTERL
               "strips": "ANS_LAYOUT_STRIPS"}
 
 
-def build_case(ans, args, workload, layout_name, lanes, table_log=0, chunk=0, local=0, by_channel=False, settled=True):
+def build_case(ans, args, workload, layout_name, lanes, table_log=0, chunk=0, local=0, by_channel=False, flags=3):
     """Draw the workload's symbols, pack them with the library's host packer, put everything on
     the device.  Returns (specs, syms, layers, db, n_sets, working-set text)."""
     import copy
@@ -337,9 +337,9 @@ def build_case(ans, args, workload, layout_name, lanes, table_log=0, chunk=0, lo
     # change: the descriptors say so (ANS_DESC_INPUTS_SETTLED), which lets a strips launch fetch them
     # and begin while the launch before it drains; where the launches rotate over several output
     # sets, a launch writes a set that the launch before it does not touch (ANS_DESC_OUTPUT_IDLE)
-    settled = settled and not args.no_settled
+    settled = bool(flags & 1) and not args.no_settled
     db = DeviceBatch(layers, f"cuda:{local}", n_out_sets=n_sets, inputs_settled=settled,
-                     output_idle=n_sets >= 2 and settled)
+                     output_idle=bool(flags & 2) and n_sets >= 2 and settled and not args.no_idle)
     policy = (f"inputs larger than L2: launches rotate over {n_sets} full copies of the workload "
               f"({n_sets * ws / 2**20:.0f} MB in all)" if small
               else f"working set (compressed + output) is larger than L2; launches alternate between {n_sets} full copies")
@@ -374,13 +374,13 @@ def entropy_bits(specs, syms):
 
 # (workload, container, lanes, table_log, chunk) measured beside the headline: the other table size
 # quoted for the large layers, the two ResNets, one cell of the granularity sweep
-# last field: whether the descriptors carry ANS_DESC_INPUTS_SETTLED / ANS_DESC_OUTPUT_IDLE (only the strips
-# kernel reads them); resnet50 is measured both ways
-VARIANTS = [("large", "quads", 32, 12, 0, True), ("resnet50", "strips", 32, 0, 0, True),
-            ("resnet50", "strips", 64, 0, 0, True), ("resnet50", "strips", 64, 0, 0, False),
-            ("resnet50", "strips", 32, 0, 0, False), ("resnet50", "quads", 32, 0, 0, True),
-            ("resnet50", "strips", 64, 12, 0, True), ("resnet18", "strips", 64, 0, 0, True),
-            ("resnet18", "quads", 32, 0, 0, True), ("sweep", "quads", 32, 12, 16384, True)]
+# last field: the descriptor flags (3: ANS_DESC_INPUTS_SETTLED | ANS_DESC_OUTPUT_IDLE, 1: the first only,
+# 0: none: every launch waits for the one before it); resnet50 is measured all three ways
+VARIANTS = [("large", "quads", 32, 12, 0, 3), ("resnet50", "strips", 32, 0, 0, 3),
+            ("resnet50", "strips", 64, 0, 0, 3), ("resnet50", "strips", 64, 0, 0, 1), ("resnet50", "strips", 64, 0, 0, 0),
+            ("resnet50", "strips", 32, 0, 0, 0), ("resnet50", "quads", 32, 0, 0, 3),
+            ("resnet50", "strips", 64, 12, 0, 3), ("resnet18", "strips", 64, 0, 0, 3),
+            ("resnet18", "quads", 32, 0, 0, 3), ("sweep", "quads", 32, 12, 16384, 3)]
 
 
 FUSED_COPIES = 12           # device copies of the compressed matrix the fused launches rotate over (> L2 in all)
@@ -557,7 +557,7 @@ def run_ours(args):
         del db
         torch.cuda.empty_cache()
         for wl, lay, ln, tl, ck, vflag in VARIANTS:
-            vs, vy, vl, vdb, vsets, vpol = build_case(ans, args, wl, lay, ln, tl, ck, local, settled=vflag)
+            vs, vy, vl, vdb, vsets, vpol = build_case(ans, args, wl, lay, ln, tl, ck, local, flags=vflag)
             sampler.first = len(sampler.rows)
             vr, ve = time_workload(vdb, min(args.steps, 200) if wl in ("large", "sweep") else max(args.steps, 100), 5, vsets, 1,
                                    min_region_s=0.3)
@@ -689,6 +689,8 @@ def main():
     ap.add_argument("--no-settled", action="store_true",
                     help="set neither ANS_DESC_INPUTS_SETTLED nor ANS_DESC_OUTPUT_IDLE: every launch waits for the one "
                          "before it before it reads anything")
+    ap.add_argument("--no-idle", action="store_true",
+                    help="set ANS_DESC_INPUTS_SETTLED only: a launch waits for the one before it before its first write")
     ap.add_argument("--fused-only", action="store_true",
                     help="only the fused decode + matrix product measurement (one short region), as one JSON line")
     args = ap.parse_args()
