@@ -370,6 +370,14 @@ int ans_normalize_freqs_device(const uint64_t* d_counts, int alphabet, int table
  * written), bit 4 = a symbol without a state in the table, or a lane longer than 65535 bits.
  */
 int ans_encode_scratch_bytes(uint64_t n_symbols, uint32_t chunk_symbols, uint32_t lanes, size_t* h_bytes_out);
+/* The same for the channels container (Section III-B: one stream per input channel of a tensor
+ * stored O x I x H x W): byte for byte what ans_host_pack_channels writes; sizes as there
+ * (piece_symbols = H * W in 1 .. ANS_MAX_PIECE_SYMBOLS, lanes = I, chunk_symbols and n_symbols
+ * multiples of lanes * piece_symbols); buffers, scratch and status as for ans_encode_layer_device. */
+int ans_encode_channels_device(const uint8_t* d_symbols, uint64_t n_symbols, const void* d_table, int table_log,
+                               uint32_t chunk_symbols, uint32_t lanes, uint32_t piece_symbols,
+                               uint8_t* d_stream_out, uint64_t stream_cap, uint64_t* d_sub_offsets_out,
+                               void* d_scratch, size_t d_scratch_bytes, uint32_t* d_status, void* stream);
 int ans_encode_layer_device(const uint8_t* d_symbols, uint64_t n_symbols, const void* d_table, int table_log,
                             uint32_t chunk_symbols, uint32_t lanes, int layout, uint8_t* d_stream_out,
                             uint64_t stream_cap, uint64_t* d_sub_offsets_out, void* d_scratch,

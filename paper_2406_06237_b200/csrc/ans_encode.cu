@@ -142,6 +142,7 @@ struct EncArgs {
   int R;
   uint32_t chunk;
   uint32_t G;                  // lanes / 32
+  uint32_t piece;              // channels container: symbols of a piece; 0: strips
   uint64_t n_sub;
   uint16_t* lens;              // [n_sub][32] bit length of every lane's string
   unsigned long long* sizes;   // [n_sub] bytes of every sub-stream
@@ -182,10 +183,14 @@ __device__ __forceinline__ void build_enc_tables(const uint8_t* blob, int R, Enc
 // One lane's encoding, backwards from state index 0 (so that its decoder ends there).  With WRITE
 // the fields go to their places: the string ends at bit `end` of the sub-stream's body and is
 // filled from the back; bit p of the body is bit 31 - p % 32 of its 32-bit little-endian word p / 32.
+// strip: the lane's symbol t is strip[t * 32 + lane] (strips: `strip` is the sub-stream's first
+// symbol), or, with piece = E > 0 (channels), strip[((t / E) * row + lane) * E + t % E], `strip`
+// being the first symbol of the sub-stream's first lane and row = lanes per chunk.
 template <bool WRITE>
 __device__ __forceinline__ uint32_t encode_lane(const EncTables& T, int R, const uint8_t* strip, uint32_t count,
                                                 uint32_t lane, uint32_t* body, uint64_t body_words, uint32_t end,
-                                                uint32_t& state_out, bool& bad_symbol) {
+                                                uint32_t& state_out, bool& bad_symbol, uint32_t piece = 0,
+                                                uint32_t row = 0) {
   const uint32_t L = 1u << R;
   uint32_t x = L, bits = 0;
   uint32_t word = 0, acc = 0;            // WRITE: the word being filled and the bits collected for it
@@ -201,7 +206,7 @@ __device__ __forceinline__ uint32_t encode_lane(const EncTables& T, int R, const
     }
   };
   for (uint32_t t = count; t-- > 0;) {
-    const uint32_t s = strip[size_t(t) * 32u + lane];
+    const uint32_t s = piece ? strip[(size_t(t / piece) * row + lane) * piece + t % piece] : strip[size_t(t) * 32u + lane];
     const uint32_t f = T.f[s];
     if (!f) { bad_symbol = true; break; }
     const uint32_t maxb = static_cast<uint32_t>(R) - (31u - static_cast<uint32_t>(__clz(f)));
@@ -236,12 +241,17 @@ __global__ void __launch_bounds__(kEncWarps * 32) encode_strips_kernel(const Enc
   const uint64_t nc = min(uint64_t(a.chunk), a.n - c0);
   const uint64_t sfirst = uint64_t(g) * 32u * S;
   const uint32_t ns = nc > sfirst ? static_cast<uint32_t>(min(nc - sfirst, uint64_t(32u) * S)) : 0u;
-  const uint32_t count = ns > lane ? (ns - lane + 31u) / 32u : 0u;
+  uint32_t count = ns > lane ? (ns - lane + 31u) / 32u : 0u;
   const uint8_t* strip = a.sym + c0 + sfirst;
+  const uint32_t row = 32u * a.G;
+  if (a.piece) {               // channels: lanes 32 g .. 32 g + 31 of the chunk, every lane nc / W symbols in pieces
+    count = static_cast<uint32_t>(nc / row);
+    strip = a.sym + c0 + size_t(32u * g) * a.piece;
+  }
   uint32_t state = 0;
   bool bad = false;
   if (!WRITE) {
-    const uint32_t len = encode_lane<false>(T, a.R, strip, count, lane, nullptr, 0, 0, state, bad);
+    const uint32_t len = encode_lane<false>(T, a.R, strip, count, lane, nullptr, 0, 0, state, bad, a.piece, row);
     a.lens[sub * 32 + lane] = static_cast<uint16_t>(len);
     uint32_t total = len;
 #pragma unroll
@@ -262,7 +272,7 @@ __global__ void __launch_bounds__(kEncWarps * 32) encode_strips_kernel(const Enc
       reinterpret_cast<uint16_t*>(dst)[lane] = static_cast<uint16_t>(len);
       uint32_t* body = reinterpret_cast<uint32_t*>(dst + kEncHeader);
       const uint64_t body_words = (off1 - off0 - kEncHeader) / 4;
-      encode_lane<true>(T, a.R, strip, count, lane, body, body_words, incl, state, bad);
+      encode_lane<true>(T, a.R, strip, count, lane, body, body_words, incl, state, bad, a.piece, row);
     } else if (lane == 0 && a.status) {
       atomicOr(a.status, 2u);
     }
@@ -341,16 +351,21 @@ ANS_EXPORT int ans_encode_scratch_bytes(uint64_t n_symbols, uint32_t chunk_symbo
   return ANS_OK;
 }
 
-ANS_EXPORT int ans_encode_layer_device(const uint8_t* d_symbols, uint64_t n_symbols, const void* d_table, int table_log,
-                                       uint32_t chunk_symbols, uint32_t lanes, int layout, uint8_t* d_stream_out,
-                                       uint64_t stream_cap, uint64_t* d_sub_offsets_out, void* d_scratch,
-                                       size_t d_scratch_bytes, uint32_t* d_status, void* stream) {
+static int encode_device(const uint8_t* d_symbols, uint64_t n_symbols, const void* d_table, int table_log,
+                         uint32_t chunk_symbols, uint32_t lanes, uint32_t piece, uint8_t* d_stream_out,
+                         uint64_t stream_cap, uint64_t* d_sub_offsets_out, void* d_scratch,
+                         size_t d_scratch_bytes, uint32_t* d_status, void* stream) {
   if (!d_sub_offsets_out || !d_status) return ANS_ERR_INVALID_ARG;
-  if (layout != ANS_LAYOUT_STRIPS) return ANS_ERR_UNSUPPORTED;
   if (table_log < 1 || table_log > ANS_MAX_TABLE_LOG) return ANS_ERR_UNSUPPORTED;
-  if (lanes < 32 || lanes > ANS_MAX_LANES || lanes % 32 || chunk_symbols == 0 || chunk_symbols % lanes ||
-      chunk_symbols / lanes > ANS_MAX_STRIP_LANE_SYMBOLS)
+  if (lanes < 32 || lanes > ANS_MAX_LANES || lanes % 32 || chunk_symbols == 0) return ANS_ERR_UNSUPPORTED;
+  if (piece) {                                             // channels container
+    if (piece > ANS_MAX_PIECE_SYMBOLS) return ANS_ERR_UNSUPPORTED;
+    const uint64_t unit = uint64_t(lanes) * piece;
+    if (chunk_symbols % unit || n_symbols % unit || chunk_symbols / lanes > ANS_MAX_CHANNEL_LANE_SYMBOLS)
+      return ANS_ERR_UNSUPPORTED;
+  } else if (chunk_symbols % lanes || chunk_symbols / lanes > ANS_MAX_STRIP_LANE_SYMBOLS) {
     return ANS_ERR_UNSUPPORTED;
+  }
   size_t need = 0;
   int rc = ans_encode_scratch_bytes(n_symbols, chunk_symbols, lanes, &need);
   if (rc != ANS_OK) return rc;
@@ -372,6 +387,7 @@ ANS_EXPORT int ans_encode_layer_device(const uint8_t* d_symbols, uint64_t n_symb
   a.R = table_log;
   a.chunk = chunk_symbols;
   a.G = lanes / 32;
+  a.piece = piece;
   a.n_sub = ((n_symbols + chunk_symbols - 1) / chunk_symbols) * a.G;
   if (a.n_sub > 0x7FFFFFFFull * kEncWarps) return ANS_ERR_UNSUPPORTED;
   uint8_t* p = static_cast<uint8_t*>(d_scratch);
@@ -392,4 +408,22 @@ ANS_EXPORT int ans_encode_layer_device(const uint8_t* d_symbols, uint64_t n_symb
   encode_strips_kernel<true><<<blocks, kEncWarps * 32, smem, st>>>(a);
   ANSB_CUDA(cudaGetLastError());
   return ANS_OK;
+}
+
+ANS_EXPORT int ans_encode_layer_device(const uint8_t* d_symbols, uint64_t n_symbols, const void* d_table, int table_log,
+                                       uint32_t chunk_symbols, uint32_t lanes, int layout, uint8_t* d_stream_out,
+                                       uint64_t stream_cap, uint64_t* d_sub_offsets_out, void* d_scratch,
+                                       size_t d_scratch_bytes, uint32_t* d_status, void* stream) {
+  if (layout != ANS_LAYOUT_STRIPS) return ANS_ERR_UNSUPPORTED;
+  return encode_device(d_symbols, n_symbols, d_table, table_log, chunk_symbols, lanes, 0, d_stream_out, stream_cap,
+                       d_sub_offsets_out, d_scratch, d_scratch_bytes, d_status, stream);
+}
+
+ANS_EXPORT int ans_encode_channels_device(const uint8_t* d_symbols, uint64_t n_symbols, const void* d_table, int table_log,
+                                          uint32_t chunk_symbols, uint32_t lanes, uint32_t piece_symbols,
+                                          uint8_t* d_stream_out, uint64_t stream_cap, uint64_t* d_sub_offsets_out,
+                                          void* d_scratch, size_t d_scratch_bytes, uint32_t* d_status, void* stream) {
+  if (piece_symbols < 1) return ANS_ERR_UNSUPPORTED;
+  return encode_device(d_symbols, n_symbols, d_table, table_log, chunk_symbols, lanes, piece_symbols, d_stream_out,
+                       stream_cap, d_sub_offsets_out, d_scratch, d_scratch_bytes, d_status, stream);
 }

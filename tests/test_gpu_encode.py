@@ -127,6 +127,49 @@ def test_device_encoder_writes_the_oracles_bytes(n, C, lanes, R, b, pzp):
     assert got.size == P.stream.size and (got == P.stream).all()
 
 
+@pytest.mark.parametrize("shape,b,pzp,R,rows", [((64, 64, 3, 3), 3, 0.8, 8, 0), ((128, 32, 1, 1), 4, 0.6, 10, 0),
+                                                ((16, 96, 7, 7), 2, 0.9, 6, 0), ((40, 128, 3, 3), 5, 0.7, 12, 8),
+                                                ((512, 256, 3, 3), 3, 0.93, 8, 64)])
+def test_device_encoder_writes_the_oracles_bytes_for_the_channels_container(shape, b, pzp, R, rows):
+    """One stream per input channel of an O x I x H x W tensor (Section III-B), encoded on the
+    device: bytes and offsets equal to the oracle's."""
+    O, I, H, Wd = shape
+    n, E = O * I * H * Wd, H * Wd
+    C = n if not rows else rows * I * E
+    spec = tiny_spec(n, bitwidth=b, pzp=pzp, table_log=R, chunk=C)
+    sym = sg.draw_symbols(spec)
+    f = oracle.normalize_freqs(oracle.histogram(sym), spec.alphabet, R)
+    T = oracle.Table(f, R)
+    P = oracle.pack(T, sym, C, I // 32, oracle.CHANNELS, piece=E)
+    f256 = np.zeros(256, dtype=np.uint32)
+    f256[:spec.alphabet] = f
+    tables = torch.zeros(max(ans.ans_table_bytes(R), 256), dtype=torch.uint8, device="cuda")
+    ans.ans_build_decode_tables(f256[None, :], [spec.alphabet], [R], tables.data_ptr(), tables.numel(), _stream())
+    n_sub = -(-n // C) * (I // 32)
+    cap = ans.ans_host_pack_bound(n, C, I, ans.ANS_LAYOUT_CHANNELS)
+    out = torch.full((cap + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+    offs = torch.full((n_sub + 1,), -1, dtype=torch.int64, device="cuda")
+    need = ans.ans_encode_scratch_bytes(n, C, I)
+    scratch = torch.empty(need, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ans.ans_encode_channels_device(_dev(sym).data_ptr(), n, tables.data_ptr(), R, C, I, E, out.data_ptr(), cap,
+                                   offs.data_ptr(), scratch.data_ptr(), need, status.data_ptr(), _stream())
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    o = offs.cpu().numpy().astype(np.uint64)
+    assert (o == P.sub_offsets).all()
+    got = out[:int(o[-1])].cpu().numpy()
+    assert got.size == P.stream.size and (got == P.stream).all()
+    assert (out[cap:].cpu().numpy() == 0xA5).all()
+    # sizes the container does not take are refused
+    with pytest.raises(ans.AnsError):
+        ans.ans_encode_channels_device(_dev(sym).data_ptr(), n, tables.data_ptr(), R, C, I, 0, out.data_ptr(), cap,
+                                       offs.data_ptr(), scratch.data_ptr(), need, status.data_ptr(), _stream())
+    with pytest.raises(ans.AnsError):
+        ans.ans_encode_channels_device(_dev(sym).data_ptr(), n - 1, tables.data_ptr(), R, C, I, E, out.data_ptr(), cap,
+                                       offs.data_ptr(), scratch.data_ptr(), need, status.data_ptr(), _stream())
+
+
 def test_compress_then_decode_on_the_device():
     """The whole loop without the host: histogram, normalise, build the table, encode, decode +
     dequantise; the output is the oracle's dequantisation of the symbols."""
