@@ -378,6 +378,13 @@ int ans_encode_channels_device(const uint8_t* d_symbols, uint64_t n_symbols, con
                                uint32_t chunk_symbols, uint32_t lanes, uint32_t piece_symbols,
                                uint8_t* d_stream_out, uint64_t stream_cap, uint64_t* d_sub_offsets_out,
                                void* d_scratch, size_t d_scratch_bytes, uint32_t* d_status, void* stream);
+/* The same for the quads container: byte for byte what ans_host_pack_layer writes for
+ * ANS_LAYOUT_QUADS, d_lane_meta_out[n_sub][32] included (initial state | first word << 16).  Any
+ * chunk_symbols >= 1; bit 4 of *d_status also if a sub-stream is longer than 65535 words. */
+int ans_encode_quads_device(const uint8_t* d_symbols, uint64_t n_symbols, const void* d_table, int table_log,
+                            uint32_t chunk_symbols, uint32_t lanes, uint8_t* d_stream_out, uint64_t stream_cap,
+                            uint64_t* d_sub_offsets_out, uint32_t* d_lane_meta_out, void* d_scratch,
+                            size_t d_scratch_bytes, uint32_t* d_status, void* stream);
 int ans_encode_layer_device(const uint8_t* d_symbols, uint64_t n_symbols, const void* d_table, int table_log,
                             uint32_t chunk_symbols, uint32_t lanes, int layout, uint8_t* d_stream_out,
                             uint64_t stream_cap, uint64_t* d_sub_offsets_out, void* d_scratch,

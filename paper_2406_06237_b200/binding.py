@@ -29,7 +29,8 @@ EXPORTS = [
     "ans_host_normalize_freqs", "ans_host_pack_bound", "ans_host_pack_layer", "ans_host_pack_channels",
     "ans_noalloc_max_bytes", "ans_decode_dequant_host_noalloc",
     "ans_histogram_device", "ans_entropy_device", "ans_normalize_freqs_device",
-    "ans_encode_scratch_bytes", "ans_encode_layer_device", "ans_encode_channels_device", "ans_decode_gemm_bf16",
+    "ans_encode_scratch_bytes", "ans_encode_layer_device", "ans_encode_channels_device", "ans_encode_quads_device",
+    "ans_decode_gemm_bf16",
 ]
 
 
@@ -95,6 +96,7 @@ def lib():
         L.ans_encode_scratch_bytes.argtypes = [u64, u32, u32, P(sz)]
         L.ans_encode_layer_device.argtypes = [vp, u64, vp, i32, u32, u32, i32, vp, u64, vp, vp, sz, vp, vp]
         L.ans_encode_channels_device.argtypes = [vp, u64, vp, i32, u32, u32, u32, vp, u64, vp, vp, sz, vp, vp]
+        L.ans_encode_quads_device.argtypes = [vp, u64, vp, i32, u32, u32, vp, u64, vp, vp, vp, sz, vp, vp]
         _LIB = L
     return _LIB
 
@@ -277,6 +279,15 @@ def ans_encode_channels_device(d_symbols: int, n_symbols: int, d_table: int, tab
     _check(lib().ans_encode_channels_device(d_symbols, n_symbols, d_table, table_log, chunk_symbols, lanes,
                                             piece_symbols, d_stream_out, stream_cap, d_sub_offsets_out, d_scratch,
                                             d_scratch_bytes, d_status, stream), "ans_encode_channels_device")
+
+
+def ans_encode_quads_device(d_symbols: int, n_symbols: int, d_table: int, table_log: int, chunk_symbols: int,
+                            lanes: int, d_stream_out: int, stream_cap: int, d_sub_offsets_out: int,
+                            d_lane_meta_out: int, d_scratch: int, d_scratch_bytes: int, d_status: int,
+                            stream: int = 0) -> None:
+    _check(lib().ans_encode_quads_device(d_symbols, n_symbols, d_table, table_log, chunk_symbols, lanes, d_stream_out,
+                                         stream_cap, d_sub_offsets_out, d_lane_meta_out, d_scratch, d_scratch_bytes,
+                                         d_status, stream), "ans_encode_quads_device")
 
 
 def ans_host_pack_channels(symbols: np.ndarray, freqs: np.ndarray, alphabet: int, table_log: int,

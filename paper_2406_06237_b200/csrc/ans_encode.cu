@@ -143,8 +143,9 @@ struct EncArgs {
   uint32_t chunk;
   uint32_t G;                  // lanes / 32
   uint32_t piece;              // channels container: symbols of a piece; 0: strips
+  uint32_t* meta;              // quads container (not null): [n_sub][32] initial state | first word << 16
   uint64_t n_sub;
-  uint16_t* lens;              // [n_sub][32] bit length of every lane's string
+  uint32_t* lens;              // [n_sub][32] bit length of every lane's string
   unsigned long long* sizes;   // [n_sub] bytes of every sub-stream
   const unsigned long long* offsets;   // [n_sub + 1], for the writing pass
   uint8_t* out;
@@ -190,7 +191,7 @@ template <bool WRITE>
 __device__ __forceinline__ uint32_t encode_lane(const EncTables& T, int R, const uint8_t* strip, uint32_t count,
                                                 uint32_t lane, uint32_t* body, uint64_t body_words, uint32_t end,
                                                 uint32_t& state_out, bool& bad_symbol, uint32_t piece = 0,
-                                                uint32_t row = 0) {
+                                                uint32_t row = 0, bool state_in_stream = true) {
   const uint32_t L = 1u << R;
   uint32_t x = L, bits = 0;
   uint32_t word = 0, acc = 0;            // WRITE: the word being filled and the bits collected for it
@@ -217,10 +218,10 @@ __device__ __forceinline__ uint32_t encode_lane(const EncTables& T, int R, const
   }
   state_out = x - L;
   if (WRITE && count) {
-    put(x - L, static_cast<uint32_t>(R));
+    if (state_in_stream) put(x - L, static_cast<uint32_t>(R));
     if (have && word < body_words) atomicOr(body + word, acc);
   }
-  return count ? bits + static_cast<uint32_t>(R) : 0u;
+  return count ? bits + (state_in_stream ? static_cast<uint32_t>(R) : 0u) : 0u;
 }
 
 template <bool WRITE>
@@ -250,9 +251,47 @@ __global__ void __launch_bounds__(kEncWarps * 32) encode_strips_kernel(const Enc
   }
   uint32_t state = 0;
   bool bad = false;
+  if (a.meta) {
+    // quads: the chunk is dealt in pieces of four to its lanes, the last piece may be short and the
+    // lanes own different numbers of pieces; a lane's string is its fields alone, padded to a whole
+    // 32-bit word, the strings one after the other, the state in the lane metadata
+    const uint32_t lambda = 32u * g + lane;
+    const uint64_t full = nc / 4u, rem = nc % 4u;
+    count = 4u * static_cast<uint32_t>(full > lambda ? (full - lambda + row - 1u) / row : 0u) +
+            ((rem && full % row == lambda) ? static_cast<uint32_t>(rem) : 0u);
+    strip = a.sym + c0 + size_t(32u * g) * 4u;
+    uint32_t len = WRITE ? a.lens[sub * 32 + lane] : 0u;
+    if (!WRITE) {
+      len = encode_lane<false>(T, a.R, strip, count, lane, nullptr, 0, 0, state, bad, 4u, row, false);
+      a.lens[sub * 32 + lane] = len;
+    }
+    const uint32_t words = (len + 31u) >> 5;
+    uint32_t incl = words;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+      if (lane >= static_cast<uint32_t>(d)) incl += up;
+    }
+    const uint32_t word0 = incl - words, total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    if (!WRITE) {
+      if (lane == 0) a.sizes[sub] = (uint64_t(total) * 4u + 15u) & ~15ull;
+      if (word0 > 0xFFFFu) bad = true;
+    } else {
+      const unsigned long long off0 = a.offsets[sub], off1 = a.offsets[sub + 1];
+      if (off1 <= a.cap) {
+        uint32_t* body = reinterpret_cast<uint32_t*>(a.out + off0);
+        encode_lane<true>(T, a.R, strip, count, lane, body, (off1 - off0) / 4, word0 * 32u + len, state, bad, 4u, row, false);
+        a.meta[sub * 32 + lane] = state | (word0 << 16);
+      } else if (lane == 0 && a.status) {
+        atomicOr(a.status, 2u);
+      }
+    }
+    if (bad && a.status) atomicOr(a.status, 4u);
+    return;
+  }
   if (!WRITE) {
     const uint32_t len = encode_lane<false>(T, a.R, strip, count, lane, nullptr, 0, 0, state, bad, a.piece, row);
-    a.lens[sub * 32 + lane] = static_cast<uint16_t>(len);
+    a.lens[sub * 32 + lane] = len;
     uint32_t total = len;
 #pragma unroll
     for (int d = 16; d; d >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, d);
@@ -347,12 +386,12 @@ ANS_EXPORT int ans_encode_scratch_bytes(uint64_t n_symbols, uint32_t chunk_symbo
   if (n_symbols > (uint64_t(1) << 46)) return ANS_ERR_INVALID_ARG;
   const uint64_t chunks = n_symbols ? (n_symbols + chunk_symbols - 1) / chunk_symbols : 0;
   const uint64_t n_sub = chunks * (lanes / 32);
-  *h_bytes_out = up256(n_sub * 64) + up256(n_sub * 8) + 256;
+  *h_bytes_out = up256(n_sub * 128) + up256(n_sub * 8) + 256;
   return ANS_OK;
 }
 
 static int encode_device(const uint8_t* d_symbols, uint64_t n_symbols, const void* d_table, int table_log,
-                         uint32_t chunk_symbols, uint32_t lanes, uint32_t piece, uint8_t* d_stream_out,
+                         uint32_t chunk_symbols, uint32_t lanes, uint32_t piece, uint32_t* d_lane_meta_out, uint8_t* d_stream_out,
                          uint64_t stream_cap, uint64_t* d_sub_offsets_out, void* d_scratch,
                          size_t d_scratch_bytes, uint32_t* d_status, void* stream) {
   if (!d_sub_offsets_out || !d_status) return ANS_ERR_INVALID_ARG;
@@ -363,7 +402,7 @@ static int encode_device(const uint8_t* d_symbols, uint64_t n_symbols, const voi
     const uint64_t unit = uint64_t(lanes) * piece;
     if (chunk_symbols % unit || n_symbols % unit || chunk_symbols / lanes > ANS_MAX_CHANNEL_LANE_SYMBOLS)
       return ANS_ERR_UNSUPPORTED;
-  } else if (chunk_symbols % lanes || chunk_symbols / lanes > ANS_MAX_STRIP_LANE_SYMBOLS) {
+  } else if (!d_lane_meta_out && (chunk_symbols % lanes || chunk_symbols / lanes > ANS_MAX_STRIP_LANE_SYMBOLS)) {
     return ANS_ERR_UNSUPPORTED;
   }
   size_t need = 0;
@@ -388,10 +427,11 @@ static int encode_device(const uint8_t* d_symbols, uint64_t n_symbols, const voi
   a.chunk = chunk_symbols;
   a.G = lanes / 32;
   a.piece = piece;
+  a.meta = d_lane_meta_out;
   a.n_sub = ((n_symbols + chunk_symbols - 1) / chunk_symbols) * a.G;
   if (a.n_sub > 0x7FFFFFFFull * kEncWarps) return ANS_ERR_UNSUPPORTED;
   uint8_t* p = static_cast<uint8_t*>(d_scratch);
-  a.lens = reinterpret_cast<uint16_t*>(p); p += up256(a.n_sub * 64);
+  a.lens = reinterpret_cast<uint32_t*>(p); p += up256(a.n_sub * 128);
   a.sizes = reinterpret_cast<unsigned long long*>(p);
   a.offsets = reinterpret_cast<const unsigned long long*>(d_sub_offsets_out);
   a.out = d_stream_out;
@@ -415,7 +455,7 @@ ANS_EXPORT int ans_encode_layer_device(const uint8_t* d_symbols, uint64_t n_symb
                                        uint64_t stream_cap, uint64_t* d_sub_offsets_out, void* d_scratch,
                                        size_t d_scratch_bytes, uint32_t* d_status, void* stream) {
   if (layout != ANS_LAYOUT_STRIPS) return ANS_ERR_UNSUPPORTED;
-  return encode_device(d_symbols, n_symbols, d_table, table_log, chunk_symbols, lanes, 0, d_stream_out, stream_cap,
+  return encode_device(d_symbols, n_symbols, d_table, table_log, chunk_symbols, lanes, 0, nullptr, d_stream_out, stream_cap,
                        d_sub_offsets_out, d_scratch, d_scratch_bytes, d_status, stream);
 }
 
@@ -424,6 +464,17 @@ ANS_EXPORT int ans_encode_channels_device(const uint8_t* d_symbols, uint64_t n_s
                                           uint8_t* d_stream_out, uint64_t stream_cap, uint64_t* d_sub_offsets_out,
                                           void* d_scratch, size_t d_scratch_bytes, uint32_t* d_status, void* stream) {
   if (piece_symbols < 1) return ANS_ERR_UNSUPPORTED;
-  return encode_device(d_symbols, n_symbols, d_table, table_log, chunk_symbols, lanes, piece_symbols, d_stream_out,
+  return encode_device(d_symbols, n_symbols, d_table, table_log, chunk_symbols, lanes, piece_symbols, nullptr, d_stream_out,
                        stream_cap, d_sub_offsets_out, d_scratch, d_scratch_bytes, d_status, stream);
+}
+
+ANS_EXPORT int ans_encode_quads_device(const uint8_t* d_symbols, uint64_t n_symbols, const void* d_table, int table_log,
+                                       uint32_t chunk_symbols, uint32_t lanes, uint8_t* d_stream_out, uint64_t stream_cap,
+                                       uint64_t* d_sub_offsets_out, uint32_t* d_lane_meta_out, void* d_scratch,
+                                       size_t d_scratch_bytes, uint32_t* d_status, void* stream) {
+  if (n_symbols && (!d_lane_meta_out || (reinterpret_cast<uintptr_t>(d_lane_meta_out) & 3))) return ANS_ERR_INVALID_ARG;
+  static uint32_t dummy = 0;                               // (an empty layer writes no metadata)
+  return encode_device(d_symbols, n_symbols, d_table, table_log, chunk_symbols, lanes, 0,
+                       d_lane_meta_out ? d_lane_meta_out : &dummy, d_stream_out, stream_cap, d_sub_offsets_out, d_scratch,
+                       d_scratch_bytes, d_status, stream);
 }

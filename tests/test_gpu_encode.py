@@ -170,6 +170,42 @@ def test_device_encoder_writes_the_oracles_bytes_for_the_channels_container(shap
                                        offs.data_ptr(), scratch.data_ptr(), need, status.data_ptr(), _stream())
 
 
+@pytest.mark.parametrize("n,C,lanes,R,b,pzp", [(36864, 4096, 32, 12, 4, 0.6), (5000, 1024, 64, 8, 3, 0.9),
+                                               (100_003, 16384, 128, 11, 6, 0.8), (33, 128, 32, 6, 2, 0.7),
+                                               (70_001, 65536, 256, 14, 8, 0.3), (4097, 4096, 32, 12, 1, 0.6),
+                                               (131, 512, 32, 5, 3, 0.7), (1_300_002, 32768, 32, 8, 3, 0.7),
+                                               (0, 4096, 32, 8, 4, 0.6), (1, 32, 32, 1, 1, 0.6), (7, 1000, 96, 4, 2, 0.6)])
+def test_device_encoder_writes_the_oracles_bytes_for_the_quads_container(n, C, lanes, R, b, pzp):
+    """Bytes, offsets and lane metadata (initial state, first word) equal to the oracle's."""
+    spec = tiny_spec(max(n, 1), bitwidth=b, pzp=pzp, table_log=R, chunk=C)
+    sym = sg.draw_symbols(spec)
+    T, _, f256 = oracle_pack_spec(spec, sym, oracle.QUADS, lanes)
+    sym = sym[:n]
+    P = oracle.pack(T, sym, C, lanes // 32, oracle.QUADS)
+    tables = torch.zeros(max(ans.ans_table_bytes(R), 256), dtype=torch.uint8, device="cuda")
+    ans.ans_build_decode_tables(f256[None, :], [spec.alphabet], [R], tables.data_ptr(), tables.numel(), _stream())
+    n_sub = -(-n // C) * (lanes // 32)
+    cap = ans.ans_host_pack_bound(n, C, lanes, ans.ANS_LAYOUT_QUADS)
+    out = torch.full((cap + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+    offs = torch.full((n_sub + 1,), -1, dtype=torch.int64, device="cuda")
+    meta = torch.full((max(n_sub, 1), 32), -1, dtype=torch.int32, device="cuda")
+    need = ans.ans_encode_scratch_bytes(n, C, lanes)
+    scratch = torch.empty(need, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    d = _dev(sym) if n else torch.zeros(1, dtype=torch.uint8, device="cuda")
+    ans.ans_encode_quads_device(d.data_ptr(), n, tables.data_ptr(), R, C, lanes, out.data_ptr(), cap, offs.data_ptr(),
+                                meta.data_ptr(), scratch.data_ptr(), need, status.data_ptr(), _stream())
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    o = offs.cpu().numpy().astype(np.uint64)
+    assert (o == P.sub_offsets).all()
+    got = out[:int(o[-1])].cpu().numpy()
+    assert got.size == P.stream.size and (got == P.stream).all()
+    if n:
+        assert (meta.cpu().numpy().view(np.uint32)[:n_sub] == P.lane_meta.reshape(n_sub, 32)).all()
+    assert (out[cap:].cpu().numpy() == 0xA5).all()
+
+
 def test_compress_then_decode_on_the_device():
     """The whole loop without the host: histogram, normalise, build the table, encode, decode +
     dequantise; the output is the oracle's dequantisation of the symbols."""
