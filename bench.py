@@ -5,9 +5,18 @@ One step = one pass of the whole hot path (stage tables, read compressed streams
 dequantise, store) over one synthetic workload, as ONE batched kernel launch.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload large|resnet50|resnet18|conv3x3|sweep]
-                  [--layout private|interleaved|quads] [--lanes 32|64|128|256] [--impl ours|reference]
+                  [--layout private|interleaved|quads|strips] [--lanes 32|64|128|256] [--impl ours|reference]
+                  [--no-settled | --no-idle] [--no-variants] [--no-fused] [--fused-only]
 
 Prints one JSON line (rank 0).  With --impl reference the CPU oracle is timed instead.
+
+The timed launches are queued back to back and rotate over at least two full sets of buffers; the
+layer descriptors say that the inputs were settled before the timing began and that a launch does not
+touch the output set of the launch before it (ANS_DESC_INPUTS_SETTLED | ANS_DESC_OUTPUT_IDLE), so
+consecutive launches may overlap at their ends and the per-launch time is the rate of a stream of
+decode calls.  --no-idle keeps the first flag only (a launch waits for the one before it before its
+first write), --no-settled neither (it waits before it reads anything); the line also carries the
+headline workload timed without the flags, and a launch bracketed alone by its own pair of events.
 """
 from __future__ import annotations
 
