@@ -34,8 +34,7 @@ namespace ansb {
   "setp.ne.u32 q, t, 0;\n\t"                                      \
   "@q mov.u32 %2, %3;\n\t"                                        \
   "@q mov.u32 %3, %4;\n\t"                                        \
-  "@q ld.shared.u32 nw, [%5];\n\t"                                \
-  "@q mov.u32 %4, nw;\n\t"                                        \
+  "@q ld.shared.u32 %4, [%5];\n\t"                                \
   "@q add.u32 %5, %5, 4;\n\t"                                     \
   "and.b32 %1, %1, 31;\n\t"
 #define ANSB_LS_G4(S_, A0, A1, A2, A3)                            \

@@ -31,8 +31,7 @@ __device__ __forceinline__ uint32_t to_strip_entry_short(uint32_t g, uint32_t va
   "setp.ne.u32 pq, tt, 0;\n\t"                                    \
   "@pq mov.u32 %2, %3;\n\t"                                       \
   "@pq mov.u32 %3, %4;\n\t"                                       \
-  "@pq ld.shared.u32 nw, [%5];\n\t"                               \
-  "@pq mov.u32 %4, nw;\n\t"                                       \
+  "@pq ld.shared.u32 %4, [%5];\n\t"                               \
   "@pq add.u32 %5, %5, 4;\n\t"                                    \
   "and.b32 %1, %1, 31;\n\t"
 // One look-up.  %6: the lane's next position; zn: the position of the symbol that ends the run;
