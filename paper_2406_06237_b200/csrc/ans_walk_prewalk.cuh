@@ -102,8 +102,7 @@ __device__ __forceinline__ void pair_steps(uint32_t& st, uint32_t& tbm, uint32_t
       "setp.ne.u32 q, t, 0;\n\t"                                                           \
       "@q mov.u32 %3, %4;\n\t"                                                             \
       "@q mov.u32 %4, %5;\n\t"                                                             \
-      "@q ld.shared.u32 nw, [%6];\n\t"                                                     \
-      "@q mov.u32 %5, nw;\n\t"                                                             \
+      "@q ld.shared.u32 %5, [%6];\n\t"                                                     \
       "@q add.u32 %6, %6, 4;\n\t"
 #define ANSB_PAIRS(ADV_, STOP_)                                                            \
   asm volatile(                                                                            \
