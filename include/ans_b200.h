@@ -168,6 +168,7 @@ typedef struct ans_layer_desc {
  * kernel then does not wait for the preceding work at all, except before it sets a bit in
  * *d_status.  Work that follows the call on the stream is ordered after it as always.
  *
+ * ans_decode_layer, which writes d_symbols_out and not d_out, honours the first flag only.
  * The host-buffer calls (ans_decode_dequant_host, ans_decode_dequant_host_noalloc) copy their
  * inputs in on the same stream and ignore the flags; so do the encoder and ans_decode_gemm_bf16. */
 #define ANS_DESC_INPUTS_SETTLED 1u

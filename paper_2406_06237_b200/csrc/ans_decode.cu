@@ -562,6 +562,7 @@ ANS_EXPORT int ans_decode_layer(const ans_layer_desc* h_desc, uint8_t* d_symbols
   if (!h_desc || !d_status) return ANS_ERR_INVALID_ARG;
   if (!d_symbols_out && h_desc->n_symbols) return ANS_ERR_INVALID_ARG;
   ans_layer_desc d = *h_desc;
+  d.flags &= ~ANS_DESC_OUTPUT_IDLE;                        // (that flag speaks of d_out, which this call does not write)
   const int rc = ans_plan_batch(&d, 1, nullptr);
   if (rc != ANS_OK) return rc;
   if (d.n_symbols == 0) return validate_desc(d, false);
