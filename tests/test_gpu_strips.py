@@ -148,6 +148,39 @@ def test_launches_queued_back_to_back_with_the_settled_inputs_flags(idle):
     assert db2.read_status() != 0
 
 
+@pytest.mark.parametrize("layout,lanes", [(STRIPS, 64), (ans.ANS_LAYOUT_QUADS, 32)])
+def test_decode_launches_captured_in_a_cuda_graph(layout, lanes):
+    """Six batched decode launches (descriptor flags set, rotating over three output sets) captured
+    from a stream into a CUDA graph and replayed three times; every set holds the oracle's bits."""
+    specs = [tiny_spec(300_000, 3, 0.9, 8, 16384, "bf16", index=0), tiny_spec(70_001, 4, 0.7, 8, 4096, "f32", index=1),
+             tiny_spec(150_000, 2, 0.95, 7, 8192, "u8", index=3)]
+    prepared = []
+    for spec in specs:
+        sym = sg.draw_symbols(spec)
+        T, P, f256 = oracle_pack_spec(spec, sym, layout, lanes)
+        prepared.append((to_packed_layer(spec, P, f256), oracle_expected(spec, T, P)[1]))
+    db = DeviceBatch([p[0] for p in prepared], n_out_sets=3, inputs_settled=True, output_idle=True)
+    db.decode(0)                                          # the first call sets the kernels' attributes: outside the capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(6):
+                db.decode(i % 3, stream=side.cuda_stream)
+    for outs in db.out_sets:
+        for o in outs:
+            o.view(torch.uint8).fill_(0xA5)
+    torch.cuda.synchronize()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert db.read_status() == 0
+    for k in range(3):
+        for i, (pl, want) in enumerate(prepared):
+            assert (bits_view(db.output(i, k)) == expected_bits(want)).all(), (k, i)
+
+
 def test_long_substreams_read_from_global_memory():
     """Sub-streams too long for the shared-memory staging buffer (here beside short ones of another
     layer, which size the buffer) are read word by word from global memory."""
