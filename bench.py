@@ -388,7 +388,7 @@ def entropy_bits(specs, syms):
 VARIANTS = [("large", "quads", 32, 12, 0, 3), ("resnet50", "strips", 32, 0, 0, 3),
             ("resnet50", "strips", 64, 0, 0, 3), ("resnet50", "strips", 64, 0, 0, 1), ("resnet50", "strips", 64, 0, 0, 0),
             ("resnet50", "strips", 32, 0, 0, 0), ("resnet50", "quads", 32, 0, 0, 3),
-            ("resnet50", "strips", 64, 12, 0, 3), ("resnet18", "strips", 64, 0, 0, 3),
+            ("resnet50", "strips", 32, 12, 0, 3), ("resnet18", "strips", 64, 0, 0, 3),
             ("resnet18", "quads", 32, 0, 0, 3), ("sweep", "quads", 32, 12, 16384, 3)]
 
 
