@@ -237,19 +237,23 @@ def reduce_max(x: float, world: int) -> float:
 
 
 MIN_REGION_S = 0.5          # device time the timed rounds of a workload add up to, at least
+LATER_ROUND = 100           # launches of every timed round after the first, at least
 
 
 def time_workload(db, steps, warmup, n_sets, world, min_region_s=MIN_REGION_S, max_rounds=2000):
     """Rounds of K back-to-back launches, each round bracketed by CUDA events on the launching
     stream.  The host must not be what is timed, so every round goes behind a device-side spin of
     a few milliseconds (outside the brackets): by the time the device reaches the first launch all
-    K are queued.  The first round is the K steps the command line asked for; further rounds
-    repeat them until the rounds add up to min_region_s of device time, so that clock samples
-    fall inside the timed region.  A last round brackets every launch by itself.
-    Returns (per-round milliseconds per step, per-launch milliseconds of the last round)."""
+    K are queued.  The first round is the K steps the command line asked for; further rounds (of
+    at least LATER_ROUND launches each, so that a round's first and last launch, which overlap
+    nothing, weigh little) repeat until the rounds add up to min_region_s of device time, so that
+    clock samples fall inside the timed region.  A last round brackets every launch by itself.
+    Returns (per-round milliseconds per step, per-launch milliseconds of the last round); the
+    launches made are counted in time_workload.launches."""
     import torch
     import torch.distributed as dist
     st = torch.cuda.current_stream()
+    time_workload.launches = warmup * db.launches_per_decode()
     for i in range(warmup):
         db.decode(i % n_sets)
     torch.cuda.synchronize()
@@ -258,9 +262,10 @@ def time_workload(db, steps, warmup, n_sets, world, min_region_s=MIN_REGION_S, m
     torch.cuda.synchronize()
     spin = int(2e7)                                       # cycles: about 10 ms
 
-    def one_round(per_launch=False):
+    def one_round(per_launch=False, n=steps):
         evs = []
         torch.cuda._sleep(spin)
+        time_workload.launches += n * db.launches_per_decode()
         if per_launch:
             for i in range(steps):
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -271,7 +276,7 @@ def time_workload(db, steps, warmup, n_sets, world, min_region_s=MIN_REGION_S, m
         else:
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(st)
-            for i in range(steps):
+            for i in range(n):
                 db.decode(i % n_sets)
             b.record(st)
             evs.append((a, b))
@@ -279,10 +284,11 @@ def time_workload(db, steps, warmup, n_sets, world, min_region_s=MIN_REGION_S, m
 
     rounds, total_ms = [], 0.0
     while True:
-        ev = one_round()
+        n = steps if not rounds else max(steps, LATER_ROUND)
+        ev = one_round(n=n)
         torch.cuda.synchronize()
         ms = ev[0][0].elapsed_time(ev[0][1])
-        rounds.append(ms / steps)
+        rounds.append(ms / n)
         total_ms += ms
         if total_ms >= min_region_s * 1e3 or len(rounds) >= max_rounds:
             break
@@ -515,6 +521,7 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     sampler.first = len(sampler.rows)
     rounds, each = time_workload(db, args.steps, args.warmup, n_sets, world)
+    launches = time_workload.launches
     sampler.last = len(sampler.rows)
     db_flags = db.h_descs[0][0].flags if layers else 0
     clocks = sampler.summary() if rank == 0 else None
@@ -523,6 +530,7 @@ def run_ours(args):
     if db_flags and world == 1:
         db.set_flags(0)
         wr, _ = time_workload(db, args.steps, 3, n_sets, world, min_region_s=0.15)
+        launches += time_workload.launches + 3
         waiting_ms = sum(wr) / len(wr)
         db.set_flags(int(db_flags))
     ms_per_step = reduce_max(rounds[0], world)          # the K steps asked for: the first round
@@ -537,7 +545,7 @@ def run_ours(args):
     roofline = {"bound": "hbm", "achieved": fg["achieved"], "peak": peak, "unit": "GB/s", "frac": fg["frac"],
                 "traffic": traffic, "kernel": kname, "peak_kind": f"of {peak_kind}",
                 "algorithmic_bytes_per_launch": fg["algo_bytes"], "kernel_ms_mean": fg["kernel_ms"],
-                "timed_rounds": len(rounds), "launches_per_round": args.steps,
+                "timed_rounds": len(rounds), "launches_per_round": [args.steps, max(args.steps, LATER_ROUND)],
                 "round_ms_per_launch_min": min(rounds), "round_ms_per_launch_max": max(rounds),
                 "launch_bracketed_alone_ms_median": statistics.median(each), "launch_bracketed_alone_ms_min": min(each),
                 "frac_of_nominal_8TBs": fg["frac_nominal"],
@@ -555,9 +563,6 @@ def run_ours(args):
     ent_bits = entropy_bits(specs, syms)
     cpu = cpu_baseline(specs, syms, args.layout, args.lanes) if world == 1 and rank == 0 and not args.no_cpu_baseline else None
     head_specs = specs
-    launches = (len(rounds) + 1) * args.steps * db.launches_per_decode()
-    if waiting_ms is not None:
-        launches += (len(wr) + 1) * args.steps * db.launches_per_decode() + 3
 
     # the other workloads and table sizes, each measured the same way (shorter regions)
     variants = []
@@ -582,7 +587,7 @@ def run_ours(args):
                              "entropy_bits_per_weight": entropy_bits(vs, vy) / max(1, vf["n_w"]),
                              "desc_flags": int(vdb.h_descs[0][0].flags),
                              "l2_policy": vpol, "clocks": sampler.summary()})
-            launches += (len(vr) + 1) * (min(args.steps, 200) if wl in ("large", "sweep") else max(args.steps, 100)) * vdb.launches_per_decode()
+            launches += time_workload.launches
             del vdb
             torch.cuda.empty_cache()
     fused = None
