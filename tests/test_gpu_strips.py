@@ -148,6 +148,31 @@ def test_launches_queued_back_to_back_with_the_settled_inputs_flags(idle):
     assert db2.read_status() != 0
 
 
+def test_a_batch_of_more_layers_than_one_launch_holds_with_the_flags_set():
+    """70 small layers are two launches of the strips kernel per call; with both flags set the
+    second does not wait for the first.  Four calls queued back to back over two output sets."""
+    specs = [tiny_spec(3000 + 517 * i, 1 + i % 6, 0.6 + 0.005 * i, 5 + i % 4, 2048, ("bf16", "u8", "f32")[i % 3], index=i)
+             for i in range(70)]
+    prepared = []
+    for spec in specs:
+        sym = sg.draw_symbols(spec)
+        T, P, f256 = oracle_pack_spec(spec, sym, STRIPS, 64)
+        prepared.append((to_packed_layer(spec, P, f256), oracle_expected(spec, T, P)[1]))
+    db = DeviceBatch([p[0] for p in prepared], n_out_sets=2, inputs_settled=True, output_idle=True)
+    assert db.launches_per_decode() == 2
+    for outs in db.out_sets:
+        for o in outs:
+            o.view(torch.uint8).fill_(0xA5)
+    torch.cuda.synchronize()
+    torch.cuda._sleep(10_000_000)
+    for i in range(4):
+        db.decode(i % 2)
+    assert db.read_status() == 0
+    for k in range(2):
+        for i, (pl, want) in enumerate(prepared):
+            assert (bits_view(db.output(i, k)) == expected_bits(want)).all(), (k, i)
+
+
 @pytest.mark.parametrize("layout,lanes", [(STRIPS, 64), (ans.ANS_LAYOUT_QUADS, 32)])
 def test_decode_launches_captured_in_a_cuda_graph(layout, lanes):
     """Six batched decode launches (descriptor flags set, rotating over three output sets) captured
