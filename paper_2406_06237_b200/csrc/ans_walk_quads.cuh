@@ -59,21 +59,23 @@ __device__ __forceinline__ uint2 to_quads_entry(uint32_t g, uint32_t val, bool n
 // four look-ups of one turn: one refill check when a symbol takes at most 8 bits, else two
 #define ANSB_QD_TURN4(ST_) ANSB_QD_BEGIN ST_("0") ST_("1") ST_("2") ST_("3") ANSB_LS_END
 #define ANSB_QD_TURN2(ST_) ANSB_QD_BEGIN ST_("0") ST_("1") ANSB_LS_END ANSB_QD_BEGIN ST_("2") ST_("3") ANSB_LS_END
+// (the stores carry the streaming hint: an output line is written once and not read again by
+// this kernel, and evicting it first leaves L2 to the compressed bytes and to the other writes)
 #define ANSB_QD_OUT1(A_)                                          \
   "prmt.b32 v0, ea0, ea1, 0x0062;\n\t"                            \
   "prmt.b32 v1, ea2, ea3, 0x0062;\n\t"                            \
   "prmt.b32 v0, v0, v1, 0x5410;\n\t"                              \
-  "st.global.u32 " A_ ", v0;\n\t"
+  "st.global.cs.u32 " A_ ", v0;\n\t"
 #define ANSB_QD_OUT1S(A_)                                         \
   "prmt.b32 v0, ea0, ea1, 0x0073;\n\t"                            \
   "prmt.b32 v1, ea2, ea3, 0x0073;\n\t"                            \
   "prmt.b32 v0, v0, v1, 0x5410;\n\t"                              \
-  "st.global.u32 " A_ ", v0;\n\t"
+  "st.global.cs.u32 " A_ ", v0;\n\t"
 #define ANSB_QD_OUT2(A_)                                          \
   "prmt.b32 v0, ea0, ea1, 0x7632;\n\t"                            \
   "prmt.b32 v1, ea2, ea3, 0x7632;\n\t"                            \
-  "st.global.v2.u32 " A_ ", {v0, v1};\n\t"
-#define ANSB_QD_OUT4(A_) "st.global.v4.u32 " A_ ", {eb0, eb1, eb2, eb3};\n\t"
+  "st.global.cs.v2.u32 " A_ ", {v0, v1};\n\t"
+#define ANSB_QD_OUT4(A_) "st.global.cs.v4.u32 " A_ ", {eb0, eb1, eb2, eb3};\n\t"
 
 constexpr uint32_t kQuadTurns = 4;     // turns (of four symbols per lane) per trip of the PTX loop
 
