@@ -120,9 +120,11 @@ __global__ void __launch_bounds__(MANY ? 896 : 512, 1) ans_decode_kernel(const L
         if (lane == 0) {
           const uint32_t bytes = static_cast<uint32_t>(it.extent);
           asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+          uint64_t pol;                                   // (the bytes are read once: they need not stay in L2)
+          asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
           asm volatile(
-              "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-              :: "r"(stage_abs), "l"(L.d_stream + it.off0), "r"(bytes), "r"(bar) : "memory");
+              "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+              :: "r"(stage_abs), "l"(L.d_stream + it.off0), "r"(bytes), "r"(bar), "l"(pol) : "memory");
         }
         for (uint32_t i = lane; i < kStagePad / 4u; i += 32u) reinterpret_cast<uint32_t*>(stage + it.extent)[i] = 0u;
       }
