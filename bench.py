@@ -42,10 +42,10 @@ FALLBACK_PEAK_GBS = 6650.0
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the 8 matrices, from the 2-matrix capture in
-# profiles/ans_decode_kernel_quads_large.md: reads scale with the matrices (4 x 25.41 MB); writes are the
+# profiles/ans_decode_kernel_quads_large.md: reads scale with the matrices (4 x 25.20 MB); writes are the
 # output (1073.74 MB) less what is still in L2 when the kernel ends, which the capture shows as
-# 268.44 - 217.76 = 50.68 MB (40-51 MB from capture to capture, whatever the size)
-NCU_TRAFFIC = {("large", "quads", 32, 8, 8192, 0, 0): 4 * 25.41e6 + 1073.74e6 - 50.68e6}      # 256-state table (the default)
+# 268.44 - 217.17 = 51.27 MB (40-51 MB from capture to capture, whatever the size)
+NCU_TRAFFIC = {("large", "quads", 32, 8, 8192, 0, 0): 4 * 25.20e6 + 1073.74e6 - 51.27e6}      # 256-state table (the default)
 
 
 def measured_peak():
